@@ -1,0 +1,225 @@
+/*
+ * pc.h -- C ABI of the Pilot-Commit group-rollout engine for NVIDIA B200 (sm_100a).
+ *
+ * The library generates the rollouts of group-based RL post-training the way the
+ * Pilot-Commit method spends them (Section 3.3 of the paper): every prompt of a
+ * sampling batch is evaluated once, its key/value cache stays resident and is
+ * shared by all rollouts of its group in both the pilot stage (n_pilot rollouts per
+ * prompt) and the commit stage (n_commit more rollouts for the prompts that pass the
+ * pilot filter); rewards of each group are reduced to the statistics of Eq. 3, the
+ * pilot filter / eviction / commit allocation of Algorithm 1 is evaluated on the
+ * device, and the group-relative advantages of Section 3.1 are produced for the
+ * union of pilot and commit rollouts.
+ *
+ * Conventions
+ *  - Every function returns an int status (PC_OK = 0).  Errors found on the host
+ *    (bad arguments, shapes, alignment, capacity) are returned before anything is
+ *    launched.  Nothing here synchronises the stream: work is asynchronous.
+ *  - The caller owns all device memory: weights, KV arenas, workspace, inputs,
+ *    outputs.  The library never allocates or frees device memory.
+ *  - "device" / "host" in a comment says where a pointer must point.
+ *  - Matrices are row-major [out_features, in_features] in the model's storage type
+ *    (dtype): float (PC_DTYPE_F32) or bfloat16 (PC_DTYPE_BF16).  Norm gains and
+ *    biases are always float arrays.  The residual stream, softmax, logits and all
+ *    statistics are float; dot products accumulate in float.
+ *  - KV arena layout (prompt arena and suffix arena alike):
+ *        [n_layers][2 (0 = K after RoPE, 1 = V)][n_kv_heads][n_slots][head_dim]
+ *    in the model's storage type; a "slot" holds one token position.  A prompt or a
+ *    rollout owns a contiguous range of slots given by its first slot (int64).
+ *  - Index arrays are int32, slot numbers and token-buffer indices int64.
+ *  - Device-side anomalies (an index outside its arena, a wait that ran out) set
+ *    *dev_error_flag (see pc_set_workspace) to a non-zero code and skip the access;
+ *    no kernel traps.
+ */
+#ifndef PC_H_
+#define PC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(PC_BUILDING_LIB) && defined(__GNUC__)
+#define PC_API __attribute__((visibility("default")))
+#else
+#define PC_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    PC_OK = 0,
+    PC_ERR_INVALID_ARG = 1,   /* null pointer, negative count, bad enum                      */
+    PC_ERR_SHAPE = 2,         /* model dimensions the kernels do not support                 */
+    PC_ERR_ALIGNMENT = 3,     /* a pointer is not aligned to 16 bytes (256 for the workspace) */
+    PC_ERR_CAPACITY = 4,      /* more rows / tokens than the workspace was sized for         */
+    PC_ERR_UNSUPPORTED = 5,
+    PC_ERR_CUDA = 6,          /* a CUDA runtime / driver call failed; see pc_last_cuda_error */
+    PC_ERR_NO_WORKSPACE = 7
+};
+
+enum { PC_DTYPE_F32 = 0, PC_DTYPE_BF16 = 1 };
+
+/* Status of a prompt after the pilot stage (Section 3.3; Algorithm 1, Filter / Commit). */
+enum {
+    PC_STATUS_COMMIT = 0,      /* passed the filter and received n_commit more rollouts          */
+    PC_STATUS_BUFFERED = 1,    /* passed the filter but b_t prompts were already selected         */
+    PC_STATUS_DEFER_HARD = 2,  /* p_hat < p_lower                                                */
+    PC_STATUS_SKIP_EASY = 3    /* p_hat > p_upper                                                */
+};
+
+typedef struct pc_ctx pc_ctx;
+
+/* Qwen2/3-style pre-norm decoder (the model families of Section 4.1). */
+typedef struct pc_model_desc {
+    int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab;
+    float rms_eps;
+    float rope_theta;
+    int32_t dtype;       /* PC_DTYPE_*: type of matrices, embedding and KV arenas          */
+    int32_t tied_embed;  /* 1: the LM head is the embedding matrix                         */
+    int32_t qk_norm;     /* 1: per-head RMSNorm of q and k over head_dim, before RoPE      */
+    int32_t qkv_bias;    /* 1: q/k/v projections have a bias                               */
+} pc_model_desc;
+
+/* Device pointers to the weights.  The per-layer members are HOST arrays of n_layers
+ * DEVICE pointers; the arrays are copied by pc_create, the tensors are not.
+ *   embed      [vocab, d_model]                      lm_head [vocab, d_model] or NULL if tied
+ *   final_norm [d_model] float
+ *   attn_norm  [d_model] float                       mlp_norm [d_model] float
+ *   wqkv       [(Hq + 2 Hkv) * head_dim, d_model]    rows: all q heads, then k heads, then v heads
+ *   bqkv       [(Hq + 2 Hkv) * head_dim] float, or NULL array when qkv_bias = 0
+ *   q_norm, k_norm [head_dim] float, or NULL arrays when qk_norm = 0
+ *   wo         [d_model, Hq * head_dim]
+ *   w_gate_up  [2 * d_ff, d_model]   INTERLEAVED: row 2j = gate row j, row 2j+1 = up row j
+ *   w_down     [d_model, d_ff]
+ */
+typedef struct pc_weights {
+    const void* embed;
+    const void* lm_head;
+    const float* final_norm;
+    const float* const* attn_norm;
+    const void* const* wqkv;
+    const float* const* bqkv;
+    const float* const* q_norm;
+    const float* const* k_norm;
+    const void* const* wo;
+    const float* const* mlp_norm;
+    const void* const* w_gate_up;
+    const void* const* w_down;
+} pc_weights;
+
+/* Seeded sampling (Section 4.2: temperature 1.0, top_p 1.0 in training). */
+typedef struct pc_sample_params {
+    float temperature;   /* > 0 */
+    uint64_t seed;
+} pc_sample_params;
+
+/* Pilot filter, eviction and commit allocation (Section 3.3, 3.4; defaults of Section 4.2:
+ * p_lower 0.125, p_upper 0.75, p_solve 1.0). */
+typedef struct pc_alloc_params {
+    double p_lower, p_upper, p_solve;
+    int32_t n_commit;   /* rollouts added to a committed prompt */
+    int32_t b_t;        /* at most this many prompts commit     */
+} pc_alloc_params;
+
+PC_API const char* pc_status_string(int status);
+/* Text of the last CUDA error seen by this thread inside the library (host pointer, static storage). */
+PC_API const char* pc_last_cuda_error(void);
+
+/* Builds a context: copies the description and the pointer tables (host memory only)
+ * and, for bf16 models, encodes the TMA descriptors of the weight matrices.  Needs a
+ * current CUDA device for bf16 models.  Shapes: head_dim in {64, 128}; n_q_heads a
+ * multiple of n_kv_heads with ratio <= 8; d_model, d_ff, q/kv widths multiples of 8;
+ * bf16 additionally needs d_model, d_ff and Hq*head_dim multiples of 64. */
+PC_API int pc_create(const pc_model_desc* desc, const pc_weights* weights, pc_ctx** out);
+PC_API void pc_destroy(pc_ctx* ctx);
+
+/* Scratch the kernels need for at most max_rows concurrent rollouts per decode step and
+ * max_prefill_tokens packed prompt tokens per prefill call. */
+PC_API int pc_workspace_bytes(const pc_ctx* ctx, int max_rows, int max_prefill_tokens, size_t* out_bytes);
+/* dev_ws: device, 256-byte aligned, at least `bytes` long, untouched by the caller while
+ * work of this context is in flight.  dev_error_flag: device int32, zeroed by the caller;
+ * kernels store a non-zero code there when they meet an out-of-range index. */
+PC_API int pc_set_workspace(pc_ctx* ctx, void* dev_ws, size_t bytes, int max_rows, int max_prefill_tokens,
+                     int32_t* dev_error_flag);
+
+/* Shared prefill (Section 3.1: o ~ pi_theta(. | q); Section 3.3: pilot and commit rollouts of a
+ * prompt are drawn from the same pi_theta(. | q), so q is evaluated once).
+ * Full causal forward over every prompt of the batch; writes K (after RoPE) and V of every
+ * prompt position and layer into the prompt arena and the logits at each prompt's last
+ * position.
+ *   prompt_tokens   device [total_tokens] int32, prompts packed back to back
+ *   prompt_offsets  device [n_prompts + 1] int32, prompt p = tokens[offsets[p] : offsets[p+1]]
+ *   total_tokens, max_prompt_len   host scalars describing the same arrays
+ *   prompt_kv       device, arena with prompt_slots slots
+ *   prompt_kv_start device [n_prompts] int64, first slot of each prompt
+ *   last_logits     device [n_prompts, vocab] float, written */
+PC_API int pc_prefill_shared(pc_ctx* ctx, void* stream, int n_prompts, const int32_t* prompt_tokens,
+                      const int32_t* prompt_offsets, int total_tokens, int max_prompt_len,
+                      void* prompt_kv, int64_t prompt_slots, const int64_t* prompt_kv_start,
+                      float* last_logits);
+
+/* One autoregressive step for n_rows live rollouts (Section 3.1: pi_theta(o_t | q, o_<t)).
+ * Row r belongs to prompt row_prompt[r], is rollout row_rollout[r] of its group and has
+ * row_step[r] suffix tokens cached already.  Its input token is tokens[row_tok_index[r]]; the
+ * step appends that token's K/V at suffix slot row_kv_start[r] + row_step[r], attends over the
+ * prompt's shared KV (prompt_len[p] slots from prompt_kv_start[p]) followed by the rollout's own
+ * row_step[r] + 1 suffix slots, and produces the logits of the next token.
+ *   logits_out  device [n_rows, vocab] float or NULL
+ *   sample      host or NULL.  When given, the next token is drawn as in pc_sample with
+ *               step key row_step[r] + 1 and stored at tokens[row_tok_index[r] + 1].
+ * Rows of one prompt must be contiguous; group g covers rows
+ * group_row_start[g] .. group_row_start[g+1]-1 (device [n_groups + 1] int32), none longer
+ * than max_group_rows (host scalar).  All row_* arrays are device [n_rows]. */
+PC_API int pc_decode_step(pc_ctx* ctx, void* stream, int n_rows,
+                   const int32_t* row_prompt, const int32_t* row_rollout, const int32_t* row_step,
+                   const int64_t* row_kv_start, int32_t* tokens, const int64_t* row_tok_index,
+                   int n_groups, const int32_t* group_row_start, int max_group_rows,
+                   const int32_t* prompt_len, const void* prompt_kv, int64_t prompt_slots,
+                   const int64_t* prompt_kv_start, void* suffix_kv, int64_t suffix_slots,
+                   float* logits_out, const pc_sample_params* sample);
+
+/* Seeded draw from softmax(logits / T) by Gumbel-max (Section 4.2: T = 1.0, top_p = 1.0):
+ *   token = argmin-index argmax_v ( logits[v] / T + g_v ),   g_v = -ln(-ln u_v),
+ *   u_v = ((w_v >> 9) + 0.5) * 2^-23, w_v = word (v & 3) of Philox4x32-10 with
+ *   key (seed lo, seed hi) and counter (v >> 2, step, rollout, prompt).
+ * Row r reads logits row logits_row[r] (NULL: row r), so all rollouts of a group can draw
+ * their first token from their prompt's single prefill row.
+ *   out_tokens  device int32; token of row r is stored at out_tokens[out_index[r]] (NULL: [r])
+ *   out_top2_gap device [n_rows] float or NULL: largest minus second-largest perturbed score */
+PC_API int pc_sample(void* stream, int n_rows, int vocab, const float* logits, const int32_t* logits_row,
+              float temperature, uint64_t seed, const int32_t* row_prompt, const int32_t* row_rollout,
+              const int32_t* row_step, int32_t* out_tokens, const int64_t* out_index, float* out_top2_gap);
+
+/* Binary reward of the synthetic workloads, standing in for the verifier R(q, o) in {0, 1} of
+ * Section 3.3: reward[i] = 1 if tokens[last_index[i]] < threshold[i] else 0.  All device. */
+PC_API int pc_reward_last_token(void* stream, int n, const int32_t* tokens, const int64_t* last_index,
+                         const int32_t* threshold, float* reward);
+
+/* Group statistics (Eq. 3, population form) and the pilot estimate p_hat = n_success / n
+ * (Section 3.3).  Group g is rewards[group_start[g] : group_start[g] + group_count[g]].
+ * Outputs, device [n_groups]: n, n_success (number of rewards equal to 1), mean, var. */
+PC_API int pc_group_stats(void* stream, int n_groups, const float* rewards, const int32_t* group_start,
+                   const int32_t* group_count, int32_t* n, int32_t* n_success, float* mean, float* var);
+
+/* Pilot filter, eviction and commit allocation (Section 3.3, 3.4; Algorithm 1: Filter, Evict,
+ * Commit).  p_hat = (double) pilot_success / pilot_n; keep iff p_lower <= p_hat <= p_upper;
+ * evict iff p_hat >= p_solve (independent of the filter); the first b_t kept prompts in batch
+ * order get status COMMIT and extra_rollouts = n_commit, later ones BUFFERED.
+ * Outputs device: status, extra_rollouts, evict [n_prompts] int32; n_selected [1] int32;
+ * total_rollouts [1] int64 = sum(pilot_n) + n_selected * n_commit (the cost of Section 4.3). */
+PC_API int pc_allocate(void* stream, int n_prompts, const int32_t* pilot_success, const int32_t* pilot_n,
+                const pc_alloc_params* params, int32_t* status, int32_t* extra_rollouts, int32_t* evict,
+                int32_t* n_selected, int64_t* total_rollouts);
+
+/* Group-relative advantage A_i = (r_i - mu) / sigma (Section 3.1) over group g =
+ * rewards[group_start[g] : +group_count[g]]; 0 when all rewards of the group are equal, and
+ * for groups whose status (device [n_groups] or NULL) is not PC_STATUS_COMMIT.
+ * adv: device, same indexing as rewards; only elements inside a group are written. */
+PC_API int pc_grpo_advantage(void* stream, int n_groups, const float* rewards, const int32_t* group_start,
+                      const int32_t* group_count, const int32_t* status, float* adv);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PC_H_ */

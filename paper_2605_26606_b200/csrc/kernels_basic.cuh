@@ -1,0 +1,173 @@
+// Row bookkeeping, embedding gather, RMSNorm, rotary tables, q/k/v post-processing, reward rule.
+#pragma once
+
+#include "common.cuh"
+
+namespace pc {
+
+// Per-row attention geometry shared by prefill and decode.
+struct RowGeom {
+    int32_t* pos;        // [M] absolute position of the row's token
+    int64_t* wslot;      // [M] slot the row's K/V is written to
+    int32_t* warena;     // [M] 0: write into the prompt arena, 1: into the suffix arena
+    int64_t* p_start;    // [M] first prompt-arena slot attended
+    int32_t* p_len;      // [M] number of prompt-arena slots attended
+    int64_t* s_start;    // [M] first suffix-arena slot attended
+    int32_t* s_len;      // [M] number of suffix-arena slots attended
+    int32_t* token;      // [M] input token id
+};
+
+// Decode: row r of prompt p with `step` suffix tokens cached attends prompt slots [start_p, start_p + Lp)
+// and suffix slots [kv_start_r, kv_start_r + step + 1); its own K/V goes to suffix slot kv_start_r + step.
+__global__ void prep_decode_rows(int n_rows, const int32_t* row_prompt, const int32_t* row_step,
+                                 const int64_t* row_kv_start, const int32_t* tokens, const int64_t* row_tok_index,
+                                 const int32_t* prompt_len, const int64_t* prompt_kv_start, int64_t prompt_slots,
+                                 int64_t suffix_slots, int vocab, RowGeom g, int32_t* err) {
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= n_rows) return;
+    const int p = row_prompt[r];
+    const int step = row_step[r];
+    const int Lp = prompt_len[p];
+    const int64_t ps = prompt_kv_start[p];
+    const int64_t ss = row_kv_start[r];
+    int tok = tokens[row_tok_index[r]];
+    bool ok = true;
+    if (tok < 0 || tok >= vocab) { set_error(err, DEV_ERR_TOKEN_RANGE); tok = 0; }
+    if (ps < 0 || Lp < 0 || ps + Lp > prompt_slots || ss < 0 || step < 0 || ss + step + 1 > suffix_slots) {
+        set_error(err, DEV_ERR_SLOT_RANGE);
+        ok = false;
+    }
+    g.pos[r] = Lp + step;
+    g.token[r] = tok;
+    g.warena[r] = 1;
+    g.wslot[r] = ok ? ss + step : -1;
+    g.p_start[r] = ps;
+    g.p_len[r] = ok ? Lp : 0;
+    g.s_start[r] = ss;
+    g.s_len[r] = ok ? step + 1 : 0;
+}
+
+// Prefill: packed token t of prompt p at position i attends prompt slots [start_p, start_p + i + 1).
+__global__ void prep_prefill_rows(int n_prompts, const int32_t* prompt_tokens, const int32_t* prompt_offsets,
+                                  const int64_t* prompt_kv_start, int64_t prompt_slots, int vocab, RowGeom g,
+                                  int32_t* last_row, int32_t* err) {
+    const int p = blockIdx.x;
+    const int b = prompt_offsets[p], e = prompt_offsets[p + 1];
+    const int64_t ps = prompt_kv_start[p];
+    const bool ok = ps >= 0 && ps + (e - b) <= prompt_slots;
+    if (!ok && threadIdx.x == 0) set_error(err, DEV_ERR_SLOT_RANGE);
+    if (threadIdx.x == 0) last_row[p] = e - 1;
+    for (int t = b + threadIdx.x; t < e; t += blockDim.x) {
+        int tok = prompt_tokens[t];
+        if (tok < 0 || tok >= vocab) { set_error(err, DEV_ERR_TOKEN_RANGE); tok = 0; }
+        const int i = t - b;
+        g.pos[t] = i;
+        g.token[t] = tok;
+        g.warena[t] = 0;
+        g.wslot[t] = ok ? ps + i : -1;
+        g.p_start[t] = ps;
+        g.p_len[t] = ok ? i + 1 : 0;
+        g.s_start[t] = 0;
+        g.s_len[t] = 0;
+    }
+}
+
+// cos/sin of pos * theta^(-2i/hd), evaluated in double so that long positions keep float accuracy.
+__global__ void rope_table_kernel(int M, int half, double theta, const int32_t* pos, float2* table) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= M * half) return;
+    const int r = idx / half, i = idx - r * half;
+    const double inv_freq = pow(theta, -(double)i / (double)half);
+    double s, c;
+    sincos((double)pos[r] * inv_freq, &s, &c);
+    table[idx] = make_float2((float)c, (float)s);
+}
+
+// h[r, :] = E[token[r], :] (float residual stream); a[r, :] = RMSNorm(h[r, :]; gain) in storage type T.
+template <typename T>
+__global__ void embed_rmsnorm_kernel(int d, const int32_t* token, const T* __restrict__ embed, const float* __restrict__ gain,
+                                     float eps, float* __restrict__ h, T* __restrict__ a) {
+    __shared__ float red[33];
+    const int r = blockIdx.x;
+    const T* e = embed + (size_t)token[r] * d;
+    float ss = 0.f;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        const float v = to_f32<T>(e[i]);
+        h[(size_t)r * d + i] = v;
+        ss += v * v;
+    }
+    ss = block_sum(ss, red);
+    const float rstd = rsqrtf(ss / (float)d + eps);
+    for (int i = threadIdx.x; i < d; i += blockDim.x)
+        a[(size_t)r * d + i] = from_f32<T>(h[(size_t)r * d + i] * rstd * gain[i]);
+}
+
+// a[r, :] = RMSNorm(h[src[r], :]; gain);  src == nullptr means row r.
+template <typename T>
+__global__ void rmsnorm_kernel(int d, const float* __restrict__ h, const int32_t* __restrict__ src,
+                               const float* __restrict__ gain, float eps, T* __restrict__ a) {
+    __shared__ float red[33];
+    const int r = blockIdx.x;
+    const float* x = h + (size_t)(src ? src[r] : r) * d;
+    float ss = 0.f;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) { const float v = x[i]; ss += v * v; }
+    ss = block_sum(ss, red);
+    const float rstd = rsqrtf(ss / (float)d + eps);
+    for (int i = threadIdx.x; i < d; i += blockDim.x) a[(size_t)r * d + i] = from_f32<T>(x[i] * rstd * gain[i]);
+}
+
+struct KvArena {
+    void* base;
+    int64_t n_slots;
+};
+
+// One block per (row, head of the fused q|k|v projection); thread i handles the rotary pair (i, i + hd/2).
+// q heads: optional RMSNorm over head_dim, RoPE, stored to q_out [M, Hq*hd] as T.
+// k heads: optional RMSNorm, RoPE, stored to the row's KV slot.  v heads: stored to the row's KV slot.
+template <typename T>
+__global__ void qkv_post_kernel(int Hq, int Hkv, int hd, int layer, const float* __restrict__ qkv,
+                                const float* __restrict__ q_gain, const float* __restrict__ k_gain, float eps,
+                                const float2* __restrict__ rope, RowGeom g, KvArena prompt_arena, KvArena suffix_arena,
+                                T* __restrict__ q_out) {
+    __shared__ float red[33];
+    const int r = blockIdx.x, head = blockIdx.y, i = threadIdx.x, half = hd >> 1;
+    const int n_tot = (Hq + 2 * Hkv) * hd;
+    const float* src = qkv + (size_t)r * n_tot + (size_t)head * hd;
+    float x1 = src[i], x2 = src[i + half];
+    const bool is_q = head < Hq, is_k = !is_q && head < Hq + Hkv;
+    if (is_q || is_k) {
+        const float* gain = is_q ? q_gain : k_gain;
+        if (gain != nullptr) {
+            const float ss = block_sum(x1 * x1 + x2 * x2, red);
+            const float rstd = rsqrtf(ss / (float)hd + eps);
+            x1 = x1 * rstd * gain[i];
+            x2 = x2 * rstd * gain[i + half];
+        }
+        const float2 cs = rope[(size_t)r * half + i];
+        const float y1 = x1 * cs.x - x2 * cs.y;
+        const float y2 = x2 * cs.x + x1 * cs.y;
+        x1 = y1; x2 = y2;
+    }
+    if (is_q) {
+        T* dst = q_out + (size_t)r * Hq * hd + (size_t)head * hd;
+        dst[i] = from_f32<T>(x1);
+        dst[i + half] = from_f32<T>(x2);
+        return;
+    }
+    const int64_t slot = g.wslot[r];
+    if (slot < 0) return;
+    const KvArena ar = g.warena[r] ? suffix_arena : prompt_arena;
+    const int kvh = is_k ? head - Hq : head - Hq - Hkv;
+    const int64_t plane = ((int64_t)layer * 2 + (is_k ? 0 : 1)) * Hkv + kvh;
+    T* dst = reinterpret_cast<T*>(ar.base) + (plane * ar.n_slots + slot) * hd;
+    dst[i] = from_f32<T>(x1);
+    dst[i + half] = from_f32<T>(x2);
+}
+
+__global__ void reward_last_token_kernel(int n, const int32_t* tokens, const int64_t* last_index,
+                                         const int32_t* threshold, float* reward) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) reward[i] = tokens[last_index[i]] < threshold[i] ? 1.f : 0.f;
+}
+
+}  // namespace pc

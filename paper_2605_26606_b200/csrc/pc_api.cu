@@ -1,0 +1,391 @@
+// C ABI of the Pilot-Commit rollout engine: argument checks, workspace carving and kernel sequencing.
+// See include/pc.h for the contract of every entry point.
+#include "../../include/pc.h"
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "attention_simt.cuh"
+#include "common.cuh"
+#include "gemm_simt.cuh"
+#include "kernels_basic.cuh"
+#include "sampler.cuh"
+#include "stats.cuh"
+
+namespace {
+
+thread_local std::string g_cuda_error;
+
+int cuda_fail(cudaError_t e, const char* what) {
+    g_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
+    return PC_ERR_CUDA;
+}
+
+#define PC_CUDA_CHECK_LAUNCH(what)                                  \
+    do {                                                            \
+        cudaError_t e__ = cudaGetLastError();                       \
+        if (e__ != cudaSuccess) return cuda_fail(e__, what);        \
+    } while (0)
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Carve {
+    size_t h, a, qkv, q, attn, act, logits, rope, pos, wslot, warena, p_start, p_len, s_start, s_len, token, last_row, total;
+};
+
+}  // namespace
+
+struct pc_ctx {
+    pc_model_desc d;
+    const void* embed;
+    const void* lm_head;
+    const float* final_norm;
+    std::vector<const float*> attn_norm, bqkv, q_norm, k_norm, mlp_norm;
+    std::vector<const void*> wqkv, wo, w_gate_up, w_down;
+    // workspace
+    char* ws = nullptr;
+    size_t ws_bytes = 0;
+    int max_rows = 0, max_prefill = 0;
+    int32_t* err = nullptr;
+    Carve cv{};
+
+    int n_qkv() const { return (d.n_q_heads + 2 * d.n_kv_heads) * d.head_dim; }
+    int q_dim() const { return d.n_q_heads * d.head_dim; }
+    size_t eb() const { return d.dtype == PC_DTYPE_F32 ? 4 : 2; }
+};
+
+namespace {
+
+Carve carve(const pc_ctx* c, int max_rows, int max_prefill) {
+    const pc_model_desc& d = c->d;
+    const size_t M = (size_t)std::max(max_rows, max_prefill), eb = c->eb();
+    Carve v{};
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    v.h = take(M * d.d_model * 4);
+    v.a = take(M * d.d_model * eb);
+    v.qkv = take(M * c->n_qkv() * 4);
+    v.q = take(M * c->q_dim() * eb);
+    v.attn = take(M * c->q_dim() * eb);
+    v.act = take(M * (size_t)d.d_ff * eb);
+    v.logits = take((size_t)std::max(max_rows, 1) * d.vocab * 4);
+    v.rope = take(M * (d.head_dim / 2) * 8);
+    v.pos = take(M * 4);
+    v.wslot = take(M * 8);
+    v.warena = take(M * 4);
+    v.p_start = take(M * 8);
+    v.p_len = take(M * 4);
+    v.s_start = take(M * 8);
+    v.s_len = take(M * 4);
+    v.token = take(M * 4);
+    v.last_row = take(M * 4);
+    v.total = off;
+    return v;
+}
+
+pc::RowGeom geom(const pc_ctx* c) {
+    pc::RowGeom g;
+    char* w = c->ws;
+    g.pos = reinterpret_cast<int32_t*>(w + c->cv.pos);
+    g.wslot = reinterpret_cast<int64_t*>(w + c->cv.wslot);
+    g.warena = reinterpret_cast<int32_t*>(w + c->cv.warena);
+    g.p_start = reinterpret_cast<int64_t*>(w + c->cv.p_start);
+    g.p_len = reinterpret_cast<int32_t*>(w + c->cv.p_len);
+    g.s_start = reinterpret_cast<int64_t*>(w + c->cv.s_start);
+    g.s_len = reinterpret_cast<int32_t*>(w + c->cv.s_len);
+    g.token = reinterpret_cast<int32_t*>(w + c->cv.token);
+    return g;
+}
+
+// The decoder layers over M rows whose geometry is already in the workspace; leaves the residual stream in ws.h.
+template <typename T>
+int run_layers(pc_ctx* c, cudaStream_t st, int M, pc::KvArena prompt_arena, pc::KvArena suffix_arena) {
+    using namespace pc;
+    const pc_model_desc& d = c->d;
+    char* w = c->ws;
+    float* h = reinterpret_cast<float*>(w + c->cv.h);
+    T* a = reinterpret_cast<T*>(w + c->cv.a);
+    float* qkv = reinterpret_cast<float*>(w + c->cv.qkv);
+    T* q = reinterpret_cast<T*>(w + c->cv.q);
+    T* attn = reinterpret_cast<T*>(w + c->cv.attn);
+    T* act = reinterpret_cast<T*>(w + c->cv.act);
+    float2* rope = reinterpret_cast<float2*>(w + c->cv.rope);
+    const RowGeom g = geom(c);
+    const int half = d.head_dim / 2;
+    const float scale = 1.0f / sqrtf((float)d.head_dim);
+
+    rope_table_kernel<<<(M * half + 255) / 256, 256, 0, st>>>(M, half, (double)d.rope_theta, g.pos, rope);
+    embed_rmsnorm_kernel<T><<<M, 256, 0, st>>>(d.d_model, g.token, reinterpret_cast<const T*>(c->embed), c->attn_norm[0],
+                                               d.rms_eps, h, a);
+    PC_CUDA_CHECK_LAUNCH("embed_rmsnorm");
+    for (int l = 0; l < d.n_layers; ++l) {
+        if (l > 0) rmsnorm_kernel<T><<<M, 256, 0, st>>>(d.d_model, h, nullptr, c->attn_norm[l], d.rms_eps, a);
+        launch_gemm_simt<T>(st, a, reinterpret_cast<const T*>(c->wqkv[l]), M, c->n_qkv(), d.d_model,
+                            EpiStoreF32{qkv, c->n_qkv(), d.qkv_bias ? c->bqkv[l] : nullptr});
+        qkv_post_kernel<T><<<dim3(M, d.n_q_heads + 2 * d.n_kv_heads), half, 0, st>>>(
+            d.n_q_heads, d.n_kv_heads, d.head_dim, l, qkv, d.qk_norm ? c->q_norm[l] : nullptr,
+            d.qk_norm ? c->k_norm[l] : nullptr, d.rms_eps, rope, g, prompt_arena, suffix_arena, q);
+        if (d.head_dim == 128)
+            attn_row_simt_kernel<T, 128><<<dim3(M, d.n_kv_heads), 128, 0, st>>>(d.n_q_heads, d.n_kv_heads, l, q, g, prompt_arena,
+                                                                               suffix_arena, scale, attn);
+        else
+            attn_row_simt_kernel<T, 64><<<dim3(M, d.n_kv_heads), 128, 0, st>>>(d.n_q_heads, d.n_kv_heads, l, q, g, prompt_arena,
+                                                                              suffix_arena, scale, attn);
+        launch_gemm_simt<T>(st, attn, reinterpret_cast<const T*>(c->wo[l]), M, d.d_model, c->q_dim(), EpiResidual{h, d.d_model});
+        rmsnorm_kernel<T><<<M, 256, 0, st>>>(d.d_model, h, nullptr, c->mlp_norm[l], d.rms_eps, a);
+        launch_gemm_simt<T>(st, a, reinterpret_cast<const T*>(c->w_gate_up[l]), M, 2 * d.d_ff, d.d_model,
+                            EpiSwiGLU<T>{act, d.d_ff});
+        launch_gemm_simt<T>(st, act, reinterpret_cast<const T*>(c->w_down[l]), M, d.d_model, d.d_ff, EpiResidual{h, d.d_model});
+        PC_CUDA_CHECK_LAUNCH("decoder layer");
+    }
+    return PC_OK;
+}
+
+// logits[n, V] = RMSNorm(h[src[r]]; final_norm) * W_lm^T
+template <typename T>
+int run_lm_head(pc_ctx* c, cudaStream_t st, int n, const int32_t* src, float* logits) {
+    using namespace pc;
+    const pc_model_desc& d = c->d;
+    float* h = reinterpret_cast<float*>(c->ws + c->cv.h);
+    T* a = reinterpret_cast<T*>(c->ws + c->cv.a);
+    rmsnorm_kernel<T><<<n, 256, 0, st>>>(d.d_model, h, src, c->final_norm, d.rms_eps, a);
+    const T* wlm = reinterpret_cast<const T*>(d.tied_embed ? c->embed : c->lm_head);
+    launch_gemm_simt<T>(st, a, wlm, n, d.vocab, d.d_model, EpiStoreF32{logits, d.vocab, nullptr});
+    PC_CUDA_CHECK_LAUNCH("lm head");
+    return PC_OK;
+}
+
+int check_ready(const pc_ctx* c) {
+    if (c == nullptr) return PC_ERR_INVALID_ARG;
+    if (c->ws == nullptr) return PC_ERR_NO_WORKSPACE;
+    return PC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* pc_status_string(int status) {
+    switch (status) {
+        case PC_OK: return "ok";
+        case PC_ERR_INVALID_ARG: return "invalid argument";
+        case PC_ERR_SHAPE: return "unsupported model shape";
+        case PC_ERR_ALIGNMENT: return "misaligned pointer";
+        case PC_ERR_CAPACITY: return "workspace capacity exceeded";
+        case PC_ERR_UNSUPPORTED: return "unsupported";
+        case PC_ERR_CUDA: return "CUDA error";
+        case PC_ERR_NO_WORKSPACE: return "workspace not set";
+        default: return "unknown status";
+    }
+}
+
+const char* pc_last_cuda_error(void) { return g_cuda_error.c_str(); }
+
+int pc_create(const pc_model_desc* desc, const pc_weights* wts, pc_ctx** out) {
+    if (desc == nullptr || wts == nullptr || out == nullptr) return PC_ERR_INVALID_ARG;
+    *out = nullptr;
+    const pc_model_desc& d = *desc;
+    if (d.dtype != PC_DTYPE_F32 && d.dtype != PC_DTYPE_BF16) return PC_ERR_INVALID_ARG;
+    if (d.n_layers <= 0 || d.d_model <= 0 || d.n_q_heads <= 0 || d.n_kv_heads <= 0 || d.d_ff <= 0 || d.vocab <= 0 ||
+        !(d.rms_eps >= 0.f) || !(d.rope_theta > 0.f))
+        return PC_ERR_INVALID_ARG;
+    if (d.head_dim != 64 && d.head_dim != 128) return PC_ERR_SHAPE;
+    if (d.n_q_heads % d.n_kv_heads != 0 || d.n_q_heads / d.n_kv_heads > pc::ATTN_MAX_REP) return PC_ERR_SHAPE;
+    if (d.d_model % 8 != 0 || d.d_ff % 8 != 0) return PC_ERR_SHAPE;
+    if (d.dtype == PC_DTYPE_BF16 && (d.d_model % 64 != 0 || d.d_ff % 64 != 0)) return PC_ERR_SHAPE;
+    if (wts->embed == nullptr || wts->final_norm == nullptr || (!d.tied_embed && wts->lm_head == nullptr)) return PC_ERR_INVALID_ARG;
+    if (wts->attn_norm == nullptr || wts->wqkv == nullptr || wts->wo == nullptr || wts->mlp_norm == nullptr ||
+        wts->w_gate_up == nullptr || wts->w_down == nullptr)
+        return PC_ERR_INVALID_ARG;
+    if (d.qkv_bias && wts->bqkv == nullptr) return PC_ERR_INVALID_ARG;
+    if (d.qk_norm && (wts->q_norm == nullptr || wts->k_norm == nullptr)) return PC_ERR_INVALID_ARG;
+    pc_ctx* c = new (std::nothrow) pc_ctx();
+    if (c == nullptr) return PC_ERR_INVALID_ARG;
+    c->d = d;
+    c->embed = wts->embed;
+    c->lm_head = wts->lm_head;
+    c->final_norm = wts->final_norm;
+    if (!aligned(c->embed, 16) || (c->lm_head && !aligned(c->lm_head, 16))) { delete c; return PC_ERR_ALIGNMENT; }
+    for (int l = 0; l < d.n_layers; ++l) {
+        const void* mats[4] = {wts->wqkv[l], wts->wo[l], wts->w_gate_up[l], wts->w_down[l]};
+        for (const void* m : mats) {
+            if (m == nullptr) { delete c; return PC_ERR_INVALID_ARG; }
+            if (!aligned(m, 16)) { delete c; return PC_ERR_ALIGNMENT; }
+        }
+        if (wts->attn_norm[l] == nullptr || wts->mlp_norm[l] == nullptr) { delete c; return PC_ERR_INVALID_ARG; }
+        if (d.qkv_bias && wts->bqkv[l] == nullptr) { delete c; return PC_ERR_INVALID_ARG; }
+        if (d.qk_norm && (wts->q_norm[l] == nullptr || wts->k_norm[l] == nullptr)) { delete c; return PC_ERR_INVALID_ARG; }
+        c->attn_norm.push_back(wts->attn_norm[l]);
+        c->mlp_norm.push_back(wts->mlp_norm[l]);
+        c->bqkv.push_back(d.qkv_bias ? wts->bqkv[l] : nullptr);
+        c->q_norm.push_back(d.qk_norm ? wts->q_norm[l] : nullptr);
+        c->k_norm.push_back(d.qk_norm ? wts->k_norm[l] : nullptr);
+        c->wqkv.push_back(wts->wqkv[l]);
+        c->wo.push_back(wts->wo[l]);
+        c->w_gate_up.push_back(wts->w_gate_up[l]);
+        c->w_down.push_back(wts->w_down[l]);
+    }
+    *out = c;
+    return PC_OK;
+}
+
+void pc_destroy(pc_ctx* ctx) { delete ctx; }
+
+int pc_workspace_bytes(const pc_ctx* ctx, int max_rows, int max_prefill_tokens, size_t* out_bytes) {
+    if (ctx == nullptr || out_bytes == nullptr || max_rows < 0 || max_prefill_tokens < 0) return PC_ERR_INVALID_ARG;
+    *out_bytes = carve(ctx, max_rows, max_prefill_tokens).total;
+    return PC_OK;
+}
+
+int pc_set_workspace(pc_ctx* ctx, void* dev_ws, size_t bytes, int max_rows, int max_prefill_tokens, int32_t* dev_error_flag) {
+    if (ctx == nullptr || dev_ws == nullptr || dev_error_flag == nullptr || max_rows < 0 || max_prefill_tokens < 0)
+        return PC_ERR_INVALID_ARG;
+    if (!aligned(dev_ws, 256) || !aligned(dev_error_flag, 4)) return PC_ERR_ALIGNMENT;
+    const Carve cv = carve(ctx, max_rows, max_prefill_tokens);
+    if (bytes < cv.total) return PC_ERR_CAPACITY;
+    ctx->ws = static_cast<char*>(dev_ws);
+    ctx->ws_bytes = bytes;
+    ctx->max_rows = max_rows;
+    ctx->max_prefill = max_prefill_tokens;
+    ctx->err = dev_error_flag;
+    ctx->cv = cv;
+    return PC_OK;
+}
+
+int pc_prefill_shared(pc_ctx* ctx, void* stream, int n_prompts, const int32_t* prompt_tokens, const int32_t* prompt_offsets,
+                      int total_tokens, int max_prompt_len, void* prompt_kv, int64_t prompt_slots,
+                      const int64_t* prompt_kv_start, float* last_logits) {
+    if (int rc = check_ready(ctx)) return rc;
+    if (n_prompts < 0 || total_tokens < 0 || max_prompt_len < 0 || prompt_slots < 0) return PC_ERR_INVALID_ARG;
+    if (n_prompts == 0 || total_tokens == 0) return PC_OK;
+    if (prompt_tokens == nullptr || prompt_offsets == nullptr || prompt_kv == nullptr || prompt_kv_start == nullptr ||
+        last_logits == nullptr)
+        return PC_ERR_INVALID_ARG;
+    if (!aligned(prompt_kv, 16) || !aligned(last_logits, 16)) return PC_ERR_ALIGNMENT;
+    if (total_tokens > ctx->max_prefill || n_prompts > total_tokens || max_prompt_len > total_tokens) return PC_ERR_CAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const pc::RowGeom g = geom(ctx);
+    int32_t* last_row = reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.last_row);
+    pc::prep_prefill_rows<<<n_prompts, 256, 0, st>>>(n_prompts, prompt_tokens, prompt_offsets, prompt_kv_start, prompt_slots,
+                                                     ctx->d.vocab, g, last_row, ctx->err);
+    PC_CUDA_CHECK_LAUNCH("prep_prefill_rows");
+    const pc::KvArena pa{prompt_kv, prompt_slots}, sa{prompt_kv, prompt_slots};
+    int rc = ctx->d.dtype == PC_DTYPE_F32 ? run_layers<float>(ctx, st, total_tokens, pa, sa)
+                                          : run_layers<__nv_bfloat16>(ctx, st, total_tokens, pa, sa);
+    if (rc) return rc;
+    return ctx->d.dtype == PC_DTYPE_F32 ? run_lm_head<float>(ctx, st, n_prompts, last_row, last_logits)
+                                        : run_lm_head<__nv_bfloat16>(ctx, st, n_prompts, last_row, last_logits);
+}
+
+int pc_decode_step(pc_ctx* ctx, void* stream, int n_rows, const int32_t* row_prompt, const int32_t* row_rollout,
+                   const int32_t* row_step, const int64_t* row_kv_start, int32_t* tokens, const int64_t* row_tok_index,
+                   int n_groups, const int32_t* group_row_start, int max_group_rows, const int32_t* prompt_len,
+                   const void* prompt_kv, int64_t prompt_slots, const int64_t* prompt_kv_start, void* suffix_kv,
+                   int64_t suffix_slots, float* logits_out, const pc_sample_params* sample) {
+    if (int rc = check_ready(ctx)) return rc;
+    if (n_rows < 0 || n_groups < 0 || max_group_rows < 0 || prompt_slots < 0 || suffix_slots < 0) return PC_ERR_INVALID_ARG;
+    if (n_rows == 0) return PC_OK;
+    if (row_prompt == nullptr || row_rollout == nullptr || row_step == nullptr || row_kv_start == nullptr || tokens == nullptr ||
+        row_tok_index == nullptr || group_row_start == nullptr || prompt_len == nullptr || prompt_kv == nullptr ||
+        prompt_kv_start == nullptr || suffix_kv == nullptr)
+        return PC_ERR_INVALID_ARG;
+    if (n_groups == 0 || max_group_rows == 0 || max_group_rows > n_rows || n_groups > n_rows) return PC_ERR_INVALID_ARG;
+    if (logits_out == nullptr && sample == nullptr) return PC_ERR_INVALID_ARG;
+    if (sample != nullptr && !(sample->temperature > 0.f)) return PC_ERR_INVALID_ARG;
+    if (!aligned(prompt_kv, 16) || !aligned(suffix_kv, 16) || (logits_out && !aligned(logits_out, 16))) return PC_ERR_ALIGNMENT;
+    if (n_rows > ctx->max_rows) return PC_ERR_CAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const pc::RowGeom g = geom(ctx);
+    pc::prep_decode_rows<<<(n_rows + 127) / 128, 128, 0, st>>>(n_rows, row_prompt, row_step, row_kv_start, tokens, row_tok_index,
+                                                               prompt_len, prompt_kv_start, prompt_slots, suffix_slots,
+                                                               ctx->d.vocab, g, ctx->err);
+    PC_CUDA_CHECK_LAUNCH("prep_decode_rows");
+    const pc::KvArena pa{const_cast<void*>(prompt_kv), prompt_slots}, sa{suffix_kv, suffix_slots};
+    const bool f32 = ctx->d.dtype == PC_DTYPE_F32;
+    int rc = f32 ? run_layers<float>(ctx, st, n_rows, pa, sa) : run_layers<__nv_bfloat16>(ctx, st, n_rows, pa, sa);
+    if (rc) return rc;
+    float* logits = logits_out ? logits_out : reinterpret_cast<float*>(ctx->ws + ctx->cv.logits);
+    rc = f32 ? run_lm_head<float>(ctx, st, n_rows, nullptr, logits) : run_lm_head<__nv_bfloat16>(ctx, st, n_rows, nullptr, logits);
+    if (rc) return rc;
+    if (sample != nullptr) {
+        pc::sample_kernel<<<n_rows, 256, 0, st>>>(ctx->d.vocab, logits, nullptr, sample->temperature,
+                                                  (uint32_t)(sample->seed & 0xffffffffu), (uint32_t)(sample->seed >> 32), row_prompt,
+                                                  row_rollout, row_step, 1, tokens, row_tok_index, 1, nullptr);
+        PC_CUDA_CHECK_LAUNCH("sample");
+    }
+    return PC_OK;
+}
+
+int pc_sample(void* stream, int n_rows, int vocab, const float* logits, const int32_t* logits_row, float temperature,
+              uint64_t seed, const int32_t* row_prompt, const int32_t* row_rollout, const int32_t* row_step,
+              int32_t* out_tokens, const int64_t* out_index, float* out_top2_gap) {
+    if (n_rows < 0 || vocab <= 0 || !(temperature > 0.f)) return PC_ERR_INVALID_ARG;
+    if (n_rows == 0) return PC_OK;
+    if (logits == nullptr || row_prompt == nullptr || row_rollout == nullptr || row_step == nullptr || out_tokens == nullptr)
+        return PC_ERR_INVALID_ARG;
+    pc::sample_kernel<<<n_rows, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        vocab, logits, logits_row, temperature, (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32), row_prompt, row_rollout,
+        row_step, 0, out_tokens, out_index, 0, out_top2_gap);
+    PC_CUDA_CHECK_LAUNCH("sample");
+    return PC_OK;
+}
+
+int pc_reward_last_token(void* stream, int n, const int32_t* tokens, const int64_t* last_index, const int32_t* threshold,
+                         float* reward) {
+    if (n < 0) return PC_ERR_INVALID_ARG;
+    if (n == 0) return PC_OK;
+    if (tokens == nullptr || last_index == nullptr || threshold == nullptr || reward == nullptr) return PC_ERR_INVALID_ARG;
+    pc::reward_last_token_kernel<<<(n + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(n, tokens, last_index, threshold,
+                                                                                                reward);
+    PC_CUDA_CHECK_LAUNCH("reward");
+    return PC_OK;
+}
+
+int pc_group_stats(void* stream, int n_groups, const float* rewards, const int32_t* group_start, const int32_t* group_count,
+                   int32_t* n, int32_t* n_success, float* mean, float* var) {
+    if (n_groups < 0) return PC_ERR_INVALID_ARG;
+    if (n_groups == 0) return PC_OK;
+    if (rewards == nullptr || group_start == nullptr || group_count == nullptr || n == nullptr || n_success == nullptr ||
+        mean == nullptr || var == nullptr)
+        return PC_ERR_INVALID_ARG;
+    const int threads = 128, groups_per_block = threads / 32;
+    pc::group_stats_kernel<<<(n_groups + groups_per_block - 1) / groups_per_block, threads, 0, static_cast<cudaStream_t>(stream)>>>(
+        n_groups, rewards, group_start, group_count, n, n_success, mean, var);
+    PC_CUDA_CHECK_LAUNCH("group_stats");
+    return PC_OK;
+}
+
+int pc_allocate(void* stream, int n_prompts, const int32_t* pilot_success, const int32_t* pilot_n, const pc_alloc_params* params,
+                int32_t* status, int32_t* extra_rollouts, int32_t* evict, int32_t* n_selected, int64_t* total_rollouts) {
+    if (n_prompts < 0 || params == nullptr || n_selected == nullptr || total_rollouts == nullptr) return PC_ERR_INVALID_ARG;
+    if (params->n_commit < 0 || params->b_t < 0 || !(params->p_lower <= params->p_upper)) return PC_ERR_INVALID_ARG;
+    if (n_prompts > 0 && (pilot_success == nullptr || pilot_n == nullptr || status == nullptr || extra_rollouts == nullptr ||
+                          evict == nullptr))
+        return PC_ERR_INVALID_ARG;
+    pc::allocate_kernel<<<1, 1024, 0, static_cast<cudaStream_t>(stream)>>>(
+        n_prompts, pilot_success, pilot_n, params->p_lower, params->p_upper, params->p_solve, params->n_commit, params->b_t, status,
+        extra_rollouts, evict, n_selected, reinterpret_cast<long long*>(total_rollouts));
+    PC_CUDA_CHECK_LAUNCH("allocate");
+    return PC_OK;
+}
+
+int pc_grpo_advantage(void* stream, int n_groups, const float* rewards, const int32_t* group_start, const int32_t* group_count,
+                      const int32_t* status, float* adv) {
+    if (n_groups < 0) return PC_ERR_INVALID_ARG;
+    if (n_groups == 0) return PC_OK;
+    if (rewards == nullptr || group_start == nullptr || group_count == nullptr || adv == nullptr) return PC_ERR_INVALID_ARG;
+    const int threads = 128, groups_per_block = threads / 32;
+    pc::grpo_advantage_kernel<<<(n_groups + groups_per_block - 1) / groups_per_block, threads, 0, static_cast<cudaStream_t>(stream)>>>(
+        n_groups, rewards, group_start, group_count, status, adv);
+    PC_CUDA_CHECK_LAUNCH("grpo_advantage");
+    return PC_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,255 @@
+"""Thin driver of one Pilot-Commit step on one GPU (Section 3.3; Algorithm 1, one iteration).
+
+It only owns device memory (torch tensors), lays out the weights the way the C ABI
+wants them, decides which rollouts are live at which step (known in advance: the
+synthetic workloads end a rollout at its length cap, there is no end-of-sequence
+token) and calls the library: pc_prefill_shared once per batch, then for the pilot
+and for the commit stage pc_sample for the first token, pc_decode_step per step,
+pc_reward_last_token, pc_group_stats, pc_allocate, pc_grpo_advantage.  No arithmetic
+of the method happens here.
+"""
+from __future__ import annotations
+
+import dataclasses
+from typing import Dict, List, Optional
+
+import numpy as np
+import torch
+
+from . import binding as B
+from .workloads import DTYPE_BF16, DTYPE_F32, Batch, ModelShape, Weights, Workload
+
+
+def _dev_matrix(w: Weights, names: List[str], model: ModelShape, device, interleave: bool = False) -> torch.Tensor:
+    """Concatenates (or row-interleaves) matrices and uploads them in the model's storage type."""
+    if model.dtype == DTYPE_BF16:
+        parts = [torch.from_numpy(w.bits(n).view(np.int16)) for n in names]
+    else:
+        parts = [torch.from_numpy(w[n]) for n in names]
+    if interleave:
+        assert len(parts) == 2
+        t = torch.stack(parts, dim=1).reshape(-1, parts[0].shape[1])
+    else:
+        t = torch.cat(parts, dim=0) if len(parts) > 1 else parts[0]
+    t = t.contiguous().to(device)
+    return t.view(torch.bfloat16) if model.dtype == DTYPE_BF16 else t
+
+
+@dataclasses.dataclass
+class StageSchedule:
+    """Which rollouts are live at every decode step of one stage, flattened over steps and uploaded once."""
+    n_steps: int
+    rows_per_step: np.ndarray         # [n_steps]
+    row_off: np.ndarray               # [n_steps] offset of the step's rows in the flat row arrays
+    groups_per_step: np.ndarray       # [n_steps]
+    group_off: np.ndarray             # [n_steps] offset in the flat group_row_start array
+    max_group_rows: np.ndarray        # [n_steps]
+    row_prompt: torch.Tensor
+    row_rollout: torch.Tensor
+    row_step: torch.Tensor
+    row_kv_start: torch.Tensor
+    row_tok_index: torch.Tensor
+    group_row_start: torch.Tensor
+    total_rows: int
+
+
+class RolloutEngine:
+    def __init__(self, model: ModelShape, weights: Weights, max_rows: int, max_prefill_tokens: int, device="cuda:0"):
+        self.model = model
+        self.device = torch.device(device)
+        torch.cuda.set_device(self.device)
+        m, dev = model, self.device
+        f32 = lambda n: torch.from_numpy(np.ascontiguousarray(weights[n], dtype=np.float32)).to(dev)
+        L = range(m.n_layers)
+        self.embed = _dev_matrix(weights, ["embed"], m, dev)
+        self.lm_head = None if m.tied_embed else _dev_matrix(weights, ["lm_head"], m, dev)
+        self.final_norm = f32("final_norm")
+        self.attn_norm = [f32(f"layers.{l}.attn_norm") for l in L]
+        self.mlp_norm = [f32(f"layers.{l}.mlp_norm") for l in L]
+        self.wqkv = [_dev_matrix(weights, [f"layers.{l}.wq", f"layers.{l}.wk", f"layers.{l}.wv"], m, dev) for l in L]
+        self.bqkv = [torch.cat([f32(f"layers.{l}.bq"), f32(f"layers.{l}.bk"), f32(f"layers.{l}.bv")]) for l in L] \
+            if m.qkv_bias else None
+        self.q_norm = [f32(f"layers.{l}.q_norm") for l in L] if m.qk_norm else None
+        self.k_norm = [f32(f"layers.{l}.k_norm") for l in L] if m.qk_norm else None
+        self.wo = [_dev_matrix(weights, [f"layers.{l}.wo"], m, dev) for l in L]
+        self.w_gate_up = [_dev_matrix(weights, [f"layers.{l}.w_gate", f"layers.{l}.w_up"], m, dev, interleave=True) for l in L]
+        self.w_down = [_dev_matrix(weights, [f"layers.{l}.w_down"], m, dev) for l in L]
+        desc = B.ModelDesc(m.n_layers, m.d_model, m.n_q_heads, m.n_kv_heads, m.head_dim, m.d_ff, m.vocab, m.rms_eps,
+                           m.rope_theta, m.dtype, int(m.tied_embed), int(m.qk_norm), int(m.qkv_bias))
+        self.ctx = B.pc_create(desc, self.embed, self.lm_head, self.final_norm, self.attn_norm, self.wqkv, self.bqkv,
+                               self.q_norm, self.k_norm, self.wo, self.mlp_norm, self.w_gate_up, self.w_down)
+        self.max_rows, self.max_prefill = max_rows, max_prefill_tokens
+        nbytes = B.pc_workspace_bytes(self.ctx, max_rows, max_prefill_tokens)
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        self.err_flag = torch.zeros(1, dtype=torch.int32, device=dev)
+        B.pc_set_workspace(self.ctx, self.workspace, max_rows, max_prefill_tokens, self.err_flag)
+        self.kv_dtype = torch.float32 if m.dtype == DTYPE_F32 else torch.bfloat16
+
+    # ------------------------------------------------------------------------------------------
+    def kv_arena(self, n_slots: int) -> torch.Tensor:
+        m = self.model
+        return torch.empty((m.n_layers, 2, m.n_kv_heads, max(n_slots, 1), m.head_dim), dtype=self.kv_dtype, device=self.device)
+
+    def check_error_flag(self) -> None:
+        code = int(self.err_flag.item())
+        if code != 0:
+            raise RuntimeError(f"device error flag = {code}")
+
+    # ------------------------------------------------------------------------------------------
+    def load_batch(self, wl: Workload, batch: Batch, host_inputs: Optional[Dict[str, torch.Tensor]] = None) -> None:
+        """Uploads the batch and allocates the KV arenas and every output buffer of the step."""
+        dev, P, G = self.device, wl.n_prompts, wl.group_size
+        self.wl, self.batch = wl, batch
+        up = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a)).to(dev, dtype=dt, non_blocking=True)
+        if host_inputs is not None:           # pinned host buffers prepared by the caller (end-to-end timing)
+            self.prompt_tokens = host_inputs["prompt_tokens"].to(dev, non_blocking=True)
+            self.prompt_offsets = host_inputs["prompt_offsets"].to(dev, non_blocking=True)
+        else:
+            self.prompt_tokens = up(batch.prompt_tokens, torch.int32)
+            self.prompt_offsets = up(batch.prompt_offsets, torch.int32)
+        self.prompt_len = up(batch.prompt_lens, torch.int32)
+        self.prompt_kv_start = up(batch.prompt_offsets[:-1].astype(np.int64), torch.int64)
+        self.total_prompt_tokens = int(batch.prompt_offsets[-1])
+        self.prompt_kv = self.kv_arena(self.total_prompt_tokens)
+        # every rollout (p, i) owns caps[p, i] suffix slots and max_new token cells
+        caps = batch.caps.astype(np.int64)
+        kv_start = np.zeros(P * G, dtype=np.int64)
+        kv_start[1:] = np.cumsum(caps.reshape(-1))[:-1]
+        self.kv_start_host = kv_start.reshape(P, G)
+        self.suffix_slots = int(caps.sum())
+        self.suffix_kv = self.kv_arena(self.suffix_slots)
+        self.tokens = torch.full((P * G * wl.max_new,), -1, dtype=torch.int32, device=dev)
+        self.last_logits = torch.empty((P, self.model.vocab), dtype=torch.float32, device=dev)
+        self.rewards = torch.zeros(P * G, dtype=torch.float32, device=dev)
+        self.adv = torch.zeros(P * G, dtype=torch.float32, device=dev)
+        self.thresholds = up(np.repeat(batch.reward_threshold, G), torch.int32)
+        self.last_index = up((np.arange(P * G, dtype=np.int64) * wl.max_new + caps.reshape(-1) - 1), torch.int64)
+        self.group_start = up(np.arange(P, dtype=np.int32) * G, torch.int32)
+        i32 = lambda: torch.zeros(P, dtype=torch.int32, device=dev)
+        f32 = lambda: torch.zeros(P, dtype=torch.float32, device=dev)
+        self.pilot_n, self.pilot_success, self.pilot_mean, self.pilot_var = i32(), i32(), f32(), f32()
+        self.union_n, self.union_success, self.union_mean, self.union_var = i32(), i32(), f32(), f32()
+        self.status, self.extra, self.evict = i32(), i32(), i32()
+        self.n_selected = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.total_rollouts = torch.zeros(1, dtype=torch.int64, device=dev)
+
+    def prefill(self) -> None:
+        b = self.batch
+        B.pc_prefill_shared(self.ctx, self.wl.n_prompts, self.prompt_tokens, self.prompt_offsets, self.total_prompt_tokens,
+                            int(b.prompt_lens.max()), self.prompt_kv, self.total_prompt_tokens, self.prompt_kv_start,
+                            self.last_logits)
+
+    # ------------------------------------------------------------------------------------------
+    def build_schedule(self, prompts: np.ndarray, rollouts: np.ndarray) -> StageSchedule:
+        """Rollouts (prompts[j], rollouts[j]), sorted by (prompt, rollout), all starting together.
+
+        A rollout with cap c takes part in decode steps 0 .. c-2 (its c-th token needs no further forward)."""
+        wl, dev = self.wl, self.device
+        caps = self.batch.caps[prompts, rollouts].astype(np.int64)
+        rid = prompts.astype(np.int64) * wl.group_size + rollouts
+        kv0 = self.kv_start_host[prompts, rollouts]
+        n_steps = int(max(caps.max() - 1, 0)) if len(caps) else 0
+        rp, rr, rs, rk, rt, gs = [], [], [], [], [], []
+        rows_per_step = np.zeros(n_steps, dtype=np.int64)
+        groups_per_step = np.zeros(n_steps, dtype=np.int64)
+        max_group = np.zeros(n_steps, dtype=np.int64)
+        for s in range(n_steps):
+            live = caps > s + 1
+            p = prompts[live]
+            rows_per_step[s] = p.shape[0]
+            rp.append(p); rr.append(rollouts[live]); rk.append(kv0[live]); rt.append(rid[live] * wl.max_new + s)
+            rs.append(np.full(p.shape[0], s, dtype=np.int32))
+            starts = np.flatnonzero(np.r_[True, p[1:] != p[:-1]])
+            bounds = np.r_[starts, p.shape[0]]
+            groups_per_step[s] = starts.shape[0]
+            max_group[s] = int(np.max(np.diff(bounds)))
+            gs.append(bounds.astype(np.int32))
+        cat = lambda xs, dt: torch.from_numpy(np.concatenate(xs).astype(dt) if xs else np.zeros(0, dt)).to(dev)
+        row_off = np.r_[0, np.cumsum(rows_per_step)[:-1]] if n_steps else np.zeros(0, np.int64)
+        group_off = np.r_[0, np.cumsum(groups_per_step + 1)[:-1]] if n_steps else np.zeros(0, np.int64)
+        return StageSchedule(n_steps, rows_per_step, row_off, groups_per_step, group_off, max_group,
+                             cat(rp, np.int32), cat(rr, np.int32), cat(rs, np.int32), cat(rk, np.int64), cat(rt, np.int64),
+                             cat(gs, np.int32), int(rows_per_step.sum()))
+
+    def run_stage(self, prompts: np.ndarray, rollouts: np.ndarray, record_logits: Optional[dict] = None,
+                  teacher_forced: bool = False) -> int:
+        """First token from the prompt's prefill logits, then the decode steps.  Returns tokens generated.
+
+        record_logits: {step: None} asks for the logits of those decode steps (filled in place with
+        (logits tensor, row prompts, row rollouts)).  teacher_forced: nothing is sampled; the token
+        buffer must already hold every rollout's tokens and every step's logits must be recorded."""
+        wl, dev = self.wl, self.device
+        n = int(prompts.shape[0])
+        if n == 0:
+            return 0
+        sp = B.SampleParams(wl.temperature, wl.sample_seed)
+        d_p = torch.from_numpy(prompts.astype(np.int32)).to(dev)
+        d_r = torch.from_numpy(rollouts.astype(np.int32)).to(dev)
+        d_zero = torch.zeros(n, dtype=torch.int32, device=dev)
+        rid = prompts.astype(np.int64) * wl.group_size + rollouts
+        d_first = torch.from_numpy(rid * wl.max_new).to(dev)
+        if not teacher_forced:
+            B.pc_sample(n, self.model.vocab, self.last_logits, d_p, wl.temperature, wl.sample_seed, d_p, d_r, d_zero,
+                        self.tokens, out_index=d_first)
+        sch = self.build_schedule(prompts, rollouts)
+        pr, rr, rs = sch.row_prompt.data_ptr(), sch.row_rollout.data_ptr(), sch.row_step.data_ptr()
+        rk, rt, gs = sch.row_kv_start.data_ptr(), sch.row_tok_index.data_ptr(), sch.group_row_start.data_ptr()
+        for s in range(sch.n_steps):
+            nr, o, go = int(sch.rows_per_step[s]), int(sch.row_off[s]), int(sch.group_off[s])
+            logits_out = None
+            if record_logits is not None and s in record_logits:
+                logits_out = torch.empty((nr, self.model.vocab), dtype=torch.float32, device=dev)
+                record_logits[s] = (logits_out, sch.row_prompt[o:o + nr].cpu().numpy(), sch.row_rollout[o:o + nr].cpu().numpy())
+            B.pc_decode_step(self.ctx, nr, pr + 4 * o, rr + 4 * o, rs + 4 * o, rk + 8 * o, self.tokens, rt + 8 * o,
+                             int(sch.groups_per_step[s]), gs + 4 * go, int(sch.max_group_rows[s]), self.prompt_len,
+                             self.prompt_kv, self.total_prompt_tokens, self.prompt_kv_start, self.suffix_kv,
+                             self.suffix_slots, logits_out, None if teacher_forced else sp)
+        self._keep_schedule = sch
+        return int(self.batch.caps[prompts, rollouts].sum())
+
+    # ------------------------------------------------------------------------------------------
+    def pilot_commit_step(self, wl: Workload, batch: Batch, b_t: Optional[int] = None,
+                          host_inputs: Optional[Dict[str, torch.Tensor]] = None) -> dict:
+        """The whole step.  Returns host copies of every output plus token counts."""
+        P, G, k = wl.n_prompts, wl.group_size, wl.n_pilot
+        b_t = P if b_t is None else b_t
+        self.load_batch(wl, batch, host_inputs)
+        self.prefill()
+        pp, rr = np.repeat(np.arange(P), k), np.tile(np.arange(k), P)
+        n_tok = self.run_stage(pp, rr)
+        pilot_count = torch.full((P,), k, dtype=torch.int32, device=self.device)
+        B.pc_reward_last_token(P * G, self.tokens, self.last_index, self.thresholds, self.rewards)
+        B.pc_group_stats(P, self.rewards, self.group_start, pilot_count, self.pilot_n, self.pilot_success, self.pilot_mean,
+                         self.pilot_var)
+        B.pc_allocate(P, self.pilot_success, self.pilot_n, B.AllocParams(wl.p_lower, wl.p_upper, wl.p_solve, G - k, b_t),
+                      self.status, self.extra, self.evict, self.n_selected, self.total_rollouts)
+        status = self.status.cpu().numpy()            # the commit stage's row set depends on it
+        commit = np.flatnonzero(status == B.PC_STATUS_COMMIT)
+        if G > k and commit.size:
+            n_tok += self.run_stage(np.repeat(commit, G - k), np.tile(np.arange(k, G), commit.size))
+        B.pc_reward_last_token(P * G, self.tokens, self.last_index, self.thresholds, self.rewards)
+        union_count = torch.from_numpy(np.where(status == B.PC_STATUS_COMMIT, G, k).astype(np.int32)).to(self.device)
+        B.pc_group_stats(P, self.rewards, self.group_start, union_count, self.union_n, self.union_success, self.union_mean,
+                         self.union_var)
+        B.pc_grpo_advantage(P, self.rewards, self.group_start, union_count, self.status, self.adv)
+        out = self.collect(status)
+        out["generated_tokens"] = n_tok
+        return out
+
+    def collect(self, status: np.ndarray) -> dict:
+        wl, P, G, k = self.wl, self.wl.n_prompts, self.wl.group_size, self.wl.n_pilot
+        self.check_error_flag()
+        toks = self.tokens.cpu().numpy().reshape(P, G, wl.max_new)
+        generated = np.zeros((P, G), dtype=bool)
+        generated[:, :k] = True
+        generated[status == B.PC_STATUS_COMMIT, :] = True
+        tokens = [[toks[p, i, :self.batch.caps[p, i]].copy() if generated[p, i] else None for i in range(G)] for p in range(P)]
+        rewards = self.rewards.cpu().numpy().reshape(P, G).copy()
+        rewards[~generated] = 0.0          # cells of rollouts that were never generated hold no reward
+        h = lambda t: t.cpu().numpy()
+        return dict(tokens=tokens, rewards=rewards, generated=generated,
+                    pilot_n=h(self.pilot_n), pilot_success=h(self.pilot_success), pilot_mean=h(self.pilot_mean),
+                    pilot_var=h(self.pilot_var), status=status, extra=h(self.extra), evict=h(self.evict),
+                    n_selected=int(self.n_selected.item()), total_rollouts=int(self.total_rollouts.item()),
+                    union_n=h(self.union_n), union_success=h(self.union_success), union_mean=h(self.union_mean),
+                    union_var=h(self.union_var), advantages=h(self.adv).reshape(P, G))

@@ -114,7 +114,7 @@ QWEN3_14B = ModelShape("qwen3-14b-shape", 40, 5120, 40, 8, 128, 17408, 151936,
 
 WORKLOADS: Dict[str, Workload] = {
     "config0": Workload("config0", TINY, 4, 32, 32, 8, 2, 16, 16, 16, 0.0,
-                        forced_explicit=((0, 0.0), (3, 1.0))),
+                        forced_explicit=((0, 0.0), (3, 1.0)), data_seed=6),
     "config1": Workload("config1", QWEN25_1P5B, 32, 256, 256, 16, 4, 512, 128, 512, 0.0),
     "config2": Workload("config2", QWEN25_1P5B, 16, 256, 1024, 128, 16, 2048, 512, 2048, 0.3),
     "config3": Workload("config3", QWEN3_8B, 8, 512, 512, 64, 8, 1024, 256, 1024, 0.3),

@@ -1,0 +1,113 @@
+"""End-to-end parity of the CUDA rollout path with the CPU oracle (through the C ABI)."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import rollout as orollout
+from oracle import stats as ostats
+from oracle.decoder import Decoder
+from paper_2605_26606_b200 import workloads as wl
+from paper_2605_26606_b200.engine import RolloutEngine
+
+from gpu_util import ensure_built, oracle_group_tokens, teacher_forced_compare
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built(cuda_device):
+    ensure_built()
+
+
+def _compare_step(got, want, w):
+    P, G = w.n_prompts, w.group_size
+    assert np.array_equal(got["status"], want["status"]) and np.array_equal(got["extra"], want["extra"])
+    assert np.array_equal(got["evict"], want["evict"])
+    assert got["n_selected"] == want["n_selected"] and got["total_rollouts"] == want["total_rollouts"]
+    assert np.array_equal(got["generated"], want["generated"])
+    for p in range(P):
+        for i in range(G):
+            if want["generated"][p, i]:
+                assert np.array_equal(got["tokens"][p][i], want["tokens"][p][i]), (p, i)
+    assert np.array_equal(got["rewards"], want["rewards"])
+    for key in ("pilot_n", "pilot_success", "union_n", "union_success"):
+        assert np.array_equal(got[key], want[key]), key
+    for key in ("pilot_mean", "pilot_var", "union_mean", "union_var"):
+        assert np.max(np.abs(got[key] - want[key])) < 1e-6, key
+    assert np.max(np.abs(got["advantages"] - want["advantages"])) < 1e-5
+
+
+@pytest.mark.parametrize("variant", ["config0", "all_mid", "bt1", "k_eq_G", "ragged"])
+def test_config0_free_running_step_is_bit_exact(variant):
+    """Tiny fp32 decoder: tokens, rewards, counts, statuses and allocations identical; advantages within 1e-5."""
+    w = wl.WORKLOADS["config0"]
+    b_t = None
+    if variant == "all_mid":
+        w = dataclasses.replace(w, forced_explicit=((0, 0.5), (1, 0.5), (2, 0.45), (3, 0.55)))
+    elif variant == "bt1":
+        w = dataclasses.replace(w, forced_explicit=((0, 0.5), (1, 0.5), (2, 0.5), (3, 0.5)), sample_seed=99)
+        b_t = 1
+    elif variant == "k_eq_G":
+        w = dataclasses.replace(w, n_pilot=8)                     # GRPO-style: every rollout in one stage
+    elif variant == "ragged":
+        w = dataclasses.replace(w, n_prompts=5, prompt_len_lo=1, prompt_len_hi=40, cap_lo=1, cap_hi=16, data_seed=3,
+                                forced_explicit=((0, 0.5), (1, 0.5), (2, 0.5), (3, 0.5), (4, 0.5)))
+    weights = wl.gen_weights(w.model, seed=0, threads=2, gain_jitter=0.1)
+    batch = wl.gen_batch(w)
+    dec = Decoder(w.model, weights)
+    want = orollout.pilot_commit_step(dec, w, batch, b_t=b_t)
+    eng = RolloutEngine(w.model, weights, max_rows=w.n_prompts * w.group_size, max_prefill_tokens=int(batch.prompt_offsets[-1]))
+    got = eng.pilot_commit_step(w, batch, b_t=b_t)
+    _compare_step(got, want, w)
+    if variant in ("all_mid", "ragged"):
+        assert np.any(want["status"] == ostats.COMMIT)
+
+
+def test_config0_teacher_forced_logits_within_1e_4():
+    w = wl.WORKLOADS["config0"]
+    weights = wl.gen_weights(w.model, seed=0, threads=2, gain_jitter=0.1)
+    batch = wl.gen_batch(w)
+    dec = Decoder(w.model, weights)
+    P, G = w.n_prompts, w.group_size
+    prompts, rollouts = np.repeat(np.arange(P), G), np.tile(np.arange(G), P)
+    ref = oracle_group_tokens(dec, w, batch, prompts, rollouts)
+    eng = RolloutEngine(w.model, weights, max_rows=P * G, max_prefill_tokens=int(batch.prompt_offsets[-1]))
+    worst, n_cmp, n_exempt = teacher_forced_compare(eng, w, batch, ref, prompts, rollouts, logit_tol=1e-4, gap_tol=1e-3)
+    assert n_cmp == P * G * 16 and n_exempt <= 2
+
+
+@pytest.mark.parametrize("model", [wl.TINY_BF16, wl.SMALL_BF16, wl.SMALL_QKNORM_BF16], ids=lambda m: m.name)
+def test_small_bf16_models_teacher_forced(model):
+    """bf16 storage: logits within 5e-2; sampled token identical wherever the oracle's top-two gap exceeds 1e-1."""
+    w = dataclasses.replace(wl.WORKLOADS["config0"], model=model, n_prompts=3, prompt_len_lo=5, prompt_len_hi=70,
+                            group_size=6, n_pilot=2, max_new=12, cap_lo=3, cap_hi=12, data_seed=11)
+    weights = wl.gen_weights(model, seed=1, threads=2, gain_jitter=0.1)
+    batch = wl.gen_batch(w)
+    dec = Decoder(model, weights)
+    P, G = w.n_prompts, w.group_size
+    prompts, rollouts = np.repeat(np.arange(P), G), np.tile(np.arange(G), P)
+    ref = oracle_group_tokens(dec, w, batch, prompts, rollouts)
+    eng = RolloutEngine(model, weights, max_rows=P * G, max_prefill_tokens=int(batch.prompt_offsets[-1]))
+    worst, n_cmp, n_exempt = teacher_forced_compare(eng, w, batch, ref, prompts, rollouts, logit_tol=5e-2, gap_tol=1e-1)
+    assert n_cmp == int(batch.caps.sum())
+
+
+def test_run_twice_is_deterministic_and_batch_invariant():
+    """Same inputs give bit-identical tokens; a rollout's tokens do not depend on its batch mates."""
+    w = dataclasses.replace(wl.WORKLOADS["config0"], model=wl.TINY_BF16, n_pilot=8)
+    weights = wl.gen_weights(w.model, seed=0, threads=2)
+    batch = wl.gen_batch(w)
+    eng = RolloutEngine(w.model, weights, max_rows=64, max_prefill_tokens=int(batch.prompt_offsets[-1]))
+    a = eng.pilot_commit_step(w, batch)
+    b = eng.pilot_commit_step(w, batch)
+    for p in range(w.n_prompts):
+        for i in range(w.group_size):
+            assert np.array_equal(a["tokens"][p][i], b["tokens"][p][i])
+    w2 = dataclasses.replace(w, n_pilot=2, forced_explicit=((0, 0.5), (1, 0.5), (2, 0.5), (3, 0.5)))
+    c = eng.pilot_commit_step(w2, wl.gen_batch(w2))
+    for p in range(w.n_prompts):
+        for i in range(w.group_size):
+            if c["generated"][p, i]:
+                assert np.array_equal(a["tokens"][p][i], c["tokens"][p][i])

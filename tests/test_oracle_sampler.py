@@ -8,33 +8,49 @@ import pytest
 from oracle import philox, sampler
 
 
+_TRITON_SCRIPT = r"""
+import json, sys
+import numpy as np, torch, triton, triton.language as tl
+
+@triton.jit
+def kern(out, c0_ptr, c1, c2, c3, k0, k1, n: tl.constexpr):
+    i = tl.arange(0, n)
+    c0 = tl.load(c0_ptr + i).to(tl.uint32, bitcast=True)
+    z = c0 * 0
+    a, b, c, d = tl.philox_impl(c0, z + c1, z + c2, z + c3, z + k0, z + k1, 10)
+    tl.store(out + i * 4 + 0, a.to(tl.int32, bitcast=True)); tl.store(out + i * 4 + 1, b.to(tl.int32, bitcast=True))
+    tl.store(out + i * 4 + 2, c.to(tl.int32, bitcast=True)); tl.store(out + i * 4 + 3, d.to(tl.int32, bitcast=True))
+
+cases = json.loads(sys.argv[1]); n = 256
+c0 = (np.arange(n, dtype=np.uint64) * np.uint64(2654435761) + np.uint64(12345)) & np.uint64(0xFFFFFFFF)
+c0[:4] = [0, 1, 0xFFFFFFFF, 0x80000000]
+res = []
+for (c1, c2, c3, k0, k1) in cases:
+    out = torch.zeros(n * 4, dtype=torch.int32)
+    kern[(1,)](out, torch.from_numpy(c0.astype(np.uint32).view(np.int32)), c1, c2, c3, k0, k1, n)
+    res.append(out.numpy().view(np.uint32).tolist())
+print(json.dumps(res))
+"""
+
+
 def test_philox_matches_independent_library_implementation():
-    """Triton ships its own Philox4x32 (`philox_impl`); its CPU interpreter runs it without a GPU."""
-    os.environ["TRITON_INTERPRET"] = "1"
-    try:
-        import torch
-        import triton
-        import triton.language as tl
-    except Exception as e:                       # pragma: no cover
-        pytest.skip(f"triton interpreter unavailable: {e}")
-
-    @triton.jit
-    def kern(out, c0_ptr, c1, c2, c3, k0, k1, n: tl.constexpr):
-        i = tl.arange(0, n)
-        c0 = tl.load(c0_ptr + i).to(tl.uint32, bitcast=True)
-        z = c0 * 0
-        a, b, c, d = tl.philox_impl(c0, z + c1, z + c2, z + c3, z + k0, z + k1, 10)
-        tl.store(out + i * 4 + 0, a.to(tl.int32, bitcast=True)); tl.store(out + i * 4 + 1, b.to(tl.int32, bitcast=True))
-        tl.store(out + i * 4 + 2, c.to(tl.int32, bitcast=True)); tl.store(out + i * 4 + 3, d.to(tl.int32, bitcast=True))
-
+    """Triton ships its own Philox4x32 (`philox_impl`); its CPU interpreter runs it without a GPU.
+    It runs in a fresh process because the interpreter mode must be chosen before triton is imported."""
+    import json
+    import subprocess
+    import sys
+    cases = [(0, 0, 0, 0, 0), (7, 3, 1, 5, 9), (2047, 127, 15, 0x7FFFFFFF, 0x12345678)]
+    env = dict(os.environ, TRITON_INTERPRET="1", CUDA_VISIBLE_DEVICES="")
+    res = subprocess.run([sys.executable, "-c", _TRITON_SCRIPT, json.dumps(cases)], capture_output=True, text=True, env=env,
+                         timeout=600)
+    assert res.returncode == 0, res.stderr[-2000:]
+    theirs = json.loads(res.stdout.strip().splitlines()[-1])
     n = 256
-    for (c1, c2, c3, k0, k1) in ((0, 0, 0, 0, 0), (7, 3, 1, 5, 9), (2047, 127, 15, 0x7FFFFFFF, 0x12345678)):
-        out = torch.zeros(n * 4, dtype=torch.int32)
-        c0 = (np.arange(n, dtype=np.uint64) * np.uint64(2654435761) + np.uint64(12345)) & np.uint64(0xFFFFFFFF)
-        c0[:4] = [0, 1, 0xFFFFFFFF, 0x80000000]
-        kern[(1,)](out, torch.from_numpy(c0.astype(np.uint32).view(np.int32)), c1, c2, c3, k0, k1, n)
+    c0 = (np.arange(n, dtype=np.uint64) * np.uint64(2654435761) + np.uint64(12345)) & np.uint64(0xFFFFFFFF)
+    c0[:4] = [0, 1, 0xFFFFFFFF, 0x80000000]
+    for (c1, c2, c3, k0, k1), ref in zip(cases, theirs):
         mine = np.stack(philox.philox4x32_10(c0, c1, c2, c3, k0, k1), axis=1).reshape(-1)
-        assert np.array_equal(mine, out.numpy().view(np.uint32))
+        assert np.array_equal(mine, np.array(ref, dtype=np.uint32))
 
 
 def test_counter_layout_and_word_selection():
