@@ -100,7 +100,7 @@ class Workload:
 
 
 TINY = ModelShape("tiny-fp32", 2, 256, 4, 2, 64, 688, 2048, dtype=DTYPE_F32)
-TINY_BF16 = dataclasses.replace(TINY, name="tiny-bf16", dtype=DTYPE_BF16, qkv_bias=True)
+TINY_BF16 = dataclasses.replace(TINY, name="tiny-bf16", dtype=DTYPE_BF16, qkv_bias=True, d_ff=704)
 SMALL_BF16 = ModelShape("small-bf16", 2, 512, 4, 2, 128, 1024, 4096, dtype=DTYPE_BF16,
                         tied_embed=True, qkv_bias=True)
 SMALL_QKNORM_BF16 = ModelShape("small-qknorm-bf16", 2, 512, 4, 2, 128, 1024, 4096, dtype=DTYPE_BF16,

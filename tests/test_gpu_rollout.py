@@ -82,7 +82,8 @@ def test_config0_teacher_forced_logits_within_1e_4():
 def test_small_bf16_models_teacher_forced(model):
     """bf16 storage: logits within 5e-2; sampled token identical wherever the oracle's top-two gap exceeds 1e-1."""
     w = dataclasses.replace(wl.WORKLOADS["config0"], model=model, n_prompts=3, prompt_len_lo=5, prompt_len_hi=70,
-                            group_size=6, n_pilot=2, max_new=12, cap_lo=3, cap_hi=12, data_seed=11)
+                            group_size=6, n_pilot=2, max_new=12, cap_lo=3, cap_hi=12, data_seed=11,
+                            forced_explicit=None)
     weights = wl.gen_weights(model, seed=1, threads=2, gain_jitter=0.1)
     batch = wl.gen_batch(w)
     dec = Decoder(model, weights)
