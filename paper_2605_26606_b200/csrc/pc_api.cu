@@ -9,14 +9,17 @@
 #include <cstring>
 #include <new>
 #include <string>
+#include <type_traits>
 #include <vector>
 
 #include "attention_simt.cuh"
 #include "common.cuh"
 #include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
 #include "kernels_basic.cuh"
 #include "sampler.cuh"
 #include "stats.cuh"
+#include "tensor_map.h"
 
 namespace {
 
@@ -40,6 +43,12 @@ struct Carve {
     size_t h, a, qkv, q, attn, act, logits, rope, pos, wslot, warena, p_start, p_len, s_start, s_len, token, last_row, total;
 };
 
+// TMA descriptors of one bf16 weight matrix [N, K], one per tile width the GEMM may pick.
+struct WMap {
+    CUtensorMap wide, narrow;   // boxes of 256 and 64 rows
+    int N = 0, K = 0;
+};
+
 }  // namespace
 
 struct pc_ctx {
@@ -55,6 +64,12 @@ struct pc_ctx {
     int max_rows = 0, max_prefill = 0;
     int32_t* err = nullptr;
     Carve cv{};
+    // bf16 models: TMA descriptors of the weights (built by pc_create) and of the activation buffers
+    // (built by pc_set_workspace over the full capacity of each buffer)
+    std::vector<WMap> m_wqkv, m_wo, m_wgu, m_wdown;
+    WMap m_lm;
+    CUtensorMap map_a, map_attn, map_act;
+    int num_sms = 148;
 
     int n_qkv() const { return (d.n_q_heads + 2 * d.n_kv_heads) * d.head_dim; }
     int q_dim() const { return d.n_q_heads * d.head_dim; }
@@ -104,10 +119,28 @@ pc::RowGeom geom(const pc_ctx* c) {
     return g;
 }
 
+bool make_wmap(WMap* w, const void* base, int N, int K) {
+    w->N = N;
+    w->K = K;
+    return pc::make_bf16_map(&w->wide, base, N, K, 256) && pc::make_bf16_map(&w->narrow, base, N, K, 64);
+}
+
+// bf16 GEMM on the tensor cores; the tile width is picked so that small batches still spread over the SMs.
+template <class Epi>
+int gemm_bf16(pc_ctx* c, cudaStream_t st, const CUtensorMap& map_a, const WMap& w, int M, Epi epi) {
+    const int tiles_m = (M + pc::tc::BM - 1) / pc::tc::BM;
+    const bool wide = tiles_m * ((w.N + 255) / 256) >= 100;
+    cudaError_t e = wide ? pc::tc::launch<256>(st, map_a, w.wide, M, w.N, w.K, epi, c->err, c->num_sms)
+                         : pc::tc::launch<64>(st, map_a, w.narrow, M, w.N, w.K, epi, c->err, c->num_sms);
+    if (e != cudaSuccess) return cuda_fail(e, "tensor-core gemm");
+    return PC_OK;
+}
+
 // The decoder layers over M rows whose geometry is already in the workspace; leaves the residual stream in ws.h.
 template <typename T>
 int run_layers(pc_ctx* c, cudaStream_t st, int M, pc::KvArena prompt_arena, pc::KvArena suffix_arena) {
     using namespace pc;
+    constexpr bool kF32 = std::is_same<T, float>::value;
     const pc_model_desc& d = c->d;
     char* w = c->ws;
     float* h = reinterpret_cast<float*>(w + c->cv.h);
@@ -127,8 +160,13 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, pc::KvArena prompt_arena, pc::
     PC_CUDA_CHECK_LAUNCH("embed_rmsnorm");
     for (int l = 0; l < d.n_layers; ++l) {
         if (l > 0) rmsnorm_kernel<T><<<M, 256, 0, st>>>(d.d_model, h, nullptr, c->attn_norm[l], d.rms_eps, a);
-        launch_gemm_simt<T>(st, a, reinterpret_cast<const T*>(c->wqkv[l]), M, c->n_qkv(), d.d_model,
-                            EpiStoreF32{qkv, c->n_qkv(), d.qkv_bias ? c->bqkv[l] : nullptr});
+        const float* bias = d.qkv_bias ? c->bqkv[l] : nullptr;
+        if constexpr (kF32) {
+            launch_gemm_simt<T>(st, a, reinterpret_cast<const T*>(c->wqkv[l]), M, c->n_qkv(), d.d_model,
+                                EpiStoreF32{qkv, c->n_qkv(), bias});
+        } else {
+            if (int rc = gemm_bf16(c, st, c->map_a, c->m_wqkv[l], M, tc::EpiStoreF32{qkv, c->n_qkv(), bias})) return rc;
+        }
         qkv_post_kernel<T><<<dim3(M, d.n_q_heads + 2 * d.n_kv_heads), half, 0, st>>>(
             d.n_q_heads, d.n_kv_heads, d.head_dim, l, qkv, d.qk_norm ? c->q_norm[l] : nullptr,
             d.qk_norm ? c->k_norm[l] : nullptr, d.rms_eps, rope, g, prompt_arena, suffix_arena, q);
@@ -138,11 +176,20 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, pc::KvArena prompt_arena, pc::
         else
             attn_row_simt_kernel<T, 64><<<dim3(M, d.n_kv_heads), 128, 0, st>>>(d.n_q_heads, d.n_kv_heads, l, q, g, prompt_arena,
                                                                               suffix_arena, scale, attn);
-        launch_gemm_simt<T>(st, attn, reinterpret_cast<const T*>(c->wo[l]), M, d.d_model, c->q_dim(), EpiResidual{h, d.d_model});
+        if constexpr (kF32) {
+            launch_gemm_simt<T>(st, attn, reinterpret_cast<const T*>(c->wo[l]), M, d.d_model, c->q_dim(), EpiResidual{h, d.d_model});
+        } else {
+            if (int rc = gemm_bf16(c, st, c->map_attn, c->m_wo[l], M, tc::EpiResidual{h, d.d_model})) return rc;
+        }
         rmsnorm_kernel<T><<<M, 256, 0, st>>>(d.d_model, h, nullptr, c->mlp_norm[l], d.rms_eps, a);
-        launch_gemm_simt<T>(st, a, reinterpret_cast<const T*>(c->w_gate_up[l]), M, 2 * d.d_ff, d.d_model,
-                            EpiSwiGLU<T>{act, d.d_ff});
-        launch_gemm_simt<T>(st, act, reinterpret_cast<const T*>(c->w_down[l]), M, d.d_model, d.d_ff, EpiResidual{h, d.d_model});
+        if constexpr (kF32) {
+            launch_gemm_simt<T>(st, a, reinterpret_cast<const T*>(c->w_gate_up[l]), M, 2 * d.d_ff, d.d_model,
+                                EpiSwiGLU<T>{act, d.d_ff});
+            launch_gemm_simt<T>(st, act, reinterpret_cast<const T*>(c->w_down[l]), M, d.d_model, d.d_ff, EpiResidual{h, d.d_model});
+        } else {
+            if (int rc = gemm_bf16(c, st, c->map_a, c->m_wgu[l], M, tc::EpiSwiGLU{act, d.d_ff})) return rc;
+            if (int rc = gemm_bf16(c, st, c->map_act, c->m_wdown[l], M, tc::EpiResidual{h, d.d_model})) return rc;
+        }
         PC_CUDA_CHECK_LAUNCH("decoder layer");
     }
     return PC_OK;
@@ -156,8 +203,12 @@ int run_lm_head(pc_ctx* c, cudaStream_t st, int n, const int32_t* src, float* lo
     float* h = reinterpret_cast<float*>(c->ws + c->cv.h);
     T* a = reinterpret_cast<T*>(c->ws + c->cv.a);
     rmsnorm_kernel<T><<<n, 256, 0, st>>>(d.d_model, h, src, c->final_norm, d.rms_eps, a);
-    const T* wlm = reinterpret_cast<const T*>(d.tied_embed ? c->embed : c->lm_head);
-    launch_gemm_simt<T>(st, a, wlm, n, d.vocab, d.d_model, EpiStoreF32{logits, d.vocab, nullptr});
+    if constexpr (std::is_same<T, float>::value) {
+        const T* wlm = reinterpret_cast<const T*>(d.tied_embed ? c->embed : c->lm_head);
+        launch_gemm_simt<T>(st, a, wlm, n, d.vocab, d.d_model, EpiStoreF32{logits, d.vocab, nullptr});
+    } else {
+        if (int rc = gemm_bf16(c, st, c->map_a, c->m_lm, n, tc::EpiStoreF32{logits, d.vocab, nullptr})) return rc;
+    }
     PC_CUDA_CHECK_LAUNCH("lm head");
     return PC_OK;
 }
@@ -232,6 +283,28 @@ int pc_create(const pc_model_desc* desc, const pc_weights* wts, pc_ctx** out) {
         c->w_gate_up.push_back(wts->w_gate_up[l]);
         c->w_down.push_back(wts->w_down[l]);
     }
+    if (d.dtype == PC_DTYPE_BF16) {
+        if (c->q_dim() % 64 != 0) { delete c; return PC_ERR_SHAPE; }
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
+            delete c;
+            return cuda_fail(cudaGetLastError(), "no CUDA device for a bf16 model");
+        }
+        c->num_sms = sms;
+        bool ok = true;
+        c->m_wqkv.resize(d.n_layers); c->m_wo.resize(d.n_layers); c->m_wgu.resize(d.n_layers); c->m_wdown.resize(d.n_layers);
+        for (int l = 0; l < d.n_layers && ok; ++l) {
+            ok = make_wmap(&c->m_wqkv[l], c->wqkv[l], c->n_qkv(), d.d_model) && make_wmap(&c->m_wo[l], c->wo[l], d.d_model, c->q_dim()) &&
+                 make_wmap(&c->m_wgu[l], c->w_gate_up[l], 2 * d.d_ff, d.d_model) && make_wmap(&c->m_wdown[l], c->w_down[l], d.d_model, d.d_ff);
+        }
+        ok = ok && make_wmap(&c->m_lm, d.tied_embed ? c->embed : c->lm_head, d.vocab, d.d_model);
+        if (!ok) {
+            delete c;
+            g_cuda_error = "cuTensorMapEncodeTiled failed for a weight matrix";
+            return PC_ERR_CUDA;
+        }
+    }
     *out = c;
     return PC_OK;
 }
@@ -256,6 +329,17 @@ int pc_set_workspace(pc_ctx* ctx, void* dev_ws, size_t bytes, int max_rows, int 
     ctx->max_prefill = max_prefill_tokens;
     ctx->err = dev_error_flag;
     ctx->cv = cv;
+    if (ctx->d.dtype == PC_DTYPE_BF16) {
+        const uint64_t cap = (uint64_t)std::max(std::max(max_rows, max_prefill_tokens), 1);
+        char* w = ctx->ws;
+        if (!pc::make_bf16_map(&ctx->map_a, w + cv.a, cap, ctx->d.d_model, 128) ||
+            !pc::make_bf16_map(&ctx->map_attn, w + cv.attn, cap, ctx->q_dim(), 128) ||
+            !pc::make_bf16_map(&ctx->map_act, w + cv.act, cap, ctx->d.d_ff, 128)) {
+            ctx->ws = nullptr;
+            g_cuda_error = "cuTensorMapEncodeTiled failed for an activation buffer";
+            return PC_ERR_CUDA;
+        }
+    }
     return PC_OK;
 }
 
