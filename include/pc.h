@@ -126,6 +126,9 @@ PC_API const char* pc_status_string(int status);
 /* Text of the last CUDA error seen by this thread inside the library (host pointer, static storage). */
 PC_API const char* pc_last_cuda_error(void);
 
+/* Number of kernels this library has launched since it was loaded (host counter, all contexts). */
+PC_API uint64_t pc_launch_count(void);
+
 /* Builds a context: copies the description and the pointer tables (host memory only)
  * and, for bf16 models, encodes the TMA descriptors of the weight matrices.  Needs a
  * current CUDA device for bf16 models.  Shapes: head_dim in {64, 128}; n_q_heads a
@@ -142,6 +145,12 @@ PC_API int pc_workspace_bytes(const pc_ctx* ctx, int max_rows, int max_prefill_t
  * kernels store a non-zero code there when they meet an out-of-range index. */
 PC_API int pc_set_workspace(pc_ctx* ctx, void* dev_ws, size_t bytes, int max_rows, int max_prefill_tokens,
                      int32_t* dev_error_flag);
+
+/* Measurement aid: in the next pc_decode_step of this context, record the two CUDA events (cudaEvent_t,
+ * created by the caller) around the attention kernel of `layer` that reads the rollouts' own suffix K/V
+ * (for float32 models: the single attention kernel).  One-shot; the caller synchronises and reads the
+ * elapsed time.  The paper has no counterpart. */
+PC_API int pc_profile_attention(pc_ctx* ctx, int layer, void* event_start, void* event_stop);
 
 /* Shared prefill (Section 3.1: o ~ pi_theta(. | q); Section 3.3: pilot and commit rollouts of a
  * prompt are drawn from the same pi_theta(. | q), so q is evaluated once).

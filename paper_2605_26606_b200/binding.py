@@ -22,7 +22,7 @@ PC_ERR_UNSUPPORTED, PC_ERR_CUDA, PC_ERR_NO_WORKSPACE = 5, 6, 7
 PC_DTYPE_F32, PC_DTYPE_BF16 = 0, 1
 PC_STATUS_COMMIT, PC_STATUS_BUFFERED, PC_STATUS_DEFER_HARD, PC_STATUS_SKIP_EASY = 0, 1, 2, 3
 
-EXPORTS = ["pc_status_string", "pc_last_cuda_error", "pc_create", "pc_destroy", "pc_workspace_bytes",
+EXPORTS = ["pc_status_string", "pc_last_cuda_error", "pc_launch_count", "pc_profile_attention", "pc_create", "pc_destroy", "pc_workspace_bytes",
            "pc_set_workspace", "pc_prefill_shared", "pc_decode_step", "pc_sample", "pc_reward_last_token",
            "pc_group_stats", "pc_allocate", "pc_grpo_advantage"]
 
@@ -71,6 +71,9 @@ def _lib():
         lib.pc_status_string.restype = C.c_char_p
         lib.pc_status_string.argtypes = [C.c_int]
         lib.pc_last_cuda_error.restype = C.c_char_p
+        lib.pc_launch_count.restype = C.c_uint64
+        lib.pc_launch_count.argtypes = []
+        lib.pc_profile_attention.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         lib.pc_destroy.restype = None
         lib.pc_destroy.argtypes = [C.c_void_p]
         p, i, i64, f, u64 = C.c_void_p, C.c_int, C.c_int64, C.c_float, C.c_uint64
@@ -84,7 +87,7 @@ def _lib():
         lib.pc_group_stats.argtypes = [p, i, p, p, p, p, p, p, p]
         lib.pc_allocate.argtypes = [p, i, p, p, C.POINTER(AllocParams), p, p, p, p, p]
         lib.pc_grpo_advantage.argtypes = [p, i, p, p, p, p, p]
-        for name in EXPORTS[2:]:
+        for name in EXPORTS[3:]:
             if name != "pc_destroy":
                 getattr(lib, name).restype = C.c_int
         _LIB = lib
@@ -121,6 +124,15 @@ def pc_status_string(status: int) -> str:
 
 def pc_last_cuda_error() -> str:
     return _lib().pc_last_cuda_error().decode()
+
+
+def pc_launch_count() -> int:
+    return int(_lib().pc_launch_count())
+
+
+def pc_profile_attention(ctx: "Context", layer: int, event_start: torch.cuda.Event, event_stop: torch.cuda.Event) -> None:
+    """The events must have been created with enable_timing=True and recorded once (so that they exist)."""
+    _check(_lib().pc_profile_attention(ctx.handle, layer, event_start.cuda_event, event_stop.cuda_event), "pc_profile_attention")
 
 
 class Context:

@@ -1,0 +1,535 @@
+// Shared-prefix decode attention for bf16 models, on tensor cores, with K/V tiles staged by TMA.
+//
+// The K/V arenas are viewed as 2-D bf16 tensors [planes * n_slots, head_dim]; a tile of TP consecutive
+// slots is fetched as head_dim/64 boxes of [TP rows x 64 columns] with the 128-byte swizzle, which makes
+// the ldmatrix reads below bank-conflict free.
+//
+//   attn_group_kernel   one CTA per (128 query rows of a group, KV head).  The query rows are all live
+//                       rollouts of the group times the query heads sharing the KV head, so the group's
+//                       prompt K/V is read once per 128 query rows instead of once per rollout
+//                       (S = Q K^T and O = P V as m16n8k16 MMAs, online softmax in registers).  Every
+//                       query row carries its own number of visible prompt slots, which also makes this
+//                       the causal prefill kernel.  Decode: leaves (m, l, unnormalised O) per query row
+//                       in scratch.  Prefill: writes the normalised output.
+//   attn_suffix_kernel  one warp per (rollout, KV head) streams the rollout's own suffix K/V through a
+//                       3-stage TMA ring at full HBM rate.  Positions sit on the MMA M axis (S^T = K Q^T,
+//                       O^T = V^T P^T), so the 6-8 query heads fill the N = 8 axis and no MMA work is
+//                       padded; P is transposed between the two MMAs with movmatrix.  At the end the
+//                       suffix part is merged with the group's prefix part by their log-sum-exp.
+//
+// Scores are kept in the log2 domain (scaled by log2(e) / sqrt(head_dim)) so that exp2f is the only
+// transcendental.  Waits on mbarriers are bounded (see gemm_tc.cuh).
+#pragma once
+
+#include "common.cuh"
+#include "gemm_tc.cuh"
+#include "kernels_basic.cuh"
+
+namespace pc {
+namespace am {
+
+using tc::mbar_arrive;
+using tc::mbar_arrive_expect_tx;
+using tc::mbar_init;
+using tc::mbar_wait;
+using tc::smem_u32;
+using tc::tma_load_2d;
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ uint32_t movmatrix_t(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+__device__ __forceinline__ void mma_bf16(float* c, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&p);
+}
+// exp2 that maps -inf to 0 without producing NaN when both operands are -inf
+__device__ __forceinline__ float exp2_safe(float x, float m) { return m == -INFINITY ? 0.f : exp2f(x - m); }
+
+// Byte offset of (row r, dim d) (d a multiple of 8) in a swizzled tile of ROWS rows: boxes of 64 dims,
+// rows of 128 bytes, 16-byte chunk index XORed with (r mod 8).
+template <int ROWS>
+__device__ __forceinline__ uint32_t tile_off(int r, int d) {
+    return (uint32_t)((d >> 6) * (ROWS * 128) + r * 128 + ((((d & 63) >> 3) ^ (r & 7)) << 4));
+}
+
+struct PrefixPartial {      // per (row, query head): running max (log2 domain), sum, unnormalised output
+    float* m;               // [rows * Hq]
+    float* l;               // [rows * Hq]
+    float* o;               // [rows * Hq * head_dim]
+};
+
+// ---------------------------------------------------------------------------------------------
+// Group (shared-prefix / causal-prefill) kernel
+// ---------------------------------------------------------------------------------------------
+constexpr int G_THREADS = 256;      // 8 warps x 16 query rows
+constexpr int G_QROWS = 128;
+constexpr int G_TK = 64;            // KV positions per stage
+constexpr int G_STAGES = 3;
+template <int HD> constexpr int group_smem_bytes() { return G_STAGES * 2 * G_TK * HD * 2 + 1024 + 128; }
+
+template <int HD, bool FINAL>
+__global__ void __launch_bounds__(G_THREADS, 1)
+attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, int64_t n_slots, int Hq, int Hkv, int layer,
+                  const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ group_row_start, RowGeom g,
+                  float scale_log2, PrefixPartial part, __nv_bfloat16* __restrict__ out, int32_t* err) {
+    constexpr int KS = HD / 16;          // k-steps of Q K^T
+    constexpr int NT = G_TK / 8;         // position n-tiles per stage
+    constexpr int DT = HD / 8;           // dim n-tiles of the output
+    constexpr int TILE_BYTES = G_TK * HD * 2;
+    const int grp = blockIdx.z, kvh = blockIdx.y;
+    const int row0 = group_row_start[grp], n_rows = group_row_start[grp + 1] - row0;
+    const int n_rep = Hq / Hkv;
+    const int q0 = blockIdx.x * G_QROWS;
+    if (q0 >= n_rows * n_rep) return;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + G_STAGES * 2 * TILE_BYTES);
+    __shared__ int s_abort;
+    __shared__ int s_maxlen;
+    const uint32_t tiles_u32 = smem_u32(tiles), full0 = smem_u32(bars), empty0 = full0 + 8 * G_STAGES;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < G_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, G_THREADS / 32); }
+        s_abort = 0;
+        s_maxlen = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    // this thread's two query rows: qr = q0 + warp*16 + lane/4 (+8); query row qr = (rollout row qr / n_rep, head qr % n_rep)
+    int lim[2], grow[2], head[2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int qr = q0 + warp * 16 + (lane >> 2) + 8 * i;
+        const bool valid = qr < n_rows * n_rep;
+        grow[i] = valid ? row0 + qr / n_rep : -1;
+        head[i] = kvh * n_rep + (valid ? qr % n_rep : 0);
+        lim[i] = valid ? g.p_len[grow[i]] : 0;
+    }
+    {
+        int mx = max(lim[0], lim[1]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        if (lane == 0) atomicMax(&s_maxlen, mx);
+    }
+    // Q fragments (A operand), straight from global memory
+    uint32_t qa[KS][4];
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            uint32_t lo = 0, hi = 0;
+            if (grow[i] >= 0) {
+                const __nv_bfloat16* p = q + ((size_t)grow[i] * Hq + head[i]) * HD + ks * 16 + (lane & 3) * 2;
+                lo = *reinterpret_cast<const uint32_t*>(p);
+                hi = *reinterpret_cast<const uint32_t*>(p + 8);
+            }
+            qa[ks][i] = lo;          // a0 (row), a1 (row + 8)
+            qa[ks][2 + i] = hi;      // a2, a3: dims + 8
+        }
+    }
+    __syncthreads();
+    const int max_len = s_maxlen;
+    const int n_tiles = (max_len + G_TK - 1) / G_TK;
+    const int64_t kv_start = g.p_start[row0];
+    const int64_t krow0 = (((int64_t)layer * 2 + 0) * Hkv + kvh) * n_slots + kv_start;
+    const int64_t vrow0 = (((int64_t)layer * 2 + 1) * Hkv + kvh) * n_slots + kv_start;
+
+    auto issue = [&](int tile, int stage) {
+        const uint32_t kb = tiles_u32 + stage * 2 * TILE_BYTES, vb = kb + TILE_BYTES;
+        mbar_arrive_expect_tx(full0 + 8 * stage, 2 * TILE_BYTES);
+#pragma unroll
+        for (int b = 0; b < HD / 64; ++b) {
+            tma_load_2d(kb + b * (G_TK * 128), &kv_map, full0 + 8 * stage, b * 64, (int)(krow0 + (int64_t)tile * G_TK));
+            tma_load_2d(vb + b * (G_TK * 128), &kv_map, full0 + 8 * stage, b * 64, (int)(vrow0 + (int64_t)tile * G_TK));
+        }
+    };
+    if (threadIdx.x == 0)
+        for (int t = 0; t < G_STAGES && t < n_tiles; ++t) issue(t, t);
+
+    float o[DT][4];
+#pragma unroll
+    for (int t = 0; t < DT; ++t) { o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f; }
+    float mrow[2] = {-INFINITY, -INFINITY}, lrow[2] = {0.f, 0.f};
+    bool ok = true;
+
+    for (int tile = 0; tile < n_tiles; ++tile) {
+        const int stage = tile % G_STAGES;
+        const uint32_t phase = (uint32_t)(tile / G_STAGES) & 1u;
+        if (!mbar_wait(full0 + 8 * stage, phase, &s_abort)) { ok = false; break; }
+        const uint32_t kb = tiles_u32 + stage * 2 * TILE_BYTES, vb = kb + TILE_BYTES;
+        // S = Q K^T for 64 positions
+        float s[NT][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) { s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f; }
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+#pragma unroll
+            for (int np = 0; np < NT / 2; ++np) {
+                const int mat = lane >> 3;
+                const int r = np * 16 + (lane & 7) + ((mat >> 1) << 3), d = ks * 16 + ((mat & 1) << 3);
+                uint32_t b0, b1, b2, b3;
+                ldsm_x4(kb + tile_off<G_TK>(r, d), b0, b1, b2, b3);
+                mma_bf16(s[2 * np], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
+                mma_bf16(s[2 * np + 1], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b2, b3);
+            }
+        }
+        // mask, online softmax (rows lane/4 and lane/4 + 8; a row lives in the four lanes of a quad)
+        const int pos0 = tile * G_TK + (lane & 3) * 2;
+        float bmax[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int pos = pos0 + nt * 8 + (c & 1);
+                const float v = pos < lim[c >> 1] ? s[nt][c] * scale_log2 : -INFINITY;
+                s[nt][c] = v;
+                bmax[c >> 1] = fmaxf(bmax[c >> 1], v);
+            }
+        }
+        float corr[2];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            bmax[i] = fmaxf(bmax[i], __shfl_xor_sync(0xffffffffu, bmax[i], 1));
+            bmax[i] = fmaxf(bmax[i], __shfl_xor_sync(0xffffffffu, bmax[i], 2));
+            const float mnew = fmaxf(mrow[i], bmax[i]);
+            corr[i] = exp2_safe(mrow[i], mnew);
+            mrow[i] = mnew;
+            lrow[i] *= corr[i];
+        }
+#pragma unroll
+        for (int t = 0; t < DT; ++t) { o[t][0] *= corr[0]; o[t][1] *= corr[0]; o[t][2] *= corr[1]; o[t][3] *= corr[1]; }
+        uint32_t pa[NT / 2][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            float p[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) { p[c] = exp2_safe(s[nt][c], mrow[c >> 1]); lrow[c >> 1] += p[c]; }
+            pa[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p[0], p[1]);
+            pa[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p[2], p[3]);
+        }
+        // rows of V beyond the longest visible prefix of this CTA may be uninitialised memory: their P is 0, but
+        // 0 * NaN would poison the sum, so positions >= max_len are never multiplied (k-steps past it are skipped)
+        const int valid_in_tile = min(G_TK, max_len - tile * G_TK);
+#pragma unroll
+        for (int kk = 0; kk < G_TK / 16; ++kk) {
+            if (kk * 16 >= valid_in_tile) break;
+            const bool ragged = kk * 16 + 16 > valid_in_tile;      // block-uniform
+#pragma unroll
+            for (int dp = 0; dp < DT / 2; ++dp) {
+                const int mat = lane >> 3;
+                const int r = kk * 16 + (lane & 7) + ((mat & 1) << 3), d = dp * 16 + ((mat >> 1) << 3);
+                uint32_t b0, b1, b2, b3;
+                ldsm_x4_t(vb + tile_off<G_TK>(r, d), b0, b1, b2, b3);
+                if (ragged) {
+                    // zero the V values of positions >= valid_in_tile: after the transposing load a thread holds
+                    // positions kk*16 + (lane%4)*2 + {0,1} in b0/b2 and + 8 in b1/b3
+                    const int p = kk * 16 + (lane & 3) * 2;
+                    const uint32_t m_lo = (p < valid_in_tile ? 0x0000ffffu : 0u) | (p + 1 < valid_in_tile ? 0xffff0000u : 0u);
+                    const uint32_t m_hi = (p + 8 < valid_in_tile ? 0x0000ffffu : 0u) | (p + 9 < valid_in_tile ? 0xffff0000u : 0u);
+                    b0 &= m_lo; b2 &= m_lo; b1 &= m_hi; b3 &= m_hi;
+                }
+                mma_bf16(o[2 * dp], pa[kk][0], pa[kk][1], pa[kk][2], pa[kk][3], b0, b1);
+                mma_bf16(o[2 * dp + 1], pa[kk][0], pa[kk][1], pa[kk][2], pa[kk][3], b2, b3);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty0 + 8 * stage);
+        if (threadIdx.x == 0 && tile + G_STAGES < n_tiles) {
+            if (!mbar_wait(empty0 + 8 * stage, phase, &s_abort)) { ok = false; break; }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            issue(tile + G_STAGES, stage);
+        }
+    }
+    if (!ok) { s_abort = 1; set_error(err, DEV_ERR_WAIT_TIMEOUT); }
+
+    // row sums live spread over the quad
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        lrow[i] += __shfl_xor_sync(0xffffffffu, lrow[i], 1);
+        lrow[i] += __shfl_xor_sync(0xffffffffu, lrow[i], 2);
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        if (grow[i] < 0) continue;
+        const size_t rh = (size_t)grow[i] * Hq + head[i];
+        if (FINAL) {
+            const float inv = lrow[i] > 0.f ? 1.f / lrow[i] : 0.f;
+#pragma unroll
+            for (int t = 0; t < DT; ++t)
+                *reinterpret_cast<uint32_t*>(out + rh * HD + t * 8 + (lane & 3) * 2) = pack_bf16(o[t][2 * i] * inv, o[t][2 * i + 1] * inv);
+        } else {
+            if ((lane & 3) == 0) { part.m[rh] = mrow[i]; part.l[rh] = lrow[i]; }
+#pragma unroll
+            for (int t = 0; t < DT; ++t)
+                *reinterpret_cast<float2*>(part.o + rh * HD + t * 8 + (lane & 3) * 2) = make_float2(o[t][2 * i], o[t][2 * i + 1]);
+        }
+    }
+    if (s_abort) {      // let copies still in flight land before the shared memory is released
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    }
+    __syncthreads();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Suffix kernel
+// ---------------------------------------------------------------------------------------------
+constexpr int S_WARPS = 4;
+constexpr int S_TP = 32;            // positions per stage
+constexpr int S_STAGES = 3;
+template <int HD> constexpr int suffix_smem_bytes() {
+    return S_WARPS * (S_STAGES * 2 * S_TP * HD * 2 + 8 * HD * 4) + 1024 + 256;
+}
+
+template <int HD>
+__global__ void __launch_bounds__(S_WARPS * 32, 1)
+attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, int64_t n_slots, int n_rows, int Hq, int Hkv, int layer,
+                   const __nv_bfloat16* __restrict__ q, RowGeom g, float scale_log2, PrefixPartial part,
+                   __nv_bfloat16* __restrict__ out, int32_t* err) {
+    constexpr int KS = HD / 16;                   // k-steps of K Q^T
+    constexpr int DT = HD / 16;                   // 16-dim m-tiles of O^T
+    constexpr int TILE_BYTES = S_TP * HD * 2;
+    constexpr int WARP_BYTES = S_STAGES * 2 * TILE_BYTES;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t* my_tiles = base + warp * WARP_BYTES;
+    float* obuf = reinterpret_cast<float*>(base + S_WARPS * WARP_BYTES) + warp * 8 * HD;      // [8 heads][HD]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base + S_WARPS * (WARP_BYTES + 8 * HD * 4)) + warp * S_STAGES;
+    __shared__ float s_ml[S_WARPS][16];
+    __shared__ int s_abort;
+    const uint32_t tiles_u32 = smem_u32(my_tiles), full0 = smem_u32(bars);
+    const int n_rep = Hq / Hkv;
+
+    if (threadIdx.x == 0) s_abort = 0;
+    if (lane == 0) {
+        for (int s = 0; s < S_STAGES; ++s) mbar_init(full0 + 8 * s, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    const int n_items = n_rows * Hkv;
+    const int item_stride = gridDim.x * S_WARPS;
+    const int first_item = blockIdx.x * S_WARPS + warp;
+
+    // producer cursor (tracked identically by every lane; lane 0 issues)
+    int p_item = first_item, p_tile = 0, p_ntiles = 0;
+    int64_t p_krow = 0, p_vrow = 0;
+    auto p_load_item = [&]() {
+        while (p_item < n_items) {
+            const int row = p_item / Hkv, kvh = p_item - row * Hkv;
+            const int n = g.s_len[row];
+            if (n > 0) {
+                p_ntiles = (n + S_TP - 1) / S_TP;
+                const int64_t st = g.s_start[row];
+                p_krow = (((int64_t)layer * 2 + 0) * Hkv + kvh) * n_slots + st;
+                p_vrow = (((int64_t)layer * 2 + 1) * Hkv + kvh) * n_slots + st;
+                p_tile = 0;
+                return;
+            }
+            p_item += item_stride;
+        }
+        p_ntiles = 0;
+    };
+    int issued = 0;
+    auto p_issue = [&]() {          // loads the producer cursor's tile into the next ring slot and advances the cursor
+        const int stage = issued % S_STAGES;
+        if (lane == 0) {
+            const uint32_t kb = tiles_u32 + stage * 2 * TILE_BYTES, vb = kb + TILE_BYTES;
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mbar_arrive_expect_tx(full0 + 8 * stage, 2 * TILE_BYTES);
+#pragma unroll
+            for (int b = 0; b < HD / 64; ++b) {
+                tma_load_2d(kb + b * (S_TP * 128), &kv_map, full0 + 8 * stage, b * 64, (int)(p_krow + (int64_t)p_tile * S_TP));
+                tma_load_2d(vb + b * (S_TP * 128), &kv_map, full0 + 8 * stage, b * 64, (int)(p_vrow + (int64_t)p_tile * S_TP));
+            }
+        }
+        ++issued;
+        if (++p_tile == p_ntiles) { p_item += item_stride; p_load_item(); }
+    };
+    p_load_item();
+    for (int i = 0; i < S_STAGES && p_item < n_items; ++i) p_issue();
+
+    int consumed = 0;
+    bool ok = true;
+    for (int item = first_item; item < n_items && ok; item += item_stride) {
+        const int row = item / Hkv, kvh = item - row * Hkv;
+        const int n = g.s_len[row];
+        const int ntiles = (n + S_TP - 1) / S_TP;
+        // Q^T fragments (B operand): head = lane / 4, dims ks*16 + (lane%4)*2 (+8)
+        uint32_t qb[KS][2];
+        {
+            const int hq = lane >> 2;
+            const __nv_bfloat16* qp = q + ((size_t)row * Hq + (size_t)kvh * n_rep + hq) * HD + (lane & 3) * 2;
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                qb[ks][0] = hq < n_rep ? *reinterpret_cast<const uint32_t*>(qp + ks * 16) : 0u;
+                qb[ks][1] = hq < n_rep ? *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8) : 0u;
+            }
+        }
+        float o[DT][4];
+#pragma unroll
+        for (int t = 0; t < DT; ++t) { o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f; }
+        float mh[2] = {-INFINITY, -INFINITY}, lh[2] = {0.f, 0.f};      // heads (lane%4)*2 + {0, 1}
+
+        for (int tile = 0; tile < ntiles; ++tile) {
+            const int stage = consumed % S_STAGES;
+            const uint32_t phase = (uint32_t)(consumed / S_STAGES) & 1u;
+            if (!mbar_wait(full0 + 8 * stage, phase, &s_abort)) { ok = false; break; }
+            const uint32_t kb = tiles_u32 + stage * 2 * TILE_BYTES, vb = kb + TILE_BYTES;
+            const int valid = min(S_TP, n - tile * S_TP);
+            // S^T = K Q^T : positions on M (two 16-row tiles), heads on N
+            float s[2][4];
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt) {
+                s[mt][0] = s[mt][1] = s[mt][2] = s[mt][3] = 0.f;
+                if (mt * 16 < valid) {
+#pragma unroll
+                    for (int ks = 0; ks < KS; ++ks) {
+                        const int mat = lane >> 3;
+                        const int r = mt * 16 + (lane & 7) + ((mat & 1) << 3), d = ks * 16 + ((mat >> 1) << 3);
+                        uint32_t a0, a1, a2, a3;
+                        ldsm_x4(kb + tile_off<S_TP>(r, d), a0, a1, a2, a3);
+                        mma_bf16(s[mt], a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
+                    }
+                }
+            }
+            // mask + per-head block max (a head's column is spread over the 8 lanes sharing lane % 4)
+            float bmax[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int pos = mt * 16 + (lane >> 2) + ((c >> 1) << 3);
+                    const float v = pos < valid ? s[mt][c] * scale_log2 : -INFINITY;
+                    s[mt][c] = v;
+                    bmax[c & 1] = fmaxf(bmax[c & 1], v);
+                }
+            }
+            float corr[2];
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                bmax[i] = fmaxf(bmax[i], __shfl_xor_sync(0xffffffffu, bmax[i], 4));
+                bmax[i] = fmaxf(bmax[i], __shfl_xor_sync(0xffffffffu, bmax[i], 8));
+                bmax[i] = fmaxf(bmax[i], __shfl_xor_sync(0xffffffffu, bmax[i], 16));
+                const float mnew = fmaxf(mh[i], bmax[i]);
+                corr[i] = exp2_safe(mh[i], mnew);
+                mh[i] = mnew;
+                lh[i] *= corr[i];
+            }
+#pragma unroll
+            for (int t = 0; t < DT; ++t) { o[t][0] *= corr[0]; o[t][1] *= corr[1]; o[t][2] *= corr[0]; o[t][3] *= corr[1]; }
+            // O^T += V^T P^T, 16 positions per k-step; P^T fragments come from S^T through movmatrix
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt) {
+                if (mt * 16 >= valid) break;
+                float p[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) { p[c] = exp2_safe(s[mt][c], mh[c & 1]); lh[c & 1] += p[c]; }
+                const uint32_t b0 = movmatrix_t(pack_bf16(p[0], p[1]));
+                const uint32_t b1 = movmatrix_t(pack_bf16(p[2], p[3]));
+                const bool ragged = mt * 16 + 16 > valid;              // warp-uniform
+#pragma unroll
+                for (int dt = 0; dt < DT; ++dt) {
+                    const int mat = lane >> 3;
+                    const int r = mt * 16 + (lane & 7) + ((mat >> 1) << 3), d = dt * 16 + ((mat & 1) << 3);
+                    uint32_t a0, a1, a2, a3;
+                    ldsm_x4_t(vb + tile_off<S_TP>(r, d), a0, a1, a2, a3);
+                    if (ragged) {
+                        // slots past the rollout's last token may be uninitialised: zero them (0 * NaN = NaN).
+                        // After the transposing load a thread holds positions mt*16 + (lane%4)*2 + {0,1} in a0/a1, + 8 in a2/a3.
+                        const int pp = mt * 16 + (lane & 3) * 2;
+                        const uint32_t m_lo = (pp < valid ? 0x0000ffffu : 0u) | (pp + 1 < valid ? 0xffff0000u : 0u);
+                        const uint32_t m_hi = (pp + 8 < valid ? 0x0000ffffu : 0u) | (pp + 9 < valid ? 0xffff0000u : 0u);
+                        a0 &= m_lo; a1 &= m_lo; a2 &= m_hi; a3 &= m_hi;
+                    }
+                    mma_bf16(o[dt], a0, a1, a2, a3, b0, b1);
+                }
+            }
+            ++consumed;
+            __syncwarp();
+            if (p_item < n_items) p_issue();      // refill the slot just drained
+        }
+        if (!ok) break;
+
+        // reduce the per-thread partial sums of each head over the 8 lanes sharing lane % 4
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            lh[i] += __shfl_xor_sync(0xffffffffu, lh[i], 4);
+            lh[i] += __shfl_xor_sync(0xffffffffu, lh[i], 8);
+            lh[i] += __shfl_xor_sync(0xffffffffu, lh[i], 16);
+        }
+        if (lane < 4) {
+            s_ml[warp][lane * 2] = mh[0]; s_ml[warp][lane * 2 + 1] = mh[1];
+            s_ml[warp][8 + lane * 2] = lh[0]; s_ml[warp][8 + lane * 2 + 1] = lh[1];
+        }
+        // O^T fragment (dims dt*16 + lane/4 (+8), heads (lane%4)*2 + {0,1}) -> obuf[head][dim]
+#pragma unroll
+        for (int dt = 0; dt < DT; ++dt) {
+            const int d = dt * 16 + (lane >> 2), hh = (lane & 3) * 2;
+            obuf[hh * HD + d] = o[dt][0];
+            obuf[(hh + 1) * HD + d] = o[dt][1];
+            obuf[hh * HD + d + 8] = o[dt][2];
+            obuf[(hh + 1) * HD + d + 8] = o[dt][3];
+        }
+        __syncwarp();
+        // merge with the prefix part and write: lane handles HD/32 consecutive dims of every head
+        constexpr int EPL = HD / 32;
+        for (int j = 0; j < n_rep; ++j) {
+            const size_t rh = (size_t)row * Hq + (size_t)kvh * n_rep + j;
+            const float ms = s_ml[warp][j], ls = s_ml[warp][8 + j];
+            const float mp = part.m[rh], lp = part.l[rh];
+            const float M = fmaxf(ms, mp);
+            const float ws = exp2_safe(ms, M), wp = exp2_safe(mp, M);
+            const float denom = ls * ws + lp * wp;
+            const float inv = denom > 0.f ? 1.f / denom : 0.f;
+            float res[EPL];
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) {
+                const float po = wp > 0.f ? part.o[rh * HD + lane * EPL + e] * wp : 0.f;
+                res[e] = (obuf[j * HD + lane * EPL + e] * ws + po) * inv;
+            }
+            __nv_bfloat16* dst = out + rh * HD + lane * EPL;
+            if (EPL == 4) {
+                *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(res[0], res[1]), pack_bf16(res[2], res[3]));
+            } else {
+                *reinterpret_cast<uint32_t*>(dst) = pack_bf16(res[0], res[1]);
+            }
+        }
+        __syncwarp();
+    }
+    if (!ok) { s_abort = 1; if (lane == 0) set_error(err, DEV_ERR_WAIT_TIMEOUT); }
+    // drain: tiles issued but not consumed must land before the shared memory is released
+    while (ok && consumed < issued) {
+        const int stage = consumed % S_STAGES;
+        if (!mbar_wait(full0 + 8 * stage, (uint32_t)(consumed / S_STAGES) & 1u, &s_abort)) break;
+        ++consumed;
+    }
+    if (s_abort) {
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    }
+    __syncthreads();
+}
+
+}  // namespace am
+}  // namespace pc

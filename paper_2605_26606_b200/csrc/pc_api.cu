@@ -12,6 +12,7 @@
 #include <type_traits>
 #include <vector>
 
+#include "attention_mma.cuh"
 #include "attention_simt.cuh"
 #include "common.cuh"
 #include "gemm_simt.cuh"
@@ -24,6 +25,8 @@
 namespace {
 
 thread_local std::string g_cuda_error;
+unsigned long long g_launches = 0;     // kernels launched by this library since it was loaded
+inline void count_launches(int n) { g_launches += (unsigned long long)n; }
 
 int cuda_fail(cudaError_t e, const char* what) {
     g_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
@@ -40,7 +43,8 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Carve {
-    size_t h, a, qkv, q, attn, act, logits, rope, pos, wslot, warena, p_start, p_len, s_start, s_len, token, last_row, total;
+    size_t h, a, qkv, q, attn, act, logits, rope, pos, wslot, warena, p_start, p_len, s_start, s_len, token, last_row,
+        part_m, part_l, part_o, total;
 };
 
 // TMA descriptors of one bf16 weight matrix [N, K], one per tile width the GEMM may pick.
@@ -70,6 +74,12 @@ struct pc_ctx {
     WMap m_lm;
     CUtensorMap map_a, map_attn, map_act;
     int num_sms = 148;
+    // TMA descriptors of the KV arenas, rebuilt when a call brings another arena
+    const void* prompt_arena_ptr = nullptr; int64_t prompt_arena_slots = -1; CUtensorMap map_prompt_kv;
+    const void* suffix_arena_ptr = nullptr; int64_t suffix_arena_slots = -1; CUtensorMap map_suffix_kv;
+    // one-shot profiling request (pc_profile_attention)
+    int prof_layer = -1;
+    cudaEvent_t prof_start = nullptr, prof_stop = nullptr;
 
     int n_qkv() const { return (d.n_q_heads + 2 * d.n_kv_heads) * d.head_dim; }
     int q_dim() const { return d.n_q_heads * d.head_dim; }
@@ -101,6 +111,11 @@ Carve carve(const pc_ctx* c, int max_rows, int max_prefill) {
     v.s_len = take(M * 4);
     v.token = take(M * 4);
     v.last_row = take(M * 4);
+    // prefix part of the shared-prefix attention: (max, sum, unnormalised output) per (row, query head)
+    const size_t R = (size_t)std::max(max_rows, 1);
+    v.part_m = take(R * d.n_q_heads * 4);
+    v.part_l = take(R * d.n_q_heads * 4);
+    v.part_o = take(R * d.n_q_heads * d.head_dim * 4);
     v.total = off;
     return v;
 }
@@ -136,9 +151,83 @@ int gemm_bf16(pc_ctx* c, cudaStream_t st, const CUtensorMap& map_a, const WMap& 
     return PC_OK;
 }
 
+// How the rows of a forward pass group for attention.
+struct AttnPlan {
+    bool prefill;                      // true: causal attention inside each prompt, no suffix part
+    int n_groups;
+    const int32_t* group_row_start;    // device [n_groups + 1]
+    int max_group_rows;
+};
+
+int arena_maps(pc_ctx* c, const void* prompt_kv, int64_t prompt_slots, const void* suffix_kv, int64_t suffix_slots) {
+    const pc_model_desc& d = c->d;
+    const uint64_t planes = (uint64_t)d.n_layers * 2 * d.n_kv_heads;
+    if (prompt_kv != c->prompt_arena_ptr || prompt_slots != c->prompt_arena_slots) {
+        if (planes * (uint64_t)prompt_slots >= (1ull << 31)) return PC_ERR_CAPACITY;
+        if (!pc::make_bf16_map(&c->map_prompt_kv, prompt_kv, planes * prompt_slots, d.head_dim, pc::am::G_TK)) {
+            g_cuda_error = "cuTensorMapEncodeTiled failed for the prompt KV arena";
+            return PC_ERR_CUDA;
+        }
+        c->prompt_arena_ptr = prompt_kv; c->prompt_arena_slots = prompt_slots;
+    }
+    if (suffix_kv != nullptr && (suffix_kv != c->suffix_arena_ptr || suffix_slots != c->suffix_arena_slots)) {
+        if (planes * (uint64_t)suffix_slots >= (1ull << 31)) return PC_ERR_CAPACITY;
+        if (!pc::make_bf16_map(&c->map_suffix_kv, suffix_kv, planes * suffix_slots, d.head_dim, pc::am::S_TP)) {
+            g_cuda_error = "cuTensorMapEncodeTiled failed for the suffix KV arena";
+            return PC_ERR_CUDA;
+        }
+        c->suffix_arena_ptr = suffix_kv; c->suffix_arena_slots = suffix_slots;
+    }
+    return PC_OK;
+}
+
+template <int HD>
+int attention_bf16(pc_ctx* c, cudaStream_t st, int M, int layer, const AttnPlan& plan, pc::KvArena prompt_arena,
+                   pc::KvArena suffix_arena, const __nv_bfloat16* q, __nv_bfloat16* attn, bool profile) {
+    using namespace pc;
+    const pc_model_desc& d = c->d;
+    const RowGeom g = geom(c);
+    const float scale_log2 = 1.4426950408889634f / sqrtf((float)d.head_dim);
+    const int n_rep = d.n_q_heads / d.n_kv_heads;
+    am::PrefixPartial part{reinterpret_cast<float*>(c->ws + c->cv.part_m), reinterpret_cast<float*>(c->ws + c->cv.part_l),
+                           reinterpret_cast<float*>(c->ws + c->cv.part_o)};
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(am::attn_group_kernel<HD, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             am::group_smem_bytes<HD>());
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(am::attn_group_kernel<HD, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     am::group_smem_bytes<HD>());
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(am::attn_suffix_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     am::suffix_smem_bytes<HD>());
+        if (e != cudaSuccess) return cuda_fail(e, "attention kernel attributes");
+        configured = true;
+    }
+    const dim3 ggrid((plan.max_group_rows * n_rep + am::G_QROWS - 1) / am::G_QROWS, d.n_kv_heads, plan.n_groups);
+    if (plan.prefill) {
+        am::attn_group_kernel<HD, true><<<ggrid, am::G_THREADS, am::group_smem_bytes<HD>(), st>>>(
+            c->map_prompt_kv, prompt_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, plan.group_row_start, g, scale_log2,
+            part, attn, c->err);
+        count_launches(1);
+        return PC_OK;
+    }
+    am::attn_group_kernel<HD, false><<<ggrid, am::G_THREADS, am::group_smem_bytes<HD>(), st>>>(
+        c->map_prompt_kv, prompt_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, plan.group_row_start, g, scale_log2, part,
+        attn, c->err);
+    const int items = M * d.n_kv_heads;
+    const int sgrid = std::min(c->num_sms, (items + am::S_WARPS - 1) / am::S_WARPS);
+    if (profile) cudaEventRecord(c->prof_start, st);
+    am::attn_suffix_kernel<HD><<<sgrid, am::S_WARPS * 32, am::suffix_smem_bytes<HD>(), st>>>(
+        c->map_suffix_kv, suffix_arena.n_slots, M, d.n_q_heads, d.n_kv_heads, layer, q, g, scale_log2, part, attn, c->err);
+    if (profile) cudaEventRecord(c->prof_stop, st);
+    count_launches(2);
+    return PC_OK;
+}
+
 // The decoder layers over M rows whose geometry is already in the workspace; leaves the residual stream in ws.h.
 template <typename T>
-int run_layers(pc_ctx* c, cudaStream_t st, int M, pc::KvArena prompt_arena, pc::KvArena suffix_arena) {
+int run_layers(pc_ctx* c, cudaStream_t st, int M, pc::KvArena prompt_arena, pc::KvArena suffix_arena, const AttnPlan& plan) {
     using namespace pc;
     constexpr bool kF32 = std::is_same<T, float>::value;
     const pc_model_desc& d = c->d;
@@ -153,13 +242,16 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, pc::KvArena prompt_arena, pc::
     const RowGeom g = geom(c);
     const int half = d.head_dim / 2;
     const float scale = 1.0f / sqrtf((float)d.head_dim);
+    const int prof_layer = plan.prefill ? -1 : c->prof_layer;
+    if (!plan.prefill) c->prof_layer = -1;           // one-shot
 
     rope_table_kernel<<<(M * half + 255) / 256, 256, 0, st>>>(M, half, (double)d.rope_theta, g.pos, rope);
     embed_rmsnorm_kernel<T><<<M, 256, 0, st>>>(d.d_model, g.token, reinterpret_cast<const T*>(c->embed), c->attn_norm[0],
                                                d.rms_eps, h, a);
+    count_launches(2);
     PC_CUDA_CHECK_LAUNCH("embed_rmsnorm");
     for (int l = 0; l < d.n_layers; ++l) {
-        if (l > 0) rmsnorm_kernel<T><<<M, 256, 0, st>>>(d.d_model, h, nullptr, c->attn_norm[l], d.rms_eps, a);
+        if (l > 0) { rmsnorm_kernel<T><<<M, 256, 0, st>>>(d.d_model, h, nullptr, c->attn_norm[l], d.rms_eps, a); count_launches(1); }
         const float* bias = d.qkv_bias ? c->bqkv[l] : nullptr;
         if constexpr (kF32) {
             launch_gemm_simt<T>(st, a, reinterpret_cast<const T*>(c->wqkv[l]), M, c->n_qkv(), d.d_model,
@@ -170,18 +262,27 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, pc::KvArena prompt_arena, pc::
         qkv_post_kernel<T><<<dim3(M, d.n_q_heads + 2 * d.n_kv_heads), half, 0, st>>>(
             d.n_q_heads, d.n_kv_heads, d.head_dim, l, qkv, d.qk_norm ? c->q_norm[l] : nullptr,
             d.qk_norm ? c->k_norm[l] : nullptr, d.rms_eps, rope, g, prompt_arena, suffix_arena, q);
-        if (d.head_dim == 128)
-            attn_row_simt_kernel<T, 128><<<dim3(M, d.n_kv_heads), 128, 0, st>>>(d.n_q_heads, d.n_kv_heads, l, q, g, prompt_arena,
-                                                                               suffix_arena, scale, attn);
-        else
-            attn_row_simt_kernel<T, 64><<<dim3(M, d.n_kv_heads), 128, 0, st>>>(d.n_q_heads, d.n_kv_heads, l, q, g, prompt_arena,
-                                                                              suffix_arena, scale, attn);
+        count_launches(2);
         if constexpr (kF32) {
+            if (l == prof_layer) cudaEventRecord(c->prof_start, st);
+            if (d.head_dim == 128)
+                attn_row_simt_kernel<T, 128><<<dim3(M, d.n_kv_heads), 128, 0, st>>>(d.n_q_heads, d.n_kv_heads, l, q, g,
+                                                                                   prompt_arena, suffix_arena, scale, attn);
+            else
+                attn_row_simt_kernel<T, 64><<<dim3(M, d.n_kv_heads), 128, 0, st>>>(d.n_q_heads, d.n_kv_heads, l, q, g,
+                                                                                  prompt_arena, suffix_arena, scale, attn);
+            if (l == prof_layer) cudaEventRecord(c->prof_stop, st);
+            count_launches(1);
             launch_gemm_simt<T>(st, attn, reinterpret_cast<const T*>(c->wo[l]), M, d.d_model, c->q_dim(), EpiResidual{h, d.d_model});
         } else {
-            if (int rc = gemm_bf16(c, st, c->map_attn, c->m_wo[l], M, tc::EpiResidual{h, d.d_model})) return rc;
+            int rc = d.head_dim == 128
+                         ? attention_bf16<128>(c, st, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer)
+                         : attention_bf16<64>(c, st, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer);
+            if (rc) return rc;
+            if (int rc2 = gemm_bf16(c, st, c->map_attn, c->m_wo[l], M, tc::EpiResidual{h, d.d_model})) return rc2;
         }
         rmsnorm_kernel<T><<<M, 256, 0, st>>>(d.d_model, h, nullptr, c->mlp_norm[l], d.rms_eps, a);
+        count_launches(2);
         if constexpr (kF32) {
             launch_gemm_simt<T>(st, a, reinterpret_cast<const T*>(c->w_gate_up[l]), M, 2 * d.d_ff, d.d_model,
                                 EpiSwiGLU<T>{act, d.d_ff});
@@ -190,6 +291,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, pc::KvArena prompt_arena, pc::
             if (int rc = gemm_bf16(c, st, c->map_a, c->m_wgu[l], M, tc::EpiSwiGLU{act, d.d_ff})) return rc;
             if (int rc = gemm_bf16(c, st, c->map_act, c->m_wdown[l], M, tc::EpiResidual{h, d.d_model})) return rc;
         }
+        count_launches(2);
         PC_CUDA_CHECK_LAUNCH("decoder layer");
     }
     return PC_OK;
@@ -209,6 +311,7 @@ int run_lm_head(pc_ctx* c, cudaStream_t st, int n, const int32_t* src, float* lo
     } else {
         if (int rc = gemm_bf16(c, st, c->map_a, c->m_lm, n, tc::EpiStoreF32{logits, d.vocab, nullptr})) return rc;
     }
+    count_launches(2);
     PC_CUDA_CHECK_LAUNCH("lm head");
     return PC_OK;
 }
@@ -238,6 +341,17 @@ const char* pc_status_string(int status) {
 }
 
 const char* pc_last_cuda_error(void) { return g_cuda_error.c_str(); }
+
+uint64_t pc_launch_count(void) { return g_launches; }
+
+int pc_profile_attention(pc_ctx* ctx, int layer, void* event_start, void* event_stop) {
+    if (ctx == nullptr || layer < 0 || layer >= ctx->d.n_layers || event_start == nullptr || event_stop == nullptr)
+        return PC_ERR_INVALID_ARG;
+    ctx->prof_layer = layer;
+    ctx->prof_start = static_cast<cudaEvent_t>(event_start);
+    ctx->prof_stop = static_cast<cudaEvent_t>(event_stop);
+    return PC_OK;
+}
 
 int pc_create(const pc_model_desc* desc, const pc_weights* wts, pc_ctx** out) {
     if (desc == nullptr || wts == nullptr || out == nullptr) return PC_ERR_INVALID_ARG;
@@ -359,10 +473,17 @@ int pc_prefill_shared(pc_ctx* ctx, void* stream, int n_prompts, const int32_t* p
     int32_t* last_row = reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.last_row);
     pc::prep_prefill_rows<<<n_prompts, 256, 0, st>>>(n_prompts, prompt_tokens, prompt_offsets, prompt_kv_start, prompt_slots,
                                                      ctx->d.vocab, g, last_row, ctx->err);
+    count_launches(1);
     PC_CUDA_CHECK_LAUNCH("prep_prefill_rows");
     const pc::KvArena pa{prompt_kv, prompt_slots}, sa{prompt_kv, prompt_slots};
-    int rc = ctx->d.dtype == PC_DTYPE_F32 ? run_layers<float>(ctx, st, total_tokens, pa, sa)
-                                          : run_layers<__nv_bfloat16>(ctx, st, total_tokens, pa, sa);
+    const AttnPlan plan{true, n_prompts, prompt_offsets, max_prompt_len};
+    int rc = PC_OK;
+    if (ctx->d.dtype == PC_DTYPE_F32) {
+        rc = run_layers<float>(ctx, st, total_tokens, pa, sa, plan);
+    } else {
+        rc = arena_maps(ctx, prompt_kv, prompt_slots, nullptr, 0);
+        if (rc == PC_OK) rc = run_layers<__nv_bfloat16>(ctx, st, total_tokens, pa, sa, plan);
+    }
     if (rc) return rc;
     return ctx->d.dtype == PC_DTYPE_F32 ? run_lm_head<float>(ctx, st, n_prompts, last_row, last_logits)
                                         : run_lm_head<__nv_bfloat16>(ctx, st, n_prompts, last_row, last_logits);
@@ -390,10 +511,18 @@ int pc_decode_step(pc_ctx* ctx, void* stream, int n_rows, const int32_t* row_pro
     pc::prep_decode_rows<<<(n_rows + 127) / 128, 128, 0, st>>>(n_rows, row_prompt, row_step, row_kv_start, tokens, row_tok_index,
                                                                prompt_len, prompt_kv_start, prompt_slots, suffix_slots,
                                                                ctx->d.vocab, g, ctx->err);
+    count_launches(1);
     PC_CUDA_CHECK_LAUNCH("prep_decode_rows");
     const pc::KvArena pa{const_cast<void*>(prompt_kv), prompt_slots}, sa{suffix_kv, suffix_slots};
     const bool f32 = ctx->d.dtype == PC_DTYPE_F32;
-    int rc = f32 ? run_layers<float>(ctx, st, n_rows, pa, sa) : run_layers<__nv_bfloat16>(ctx, st, n_rows, pa, sa);
+    const AttnPlan plan{false, n_groups, group_row_start, max_group_rows};
+    int rc = PC_OK;
+    if (f32) {
+        rc = run_layers<float>(ctx, st, n_rows, pa, sa, plan);
+    } else {
+        rc = arena_maps(ctx, prompt_kv, prompt_slots, suffix_kv, suffix_slots);
+        if (rc == PC_OK) rc = run_layers<__nv_bfloat16>(ctx, st, n_rows, pa, sa, plan);
+    }
     if (rc) return rc;
     float* logits = logits_out ? logits_out : reinterpret_cast<float*>(ctx->ws + ctx->cv.logits);
     rc = f32 ? run_lm_head<float>(ctx, st, n_rows, nullptr, logits) : run_lm_head<__nv_bfloat16>(ctx, st, n_rows, nullptr, logits);
@@ -402,6 +531,7 @@ int pc_decode_step(pc_ctx* ctx, void* stream, int n_rows, const int32_t* row_pro
         pc::sample_kernel<<<n_rows, 256, 0, st>>>(ctx->d.vocab, logits, nullptr, sample->temperature,
                                                   (uint32_t)(sample->seed & 0xffffffffu), (uint32_t)(sample->seed >> 32), row_prompt,
                                                   row_rollout, row_step, 1, tokens, row_tok_index, 1, nullptr);
+        count_launches(1);
         PC_CUDA_CHECK_LAUNCH("sample");
     }
     return PC_OK;
@@ -417,6 +547,7 @@ int pc_sample(void* stream, int n_rows, int vocab, const float* logits, const in
     pc::sample_kernel<<<n_rows, 256, 0, static_cast<cudaStream_t>(stream)>>>(
         vocab, logits, logits_row, temperature, (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32), row_prompt, row_rollout,
         row_step, 0, out_tokens, out_index, 0, out_top2_gap);
+    count_launches(1);
     PC_CUDA_CHECK_LAUNCH("sample");
     return PC_OK;
 }
@@ -428,6 +559,7 @@ int pc_reward_last_token(void* stream, int n, const int32_t* tokens, const int64
     if (tokens == nullptr || last_index == nullptr || threshold == nullptr || reward == nullptr) return PC_ERR_INVALID_ARG;
     pc::reward_last_token_kernel<<<(n + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(n, tokens, last_index, threshold,
                                                                                                 reward);
+    count_launches(1);
     PC_CUDA_CHECK_LAUNCH("reward");
     return PC_OK;
 }
@@ -442,6 +574,7 @@ int pc_group_stats(void* stream, int n_groups, const float* rewards, const int32
     const int threads = 128, groups_per_block = threads / 32;
     pc::group_stats_kernel<<<(n_groups + groups_per_block - 1) / groups_per_block, threads, 0, static_cast<cudaStream_t>(stream)>>>(
         n_groups, rewards, group_start, group_count, n, n_success, mean, var);
+    count_launches(1);
     PC_CUDA_CHECK_LAUNCH("group_stats");
     return PC_OK;
 }
@@ -456,6 +589,7 @@ int pc_allocate(void* stream, int n_prompts, const int32_t* pilot_success, const
     pc::allocate_kernel<<<1, 1024, 0, static_cast<cudaStream_t>(stream)>>>(
         n_prompts, pilot_success, pilot_n, params->p_lower, params->p_upper, params->p_solve, params->n_commit, params->b_t, status,
         extra_rollouts, evict, n_selected, reinterpret_cast<long long*>(total_rollouts));
+    count_launches(1);
     PC_CUDA_CHECK_LAUNCH("allocate");
     return PC_OK;
 }
@@ -468,6 +602,7 @@ int pc_grpo_advantage(void* stream, int n_groups, const float* rewards, const in
     const int threads = 128, groups_per_block = threads / 32;
     pc::grpo_advantage_kernel<<<(n_groups + groups_per_block - 1) / groups_per_block, threads, 0, static_cast<cudaStream_t>(stream)>>>(
         n_groups, rewards, group_start, group_count, status, adv);
+    count_launches(1);
     PC_CUDA_CHECK_LAUNCH("grpo_advantage");
     return PC_OK;
 }
