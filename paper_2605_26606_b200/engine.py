@@ -84,11 +84,26 @@ class RolloutEngine:
         self.err_flag = torch.zeros(1, dtype=torch.int32, device=dev)
         B.pc_set_workspace(self.ctx, self.workspace, max_rows, max_prefill_tokens, self.err_flag)
         self.kv_dtype = torch.float32 if m.dtype == DTYPE_F32 else torch.bfloat16
+        # measurement: every `profile_every`-th decode step, time the suffix-attention kernel of one layer
+        self._arenas: Dict[str, Optional[torch.Tensor]] = {}
+        self.profile_every = 0
+        self.profile_layer = m.n_layers // 2
+        self.profile_samples: List[tuple] = []      # (start event, stop event, rows, suffix slots read per row)
 
     # ------------------------------------------------------------------------------------------
-    def kv_arena(self, n_slots: int) -> torch.Tensor:
+    def kv_arena(self, n_slots: int, which: str) -> torch.Tensor:
+        """An arena of n_slots slots; the previous arena of the same role is reused when it has the same size
+        (two 75 GB arenas must never be alive together)."""
         m = self.model
-        return torch.empty((m.n_layers, 2, m.n_kv_heads, max(n_slots, 1), m.head_dim), dtype=self.kv_dtype, device=self.device)
+        shape = (m.n_layers, 2, m.n_kv_heads, max(n_slots, 1), m.head_dim)
+        old = self._arenas.get(which)
+        if old is not None and tuple(old.shape) == shape:
+            return old
+        self._arenas[which] = None
+        del old
+        t = torch.empty(shape, dtype=self.kv_dtype, device=self.device)
+        self._arenas[which] = t
+        return t
 
     def check_error_flag(self) -> None:
         code = int(self.err_flag.item())
@@ -110,14 +125,16 @@ class RolloutEngine:
         self.prompt_len = up(batch.prompt_lens, torch.int32)
         self.prompt_kv_start = up(batch.prompt_offsets[:-1].astype(np.int64), torch.int64)
         self.total_prompt_tokens = int(batch.prompt_offsets[-1])
-        self.prompt_kv = self.kv_arena(self.total_prompt_tokens)
+        self.prompt_kv = self.kv_arena(self.total_prompt_tokens, "prompt")
         # every rollout (p, i) owns caps[p, i] suffix slots and max_new token cells
         caps = batch.caps.astype(np.int64)
         kv_start = np.zeros(P * G, dtype=np.int64)
         kv_start[1:] = np.cumsum(caps.reshape(-1))[:-1]
         self.kv_start_host = kv_start.reshape(P, G)
         self.suffix_slots = int(caps.sum())
-        self.suffix_kv = self.kv_arena(self.suffix_slots)
+        self.prompt_kv = self.prompt_kv
+        self.suffix_kv = None
+        self.suffix_kv = self.kv_arena(self.suffix_slots, "suffix")
         self.tokens = torch.full((P * G * wl.max_new,), -1, dtype=torch.int32, device=dev)
         self.last_logits = torch.empty((P, self.model.vocab), dtype=torch.float32, device=dev)
         self.rewards = torch.zeros(P * G, dtype=torch.float32, device=dev)
@@ -200,6 +217,11 @@ class RolloutEngine:
             if record_logits is not None and s in record_logits:
                 logits_out = torch.empty((nr, self.model.vocab), dtype=torch.float32, device=dev)
                 record_logits[s] = (logits_out, sch.row_prompt[o:o + nr].cpu().numpy(), sch.row_rollout[o:o + nr].cpu().numpy())
+            if self.profile_every and s % self.profile_every == self.profile_every // 2:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); e1.record()             # creates the underlying CUDA events
+                B.pc_profile_attention(self.ctx, self.profile_layer, e0, e1)
+                self.profile_samples.append((e0, e1, nr, s + 1))
             B.pc_decode_step(self.ctx, nr, pr + 4 * o, rr + 4 * o, rs + 4 * o, rk + 8 * o, self.tokens, rt + 8 * o,
                              int(sch.groups_per_step[s]), gs + 4 * go, int(sch.max_group_rows[s]), self.prompt_len,
                              self.prompt_kv, self.total_prompt_tokens, self.prompt_kv_start, self.suffix_kv,
@@ -211,9 +233,18 @@ class RolloutEngine:
     def pilot_commit_step(self, wl: Workload, batch: Batch, b_t: Optional[int] = None,
                           host_inputs: Optional[Dict[str, torch.Tensor]] = None) -> dict:
         """The whole step.  Returns host copies of every output plus token counts."""
+        self.load_batch(wl, batch, host_inputs)
+        status, n_tok = self.run_device(b_t)
+        out = self.collect(status)
+        out["generated_tokens"] = n_tok
+        return out
+
+    def run_device(self, b_t: Optional[int] = None):
+        """Everything between the uploaded batch and the finished advantages: prefill, pilot stage, statistics,
+        allocation, commit stage, union statistics, advantages.  Returns (status on the host, tokens generated)."""
+        wl = self.wl
         P, G, k = wl.n_prompts, wl.group_size, wl.n_pilot
         b_t = P if b_t is None else b_t
-        self.load_batch(wl, batch, host_inputs)
         self.prefill()
         pp, rr = np.repeat(np.arange(P), k), np.tile(np.arange(k), P)
         n_tok = self.run_stage(pp, rr)
@@ -232,9 +263,7 @@ class RolloutEngine:
         B.pc_group_stats(P, self.rewards, self.group_start, union_count, self.union_n, self.union_success, self.union_mean,
                          self.union_var)
         B.pc_grpo_advantage(P, self.rewards, self.group_start, union_count, self.status, self.adv)
-        out = self.collect(status)
-        out["generated_tokens"] = n_tok
-        return out
+        return status, n_tok
 
     def collect(self, status: np.ndarray) -> dict:
         wl, P, G, k = self.wl, self.wl.n_prompts, self.wl.group_size, self.wl.n_pilot

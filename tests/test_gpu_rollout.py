@@ -112,3 +112,20 @@ def test_run_twice_is_deterministic_and_batch_invariant():
         for i in range(w.group_size):
             if c["generated"][p, i]:
                 assert np.array_equal(a["tokens"][p][i], c["tokens"][p][i])
+
+
+def test_bf16_many_rows_long_prefix_long_suffix():
+    """Several query tiles per group, prompt longer than the K/V ring of the group kernel, suffix longer than the
+    ring of the suffix kernel, several work items per warp, ragged tails everywhere."""
+    model = wl.SMALL_BF16
+    w = dataclasses.replace(wl.WORKLOADS["config0"], model=model, n_prompts=2, prompt_len_lo=197, prompt_len_hi=333,
+                            group_size=70, n_pilot=70, max_new=140, cap_lo=90, cap_hi=140, data_seed=5, forced_explicit=None)
+    weights = wl.gen_weights(model, seed=2, threads=2, gain_jitter=0.1)
+    batch = wl.gen_batch(w)
+    dec = Decoder(model, weights)
+    P, G = w.n_prompts, w.group_size
+    prompts, rollouts = np.repeat(np.arange(P), G), np.tile(np.arange(G), P)
+    ref = oracle_group_tokens(dec, w, batch, prompts, rollouts)
+    eng = RolloutEngine(model, weights, max_rows=P * G, max_prefill_tokens=int(batch.prompt_offsets[-1]))
+    worst, n_cmp, n_exempt = teacher_forced_compare(eng, w, batch, ref, prompts, rollouts, logit_tol=5e-2, gap_tol=1e-1)
+    assert n_cmp == int(batch.caps.sum())
