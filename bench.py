@@ -126,6 +126,50 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def run_probe(args):
+    """Decode-step microbenchmark: R rollouts in 16 groups, every rollout S tokens deep, N steps timed."""
+    import torch
+    from paper_2605_26606_b200 import binding as B
+    from paper_2605_26606_b200 import build as _build
+    from paper_2605_26606_b200.engine import RolloutEngine
+    _build.build()
+    kv = dict(x.split("=") for x in args.probe.split(","))
+    rows, suffix, steps, plen = int(kv.get("rows", 256)), int(kv.get("suffix", 512)), int(kv.get("steps", 4)), int(kv.get("prompt", 640))
+    base = wl.WORKLOADS[args.config]
+    P = min(16, rows)
+    G = rows // P
+    cap = suffix + steps + 1
+    w = dataclasses.replace(base, n_prompts=P, group_size=G, n_pilot=G, prompt_len_lo=plen, prompt_len_hi=plen, max_new=cap,
+                            cap_lo=cap, cap_hi=cap, forced_frac=0.0, forced_explicit=None)
+    weights = wl.gen_weights(w.model, seed=0)
+    batch = wl.gen_batch(w)
+    eng = RolloutEngine(w.model, weights, max_rows=P * G, max_prefill_tokens=int(batch.prompt_offsets[-1]))
+    eng.load_batch(w, batch)
+    eng.suffix_kv.zero_()
+    eng.tokens.random_(0, w.model.vocab)
+    eng.prefill()
+    pp, rr = np.repeat(np.arange(P), G), np.tile(np.arange(G), P)
+    eng.run_stage(pp, rr, step_range=(suffix, suffix + 2))            # warm-up
+    torch.cuda.synchronize()
+    l0 = B.pc_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    t0 = time.perf_counter()
+    eng.run_stage(pp, rr, step_range=(suffix, suffix + steps))
+    host_ms = (time.perf_counter() - t0) * 1e3 / steps          # time the host needs to issue one step
+    e1.record()
+    torch.cuda.synchronize()
+    eng.check_error_flag()
+    ms = e0.elapsed_time(e1) / steps
+    m = w.model
+    bytes_step = m.weight_bytes_per_decode_step() + (P * G * (suffix + 1) + P * plen) * m.kv_bytes_per_token
+    peak, kind = load_peaks()
+    print(json.dumps({"probe": {"rows": P * G, "suffix": suffix, "steps": steps, "prompt_len": plen}, "ms_per_decode_step": ms, "host_issue_ms_per_step": host_ms,
+                      "tokens_per_s": P * G / (ms * 1e-3), "launches_per_step": (B.pc_launch_count() - l0) / steps,
+                      "hbm_bytes_per_step": bytes_step, "hbm_frac": bytes_step / (ms * 1e-3) / 1e9 / peak, "peak_kind": kind}),
+          flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -134,6 +178,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="config2", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--probe", default=None, metavar="rows=R,suffix=S,steps=N,prompt=L",
+                    help="time N decode steps of R rollouts (16 groups) that already hold S suffix tokens, then exit")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -143,6 +189,10 @@ def main():
     from paper_2605_26606_b200 import binding as B
     from paper_2605_26606_b200 import build as _build
     from paper_2605_26606_b200.engine import RolloutEngine
+
+    if args.probe is not None:
+        run_probe(args)
+        return
 
     rank, local_rank, world = dist_util.init("nccl")
     torch.cuda.set_device(local_rank)

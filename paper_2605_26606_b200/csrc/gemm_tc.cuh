@@ -131,7 +131,7 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n) {
 // ---------------------------------------------------------------------------------------------
 struct EpiStoreF32 {            // C = acc (+ bias)
     float* C; int ldc; const float* bias;
-    __device__ __forceinline__ void operator()(int row, int col0, const float* v, int n_valid) const {
+    __device__ __forceinline__ void operator()(int row, int col0, const float* v, int n_valid, int /*split*/) const {
         float* dst = C + (size_t)row * ldc + col0;
         if (n_valid == 32 && (ldc & 3) == 0) {
 #pragma unroll
@@ -147,9 +147,23 @@ struct EpiStoreF32 {            // C = acc (+ bias)
         }
     }
 };
+struct EpiPartial {             // P[split][row][col] = acc   (raw K-slice sums; the consumer adds the slices in order)
+    float* P; int ld; size_t split_stride;
+    __device__ __forceinline__ void operator()(int row, int col0, const float* v, int n_valid, int split) const {
+        float* dst = P + (size_t)split * split_stride + (size_t)row * ld + col0;
+        if (n_valid == 32 && (ld & 3) == 0) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (i < n_valid) dst[i] = v[i];
+        }
+    }
+};
 struct EpiResidual {            // H += acc
     float* H; int ldc;
-    __device__ __forceinline__ void operator()(int row, int col0, const float* v, int n_valid) const {
+    __device__ __forceinline__ void operator()(int row, int col0, const float* v, int n_valid, int /*split*/) const {
         float* dst = H + (size_t)row * ldc + col0;
         if (n_valid == 32 && (ldc & 3) == 0) {
 #pragma unroll
@@ -167,7 +181,7 @@ struct EpiResidual {            // H += acc
 };
 struct EpiSwiGLU {              // columns (2j, 2j+1) = (gate_j, up_j) -> out[row, j] = silu(gate) * up, bf16
     __nv_bfloat16* out; int ld;
-    __device__ __forceinline__ void operator()(int row, int col0, const float* v, int n_valid) const {
+    __device__ __forceinline__ void operator()(int row, int col0, const float* v, int n_valid, int /*split*/) const {
         __nv_bfloat16* dst = out + (size_t)row * ld + (col0 >> 1);
         if (n_valid == 32 && (ld & 7) == 0) {
             uint32_t w[8];
@@ -193,7 +207,7 @@ struct EpiSwiGLU {              // columns (2j, 2j+1) = (gate_j, up_j) -> out[ro
 template <int BN, class Epi>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, int M, int N, int K,
-               Epi epi, int32_t* err) {
+               int splits, Epi epi, int32_t* err) {
     constexpr int STAGES = num_stages(BN);
     constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
     constexpr uint32_t TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;
@@ -222,8 +236,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN - 1) / BN, n_tiles = tiles_m * tiles_n;
-    const int k_blocks = K / BK;
+    // work item t = ((n_tile * splits) + split) * tiles_m + m_tile; split s covers k-blocks [s*KB/splits, (s+1)*KB/splits)
+    const int tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN - 1) / BN, n_tiles = tiles_m * tiles_n * splits;
+    const int k_blocks_total = K / BK;
 
     if (warp == 0) {
         if (lane == 0) {
@@ -231,8 +246,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
-                const int m0 = (t % tiles_m) * BM, n0 = (t / tiles_m) * BN;
-                for (int kb = 0; kb < k_blocks; ++kb) {
+                const int m0 = (t % tiles_m) * BM, sp = (t / tiles_m) % splits, n0 = (t / (tiles_m * splits)) * BN;
+                const int kb0 = sp * k_blocks_total / splits, kb1 = (sp + 1) * k_blocks_total / splits;
+                for (int kb = kb0; kb < kb1; ++kb) {
                     if (!mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t sa = tiles_u32 + stage * (A_BYTES + B_BYTES), sb = sa + A_BYTES;
                     mbar_arrive_expect_tx(full0 + 8 * stage, A_BYTES + B_BYTES);
@@ -253,6 +269,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
+                const int sp = (t / tiles_m) % splits;
+                const int k_blocks = (sp + 1) * k_blocks_total / splits - sp * k_blocks_total / splits;
                 for (int kb = 0; kb < k_blocks; ++kb) {
                     if (!mbar_wait(full0 + 8 * stage, phase, abort_flag)) { ok = false; break; }
                     tc_fence_after();
@@ -278,7 +296,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
-            const int m0 = (t % tiles_m) * BM, n0 = (t / tiles_m) * BN;
+            const int m0 = (t % tiles_m) * BM, sp = (t / tiles_m) % splits, n0 = (t / (tiles_m * splits)) * BN;
             if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
             tc_fence_after();
             const int row = m0 + quarter * 32 + lane;
@@ -287,7 +305,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (n0 + c >= N) break;                 // warp-uniform
                 float v[32];
                 tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + c, v);
-                if (row < M) epi(row, n0 + c, v, min(32, N - (n0 + c)));
+                if (row < M) epi(row, n0 + c, v, min(32, N - (n0 + c)), sp);
             }
             tc_fence_before();
             __syncwarp();
@@ -313,8 +331,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
 // Host launcher.  map_w must have been encoded with box_rows = BN.
 template <int BN, class Epi>
-inline cudaError_t launch(cudaStream_t st, const CUtensorMap& map_a, const CUtensorMap& map_w, int M, int N, int K, Epi epi,
-                          int32_t* err, int num_sms) {
+inline cudaError_t launch(cudaStream_t st, const CUtensorMap& map_a, const CUtensorMap& map_w, int M, int N, int K, int splits,
+                          Epi epi, int32_t* err, int num_sms) {
     auto kern = gemm_tc_kernel<BN, Epi>;
     static bool configured = false;
     if (!configured) {
@@ -322,9 +340,9 @@ inline cudaError_t launch(cudaStream_t st, const CUtensorMap& map_a, const CUten
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
+    const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN) * splits;
     if (tiles == 0) return cudaSuccess;
-    kern<<<tiles < num_sms ? tiles : num_sms, NUM_THREADS, smem_bytes(BN), st>>>(map_a, map_w, M, N, K, epi, err);
+    kern<<<tiles < num_sms ? tiles : num_sms, NUM_THREADS, smem_bytes(BN), st>>>(map_a, map_w, M, N, K, splits, epi, err);
     return cudaGetLastError();
 }
 

@@ -102,15 +102,33 @@ __global__ void embed_rmsnorm_kernel(int d, const int32_t* token, const T* __res
         a[(size_t)r * d + i] = from_f32<T>(h[(size_t)r * d + i] * rstd * gain[i]);
 }
 
-// a[r, :] = RMSNorm(h[src[r], :]; gain);  src == nullptr means row r.
+// K-slice sums left by a split GEMM: value(row, col) = sum over s < n of p[s * stride + row * ld + col], added in
+// the order s = 0, 1, ... so that the result does not depend on which CTA finished first.
+struct Partials {
+    const float* p;
+    int n;              // 0: nothing pending
+    size_t stride;
+    int ld;
+};
+
+// Optional residual update followed by the norm:  h[row, :] += pending partial sums of row r;  a[r, :] = RMSNorm(h[row, :]; gain)
+// with row = src ? src[r] : r.  The partial sums are indexed by row, like h.
 template <typename T>
-__global__ void rmsnorm_kernel(int d, const float* __restrict__ h, const int32_t* __restrict__ src,
+__global__ void rmsnorm_kernel(int d, float* __restrict__ h, const int32_t* __restrict__ src, Partials pend,
                                const float* __restrict__ gain, float eps, T* __restrict__ a) {
     __shared__ float red[33];
     const int r = blockIdx.x;
-    const float* x = h + (size_t)(src ? src[r] : r) * d;
+    const int row = src ? src[r] : r;
+    float* x = h + (size_t)row * d;
     float ss = 0.f;
-    for (int i = threadIdx.x; i < d; i += blockDim.x) { const float v = x[i]; ss += v * v; }
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        float v = x[i];
+        if (pend.n > 0) {
+            for (int s = 0; s < pend.n; ++s) v += pend.p[(size_t)s * pend.stride + (size_t)row * pend.ld + i];
+            x[i] = v;
+        }
+        ss += v * v;
+    }
     ss = block_sum(ss, red);
     const float rstd = rsqrtf(ss / (float)d + eps);
     for (int i = threadIdx.x; i < d; i += blockDim.x) a[(size_t)r * d + i] = from_f32<T>(x[i] * rstd * gain[i]);
@@ -122,18 +140,23 @@ struct KvArena {
 };
 
 // One block per (row, head of the fused q|k|v projection); thread i handles the rotary pair (i, i + hd/2).
+// The projection arrives as K-slice partial sums (one slice when the GEMM was not split); the bias is added here.
 // q heads: optional RMSNorm over head_dim, RoPE, stored to q_out [M, Hq*hd] as T.
 // k heads: optional RMSNorm, RoPE, stored to the row's KV slot.  v heads: stored to the row's KV slot.
 template <typename T>
-__global__ void qkv_post_kernel(int Hq, int Hkv, int hd, int layer, const float* __restrict__ qkv,
+__global__ void qkv_post_kernel(int Hq, int Hkv, int hd, int layer, Partials qkv, const float* __restrict__ bias,
                                 const float* __restrict__ q_gain, const float* __restrict__ k_gain, float eps,
                                 const float2* __restrict__ rope, RowGeom g, KvArena prompt_arena, KvArena suffix_arena,
                                 T* __restrict__ q_out) {
     __shared__ float red[33];
     const int r = blockIdx.x, head = blockIdx.y, i = threadIdx.x, half = hd >> 1;
-    const int n_tot = (Hq + 2 * Hkv) * hd;
-    const float* src = qkv + (size_t)r * n_tot + (size_t)head * hd;
-    float x1 = src[i], x2 = src[i + half];
+    const size_t col = (size_t)head * hd + i;
+    float x1 = bias ? bias[col] : 0.f, x2 = bias ? bias[col + half] : 0.f;
+    for (int s = 0; s < qkv.n; ++s) {
+        const float* src = qkv.p + (size_t)s * qkv.stride + (size_t)r * qkv.ld + col;
+        x1 += src[0];
+        x2 += src[half];
+    }
     const bool is_q = head < Hq, is_k = !is_q && head < Hq + Hkv;
     if (is_q || is_k) {
         const float* gain = is_q ? q_gain : k_gain;

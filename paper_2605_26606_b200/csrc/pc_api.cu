@@ -42,9 +42,12 @@ int cuda_fail(cudaError_t e, const char* what) {
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+constexpr size_t kSplitMaxRows = 512;   // GEMMs over more rows are never split along K
+constexpr int kMaxSplits = 8;
+
 struct Carve {
     size_t h, a, qkv, q, attn, act, logits, rope, pos, wslot, warena, p_start, p_len, s_start, s_len, token, last_row,
-        part_m, part_l, part_o, total;
+        part_m, part_l, part_o, res_part, total;
 };
 
 // TMA descriptors of one bf16 weight matrix [N, K], one per tile width the GEMM may pick.
@@ -72,6 +75,7 @@ struct pc_ctx {
     // (built by pc_set_workspace over the full capacity of each buffer)
     std::vector<WMap> m_wqkv, m_wo, m_wgu, m_wdown;
     WMap m_lm;
+    pc::Partials pend{nullptr, 0, 0, 0};     // residual K-slices produced by the last GEMM and not yet folded into h
     CUtensorMap map_a, map_attn, map_act;
     int num_sms = 148;
     // TMA descriptors of the KV arenas, rebuilt when a call brings another arena
@@ -96,7 +100,9 @@ Carve carve(const pc_ctx* c, int max_rows, int max_prefill) {
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
     v.h = take(M * d.d_model * 4);
     v.a = take(M * d.d_model * eb);
-    v.qkv = take(M * c->n_qkv() * 4);
+    const size_t split_rows = std::min<size_t>(M, kSplitMaxRows) * kMaxSplits;      // rows x K-slices of a split GEMM
+    v.qkv = take(std::max(M, split_rows) * c->n_qkv() * 4);
+    v.res_part = take(split_rows * d.d_model * 4);
     v.q = take(M * c->q_dim() * eb);
     v.attn = take(M * c->q_dim() * eb);
     v.act = take(M * (size_t)d.d_ff * eb);
@@ -140,13 +146,31 @@ bool make_wmap(WMap* w, const void* base, int N, int K) {
     return pc::make_bf16_map(&w->wide, base, N, K, 256) && pc::make_bf16_map(&w->narrow, base, N, K, 64);
 }
 
-// bf16 GEMM on the tensor cores; the tile width is picked so that small batches still spread over the SMs.
-template <class Epi>
-int gemm_bf16(pc_ctx* c, cudaStream_t st, const CUtensorMap& map_a, const WMap& w, int M, Epi epi) {
+// Tile width and K-split of a bf16 GEMM over M rows.  Large batches take 128 x 256 tiles.  Small batches would
+// leave most SMs idle (the weight matrix is then streamed by a few CTAs only), so they take 128 x 64 tiles and,
+// where the epilogue allows it, split K so that about one CTA per SM is busy; the K-slices are summed in a
+// fixed order by the kernel that consumes the result.
+struct GemmPlan {
+    bool wide;
+    int splits;
+};
+GemmPlan plan_gemm(const pc_ctx* c, const WMap& w, int M, bool may_split) {
     const int tiles_m = (M + pc::tc::BM - 1) / pc::tc::BM;
-    const bool wide = tiles_m * ((w.N + 255) / 256) >= 100;
-    cudaError_t e = wide ? pc::tc::launch<256>(st, map_a, w.wide, M, w.N, w.K, epi, c->err, c->num_sms)
-                         : pc::tc::launch<64>(st, map_a, w.narrow, M, w.N, w.K, epi, c->err, c->num_sms);
+    GemmPlan p{true, 1};
+    if (tiles_m * ((w.N + 255) / 256) >= c->num_sms / 2) return p;
+    p.wide = false;
+    const int tiles = tiles_m * ((w.N + 63) / 64);
+    if (may_split && (size_t)M <= kSplitMaxRows) {
+        const int k_blocks = w.K / pc::tc::BK;
+        p.splits = std::max(1, std::min(std::min(c->num_sms / tiles, kMaxSplits), k_blocks / 4));
+    }
+    return p;
+}
+
+template <class Epi>
+int gemm_bf16(pc_ctx* c, cudaStream_t st, const CUtensorMap& map_a, const WMap& w, int M, GemmPlan p, Epi epi) {
+    cudaError_t e = p.wide ? pc::tc::launch<256>(st, map_a, w.wide, M, w.N, w.K, p.splits, epi, c->err, c->num_sms)
+                           : pc::tc::launch<64>(st, map_a, w.narrow, M, w.N, w.K, p.splits, epi, c->err, c->num_sms);
     if (e != cudaSuccess) return cuda_fail(e, "tensor-core gemm");
     return PC_OK;
 }
@@ -244,6 +268,9 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, pc::KvArena prompt_arena, pc::
     const float scale = 1.0f / sqrtf((float)d.head_dim);
     const int prof_layer = plan.prefill ? -1 : c->prof_layer;
     if (!plan.prefill) c->prof_layer = -1;           // one-shot
+    float* res_part = reinterpret_cast<float*>(w + c->cv.res_part);
+    const Partials none{nullptr, 0, 0, 0};
+    Partials pend = none;
 
     rope_table_kernel<<<(M * half + 255) / 256, 256, 0, st>>>(M, half, (double)d.rope_theta, g.pos, rope);
     embed_rmsnorm_kernel<T><<<M, 256, 0, st>>>(d.d_model, g.token, reinterpret_cast<const T*>(c->embed), c->attn_norm[0],
@@ -251,16 +278,23 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, pc::KvArena prompt_arena, pc::
     count_launches(2);
     PC_CUDA_CHECK_LAUNCH("embed_rmsnorm");
     for (int l = 0; l < d.n_layers; ++l) {
-        if (l > 0) { rmsnorm_kernel<T><<<M, 256, 0, st>>>(d.d_model, h, nullptr, c->attn_norm[l], d.rms_eps, a); count_launches(1); }
+        if (l > 0) {
+            rmsnorm_kernel<T><<<M, 256, 0, st>>>(d.d_model, h, nullptr, pend, c->attn_norm[l], d.rms_eps, a);
+            pend = none;
+            count_launches(1);
+        }
         const float* bias = d.qkv_bias ? c->bqkv[l] : nullptr;
+        Partials qkv_parts{qkv, 1, (size_t)M * c->n_qkv(), c->n_qkv()};
         if constexpr (kF32) {
             launch_gemm_simt<T>(st, a, reinterpret_cast<const T*>(c->wqkv[l]), M, c->n_qkv(), d.d_model,
-                                EpiStoreF32{qkv, c->n_qkv(), bias});
+                                EpiStoreF32{qkv, c->n_qkv(), nullptr});
         } else {
-            if (int rc = gemm_bf16(c, st, c->map_a, c->m_wqkv[l], M, tc::EpiStoreF32{qkv, c->n_qkv(), bias})) return rc;
+            const GemmPlan gp = plan_gemm(c, c->m_wqkv[l], M, true);
+            qkv_parts.n = gp.splits;
+            if (int rc = gemm_bf16(c, st, c->map_a, c->m_wqkv[l], M, gp, tc::EpiPartial{qkv, c->n_qkv(), qkv_parts.stride})) return rc;
         }
         qkv_post_kernel<T><<<dim3(M, d.n_q_heads + 2 * d.n_kv_heads), half, 0, st>>>(
-            d.n_q_heads, d.n_kv_heads, d.head_dim, l, qkv, d.qk_norm ? c->q_norm[l] : nullptr,
+            d.n_q_heads, d.n_kv_heads, d.head_dim, l, qkv_parts, bias, d.qk_norm ? c->q_norm[l] : nullptr,
             d.qk_norm ? c->k_norm[l] : nullptr, d.rms_eps, rope, g, prompt_arena, suffix_arena, q);
         count_launches(2);
         if constexpr (kF32) {
@@ -279,21 +313,36 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, pc::KvArena prompt_arena, pc::
                          ? attention_bf16<128>(c, st, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer)
                          : attention_bf16<64>(c, st, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer);
             if (rc) return rc;
-            if (int rc2 = gemm_bf16(c, st, c->map_attn, c->m_wo[l], M, tc::EpiResidual{h, d.d_model})) return rc2;
+            const GemmPlan gp = plan_gemm(c, c->m_wo[l], M, true);
+            if (gp.splits == 1) {
+                if (int rc2 = gemm_bf16(c, st, c->map_attn, c->m_wo[l], M, gp, tc::EpiResidual{h, d.d_model})) return rc2;
+            } else {
+                pend = Partials{res_part, gp.splits, (size_t)M * d.d_model, d.d_model};
+                if (int rc2 = gemm_bf16(c, st, c->map_attn, c->m_wo[l], M, gp, tc::EpiPartial{res_part, d.d_model, pend.stride})) return rc2;
+            }
         }
-        rmsnorm_kernel<T><<<M, 256, 0, st>>>(d.d_model, h, nullptr, c->mlp_norm[l], d.rms_eps, a);
+        rmsnorm_kernel<T><<<M, 256, 0, st>>>(d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a);
+        pend = none;
         count_launches(2);
         if constexpr (kF32) {
             launch_gemm_simt<T>(st, a, reinterpret_cast<const T*>(c->w_gate_up[l]), M, 2 * d.d_ff, d.d_model,
                                 EpiSwiGLU<T>{act, d.d_ff});
             launch_gemm_simt<T>(st, act, reinterpret_cast<const T*>(c->w_down[l]), M, d.d_model, d.d_ff, EpiResidual{h, d.d_model});
         } else {
-            if (int rc = gemm_bf16(c, st, c->map_a, c->m_wgu[l], M, tc::EpiSwiGLU{act, d.d_ff})) return rc;
-            if (int rc = gemm_bf16(c, st, c->map_act, c->m_wdown[l], M, tc::EpiResidual{h, d.d_model})) return rc;
+            if (int rc = gemm_bf16(c, st, c->map_a, c->m_wgu[l], M, plan_gemm(c, c->m_wgu[l], M, false), tc::EpiSwiGLU{act, d.d_ff}))
+                return rc;
+            const GemmPlan gp = plan_gemm(c, c->m_wdown[l], M, true);
+            if (gp.splits == 1) {
+                if (int rc = gemm_bf16(c, st, c->map_act, c->m_wdown[l], M, gp, tc::EpiResidual{h, d.d_model})) return rc;
+            } else {
+                pend = Partials{res_part, gp.splits, (size_t)M * d.d_model, d.d_model};
+                if (int rc = gemm_bf16(c, st, c->map_act, c->m_wdown[l], M, gp, tc::EpiPartial{res_part, d.d_model, pend.stride})) return rc;
+            }
         }
         count_launches(2);
         PC_CUDA_CHECK_LAUNCH("decoder layer");
     }
+    c->pend = pend;        // folded into h by the final norm
     return PC_OK;
 }
 
@@ -304,12 +353,14 @@ int run_lm_head(pc_ctx* c, cudaStream_t st, int n, const int32_t* src, float* lo
     const pc_model_desc& d = c->d;
     float* h = reinterpret_cast<float*>(c->ws + c->cv.h);
     T* a = reinterpret_cast<T*>(c->ws + c->cv.a);
-    rmsnorm_kernel<T><<<n, 256, 0, st>>>(d.d_model, h, src, c->final_norm, d.rms_eps, a);
+    rmsnorm_kernel<T><<<n, 256, 0, st>>>(d.d_model, h, src, c->pend, c->final_norm, d.rms_eps, a);
+    c->pend = pc::Partials{nullptr, 0, 0, 0};
     if constexpr (std::is_same<T, float>::value) {
         const T* wlm = reinterpret_cast<const T*>(d.tied_embed ? c->embed : c->lm_head);
         launch_gemm_simt<T>(st, a, wlm, n, d.vocab, d.d_model, EpiStoreF32{logits, d.vocab, nullptr});
     } else {
-        if (int rc = gemm_bf16(c, st, c->map_a, c->m_lm, n, tc::EpiStoreF32{logits, d.vocab, nullptr})) return rc;
+        if (int rc = gemm_bf16(c, st, c->map_a, c->m_lm, n, plan_gemm(c, c->m_lm, n, false), tc::EpiStoreF32{logits, d.vocab, nullptr}))
+            return rc;
     }
     count_launches(2);
     PC_CUDA_CHECK_LAUNCH("lm head");

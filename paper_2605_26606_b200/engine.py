@@ -189,12 +189,14 @@ class RolloutEngine:
                              cat(gs, np.int32), int(rows_per_step.sum()))
 
     def run_stage(self, prompts: np.ndarray, rollouts: np.ndarray, record_logits: Optional[dict] = None,
-                  teacher_forced: bool = False) -> int:
+                  teacher_forced: bool = False, step_range: Optional[tuple] = None) -> int:
         """First token from the prompt's prefill logits, then the decode steps.  Returns tokens generated.
 
         record_logits: {step: None} asks for the logits of those decode steps (filled in place with
         (logits tensor, row prompts, row rollouts)).  teacher_forced: nothing is sampled; the token
-        buffer must already hold every rollout's tokens and every step's logits must be recorded."""
+        buffer must already hold every rollout's tokens and every step's logits must be recorded.
+        step_range = (first, last): run only these decode steps (measurement of a step deep into a rollout;
+        the token buffer and the KV slots before `first` must already hold finite values)."""
         wl, dev = self.wl, self.device
         n = int(prompts.shape[0])
         if n == 0:
@@ -205,13 +207,14 @@ class RolloutEngine:
         d_zero = torch.zeros(n, dtype=torch.int32, device=dev)
         rid = prompts.astype(np.int64) * wl.group_size + rollouts
         d_first = torch.from_numpy(rid * wl.max_new).to(dev)
-        if not teacher_forced:
+        if not teacher_forced and step_range is None:
             B.pc_sample(n, self.model.vocab, self.last_logits, d_p, wl.temperature, wl.sample_seed, d_p, d_r, d_zero,
                         self.tokens, out_index=d_first)
         sch = self.build_schedule(prompts, rollouts)
         pr, rr, rs = sch.row_prompt.data_ptr(), sch.row_rollout.data_ptr(), sch.row_step.data_ptr()
         rk, rt, gs = sch.row_kv_start.data_ptr(), sch.row_tok_index.data_ptr(), sch.group_row_start.data_ptr()
-        for s in range(sch.n_steps):
+        first, last = (0, sch.n_steps) if step_range is None else (step_range[0], min(step_range[1], sch.n_steps))
+        for s in range(first, last):
             nr, o, go = int(sch.rows_per_step[s]), int(sch.row_off[s]), int(sch.group_off[s])
             logits_out = None
             if record_logits is not None and s in record_logits:
