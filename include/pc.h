@@ -188,6 +188,26 @@ PC_API int pc_decode_step(pc_ctx* ctx, void* stream, int n_rows,
                    const int64_t* prompt_kv_start, void* suffix_kv, int64_t suffix_slots,
                    float* logits_out, const pc_sample_params* sample);
 
+/* One decode step of a device-resident schedule (see pc_decode_run). */
+typedef struct pc_step_desc {
+    int32_t n_rows, n_groups, max_group_rows, reserved;
+    int64_t row_offset;     /* the step's rows are entries [row_offset, row_offset + n_rows) of the row_* arrays */
+    int64_t group_offset;   /* its groups are entries [group_offset, group_offset + n_groups] of group_row_start */
+} pc_step_desc;
+
+/* n_steps consecutive decode steps (each exactly a pc_decode_step with sampling and no logits output) over a
+ * schedule that already lives on the device: the row_* arrays and group_row_start hold every step's entries back to
+ * back and step s uses the slices named by steps[s].  steps_host and steps_dev are the same n_steps descriptors in
+ * host and in device memory.  The kernels of a step are captured once per batch-size class into a CUDA graph and
+ * replayed, so the host issues one launch per step; the stream must not be capturing.  Steps with n_rows = 0 are
+ * skipped.  All other arguments as in pc_decode_step. */
+PC_API int pc_decode_run(pc_ctx* ctx, void* stream, int n_steps, const pc_step_desc* steps_host, const pc_step_desc* steps_dev,
+                         const int32_t* row_prompt, const int32_t* row_rollout, const int32_t* row_step,
+                         const int64_t* row_kv_start, int32_t* tokens, const int64_t* row_tok_index,
+                         const int32_t* group_row_start, const int32_t* prompt_len, const void* prompt_kv,
+                         int64_t prompt_slots, const int64_t* prompt_kv_start, void* suffix_kv, int64_t suffix_slots,
+                         const pc_sample_params* sample);
+
 /* Seeded draw from softmax(logits / T) by Gumbel-max (Section 4.2: T = 1.0, top_p = 1.0):
  *   token = argmin-index argmax_v ( logits[v] / T + g_v ),   g_v = -ln(-ln u_v),
  *   u_v = ((w_v >> 9) + 0.5) * 2^-23, w_v = word (v & 3) of Philox4x32-10 with

@@ -23,7 +23,7 @@ PC_DTYPE_F32, PC_DTYPE_BF16 = 0, 1
 PC_STATUS_COMMIT, PC_STATUS_BUFFERED, PC_STATUS_DEFER_HARD, PC_STATUS_SKIP_EASY = 0, 1, 2, 3
 
 EXPORTS = ["pc_status_string", "pc_last_cuda_error", "pc_launch_count", "pc_profile_attention", "pc_create", "pc_destroy", "pc_workspace_bytes",
-           "pc_set_workspace", "pc_prefill_shared", "pc_decode_step", "pc_sample", "pc_reward_last_token",
+           "pc_set_workspace", "pc_prefill_shared", "pc_decode_step", "pc_decode_run", "pc_sample", "pc_reward_last_token",
            "pc_group_stats", "pc_allocate", "pc_grpo_advantage"]
 
 
@@ -37,6 +37,11 @@ class WeightsDesc(C.Structure):
     _fields_ = [("embed", C.c_void_p), ("lm_head", C.c_void_p), ("final_norm", C.c_void_p)] + \
                [(n, C.POINTER(C.c_void_p)) for n in ("attn_norm", "wqkv", "bqkv", "q_norm", "k_norm", "wo", "mlp_norm",
                                                       "w_gate_up", "w_down")]
+
+
+class StepDesc(C.Structure):
+    _fields_ = [("n_rows", C.c_int32), ("n_groups", C.c_int32), ("max_group_rows", C.c_int32), ("reserved", C.c_int32),
+                ("row_offset", C.c_int64), ("group_offset", C.c_int64)]
 
 
 class SampleParams(C.Structure):
@@ -82,6 +87,7 @@ def _lib():
         lib.pc_set_workspace.argtypes = [p, p, C.c_size_t, i, i, p]
         lib.pc_prefill_shared.argtypes = [p, p, i, p, p, i, i, p, i64, p, p]
         lib.pc_decode_step.argtypes = [p, p, i, p, p, p, p, p, p, i, p, i, p, p, i64, p, p, i64, p, C.POINTER(SampleParams)]
+        lib.pc_decode_run.argtypes = [p, p, i, p, p, p, p, p, p, p, p, p, p, p, i64, p, p, i64, C.POINTER(SampleParams)]
         lib.pc_sample.argtypes = [p, i, i, p, p, f, u64, p, p, p, p, p, p]
         lib.pc_reward_last_token.argtypes = [p, i, p, p, p, p]
         lib.pc_group_stats.argtypes = [p, i, p, p, p, p, p, p, p]
@@ -206,6 +212,16 @@ def pc_decode_step(ctx: Context, n_rows, row_prompt, row_rollout, row_step, row_
                                  max_group_rows, _ptr(prompt_len), _ptr(prompt_kv), prompt_slots, _ptr(prompt_kv_start),
                                  _ptr(suffix_kv), suffix_slots, _ptr(logits_out),
                                  C.byref(sample) if sample is not None else None), "pc_decode_step")
+
+
+def pc_decode_run(ctx: Context, n_steps, steps_host, steps_dev, row_prompt, row_rollout, row_step, row_kv_start, tokens,
+                  row_tok_index, group_row_start, prompt_len, prompt_kv, prompt_slots, prompt_kv_start, suffix_kv, suffix_slots,
+                  sample: SampleParams) -> None:
+    """steps_host: address (int) of n_steps StepDesc records in host memory; steps_dev: the same records on the device."""
+    _check(_lib().pc_decode_run(ctx.handle, _stream(), n_steps, steps_host, _ptr(steps_dev), _ptr(row_prompt), _ptr(row_rollout),
+                                _ptr(row_step), _ptr(row_kv_start), _ptr(tokens), _ptr(row_tok_index), _ptr(group_row_start),
+                                _ptr(prompt_len), _ptr(prompt_kv), prompt_slots, _ptr(prompt_kv_start), _ptr(suffix_kv),
+                                suffix_slots, C.byref(sample)), "pc_decode_run")
 
 
 def pc_sample(n_rows, vocab, logits, logits_row, temperature, seed, row_prompt, row_rollout, row_step, out_tokens,

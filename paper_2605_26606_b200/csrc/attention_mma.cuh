@@ -85,14 +85,16 @@ template <int HD> constexpr int group_smem_bytes() { return G_STAGES * 2 * G_TK 
 
 template <int HD, bool FINAL>
 __global__ void __launch_bounds__(G_THREADS, 1)
-attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, int64_t n_slots, int Hq, int Hkv, int layer,
-                  const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ group_row_start, RowGeom g,
+attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __restrict__ sd, int64_t n_slots, int Hq, int Hkv,
+                  int layer, const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ group_row_start, RowGeom g,
                   float scale_log2, PrefixPartial part, __nv_bfloat16* __restrict__ out, int32_t* err) {
     constexpr int KS = HD / 16;          // k-steps of Q K^T
     constexpr int NT = G_TK / 8;         // position n-tiles per stage
     constexpr int DT = HD / 8;           // dim n-tiles of the output
     constexpr int TILE_BYTES = G_TK * HD * 2;
     const int grp = blockIdx.z, kvh = blockIdx.y;
+    if (grp >= sd->n_groups) return;
+    group_row_start += sd->group_off;
     const int row0 = group_row_start[grp], n_rows = group_row_start[grp + 1] - row0;
     const int n_rep = Hq / Hkv;
     const int q0 = blockIdx.x * G_QROWS;
@@ -302,8 +304,8 @@ template <int HD> constexpr int suffix_smem_bytes() {
 
 template <int HD>
 __global__ void __launch_bounds__(S_WARPS * 32, 1)
-attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, int64_t n_slots, int n_rows, int Hq, int Hkv, int layer,
-                   const __nv_bfloat16* __restrict__ q, RowGeom g, float scale_log2, PrefixPartial part,
+attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __restrict__ sd, int64_t n_slots, int Hq, int Hkv,
+                   int layer, const __nv_bfloat16* __restrict__ q, RowGeom g, float scale_log2, PrefixPartial part,
                    __nv_bfloat16* __restrict__ out, int32_t* err) {
     constexpr int KS = HD / 16;                   // k-steps of K Q^T
     constexpr int DT = HD / 16;                   // 16-dim m-tiles of O^T
@@ -328,7 +330,7 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, int64_t n_slots, 
     }
     __syncthreads();
 
-    const int n_items = n_rows * Hkv;
+    const int n_items = sd->n_rows * Hkv;
     const int item_stride = gridDim.x * S_WARPS;
     const int first_item = blockIdx.x * S_WARPS + warp;
 

@@ -13,12 +13,13 @@ constexpr int ATTN_MAX_REP = 8;   // query heads per KV head supported
 
 // HD = head_dim (64 or 128); each lane owns EPL = HD / 32 consecutive dims of every K/V row.
 template <typename T, int HD>
-__global__ void __launch_bounds__(128) attn_row_simt_kernel(int Hq, int Hkv, int layer, const T* __restrict__ q,
+__global__ void __launch_bounds__(128) attn_row_simt_kernel(const StepDesc* __restrict__ sd, int Hq, int Hkv, int layer, const T* __restrict__ q,
                                                             RowGeom g, KvArena prompt_arena, KvArena suffix_arena,
                                                             float scale, T* __restrict__ out) {
     constexpr int EPL = HD / 32;
     constexpr int NW = 4;
     const int r = blockIdx.x, kvh = blockIdx.y;
+    if (r >= sd->n_rows) return;
     const int n_rep = Hq / Hkv;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 

@@ -16,6 +16,17 @@ enum DevError : int32_t {
     DEV_ERR_GROUP_RANGE = 4,    // group / row bookkeeping inconsistent
 };
 
+// What one forward pass covers, kept in device memory so that a captured CUDA graph can be replayed for
+// every decode step: kernels are launched with grids sized for an upper bound and read the live counts here.
+struct StepDesc {
+    int32_t n_rows;           // live rows (decode) or packed prompt tokens (prefill)
+    int32_t n_groups;         // groups of contiguous rows sharing a prompt
+    int32_t max_group_rows;
+    int32_t reserved;
+    int64_t row_off;          // offset of this step's rows in the caller's flat row arrays
+    int64_t group_off;        // offset of this step's group_row_start entries
+};
+
 __device__ __forceinline__ void set_error(int32_t* flag, int32_t code) {
     if (flag != nullptr) atomicCAS(flag, 0, code);
 }

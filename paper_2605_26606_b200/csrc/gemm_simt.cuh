@@ -34,13 +34,15 @@ struct EpiSwiGLU {              // columns (2j, 2j+1) = (gate_j, up_j)  ->  out[
 };
 
 template <typename T, class Epi>
-__global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ A, const T* __restrict__ W, int M, int N, int K, Epi epi) {
+__global__ void __launch_bounds__(256) gemm_simt_kernel(const StepDesc* __restrict__ sd, const T* __restrict__ A, const T* __restrict__ W, int M, int N, int K, Epi epi) {
+    if (sd != nullptr) M = sd->n_rows;          // live row count; the grid was sized for an upper bound
     constexpr int BM = 64, BN = 64, BK = 16;
     __shared__ float As[BK][BM + 4];
     __shared__ float Ws[BK][BN + 4];
     const int tid = threadIdx.x;
     const int tx = tid & 15, ty = tid >> 4;
     const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    if (m0 >= M) return;
     const int lrow = tid >> 2, lk = (tid & 3) * 4;
     float acc[4][4] = {};
     for (int k0 = 0; k0 < K; k0 += BK) {
@@ -75,10 +77,10 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ A,
 }
 
 template <typename T, class Epi>
-inline void launch_gemm_simt(cudaStream_t st, const T* A, const T* W, int M, int N, int K, Epi epi) {
+inline void launch_gemm_simt(cudaStream_t st, const StepDesc* sd, const T* A, const T* W, int M, int N, int K, Epi epi) {
     if (M <= 0 || N <= 0) return;
     dim3 grid((N + 63) / 64, (M + 63) / 64);
-    gemm_simt_kernel<T, Epi><<<grid, 256, 0, st>>>(A, W, M, N, K, epi);
+    gemm_simt_kernel<T, Epi><<<grid, 256, 0, st>>>(sd, A, W, M, N, K, epi);
 }
 
 }  // namespace pc

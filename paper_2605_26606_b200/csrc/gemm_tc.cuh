@@ -131,6 +131,7 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n) {
 // ---------------------------------------------------------------------------------------------
 struct EpiStoreF32 {            // C = acc (+ bias)
     float* C; int ldc; const float* bias;
+    __device__ __forceinline__ void set_rows(int) {}
     __device__ __forceinline__ void operator()(int row, int col0, const float* v, int n_valid, int /*split*/) const {
         float* dst = C + (size_t)row * ldc + col0;
         if (n_valid == 32 && (ldc & 3) == 0) {
@@ -149,6 +150,7 @@ struct EpiStoreF32 {            // C = acc (+ bias)
 };
 struct EpiPartial {             // P[split][row][col] = acc   (raw K-slice sums; the consumer adds the slices in order)
     float* P; int ld; size_t split_stride;
+    __device__ __forceinline__ void set_rows(int m) { split_stride = (size_t)m * ld; }     // slices packed by live rows
     __device__ __forceinline__ void operator()(int row, int col0, const float* v, int n_valid, int split) const {
         float* dst = P + (size_t)split * split_stride + (size_t)row * ld + col0;
         if (n_valid == 32 && (ld & 3) == 0) {
@@ -163,6 +165,7 @@ struct EpiPartial {             // P[split][row][col] = acc   (raw K-slice sums;
 };
 struct EpiResidual {            // H += acc
     float* H; int ldc;
+    __device__ __forceinline__ void set_rows(int) {}
     __device__ __forceinline__ void operator()(int row, int col0, const float* v, int n_valid, int /*split*/) const {
         float* dst = H + (size_t)row * ldc + col0;
         if (n_valid == 32 && (ldc & 3) == 0) {
@@ -181,6 +184,7 @@ struct EpiResidual {            // H += acc
 };
 struct EpiSwiGLU {              // columns (2j, 2j+1) = (gate_j, up_j) -> out[row, j] = silu(gate) * up, bf16
     __nv_bfloat16* out; int ld;
+    __device__ __forceinline__ void set_rows(int) {}
     __device__ __forceinline__ void operator()(int row, int col0, const float* v, int n_valid, int /*split*/) const {
         __nv_bfloat16* dst = out + (size_t)row * ld + (col0 >> 1);
         if (n_valid == 32 && (ld & 7) == 0) {
@@ -206,8 +210,10 @@ struct EpiSwiGLU {              // columns (2j, 2j+1) = (gate_j, up_j) -> out[ro
 // ---------------------------------------------------------------------------------------------
 template <int BN, class Epi>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, int M, int N, int K,
-               int splits, Epi epi, int32_t* err) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const StepDesc* __restrict__ sd,
+               int M, int N, int K, int splits, Epi epi, int32_t* err) {
+    if (sd != nullptr) M = sd->n_rows;          // live row count; the grid was sized for an upper bound
+    epi.set_rows(M);
     constexpr int STAGES = num_stages(BN);
     constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
     constexpr uint32_t TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;
@@ -329,20 +335,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
 }
 
+// Must run once per kernel instance before its first launch (raises the dynamic shared memory limit).
+template <int BN, class Epi>
+inline cudaError_t configure() {
+    return cudaFuncSetAttribute(gemm_tc_kernel<BN, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(BN));
+}
+
 // Host launcher.  map_w must have been encoded with box_rows = BN.
 template <int BN, class Epi>
-inline cudaError_t launch(cudaStream_t st, const CUtensorMap& map_a, const CUtensorMap& map_w, int M, int N, int K, int splits,
-                          Epi epi, int32_t* err, int num_sms) {
+inline cudaError_t launch(cudaStream_t st, const CUtensorMap& map_a, const CUtensorMap& map_w, const StepDesc* sd, int M, int N,
+                          int K, int splits, Epi epi, int32_t* err, int num_sms) {
     auto kern = gemm_tc_kernel<BN, Epi>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(BN));
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
     const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN) * splits;
     if (tiles == 0) return cudaSuccess;
-    kern<<<tiles < num_sms ? tiles : num_sms, NUM_THREADS, smem_bytes(BN), st>>>(map_a, map_w, M, N, K, splits, epi, err);
+    kern<<<tiles < num_sms ? tiles : num_sms, NUM_THREADS, smem_bytes(BN), st>>>(map_a, map_w, sd, M, N, K, splits, epi, err);
     return cudaGetLastError();
 }
 

@@ -17,20 +17,32 @@ struct RowGeom {
     int32_t* token;      // [M] input token id
 };
 
+__global__ void set_step_desc(StepDesc* sd, int n_rows, int n_groups, int max_group_rows) {
+    sd->n_rows = n_rows; sd->n_groups = n_groups; sd->max_group_rows = max_group_rows; sd->reserved = 0;
+    sd->row_off = 0; sd->group_off = 0;
+}
+// First node of a captured decode step: takes the next descriptor of the caller's schedule.
+__global__ void load_step_desc(const StepDesc* __restrict__ steps, int32_t* counter, StepDesc* sd) {
+    const int i = *counter;
+    *sd = steps[i];
+    *counter = i + 1;
+}
+
 // Decode: row r of prompt p with `step` suffix tokens cached attends prompt slots [start_p, start_p + Lp)
 // and suffix slots [kv_start_r, kv_start_r + step + 1); its own K/V goes to suffix slot kv_start_r + step.
-__global__ void prep_decode_rows(int n_rows, const int32_t* row_prompt, const int32_t* row_step,
+__global__ void prep_decode_rows(const StepDesc* __restrict__ sd, const int32_t* row_prompt, const int32_t* row_step,
                                  const int64_t* row_kv_start, const int32_t* tokens, const int64_t* row_tok_index,
                                  const int32_t* prompt_len, const int64_t* prompt_kv_start, int64_t prompt_slots,
                                  int64_t suffix_slots, int vocab, RowGeom g, int32_t* err) {
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
-    if (r >= n_rows) return;
-    const int p = row_prompt[r];
-    const int step = row_step[r];
+    if (r >= sd->n_rows) return;
+    const int64_t ro = sd->row_off + r;
+    const int p = row_prompt[ro];
+    const int step = row_step[ro];
     const int Lp = prompt_len[p];
     const int64_t ps = prompt_kv_start[p];
-    const int64_t ss = row_kv_start[r];
-    int tok = tokens[row_tok_index[r]];
+    const int64_t ss = row_kv_start[ro];
+    int tok = tokens[row_tok_index[ro]];
     bool ok = true;
     if (tok < 0 || tok >= vocab) { set_error(err, DEV_ERR_TOKEN_RANGE); tok = 0; }
     if (ps < 0 || Lp < 0 || ps + Lp > prompt_slots || ss < 0 || step < 0 || ss + step + 1 > suffix_slots) {
@@ -73,9 +85,9 @@ __global__ void prep_prefill_rows(int n_prompts, const int32_t* prompt_tokens, c
 }
 
 // cos/sin of pos * theta^(-2i/hd), evaluated in double so that long positions keep float accuracy.
-__global__ void rope_table_kernel(int M, int half, double theta, const int32_t* pos, float2* table) {
+__global__ void rope_table_kernel(const StepDesc* __restrict__ sd, int half, double theta, const int32_t* pos, float2* table) {
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= M * half) return;
+    if (idx >= sd->n_rows * half) return;
     const int r = idx / half, i = idx - r * half;
     const double inv_freq = pow(theta, -(double)i / (double)half);
     double s, c;
@@ -85,10 +97,11 @@ __global__ void rope_table_kernel(int M, int half, double theta, const int32_t* 
 
 // h[r, :] = E[token[r], :] (float residual stream); a[r, :] = RMSNorm(h[r, :]; gain) in storage type T.
 template <typename T>
-__global__ void embed_rmsnorm_kernel(int d, const int32_t* token, const T* __restrict__ embed, const float* __restrict__ gain,
-                                     float eps, float* __restrict__ h, T* __restrict__ a) {
+__global__ void embed_rmsnorm_kernel(const StepDesc* __restrict__ sd, int d, const int32_t* token, const T* __restrict__ embed,
+                                     const float* __restrict__ gain, float eps, float* __restrict__ h, T* __restrict__ a) {
     __shared__ float red[33];
     const int r = blockIdx.x;
+    if (r >= sd->n_rows) return;
     const T* e = embed + (size_t)token[r] * d;
     float ss = 0.f;
     for (int i = threadIdx.x; i < d; i += blockDim.x) {
@@ -114,10 +127,12 @@ struct Partials {
 // Optional residual update followed by the norm:  h[row, :] += pending partial sums of row r;  a[r, :] = RMSNorm(h[row, :]; gain)
 // with row = src ? src[r] : r.  The partial sums are indexed by row, like h.
 template <typename T>
-__global__ void rmsnorm_kernel(int d, float* __restrict__ h, const int32_t* __restrict__ src, Partials pend,
-                               const float* __restrict__ gain, float eps, T* __restrict__ a) {
+__global__ void rmsnorm_kernel(const StepDesc* __restrict__ sd, int d, float* __restrict__ h, const int32_t* __restrict__ src,
+                               Partials pend, const float* __restrict__ gain, float eps, T* __restrict__ a) {
     __shared__ float red[33];
     const int r = blockIdx.x;
+    if (sd != nullptr && r >= sd->n_rows) return;
+    if (pend.n > 0 && sd != nullptr) pend.stride = (size_t)sd->n_rows * pend.ld;      // slices are packed by the live row count
     const int row = src ? src[r] : r;
     float* x = h + (size_t)row * d;
     float ss = 0.f;
@@ -144,12 +159,15 @@ struct KvArena {
 // q heads: optional RMSNorm over head_dim, RoPE, stored to q_out [M, Hq*hd] as T.
 // k heads: optional RMSNorm, RoPE, stored to the row's KV slot.  v heads: stored to the row's KV slot.
 template <typename T>
-__global__ void qkv_post_kernel(int Hq, int Hkv, int hd, int layer, Partials qkv, const float* __restrict__ bias,
+__global__ void qkv_post_kernel(const StepDesc* __restrict__ sd, int Hq, int Hkv, int hd, int layer, Partials qkv,
+                                const float* __restrict__ bias,
                                 const float* __restrict__ q_gain, const float* __restrict__ k_gain, float eps,
                                 const float2* __restrict__ rope, RowGeom g, KvArena prompt_arena, KvArena suffix_arena,
                                 T* __restrict__ q_out) {
     __shared__ float red[33];
     const int r = blockIdx.x, head = blockIdx.y, i = threadIdx.x, half = hd >> 1;
+    if (r >= sd->n_rows) return;
+    qkv.stride = (size_t)sd->n_rows * qkv.ld;                           // slices are packed by the live row count
     const size_t col = (size_t)head * hd + i;
     float x1 = bias ? bias[col] : 0.f, x2 = bias ? bias[col + half] : 0.f;
     for (int s = 0; s < qkv.n; ++s) {

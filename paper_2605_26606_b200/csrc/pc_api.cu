@@ -47,7 +47,19 @@ constexpr int kMaxSplits = 8;
 
 struct Carve {
     size_t h, a, qkv, q, attn, act, logits, rope, pos, wslot, warena, p_start, p_len, s_start, s_len, token, last_row,
-        part_m, part_l, part_o, res_part, total;
+        part_m, part_l, part_o, res_part, step_desc, step_counter, total;
+};
+
+// A captured decode step, replayable for every step that fits the same upper bounds and reads the same arrays.
+struct GraphKey {
+    int m_bound, groups_bound, group_rows_bound, pad;
+    const void* steps_dev;
+    unsigned char args[160];
+};
+struct GraphEntry {
+    GraphKey key;
+    cudaGraphExec_t exec;
+    int launches;       // kernels in the graph
 };
 
 // TMA descriptors of one bf16 weight matrix [N, K], one per tile width the GEMM may pick.
@@ -85,6 +97,13 @@ struct pc_ctx {
     int prof_layer = -1;
     cudaEvent_t prof_start = nullptr, prof_stop = nullptr;
 
+    std::vector<GraphEntry> graphs;
+    void drop_graphs() {
+        for (auto& g : graphs) cudaGraphExecDestroy(g.exec);
+        graphs.clear();
+    }
+    ~pc_ctx() { drop_graphs(); }
+
     int n_qkv() const { return (d.n_q_heads + 2 * d.n_kv_heads) * d.head_dim; }
     int q_dim() const { return d.n_q_heads * d.head_dim; }
     size_t eb() const { return d.dtype == PC_DTYPE_F32 ? 4 : 2; }
@@ -103,6 +122,8 @@ Carve carve(const pc_ctx* c, int max_rows, int max_prefill) {
     const size_t split_rows = std::min<size_t>(M, kSplitMaxRows) * kMaxSplits;      // rows x K-slices of a split GEMM
     v.qkv = take(std::max(M, split_rows) * c->n_qkv() * 4);
     v.res_part = take(split_rows * d.d_model * 4);
+    v.step_desc = take(sizeof(pc::StepDesc));
+    v.step_counter = take(4);
     v.q = take(M * c->q_dim() * eb);
     v.attn = take(M * c->q_dim() * eb);
     v.act = take(M * (size_t)d.d_ff * eb);
@@ -168,9 +189,9 @@ GemmPlan plan_gemm(const pc_ctx* c, const WMap& w, int M, bool may_split) {
 }
 
 template <class Epi>
-int gemm_bf16(pc_ctx* c, cudaStream_t st, const CUtensorMap& map_a, const WMap& w, int M, GemmPlan p, Epi epi) {
-    cudaError_t e = p.wide ? pc::tc::launch<256>(st, map_a, w.wide, M, w.N, w.K, p.splits, epi, c->err, c->num_sms)
-                           : pc::tc::launch<64>(st, map_a, w.narrow, M, w.N, w.K, p.splits, epi, c->err, c->num_sms);
+int gemm_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, const CUtensorMap& map_a, const WMap& w, int M, GemmPlan p, Epi epi) {
+    cudaError_t e = p.wide ? pc::tc::launch<256>(st, map_a, w.wide, sd, M, w.N, w.K, p.splits, epi, c->err, c->num_sms)
+                           : pc::tc::launch<64>(st, map_a, w.narrow, sd, M, w.N, w.K, p.splits, epi, c->err, c->num_sms);
     if (e != cudaSuccess) return cuda_fail(e, "tensor-core gemm");
     return PC_OK;
 }
@@ -178,9 +199,9 @@ int gemm_bf16(pc_ctx* c, cudaStream_t st, const CUtensorMap& map_a, const WMap& 
 // How the rows of a forward pass group for attention.
 struct AttnPlan {
     bool prefill;                      // true: causal attention inside each prompt, no suffix part
-    int n_groups;
-    const int32_t* group_row_start;    // device [n_groups + 1]
-    int max_group_rows;
+    int n_groups;                      // upper bound used for the grid; the live count is in the step descriptor
+    const int32_t* group_row_start;    // device; the step's entries start at the descriptor's group_off
+    int max_group_rows;                // upper bound
 };
 
 int arena_maps(pc_ctx* c, const void* prompt_kv, int64_t prompt_slots, const void* suffix_kv, int64_t suffix_slots) {
@@ -205,8 +226,36 @@ int arena_maps(pc_ctx* c, const void* prompt_kv, int64_t prompt_slots, const voi
     return PC_OK;
 }
 
+// Raises the dynamic shared memory limit of every tensor-core kernel instance (once per process and device).
 template <int HD>
-int attention_bf16(pc_ctx* c, cudaStream_t st, int M, int layer, const AttnPlan& plan, pc::KvArena prompt_arena,
+cudaError_t configure_attention() {
+    using namespace pc;
+    cudaError_t e = cudaFuncSetAttribute(am::attn_group_kernel<HD, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         am::group_smem_bytes<HD>());
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(am::attn_group_kernel<HD, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 am::group_smem_bytes<HD>());
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(am::attn_suffix_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, am::suffix_smem_bytes<HD>());
+    return e;
+}
+cudaError_t configure_kernels() {
+    using namespace pc;
+    cudaError_t e = tc::configure<256, tc::EpiPartial>();
+    if (e == cudaSuccess) e = tc::configure<64, tc::EpiPartial>();
+    if (e == cudaSuccess) e = tc::configure<256, tc::EpiResidual>();
+    if (e == cudaSuccess) e = tc::configure<64, tc::EpiResidual>();
+    if (e == cudaSuccess) e = tc::configure<256, tc::EpiSwiGLU>();
+    if (e == cudaSuccess) e = tc::configure<64, tc::EpiSwiGLU>();
+    if (e == cudaSuccess) e = tc::configure<256, tc::EpiStoreF32>();
+    if (e == cudaSuccess) e = tc::configure<64, tc::EpiStoreF32>();
+    if (e == cudaSuccess) e = configure_attention<128>();
+    if (e == cudaSuccess) e = configure_attention<64>();
+    return e;
+}
+
+template <int HD>
+int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, int layer, const AttnPlan& plan, pc::KvArena prompt_arena,
                    pc::KvArena suffix_arena, const __nv_bfloat16* q, __nv_bfloat16* attn, bool profile) {
     using namespace pc;
     const pc_model_desc& d = c->d;
@@ -215,43 +264,32 @@ int attention_bf16(pc_ctx* c, cudaStream_t st, int M, int layer, const AttnPlan&
     const int n_rep = d.n_q_heads / d.n_kv_heads;
     am::PrefixPartial part{reinterpret_cast<float*>(c->ws + c->cv.part_m), reinterpret_cast<float*>(c->ws + c->cv.part_l),
                            reinterpret_cast<float*>(c->ws + c->cv.part_o)};
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(am::attn_group_kernel<HD, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             am::group_smem_bytes<HD>());
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(am::attn_group_kernel<HD, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     am::group_smem_bytes<HD>());
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(am::attn_suffix_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     am::suffix_smem_bytes<HD>());
-        if (e != cudaSuccess) return cuda_fail(e, "attention kernel attributes");
-        configured = true;
-    }
     const dim3 ggrid((plan.max_group_rows * n_rep + am::G_QROWS - 1) / am::G_QROWS, d.n_kv_heads, plan.n_groups);
     if (plan.prefill) {
         am::attn_group_kernel<HD, true><<<ggrid, am::G_THREADS, am::group_smem_bytes<HD>(), st>>>(
-            c->map_prompt_kv, prompt_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, plan.group_row_start, g, scale_log2,
+            c->map_prompt_kv, sd, prompt_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, plan.group_row_start, g, scale_log2,
             part, attn, c->err);
         count_launches(1);
         return PC_OK;
     }
     am::attn_group_kernel<HD, false><<<ggrid, am::G_THREADS, am::group_smem_bytes<HD>(), st>>>(
-        c->map_prompt_kv, prompt_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, plan.group_row_start, g, scale_log2, part,
+        c->map_prompt_kv, sd, prompt_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, plan.group_row_start, g, scale_log2, part,
         attn, c->err);
     const int items = M * d.n_kv_heads;
     const int sgrid = std::min(c->num_sms, (items + am::S_WARPS - 1) / am::S_WARPS);
     if (profile) cudaEventRecord(c->prof_start, st);
     am::attn_suffix_kernel<HD><<<sgrid, am::S_WARPS * 32, am::suffix_smem_bytes<HD>(), st>>>(
-        c->map_suffix_kv, suffix_arena.n_slots, M, d.n_q_heads, d.n_kv_heads, layer, q, g, scale_log2, part, attn, c->err);
+        c->map_suffix_kv, sd, suffix_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, g, scale_log2, part, attn, c->err);
     if (profile) cudaEventRecord(c->prof_stop, st);
     count_launches(2);
     return PC_OK;
 }
 
-// The decoder layers over M rows whose geometry is already in the workspace; leaves the residual stream in ws.h.
+// The decoder layers over the rows whose geometry is already in the workspace; leaves the residual stream in ws.h.
+// M is the row count grids and GEMM plans are sized for; the live count (<= M) is read from *sd on the device.
 template <typename T>
-int run_layers(pc_ctx* c, cudaStream_t st, int M, pc::KvArena prompt_arena, pc::KvArena suffix_arena, const AttnPlan& plan) {
+int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::KvArena prompt_arena, pc::KvArena suffix_arena,
+               const AttnPlan& plan) {
     using namespace pc;
     constexpr bool kF32 = std::is_same<T, float>::value;
     const pc_model_desc& d = c->d;
@@ -266,77 +304,81 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, pc::KvArena prompt_arena, pc::
     const RowGeom g = geom(c);
     const int half = d.head_dim / 2;
     const float scale = 1.0f / sqrtf((float)d.head_dim);
-    const int prof_layer = plan.prefill ? -1 : c->prof_layer;
-    if (!plan.prefill) c->prof_layer = -1;           // one-shot
+    int prof_layer = plan.prefill ? -1 : c->prof_layer;
+    if (!plan.prefill) c->prof_layer = -1;           // one-shot (a captured step never carries the events)
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    cudaStreamIsCapturing(st, &cap);
+    const bool capturing = cap != cudaStreamCaptureStatusNone;
+    if (capturing) prof_layer = -1;
     float* res_part = reinterpret_cast<float*>(w + c->cv.res_part);
     const Partials none{nullptr, 0, 0, 0};
     Partials pend = none;
 
-    rope_table_kernel<<<(M * half + 255) / 256, 256, 0, st>>>(M, half, (double)d.rope_theta, g.pos, rope);
-    embed_rmsnorm_kernel<T><<<M, 256, 0, st>>>(d.d_model, g.token, reinterpret_cast<const T*>(c->embed), c->attn_norm[0],
+    rope_table_kernel<<<(M * half + 255) / 256, 256, 0, st>>>(sd, half, (double)d.rope_theta, g.pos, rope);
+    embed_rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, g.token, reinterpret_cast<const T*>(c->embed), c->attn_norm[0],
                                                d.rms_eps, h, a);
     count_launches(2);
     PC_CUDA_CHECK_LAUNCH("embed_rmsnorm");
     for (int l = 0; l < d.n_layers; ++l) {
         if (l > 0) {
-            rmsnorm_kernel<T><<<M, 256, 0, st>>>(d.d_model, h, nullptr, pend, c->attn_norm[l], d.rms_eps, a);
+            rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, h, nullptr, pend, c->attn_norm[l], d.rms_eps, a);
             pend = none;
             count_launches(1);
         }
         const float* bias = d.qkv_bias ? c->bqkv[l] : nullptr;
         Partials qkv_parts{qkv, 1, (size_t)M * c->n_qkv(), c->n_qkv()};
         if constexpr (kF32) {
-            launch_gemm_simt<T>(st, a, reinterpret_cast<const T*>(c->wqkv[l]), M, c->n_qkv(), d.d_model,
+            launch_gemm_simt<T>(st, sd, a, reinterpret_cast<const T*>(c->wqkv[l]), M, c->n_qkv(), d.d_model,
                                 EpiStoreF32{qkv, c->n_qkv(), nullptr});
         } else {
             const GemmPlan gp = plan_gemm(c, c->m_wqkv[l], M, true);
             qkv_parts.n = gp.splits;
-            if (int rc = gemm_bf16(c, st, c->map_a, c->m_wqkv[l], M, gp, tc::EpiPartial{qkv, c->n_qkv(), qkv_parts.stride})) return rc;
+            if (int rc = gemm_bf16(c, st, sd, c->map_a, c->m_wqkv[l], M, gp, tc::EpiPartial{qkv, c->n_qkv(), qkv_parts.stride})) return rc;
         }
         qkv_post_kernel<T><<<dim3(M, d.n_q_heads + 2 * d.n_kv_heads), half, 0, st>>>(
-            d.n_q_heads, d.n_kv_heads, d.head_dim, l, qkv_parts, bias, d.qk_norm ? c->q_norm[l] : nullptr,
+            sd, d.n_q_heads, d.n_kv_heads, d.head_dim, l, qkv_parts, bias, d.qk_norm ? c->q_norm[l] : nullptr,
             d.qk_norm ? c->k_norm[l] : nullptr, d.rms_eps, rope, g, prompt_arena, suffix_arena, q);
         count_launches(2);
         if constexpr (kF32) {
             if (l == prof_layer) cudaEventRecord(c->prof_start, st);
             if (d.head_dim == 128)
-                attn_row_simt_kernel<T, 128><<<dim3(M, d.n_kv_heads), 128, 0, st>>>(d.n_q_heads, d.n_kv_heads, l, q, g,
+                attn_row_simt_kernel<T, 128><<<dim3(M, d.n_kv_heads), 128, 0, st>>>(sd, d.n_q_heads, d.n_kv_heads, l, q, g,
                                                                                    prompt_arena, suffix_arena, scale, attn);
             else
-                attn_row_simt_kernel<T, 64><<<dim3(M, d.n_kv_heads), 128, 0, st>>>(d.n_q_heads, d.n_kv_heads, l, q, g,
+                attn_row_simt_kernel<T, 64><<<dim3(M, d.n_kv_heads), 128, 0, st>>>(sd, d.n_q_heads, d.n_kv_heads, l, q, g,
                                                                                   prompt_arena, suffix_arena, scale, attn);
             if (l == prof_layer) cudaEventRecord(c->prof_stop, st);
             count_launches(1);
-            launch_gemm_simt<T>(st, attn, reinterpret_cast<const T*>(c->wo[l]), M, d.d_model, c->q_dim(), EpiResidual{h, d.d_model});
+            launch_gemm_simt<T>(st, sd, attn, reinterpret_cast<const T*>(c->wo[l]), M, d.d_model, c->q_dim(), EpiResidual{h, d.d_model});
         } else {
             int rc = d.head_dim == 128
-                         ? attention_bf16<128>(c, st, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer)
-                         : attention_bf16<64>(c, st, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer);
+                         ? attention_bf16<128>(c, st, sd, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer)
+                         : attention_bf16<64>(c, st, sd, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer);
             if (rc) return rc;
             const GemmPlan gp = plan_gemm(c, c->m_wo[l], M, true);
             if (gp.splits == 1) {
-                if (int rc2 = gemm_bf16(c, st, c->map_attn, c->m_wo[l], M, gp, tc::EpiResidual{h, d.d_model})) return rc2;
+                if (int rc2 = gemm_bf16(c, st, sd, c->map_attn, c->m_wo[l], M, gp, tc::EpiResidual{h, d.d_model})) return rc2;
             } else {
                 pend = Partials{res_part, gp.splits, (size_t)M * d.d_model, d.d_model};
-                if (int rc2 = gemm_bf16(c, st, c->map_attn, c->m_wo[l], M, gp, tc::EpiPartial{res_part, d.d_model, pend.stride})) return rc2;
+                if (int rc2 = gemm_bf16(c, st, sd, c->map_attn, c->m_wo[l], M, gp, tc::EpiPartial{res_part, d.d_model, pend.stride})) return rc2;
             }
         }
-        rmsnorm_kernel<T><<<M, 256, 0, st>>>(d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a);
+        rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a);
         pend = none;
         count_launches(2);
         if constexpr (kF32) {
-            launch_gemm_simt<T>(st, a, reinterpret_cast<const T*>(c->w_gate_up[l]), M, 2 * d.d_ff, d.d_model,
+            launch_gemm_simt<T>(st, sd, a, reinterpret_cast<const T*>(c->w_gate_up[l]), M, 2 * d.d_ff, d.d_model,
                                 EpiSwiGLU<T>{act, d.d_ff});
-            launch_gemm_simt<T>(st, act, reinterpret_cast<const T*>(c->w_down[l]), M, d.d_model, d.d_ff, EpiResidual{h, d.d_model});
+            launch_gemm_simt<T>(st, sd, act, reinterpret_cast<const T*>(c->w_down[l]), M, d.d_model, d.d_ff, EpiResidual{h, d.d_model});
         } else {
-            if (int rc = gemm_bf16(c, st, c->map_a, c->m_wgu[l], M, plan_gemm(c, c->m_wgu[l], M, false), tc::EpiSwiGLU{act, d.d_ff}))
+            if (int rc = gemm_bf16(c, st, sd, c->map_a, c->m_wgu[l], M, plan_gemm(c, c->m_wgu[l], M, false), tc::EpiSwiGLU{act, d.d_ff}))
                 return rc;
             const GemmPlan gp = plan_gemm(c, c->m_wdown[l], M, true);
             if (gp.splits == 1) {
-                if (int rc = gemm_bf16(c, st, c->map_act, c->m_wdown[l], M, gp, tc::EpiResidual{h, d.d_model})) return rc;
+                if (int rc = gemm_bf16(c, st, sd, c->map_act, c->m_wdown[l], M, gp, tc::EpiResidual{h, d.d_model})) return rc;
             } else {
                 pend = Partials{res_part, gp.splits, (size_t)M * d.d_model, d.d_model};
-                if (int rc = gemm_bf16(c, st, c->map_act, c->m_wdown[l], M, gp, tc::EpiPartial{res_part, d.d_model, pend.stride})) return rc;
+                if (int rc = gemm_bf16(c, st, sd, c->map_act, c->m_wdown[l], M, gp, tc::EpiPartial{res_part, d.d_model, pend.stride})) return rc;
             }
         }
         count_launches(2);
@@ -348,18 +390,18 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, pc::KvArena prompt_arena, pc::
 
 // logits[n, V] = RMSNorm(h[src[r]]; final_norm) * W_lm^T
 template <typename T>
-int run_lm_head(pc_ctx* c, cudaStream_t st, int n, const int32_t* src, float* logits) {
+int run_lm_head(pc_ctx* c, cudaStream_t st, int n, const pc::StepDesc* sd, const int32_t* src, float* logits) {
     using namespace pc;
     const pc_model_desc& d = c->d;
     float* h = reinterpret_cast<float*>(c->ws + c->cv.h);
     T* a = reinterpret_cast<T*>(c->ws + c->cv.a);
-    rmsnorm_kernel<T><<<n, 256, 0, st>>>(d.d_model, h, src, c->pend, c->final_norm, d.rms_eps, a);
+    rmsnorm_kernel<T><<<n, 256, 0, st>>>(sd, d.d_model, h, src, c->pend, c->final_norm, d.rms_eps, a);
     c->pend = pc::Partials{nullptr, 0, 0, 0};
     if constexpr (std::is_same<T, float>::value) {
         const T* wlm = reinterpret_cast<const T*>(d.tied_embed ? c->embed : c->lm_head);
-        launch_gemm_simt<T>(st, a, wlm, n, d.vocab, d.d_model, EpiStoreF32{logits, d.vocab, nullptr});
+        launch_gemm_simt<T>(st, sd, a, wlm, n, d.vocab, d.d_model, EpiStoreF32{logits, d.vocab, nullptr});
     } else {
-        if (int rc = gemm_bf16(c, st, c->map_a, c->m_lm, n, plan_gemm(c, c->m_lm, n, false), tc::EpiStoreF32{logits, d.vocab, nullptr}))
+        if (int rc = gemm_bf16(c, st, sd, c->map_a, c->m_lm, n, plan_gemm(c, c->m_lm, n, false), tc::EpiStoreF32{logits, d.vocab, nullptr}))
             return rc;
     }
     count_launches(2);
@@ -494,7 +536,10 @@ int pc_set_workspace(pc_ctx* ctx, void* dev_ws, size_t bytes, int max_rows, int 
     ctx->max_prefill = max_prefill_tokens;
     ctx->err = dev_error_flag;
     ctx->cv = cv;
+    ctx->drop_graphs();
     if (ctx->d.dtype == PC_DTYPE_BF16) {
+        cudaError_t ce = configure_kernels();
+        if (ce != cudaSuccess) { ctx->ws = nullptr; return cuda_fail(ce, "kernel attributes"); }
         const uint64_t cap = (uint64_t)std::max(std::max(max_rows, max_prefill_tokens), 1);
         char* w = ctx->ws;
         if (!pc::make_bf16_map(&ctx->map_a, w + cv.a, cap, ctx->d.d_model, 128) ||
@@ -522,23 +567,84 @@ int pc_prefill_shared(pc_ctx* ctx, void* stream, int n_prompts, const int32_t* p
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const pc::RowGeom g = geom(ctx);
     int32_t* last_row = reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.last_row);
+    pc::StepDesc* sd = reinterpret_cast<pc::StepDesc*>(ctx->ws + ctx->cv.step_desc);
+    pc::set_step_desc<<<1, 1, 0, st>>>(sd, total_tokens, n_prompts, max_prompt_len);
     pc::prep_prefill_rows<<<n_prompts, 256, 0, st>>>(n_prompts, prompt_tokens, prompt_offsets, prompt_kv_start, prompt_slots,
                                                      ctx->d.vocab, g, last_row, ctx->err);
-    count_launches(1);
+    count_launches(2);
     PC_CUDA_CHECK_LAUNCH("prep_prefill_rows");
     const pc::KvArena pa{prompt_kv, prompt_slots}, sa{prompt_kv, prompt_slots};
     const AttnPlan plan{true, n_prompts, prompt_offsets, max_prompt_len};
     int rc = PC_OK;
     if (ctx->d.dtype == PC_DTYPE_F32) {
-        rc = run_layers<float>(ctx, st, total_tokens, pa, sa, plan);
+        rc = run_layers<float>(ctx, st, total_tokens, sd, pa, sa, plan);
     } else {
         rc = arena_maps(ctx, prompt_kv, prompt_slots, nullptr, 0);
-        if (rc == PC_OK) rc = run_layers<__nv_bfloat16>(ctx, st, total_tokens, pa, sa, plan);
+        if (rc == PC_OK) rc = run_layers<__nv_bfloat16>(ctx, st, total_tokens, sd, pa, sa, plan);
     }
     if (rc) return rc;
-    return ctx->d.dtype == PC_DTYPE_F32 ? run_lm_head<float>(ctx, st, n_prompts, last_row, last_logits)
-                                        : run_lm_head<__nv_bfloat16>(ctx, st, n_prompts, last_row, last_logits);
+    // only the last position of every prompt goes through the LM head: its row count is known on the host
+    return ctx->d.dtype == PC_DTYPE_F32 ? run_lm_head<float>(ctx, st, n_prompts, nullptr, last_row, last_logits)
+                                        : run_lm_head<__nv_bfloat16>(ctx, st, n_prompts, nullptr, last_row, last_logits);
 }
+
+}  // extern "C"
+
+namespace {
+
+// Everything a decode step needs besides the step descriptor; constant over a stage.
+struct DecodeArgs {
+    const int32_t* row_prompt; const int32_t* row_rollout; const int32_t* row_step; const int64_t* row_kv_start;
+    int32_t* tokens; const int64_t* row_tok_index; const int32_t* group_row_start; const int32_t* prompt_len;
+    const void* prompt_kv; int64_t prompt_slots; const int64_t* prompt_kv_start; void* suffix_kv; int64_t suffix_slots;
+    float temperature; uint64_t seed; int sample;
+};
+static_assert(sizeof(DecodeArgs) <= sizeof(GraphKey::args), "graph key too small for the decode arguments");
+
+int check_decode_args(const pc_ctx* ctx, const DecodeArgs& a) {
+    if (a.row_prompt == nullptr || a.row_rollout == nullptr || a.row_step == nullptr || a.row_kv_start == nullptr ||
+        a.tokens == nullptr || a.row_tok_index == nullptr || a.group_row_start == nullptr || a.prompt_len == nullptr ||
+        a.prompt_kv == nullptr || a.prompt_kv_start == nullptr || a.suffix_kv == nullptr)
+        return PC_ERR_INVALID_ARG;
+    if (a.prompt_slots < 0 || a.suffix_slots < 0) return PC_ERR_INVALID_ARG;
+    if (a.sample && !(a.temperature > 0.f)) return PC_ERR_INVALID_ARG;
+    if (!aligned(a.prompt_kv, 16) || !aligned(a.suffix_kv, 16)) return PC_ERR_ALIGNMENT;
+    (void)ctx;
+    return PC_OK;
+}
+
+// The kernels of one decode step.  Grids and GEMM plans are sized for (m_bound rows, groups_bound groups of at most
+// group_rows_bound rows); the live counts and the offsets into the caller's row arrays are in the step descriptor.
+int decode_launches(pc_ctx* ctx, cudaStream_t st, int m_bound, int groups_bound, int group_rows_bound, const DecodeArgs& a,
+                    float* logits_out) {
+    const pc::RowGeom g = geom(ctx);
+    const pc::StepDesc* sd = reinterpret_cast<const pc::StepDesc*>(ctx->ws + ctx->cv.step_desc);
+    pc::prep_decode_rows<<<(m_bound + 127) / 128, 128, 0, st>>>(sd, a.row_prompt, a.row_step, a.row_kv_start, a.tokens,
+                                                                a.row_tok_index, a.prompt_len, a.prompt_kv_start, a.prompt_slots,
+                                                                a.suffix_slots, ctx->d.vocab, g, ctx->err);
+    count_launches(1);
+    PC_CUDA_CHECK_LAUNCH("prep_decode_rows");
+    const pc::KvArena pa{const_cast<void*>(a.prompt_kv), a.prompt_slots}, sa{a.suffix_kv, a.suffix_slots};
+    const bool f32 = ctx->d.dtype == PC_DTYPE_F32;
+    const AttnPlan plan{false, groups_bound, a.group_row_start, group_rows_bound};
+    int rc = f32 ? run_layers<float>(ctx, st, m_bound, sd, pa, sa, plan) : run_layers<__nv_bfloat16>(ctx, st, m_bound, sd, pa, sa, plan);
+    if (rc) return rc;
+    float* logits = logits_out ? logits_out : reinterpret_cast<float*>(ctx->ws + ctx->cv.logits);
+    rc = f32 ? run_lm_head<float>(ctx, st, m_bound, sd, nullptr, logits) : run_lm_head<__nv_bfloat16>(ctx, st, m_bound, sd, nullptr, logits);
+    if (rc) return rc;
+    if (a.sample) {
+        pc::sample_kernel<<<m_bound, 256, 0, st>>>(sd, ctx->d.vocab, logits, nullptr, a.temperature, (uint32_t)(a.seed & 0xffffffffu),
+                                                   (uint32_t)(a.seed >> 32), a.row_prompt, a.row_rollout, a.row_step, 1, a.tokens,
+                                                   a.row_tok_index, 1, nullptr);
+        count_launches(1);
+        PC_CUDA_CHECK_LAUNCH("sample");
+    }
+    return PC_OK;
+}
+
+}  // namespace
+
+extern "C" {
 
 int pc_decode_step(pc_ctx* ctx, void* stream, int n_rows, const int32_t* row_prompt, const int32_t* row_rollout,
                    const int32_t* row_step, const int64_t* row_kv_start, int32_t* tokens, const int64_t* row_tok_index,
@@ -546,44 +652,92 @@ int pc_decode_step(pc_ctx* ctx, void* stream, int n_rows, const int32_t* row_pro
                    const void* prompt_kv, int64_t prompt_slots, const int64_t* prompt_kv_start, void* suffix_kv,
                    int64_t suffix_slots, float* logits_out, const pc_sample_params* sample) {
     if (int rc = check_ready(ctx)) return rc;
-    if (n_rows < 0 || n_groups < 0 || max_group_rows < 0 || prompt_slots < 0 || suffix_slots < 0) return PC_ERR_INVALID_ARG;
+    if (n_rows < 0 || n_groups < 0 || max_group_rows < 0) return PC_ERR_INVALID_ARG;
     if (n_rows == 0) return PC_OK;
-    if (row_prompt == nullptr || row_rollout == nullptr || row_step == nullptr || row_kv_start == nullptr || tokens == nullptr ||
-        row_tok_index == nullptr || group_row_start == nullptr || prompt_len == nullptr || prompt_kv == nullptr ||
-        prompt_kv_start == nullptr || suffix_kv == nullptr)
-        return PC_ERR_INVALID_ARG;
+    const DecodeArgs a{row_prompt, row_rollout, row_step, row_kv_start, tokens, row_tok_index, group_row_start, prompt_len,
+                       prompt_kv, prompt_slots, prompt_kv_start, suffix_kv, suffix_slots,
+                       sample ? sample->temperature : 1.f, sample ? sample->seed : 0, sample != nullptr};
+    if (int rc = check_decode_args(ctx, a)) return rc;
     if (n_groups == 0 || max_group_rows == 0 || max_group_rows > n_rows || n_groups > n_rows) return PC_ERR_INVALID_ARG;
     if (logits_out == nullptr && sample == nullptr) return PC_ERR_INVALID_ARG;
-    if (sample != nullptr && !(sample->temperature > 0.f)) return PC_ERR_INVALID_ARG;
-    if (!aligned(prompt_kv, 16) || !aligned(suffix_kv, 16) || (logits_out && !aligned(logits_out, 16))) return PC_ERR_ALIGNMENT;
+    if (logits_out && !aligned(logits_out, 16)) return PC_ERR_ALIGNMENT;
     if (n_rows > ctx->max_rows) return PC_ERR_CAPACITY;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const pc::RowGeom g = geom(ctx);
-    pc::prep_decode_rows<<<(n_rows + 127) / 128, 128, 0, st>>>(n_rows, row_prompt, row_step, row_kv_start, tokens, row_tok_index,
-                                                               prompt_len, prompt_kv_start, prompt_slots, suffix_slots,
-                                                               ctx->d.vocab, g, ctx->err);
+    if (ctx->d.dtype == PC_DTYPE_BF16)
+        if (int rc = arena_maps(ctx, prompt_kv, prompt_slots, suffix_kv, suffix_slots)) return rc;
+    pc::set_step_desc<<<1, 1, 0, st>>>(reinterpret_cast<pc::StepDesc*>(ctx->ws + ctx->cv.step_desc), n_rows, n_groups, max_group_rows);
     count_launches(1);
-    PC_CUDA_CHECK_LAUNCH("prep_decode_rows");
-    const pc::KvArena pa{const_cast<void*>(prompt_kv), prompt_slots}, sa{suffix_kv, suffix_slots};
-    const bool f32 = ctx->d.dtype == PC_DTYPE_F32;
-    const AttnPlan plan{false, n_groups, group_row_start, max_group_rows};
-    int rc = PC_OK;
-    if (f32) {
-        rc = run_layers<float>(ctx, st, n_rows, pa, sa, plan);
-    } else {
-        rc = arena_maps(ctx, prompt_kv, prompt_slots, suffix_kv, suffix_slots);
-        if (rc == PC_OK) rc = run_layers<__nv_bfloat16>(ctx, st, n_rows, pa, sa, plan);
+    return decode_launches(ctx, st, n_rows, n_groups, max_group_rows, a, logits_out);
+}
+
+int pc_decode_run(pc_ctx* ctx, void* stream, int n_steps, const pc_step_desc* steps_host, const pc_step_desc* steps_dev,
+                  const int32_t* row_prompt, const int32_t* row_rollout, const int32_t* row_step, const int64_t* row_kv_start,
+                  int32_t* tokens, const int64_t* row_tok_index, const int32_t* group_row_start, const int32_t* prompt_len,
+                  const void* prompt_kv, int64_t prompt_slots, const int64_t* prompt_kv_start, void* suffix_kv,
+                  int64_t suffix_slots, const pc_sample_params* sample) {
+    static_assert(sizeof(pc_step_desc) == sizeof(pc::StepDesc), "the public and the device step descriptor must agree");
+    if (int rc = check_ready(ctx)) return rc;
+    if (n_steps < 0) return PC_ERR_INVALID_ARG;
+    if (n_steps == 0) return PC_OK;
+    if (steps_host == nullptr || steps_dev == nullptr || sample == nullptr) return PC_ERR_INVALID_ARG;
+    const DecodeArgs a{row_prompt, row_rollout, row_step, row_kv_start, tokens, row_tok_index, group_row_start, prompt_len,
+                       prompt_kv, prompt_slots, prompt_kv_start, suffix_kv, suffix_slots, sample->temperature, sample->seed, 1};
+    if (int rc = check_decode_args(ctx, a)) return rc;
+    int groups_bound = 0, group_rows_bound = 0;
+    for (int s = 0; s < n_steps; ++s) {
+        const pc_step_desc& d = steps_host[s];
+        if (d.n_rows < 0 || d.n_rows > ctx->max_rows || d.n_groups < 0 || d.n_groups > d.n_rows || d.max_group_rows < 0 ||
+            d.max_group_rows > d.n_rows || d.row_offset < 0 || d.group_offset < 0 || (d.n_rows > 0 && (d.n_groups == 0 || d.max_group_rows == 0)))
+            return d.n_rows > ctx->max_rows ? PC_ERR_CAPACITY : PC_ERR_INVALID_ARG;
+        groups_bound = std::max(groups_bound, d.n_groups);
+        group_rows_bound = std::max(group_rows_bound, d.max_group_rows);
     }
-    if (rc) return rc;
-    float* logits = logits_out ? logits_out : reinterpret_cast<float*>(ctx->ws + ctx->cv.logits);
-    rc = f32 ? run_lm_head<float>(ctx, st, n_rows, nullptr, logits) : run_lm_head<__nv_bfloat16>(ctx, st, n_rows, nullptr, logits);
-    if (rc) return rc;
-    if (sample != nullptr) {
-        pc::sample_kernel<<<n_rows, 256, 0, st>>>(ctx->d.vocab, logits, nullptr, sample->temperature,
-                                                  (uint32_t)(sample->seed & 0xffffffffu), (uint32_t)(sample->seed >> 32), row_prompt,
-                                                  row_rollout, row_step, 1, tokens, row_tok_index, 1, nullptr);
-        count_launches(1);
-        PC_CUDA_CHECK_LAUNCH("sample");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (ctx->d.dtype == PC_DTYPE_BF16)
+        if (int rc = arena_maps(ctx, prompt_kv, prompt_slots, suffix_kv, suffix_slots)) return rc;
+    int32_t* counter = reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.step_counter);
+    pc::StepDesc* sd = reinterpret_cast<pc::StepDesc*>(ctx->ws + ctx->cv.step_desc);
+    cudaError_t e = cudaMemsetAsync(counter, 0, sizeof(int32_t), st);
+    if (e != cudaSuccess) return cuda_fail(e, "reset step counter");
+    for (int s = 0; s < n_steps; ++s) {
+        if (steps_host[s].n_rows == 0) {          // keep the device counter in step with the host loop
+            pc::load_step_desc<<<1, 1, 0, st>>>(reinterpret_cast<const pc::StepDesc*>(steps_dev), counter, sd);
+            count_launches(1);
+            continue;
+        }
+        const int m_bound = std::min(ctx->max_rows, (steps_host[s].n_rows + 127) / 128 * 128);
+        GraphKey key{};
+        std::memset(&key, 0, sizeof(key));
+        key.m_bound = m_bound; key.groups_bound = groups_bound; key.group_rows_bound = group_rows_bound;
+        key.steps_dev = steps_dev;
+        std::memcpy(key.args, &a, sizeof(a));
+        cudaGraphExec_t exec = nullptr;
+        for (auto& ent : ctx->graphs)
+            if (std::memcmp(&ent.key, &key, sizeof(key)) == 0) { exec = ent.exec; break; }
+        if (exec == nullptr) {
+            if (ctx->graphs.size() >= 64) ctx->drop_graphs();
+            const unsigned long long launches_before = g_launches;
+            cudaGraph_t graph = nullptr;
+            e = cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal);
+            if (e != cudaSuccess) return cuda_fail(e, "begin graph capture");
+            pc::load_step_desc<<<1, 1, 0, st>>>(reinterpret_cast<const pc::StepDesc*>(steps_dev), counter, sd);
+            count_launches(1);
+            const int rc = decode_launches(ctx, st, m_bound, groups_bound, group_rows_bound, a, nullptr);
+            e = cudaStreamEndCapture(st, &graph);
+            if (rc != PC_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
+            if (e != cudaSuccess) return cuda_fail(e, "end graph capture");
+            e = cudaGraphInstantiate(&exec, graph, 0);
+            cudaGraphDestroy(graph);
+            if (e != cudaSuccess) return cuda_fail(e, "graph instantiate");
+            GraphEntry ent;
+            ent.key = key; ent.exec = exec; ent.launches = (int)(g_launches - launches_before);
+            g_launches = launches_before;         // capturing launched nothing
+            ctx->graphs.push_back(ent);
+        }
+        e = cudaGraphLaunch(exec, st);
+        if (e != cudaSuccess) return cuda_fail(e, "graph launch");
+        for (auto& ent : ctx->graphs)
+            if (ent.exec == exec) { count_launches(ent.launches); break; }
     }
     return PC_OK;
 }
@@ -596,7 +750,7 @@ int pc_sample(void* stream, int n_rows, int vocab, const float* logits, const in
     if (logits == nullptr || row_prompt == nullptr || row_rollout == nullptr || row_step == nullptr || out_tokens == nullptr)
         return PC_ERR_INVALID_ARG;
     pc::sample_kernel<<<n_rows, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        vocab, logits, logits_row, temperature, (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32), row_prompt, row_rollout,
+        nullptr, vocab, logits, logits_row, temperature, (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32), row_prompt, row_rollout,
         row_step, 0, out_tokens, out_index, 0, out_top2_gap);
     count_launches(1);
     PC_CUDA_CHECK_LAUNCH("sample");

@@ -61,7 +61,7 @@ __device__ __forceinline__ Top2 top2_warp_reduce(Top2 t) {
 }
 
 // One block per row.
-__global__ void __launch_bounds__(256) sample_kernel(int vocab, const float* __restrict__ logits,
+__global__ void __launch_bounds__(256) sample_kernel(const StepDesc* __restrict__ sd, int vocab, const float* __restrict__ logits,
                                                      const int32_t* __restrict__ logits_row, float temperature,
                                                      uint32_t k0, uint32_t k1, const int32_t* __restrict__ row_prompt,
                                                      const int32_t* __restrict__ row_rollout, const int32_t* __restrict__ row_step,
@@ -69,8 +69,13 @@ __global__ void __launch_bounds__(256) sample_kernel(int vocab, const float* __r
                                                      const int64_t* __restrict__ out_index, int64_t out_index_offset,
                                                      float* __restrict__ out_gap) {
     const int r = blockIdx.x;
-    const float* lg = logits + (size_t)(logits_row ? logits_row[r] : r) * vocab;
-    const uint32_t c1 = (uint32_t)(row_step[r] + step_offset), c2 = (uint32_t)row_rollout[r], c3 = (uint32_t)row_prompt[r];
+    int64_t ro = r;                         // index into the caller's row arrays
+    if (sd != nullptr) {
+        if (r >= sd->n_rows) return;
+        ro += sd->row_off;
+    }
+    const float* lg = logits + (size_t)(logits_row ? logits_row[ro] : r) * vocab;
+    const uint32_t c1 = (uint32_t)(row_step[ro] + step_offset), c2 = (uint32_t)row_rollout[ro], c3 = (uint32_t)row_prompt[ro];
     Top2 t{-INFINITY, -INFINITY, 0x7fffffff};
     const int n_blocks = (vocab + 3) >> 2;
     for (int b = threadIdx.x; b < n_blocks; b += blockDim.x) {
@@ -91,7 +96,7 @@ __global__ void __launch_bounds__(256) sample_kernel(int vocab, const float* __r
         Top2 u = lane < (int)(blockDim.x >> 5) ? sh[lane] : Top2{-INFINITY, -INFINITY, 0x7fffffff};
         u = top2_warp_reduce(u);
         if (lane == 0) {
-            out_tokens[out_index ? out_index[r] + out_index_offset : (int64_t)r] = u.idx;
+            out_tokens[out_index ? out_index[ro] + out_index_offset : (int64_t)r] = u.idx;
             if (out_gap) out_gap[r] = u.best - u.second;
         }
     }

@@ -35,6 +35,10 @@ def _dev_matrix(w: Weights, names: List[str], model: ModelShape, device, interle
     return t.view(torch.bfloat16) if model.dtype == DTYPE_BF16 else t
 
 
+STEP_DESC_DTYPE = np.dtype([("n_rows", np.int32), ("n_groups", np.int32), ("max_group_rows", np.int32), ("reserved", np.int32),
+                            ("row_offset", np.int64), ("group_offset", np.int64)])
+
+
 @dataclasses.dataclass
 class StageSchedule:
     """Which rollouts are live at every decode step of one stage, flattened over steps and uploaded once."""
@@ -51,6 +55,8 @@ class StageSchedule:
     row_tok_index: torch.Tensor
     group_row_start: torch.Tensor
     total_rows: int
+    steps_host: np.ndarray            # [n_steps] records laid out like the C pc_step_desc
+    steps_dev: torch.Tensor           # the same bytes on the device
 
 
 class RolloutEngine:
@@ -87,6 +93,7 @@ class RolloutEngine:
         # measurement: every `profile_every`-th decode step, time the suffix-attention kernel of one layer
         self._arenas: Dict[str, Optional[torch.Tensor]] = {}
         self.profile_every = 0
+        self.use_graphs = True
         self.profile_layer = m.n_layers // 2
         self.profile_samples: List[tuple] = []      # (start event, stop event, rows, suffix slots read per row)
 
@@ -184,9 +191,13 @@ class RolloutEngine:
         cat = lambda xs, dt: torch.from_numpy(np.concatenate(xs).astype(dt) if xs else np.zeros(0, dt)).to(dev)
         row_off = np.r_[0, np.cumsum(rows_per_step)[:-1]] if n_steps else np.zeros(0, np.int64)
         group_off = np.r_[0, np.cumsum(groups_per_step + 1)[:-1]] if n_steps else np.zeros(0, np.int64)
+        steps = np.zeros(n_steps, dtype=STEP_DESC_DTYPE)
+        steps["n_rows"], steps["n_groups"], steps["max_group_rows"] = rows_per_step, groups_per_step, max_group
+        steps["row_offset"], steps["group_offset"] = row_off, group_off
+        steps_dev = torch.from_numpy(steps.view(np.uint8).reshape(-1).copy()).to(dev) if n_steps else torch.zeros(1, dtype=torch.uint8, device=dev)
         return StageSchedule(n_steps, rows_per_step, row_off, groups_per_step, group_off, max_group,
                              cat(rp, np.int32), cat(rr, np.int32), cat(rs, np.int32), cat(rk, np.int64), cat(rt, np.int64),
-                             cat(gs, np.int32), int(rows_per_step.sum()))
+                             cat(gs, np.int32), int(rows_per_step.sum()), steps, steps_dev)
 
     def run_stage(self, prompts: np.ndarray, rollouts: np.ndarray, record_logits: Optional[dict] = None,
                   teacher_forced: bool = False, step_range: Optional[tuple] = None) -> int:
@@ -214,13 +225,14 @@ class RolloutEngine:
         pr, rr, rs = sch.row_prompt.data_ptr(), sch.row_rollout.data_ptr(), sch.row_step.data_ptr()
         rk, rt, gs = sch.row_kv_start.data_ptr(), sch.row_tok_index.data_ptr(), sch.group_row_start.data_ptr()
         first, last = (0, sch.n_steps) if step_range is None else (step_range[0], min(step_range[1], sch.n_steps))
-        for s in range(first, last):
+
+        def eager(s):
             nr, o, go = int(sch.rows_per_step[s]), int(sch.row_off[s]), int(sch.group_off[s])
             logits_out = None
             if record_logits is not None and s in record_logits:
                 logits_out = torch.empty((nr, self.model.vocab), dtype=torch.float32, device=dev)
                 record_logits[s] = (logits_out, sch.row_prompt[o:o + nr].cpu().numpy(), sch.row_rollout[o:o + nr].cpu().numpy())
-            if self.profile_every and s % self.profile_every == self.profile_every // 2:
+            if profiled(s):
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(); e1.record()             # creates the underlying CUDA events
                 B.pc_profile_attention(self.ctx, self.profile_layer, e0, e1)
@@ -229,6 +241,28 @@ class RolloutEngine:
                              int(sch.groups_per_step[s]), gs + 4 * go, int(sch.max_group_rows[s]), self.prompt_len,
                              self.prompt_kv, self.total_prompt_tokens, self.prompt_kv_start, self.suffix_kv,
                              self.suffix_slots, logits_out, None if teacher_forced else sp)
+
+        def profiled(s):
+            return bool(self.profile_every) and s % self.profile_every == self.profile_every // 2
+
+        def needs_eager(s):
+            return teacher_forced or not self.use_graphs or (record_logits is not None and s in record_logits) or profiled(s)
+
+        s = first
+        while s < last:
+            if needs_eager(s):
+                eager(s)
+                s += 1
+                continue
+            e = s
+            while e < last and not needs_eager(e):
+                e += 1
+            # steps s .. e-1 natively: one graph launch per step, issued by the library
+            item = STEP_DESC_DTYPE.itemsize
+            B.pc_decode_run(self.ctx, e - s, sch.steps_host.ctypes.data + s * item, sch.steps_dev.data_ptr() + s * item,
+                            pr, rr, rs, rk, self.tokens, rt, gs, self.prompt_len, self.prompt_kv, self.total_prompt_tokens,
+                            self.prompt_kv_start, self.suffix_kv, self.suffix_slots, sp)
+            s = e
         self._keep_schedule = sch
         return int(self.batch.caps[prompts, rollouts].sum())
 

@@ -129,3 +129,24 @@ def test_bf16_many_rows_long_prefix_long_suffix():
     eng = RolloutEngine(model, weights, max_rows=P * G, max_prefill_tokens=int(batch.prompt_offsets[-1]))
     worst, n_cmp, n_exempt = teacher_forced_compare(eng, w, batch, ref, prompts, rollouts, logit_tol=5e-2, gap_tol=1e-1)
     assert n_cmp == int(batch.caps.sum())
+
+
+@pytest.mark.parametrize("model", [wl.TINY, wl.SMALL_BF16], ids=lambda m: m.name)
+def test_graph_replay_equals_step_by_step(model):
+    """pc_decode_run (captured steps replayed from a device-resident schedule) against one pc_decode_step per step."""
+    w = dataclasses.replace(wl.WORKLOADS["config0"], model=model, n_prompts=5, prompt_len_lo=3, prompt_len_hi=50, group_size=9,
+                            n_pilot=3, max_new=40, cap_lo=1, cap_hi=40, data_seed=21,
+                            forced_explicit=((0, 0.5), (1, 0.5), (2, 0.5), (3, 0.0), (4, 0.5)))
+    weights = wl.gen_weights(model, seed=0, threads=2)
+    batch = wl.gen_batch(w)
+    eng = RolloutEngine(model, weights, max_rows=45, max_prefill_tokens=int(batch.prompt_offsets[-1]))
+    eng.use_graphs = False
+    a = eng.pilot_commit_step(w, batch)
+    eng.use_graphs = True
+    b = eng.pilot_commit_step(w, batch)
+    assert np.array_equal(a["status"], b["status"]) and np.any(a["status"] == ostats.COMMIT)
+    for p in range(w.n_prompts):
+        for i in range(w.group_size):
+            if a["generated"][p, i]:
+                assert np.array_equal(a["tokens"][p][i], b["tokens"][p][i])
+    assert np.array_equal(a["advantages"], b["advantages"])
