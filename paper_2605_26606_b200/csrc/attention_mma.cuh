@@ -68,11 +68,17 @@ __device__ __forceinline__ uint32_t tile_off(int r, int d) {
     return (uint32_t)((d >> 6) * (ROWS * 128) + r * 128 + ((((d & 63) >> 3) ^ (r & 7)) << 4));
 }
 
-struct PrefixPartial {      // per (row, query head): running max (log2 domain), sum, unnormalised output
-    float* m;               // [rows * Hq]
-    float* l;               // [rows * Hq]
-    float* o;               // [rows * Hq * head_dim]
+// Prefix part of the attention, per (row, query head): running max (log2 domain), sum, unnormalised output.
+// When a group has few query rows its prompt is cut into n_parts ranges handled by different CTAs; every range
+// leaves its own record and the suffix kernel merges all of them.
+struct PrefixPartial {
+    float* m;               // [n_parts][stride]
+    float* l;               // [n_parts][stride]
+    float* o;               // [n_parts][stride * head_dim]
+    int n_parts;
+    size_t stride;          // rows capacity * Hq
 };
+constexpr int MAX_PREFIX_PARTS = 8;
 
 // ---------------------------------------------------------------------------------------------
 // Group (shared-prefix / causal-prefill) kernel
@@ -97,7 +103,10 @@ attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __
     group_row_start += sd->group_off;
     const int row0 = group_row_start[grp], n_rows = group_row_start[grp + 1] - row0;
     const int n_rep = Hq / Hkv;
-    const int q0 = blockIdx.x * G_QROWS;
+    const int n_parts = FINAL ? 1 : part.n_parts;
+    const int q_tiles = gridDim.x / n_parts;
+    const int my_part = blockIdx.x / q_tiles;
+    const int q0 = (blockIdx.x - my_part * q_tiles) * G_QROWS;
     if (q0 >= n_rows * n_rep) return;
 
     extern __shared__ uint8_t smem_raw[];
@@ -151,7 +160,10 @@ attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __
     }
     __syncthreads();
     const int max_len = s_maxlen;
-    const int n_tiles = (max_len + G_TK - 1) / G_TK;
+    const int n_tiles_all = (max_len + G_TK - 1) / G_TK;
+    const int tiles_per_part = (n_tiles_all + n_parts - 1) / n_parts;
+    const int tile0 = my_part * tiles_per_part;                          // this CTA covers tiles [tile0, tile0 + n_tiles)
+    const int n_tiles = max(0, min(n_tiles_all, tile0 + tiles_per_part) - tile0);
     const int64_t kv_start = g.p_start[row0];
     const int64_t krow0 = (((int64_t)layer * 2 + 0) * Hkv + kvh) * n_slots + kv_start;
     const int64_t vrow0 = (((int64_t)layer * 2 + 1) * Hkv + kvh) * n_slots + kv_start;
@@ -166,7 +178,7 @@ attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __
         }
     };
     if (threadIdx.x == 0)
-        for (int t = 0; t < G_STAGES && t < n_tiles; ++t) issue(t, t);
+        for (int t = 0; t < G_STAGES && t < n_tiles; ++t) issue(tile0 + t, t);
 
     float o[DT][4];
 #pragma unroll
@@ -174,9 +186,10 @@ attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __
     float mrow[2] = {-INFINITY, -INFINITY}, lrow[2] = {0.f, 0.f};
     bool ok = true;
 
-    for (int tile = 0; tile < n_tiles; ++tile) {
-        const int stage = tile % G_STAGES;
-        const uint32_t phase = (uint32_t)(tile / G_STAGES) & 1u;
+    for (int lt = 0; lt < n_tiles; ++lt) {
+        const int tile = tile0 + lt;
+        const int stage = lt % G_STAGES;
+        const uint32_t phase = (uint32_t)(lt / G_STAGES) & 1u;
         if (!mbar_wait(full0 + 8 * stage, phase, &s_abort)) { ok = false; break; }
         const uint32_t kb = tiles_u32 + stage * 2 * TILE_BYTES, vb = kb + TILE_BYTES;
         // S = Q K^T for 64 positions
@@ -256,7 +269,7 @@ attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8 * stage);
-        if (threadIdx.x == 0 && tile + G_STAGES < n_tiles) {
+        if (threadIdx.x == 0 && lt + G_STAGES < n_tiles) {
             if (!mbar_wait(empty0 + 8 * stage, phase, &s_abort)) { ok = false; break; }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             issue(tile + G_STAGES, stage);
@@ -280,10 +293,13 @@ attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __
             for (int t = 0; t < DT; ++t)
                 *reinterpret_cast<uint32_t*>(out + rh * HD + t * 8 + (lane & 3) * 2) = pack_bf16(o[t][2 * i] * inv, o[t][2 * i + 1] * inv);
         } else {
-            if ((lane & 3) == 0) { part.m[rh] = mrow[i]; part.l[rh] = lrow[i]; }
+            const size_t ph = (size_t)my_part * part.stride + rh;
+            if ((lane & 3) == 0) { part.m[ph] = mrow[i]; part.l[ph] = lrow[i]; }
+            if (n_tiles > 0) {          // an empty range leaves (m, l) = (-inf, 0); its output is never read
 #pragma unroll
-            for (int t = 0; t < DT; ++t)
-                *reinterpret_cast<float2*>(part.o + rh * HD + t * 8 + (lane & 3) * 2) = make_float2(o[t][2 * i], o[t][2 * i + 1]);
+                for (int t = 0; t < DT; ++t)
+                    *reinterpret_cast<float2*>(part.o + ph * HD + t * 8 + (lane & 3) * 2) = make_float2(o[t][2 * i], o[t][2 * i + 1]);
+            }
         }
     }
     if (s_abort) {      // let copies still in flight land before the shared memory is released
@@ -500,17 +516,25 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
         for (int j = 0; j < n_rep; ++j) {
             const size_t rh = (size_t)row * Hq + (size_t)kvh * n_rep + j;
             const float ms = s_ml[warp][j], ls = s_ml[warp][8 + j];
-            const float mp = part.m[rh], lp = part.l[rh];
-            const float M = fmaxf(ms, mp);
-            const float ws = exp2_safe(ms, M), wp = exp2_safe(mp, M);
-            const float denom = ls * ws + lp * wp;
-            const float inv = denom > 0.f ? 1.f / denom : 0.f;
+            float M = ms;
+            for (int pp = 0; pp < part.n_parts; ++pp) M = fmaxf(M, part.m[(size_t)pp * part.stride + rh]);
+            const float ws = exp2_safe(ms, M);
+            float denom = ls * ws;
             float res[EPL];
 #pragma unroll
-            for (int e = 0; e < EPL; ++e) {
-                const float po = wp > 0.f ? part.o[rh * HD + lane * EPL + e] * wp : 0.f;
-                res[e] = (obuf[j * HD + lane * EPL + e] * ws + po) * inv;
+            for (int e = 0; e < EPL; ++e) res[e] = obuf[j * HD + lane * EPL + e] * ws;
+            for (int pp = 0; pp < part.n_parts; ++pp) {          // fixed order: the result does not depend on CTA timing
+                const size_t ph = (size_t)pp * part.stride + rh;
+                const float wp = exp2_safe(part.m[ph], M);
+                if (wp > 0.f) {
+                    denom += part.l[ph] * wp;
+#pragma unroll
+                    for (int e = 0; e < EPL; ++e) res[e] += part.o[ph * HD + lane * EPL + e] * wp;
+                }
             }
+            const float inv = denom > 0.f ? 1.f / denom : 0.f;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) res[e] *= inv;
             __nv_bfloat16* dst = out + rh * HD + lane * EPL;
             if (EPL == 4) {
                 *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(res[0], res[1]), pack_bf16(res[2], res[3]));

@@ -126,27 +126,54 @@ struct Partials {
 
 // Optional residual update followed by the norm:  h[row, :] += pending partial sums of row r;  a[r, :] = RMSNorm(h[row, :]; gain)
 // with row = src ? src[r] : r.  The partial sums are indexed by row, like h.
+template <typename T> __device__ __forceinline__ void store4(T* p, float4 v);
+template <> __device__ __forceinline__ void store4<float>(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16* p, float4 v) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+}
+
+// One block of 256 threads per row; d is a multiple of 8 and at most 8192, so a thread keeps its <= 8 float4 of the
+// row in registers between the sum of squares and the scaling (one pass over global memory).
 template <typename T>
-__global__ void rmsnorm_kernel(const StepDesc* __restrict__ sd, int d, float* __restrict__ h, const int32_t* __restrict__ src,
-                               Partials pend, const float* __restrict__ gain, float eps, T* __restrict__ a) {
+__global__ void __launch_bounds__(256) rmsnorm_kernel(const StepDesc* __restrict__ sd, int d, float* __restrict__ h,
+                                                      const int32_t* __restrict__ src, Partials pend, const float* __restrict__ gain,
+                                                      float eps, T* __restrict__ a) {
     __shared__ float red[33];
     const int r = blockIdx.x;
     if (sd != nullptr && r >= sd->n_rows) return;
     if (pend.n > 0 && sd != nullptr) pend.stride = (size_t)sd->n_rows * pend.ld;      // slices are packed by the live row count
     const int row = src ? src[r] : r;
-    float* x = h + (size_t)row * d;
+    float4* x = reinterpret_cast<float4*>(h + (size_t)row * d);
+    const int n4 = d >> 2;
+    float4 v[8];
     float ss = 0.f;
-    for (int i = threadIdx.x; i < d; i += blockDim.x) {
-        float v = x[i];
-        if (pend.n > 0) {
-            for (int s = 0; s < pend.n; ++s) v += pend.p[(size_t)s * pend.stride + (size_t)row * pend.ld + i];
-            x[i] = v;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int i = threadIdx.x + k * 256;
+        if (i < n4) {
+            v[k] = x[i];
+            if (pend.n > 0) {
+                for (int s = 0; s < pend.n; ++s) {
+                    const float4 p = *reinterpret_cast<const float4*>(pend.p + (size_t)s * pend.stride + (size_t)row * pend.ld + 4 * i);
+                    v[k].x += p.x; v[k].y += p.y; v[k].z += p.z; v[k].w += p.w;
+                }
+                x[i] = v[k];
+            }
+            ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
         }
-        ss += v * v;
     }
     ss = block_sum(ss, red);
     const float rstd = rsqrtf(ss / (float)d + eps);
-    for (int i = threadIdx.x; i < d; i += blockDim.x) a[(size_t)r * d + i] = from_f32<T>(x[i] * rstd * gain[i]);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int i = threadIdx.x + k * 256;
+        if (i < n4) {
+            const float4 gg = *reinterpret_cast<const float4*>(gain + 4 * i);
+            store4<T>(a + (size_t)r * d + 4 * i,
+                      make_float4(v[k].x * rstd * gg.x, v[k].y * rstd * gg.y, v[k].z * rstd * gg.z, v[k].w * rstd * gg.w));
+        }
+    }
 }
 
 struct KvArena {

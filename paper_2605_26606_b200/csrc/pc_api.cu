@@ -98,11 +98,15 @@ struct pc_ctx {
     cudaEvent_t prof_start = nullptr, prof_stop = nullptr;
 
     std::vector<GraphEntry> graphs;
+    cudaStream_t capture_stream = nullptr;      // decode steps are captured here (the caller's stream may be the default one)
     void drop_graphs() {
         for (auto& g : graphs) cudaGraphExecDestroy(g.exec);
         graphs.clear();
     }
-    ~pc_ctx() { drop_graphs(); }
+    ~pc_ctx() {
+        drop_graphs();
+        if (capture_stream) cudaStreamDestroy(capture_stream);
+    }
 
     int n_qkv() const { return (d.n_q_heads + 2 * d.n_kv_heads) * d.head_dim; }
     int q_dim() const { return d.n_q_heads * d.head_dim; }
@@ -140,9 +144,9 @@ Carve carve(const pc_ctx* c, int max_rows, int max_prefill) {
     v.last_row = take(M * 4);
     // prefix part of the shared-prefix attention: (max, sum, unnormalised output) per (row, query head)
     const size_t R = (size_t)std::max(max_rows, 1);
-    v.part_m = take(R * d.n_q_heads * 4);
-    v.part_l = take(R * d.n_q_heads * 4);
-    v.part_o = take(R * d.n_q_heads * d.head_dim * 4);
+    v.part_m = take(pc::am::MAX_PREFIX_PARTS * R * d.n_q_heads * 4);
+    v.part_l = take(pc::am::MAX_PREFIX_PARTS * R * d.n_q_heads * 4);
+    v.part_o = take(pc::am::MAX_PREFIX_PARTS * R * d.n_q_heads * d.head_dim * 4);
     v.total = off;
     return v;
 }
@@ -262,9 +266,13 @@ int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, in
     const RowGeom g = geom(c);
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)d.head_dim);
     const int n_rep = d.n_q_heads / d.n_kv_heads;
+    // a group with few query rows keeps few CTAs busy: cut its prompt into ranges so that about one CTA per SM runs
+    const int q_tiles = (plan.max_group_rows * n_rep + am::G_QROWS - 1) / am::G_QROWS;
+    const int base_ctas = std::max(1, q_tiles * d.n_kv_heads * plan.n_groups);
+    const int n_parts = plan.prefill ? 1 : std::max(1, std::min(am::MAX_PREFIX_PARTS, c->num_sms / base_ctas));
     am::PrefixPartial part{reinterpret_cast<float*>(c->ws + c->cv.part_m), reinterpret_cast<float*>(c->ws + c->cv.part_l),
-                           reinterpret_cast<float*>(c->ws + c->cv.part_o)};
-    const dim3 ggrid((plan.max_group_rows * n_rep + am::G_QROWS - 1) / am::G_QROWS, d.n_kv_heads, plan.n_groups);
+                           reinterpret_cast<float*>(c->ws + c->cv.part_o), n_parts, (size_t)std::max(c->max_rows, 1) * d.n_q_heads};
+    const dim3 ggrid(q_tiles * n_parts, d.n_kv_heads, plan.n_groups);
     if (plan.prefill) {
         am::attn_group_kernel<HD, true><<<ggrid, am::G_THREADS, am::group_smem_bytes<HD>(), st>>>(
             c->map_prompt_kv, sd, prompt_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, plan.group_row_start, g, scale_log2,
@@ -456,7 +464,7 @@ int pc_create(const pc_model_desc* desc, const pc_weights* wts, pc_ctx** out) {
         return PC_ERR_INVALID_ARG;
     if (d.head_dim != 64 && d.head_dim != 128) return PC_ERR_SHAPE;
     if (d.n_q_heads % d.n_kv_heads != 0 || d.n_q_heads / d.n_kv_heads > pc::ATTN_MAX_REP) return PC_ERR_SHAPE;
-    if (d.d_model % 8 != 0 || d.d_ff % 8 != 0) return PC_ERR_SHAPE;
+    if (d.d_model % 8 != 0 || d.d_ff % 8 != 0 || d.d_model > 8192) return PC_ERR_SHAPE;
     if (d.dtype == PC_DTYPE_BF16 && (d.d_model % 64 != 0 || d.d_ff % 64 != 0)) return PC_ERR_SHAPE;
     if (wts->embed == nullptr || wts->final_norm == nullptr || (!d.tied_embed && wts->lm_head == nullptr)) return PC_ERR_INVALID_ARG;
     if (wts->attn_norm == nullptr || wts->wqkv == nullptr || wts->wo == nullptr || wts->mlp_norm == nullptr ||
@@ -599,6 +607,22 @@ struct DecodeArgs {
     const void* prompt_kv; int64_t prompt_slots; const int64_t* prompt_kv_start; void* suffix_kv; int64_t suffix_slots;
     float temperature; uint64_t seed; int sample;
 };
+// Zero-filled first (padding included) so that two equal argument sets compare equal byte by byte.
+DecodeArgs make_decode_args(const int32_t* row_prompt, const int32_t* row_rollout, const int32_t* row_step, const int64_t* row_kv_start,
+                            int32_t* tokens, const int64_t* row_tok_index, const int32_t* group_row_start, const int32_t* prompt_len,
+                            const void* prompt_kv, int64_t prompt_slots, const int64_t* prompt_kv_start, void* suffix_kv,
+                            int64_t suffix_slots, const pc_sample_params* sample) {
+    DecodeArgs a;
+    std::memset(&a, 0, sizeof(a));
+    a.row_prompt = row_prompt; a.row_rollout = row_rollout; a.row_step = row_step; a.row_kv_start = row_kv_start;
+    a.tokens = tokens; a.row_tok_index = row_tok_index; a.group_row_start = group_row_start; a.prompt_len = prompt_len;
+    a.prompt_kv = prompt_kv; a.prompt_slots = prompt_slots; a.prompt_kv_start = prompt_kv_start; a.suffix_kv = suffix_kv;
+    a.suffix_slots = suffix_slots;
+    a.temperature = sample ? sample->temperature : 1.f;
+    a.seed = sample ? sample->seed : 0;
+    a.sample = sample != nullptr;
+    return a;
+}
 static_assert(sizeof(DecodeArgs) <= sizeof(GraphKey::args), "graph key too small for the decode arguments");
 
 int check_decode_args(const pc_ctx* ctx, const DecodeArgs& a) {
@@ -654,9 +678,8 @@ int pc_decode_step(pc_ctx* ctx, void* stream, int n_rows, const int32_t* row_pro
     if (int rc = check_ready(ctx)) return rc;
     if (n_rows < 0 || n_groups < 0 || max_group_rows < 0) return PC_ERR_INVALID_ARG;
     if (n_rows == 0) return PC_OK;
-    const DecodeArgs a{row_prompt, row_rollout, row_step, row_kv_start, tokens, row_tok_index, group_row_start, prompt_len,
-                       prompt_kv, prompt_slots, prompt_kv_start, suffix_kv, suffix_slots,
-                       sample ? sample->temperature : 1.f, sample ? sample->seed : 0, sample != nullptr};
+    const DecodeArgs a = make_decode_args(row_prompt, row_rollout, row_step, row_kv_start, tokens, row_tok_index, group_row_start,
+                                          prompt_len, prompt_kv, prompt_slots, prompt_kv_start, suffix_kv, suffix_slots, sample);
     if (int rc = check_decode_args(ctx, a)) return rc;
     if (n_groups == 0 || max_group_rows == 0 || max_group_rows > n_rows || n_groups > n_rows) return PC_ERR_INVALID_ARG;
     if (logits_out == nullptr && sample == nullptr) return PC_ERR_INVALID_ARG;
@@ -680,8 +703,8 @@ int pc_decode_run(pc_ctx* ctx, void* stream, int n_steps, const pc_step_desc* st
     if (n_steps < 0) return PC_ERR_INVALID_ARG;
     if (n_steps == 0) return PC_OK;
     if (steps_host == nullptr || steps_dev == nullptr || sample == nullptr) return PC_ERR_INVALID_ARG;
-    const DecodeArgs a{row_prompt, row_rollout, row_step, row_kv_start, tokens, row_tok_index, group_row_start, prompt_len,
-                       prompt_kv, prompt_slots, prompt_kv_start, suffix_kv, suffix_slots, sample->temperature, sample->seed, 1};
+    const DecodeArgs a = make_decode_args(row_prompt, row_rollout, row_step, row_kv_start, tokens, row_tok_index, group_row_start,
+                                          prompt_len, prompt_kv, prompt_slots, prompt_kv_start, suffix_kv, suffix_slots, sample);
     if (int rc = check_decode_args(ctx, a)) return rc;
     int groups_bound = 0, group_rows_bound = 0;
     for (int s = 0; s < n_steps; ++s) {
@@ -718,12 +741,17 @@ int pc_decode_run(pc_ctx* ctx, void* stream, int n_steps, const pc_step_desc* st
             if (ctx->graphs.size() >= 64) ctx->drop_graphs();
             const unsigned long long launches_before = g_launches;
             cudaGraph_t graph = nullptr;
-            e = cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal);
+            if (ctx->capture_stream == nullptr) {
+                e = cudaStreamCreateWithFlags(&ctx->capture_stream, cudaStreamNonBlocking);
+                if (e != cudaSuccess) return cuda_fail(e, "create capture stream");
+            }
+            cudaStream_t cs = ctx->capture_stream;
+            e = cudaStreamBeginCapture(cs, cudaStreamCaptureModeThreadLocal);
             if (e != cudaSuccess) return cuda_fail(e, "begin graph capture");
-            pc::load_step_desc<<<1, 1, 0, st>>>(reinterpret_cast<const pc::StepDesc*>(steps_dev), counter, sd);
+            pc::load_step_desc<<<1, 1, 0, cs>>>(reinterpret_cast<const pc::StepDesc*>(steps_dev), counter, sd);
             count_launches(1);
-            const int rc = decode_launches(ctx, st, m_bound, groups_bound, group_rows_bound, a, nullptr);
-            e = cudaStreamEndCapture(st, &graph);
+            const int rc = decode_launches(ctx, cs, m_bound, groups_bound, group_rows_bound, a, nullptr);
+            e = cudaStreamEndCapture(cs, &graph);
             if (rc != PC_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
             if (e != cudaSuccess) return cuda_fail(e, "end graph capture");
             e = cudaGraphInstantiate(&exec, graph, 0);
