@@ -14,8 +14,10 @@
 //   attn_suffix_kernel  one warp per (rollout, KV head) streams the rollout's own suffix K/V through a
 //                       3-stage TMA ring at full HBM rate.  Positions sit on the MMA M axis (S^T = K Q^T,
 //                       O^T = V^T P^T), so the 6-8 query heads fill the N = 8 axis and no MMA work is
-//                       padded; P is transposed between the two MMAs with movmatrix.  At the end the
-//                       suffix part is merged with the group's prefix part by their log-sum-exp.
+//                       padded; P is transposed between the two MMAs with movmatrix.  It leaves its
+//                       (m, l, unnormalised O) record next to the prefix records.
+//   attn_merge_kernel   combines the prefix records and the suffix record of every (row, head) by their
+//                       log-sum-exp and writes the bf16 attention output.
 //
 // Scores are kept in the log2 domain (scaled by log2(e) / sqrt(head_dim)) so that exp2f is the only
 // transcendental.  Waits on mbarriers are bounded (see gemm_tc.cuh).
@@ -321,8 +323,7 @@ template <int HD> constexpr int suffix_smem_bytes() {
 template <int HD>
 __global__ void __launch_bounds__(S_WARPS * 32, 1)
 attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __restrict__ sd, int64_t n_slots, int Hq, int Hkv,
-                   int layer, const __nv_bfloat16* __restrict__ q, RowGeom g, float scale_log2, PrefixPartial part,
-                   __nv_bfloat16* __restrict__ out, int32_t* err) {
+                   int layer, const __nv_bfloat16* __restrict__ q, RowGeom g, float scale_log2, PrefixPartial part, int32_t* err) {
     constexpr int KS = HD / 16;                   // k-steps of K Q^T
     constexpr int DT = HD / 16;                   // 16-dim m-tiles of O^T
     constexpr int TILE_BYTES = S_TP * HD * 2;
@@ -390,21 +391,31 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
 
     int consumed = 0;
     bool ok = true;
+    // Q^T fragments (B operand): head = lane / 4, dims ks*16 + (lane%4)*2 (+8).  The next item's fragments and
+    // length are fetched while the current item streams, so that an item does not start with a global-memory stall.
+    uint32_t qn[KS][2];
+    int n_next = 0;
+    auto fetch_item = [&](int item) {
+        if (item >= n_items) return;
+        const int row = item / Hkv, kvh = item - row * Hkv;
+        n_next = g.s_len[row];
+        const int hq = lane >> 2;
+        const __nv_bfloat16* qp = q + ((size_t)row * Hq + (size_t)kvh * n_rep + hq) * HD + (lane & 3) * 2;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            qn[ks][0] = hq < n_rep ? *reinterpret_cast<const uint32_t*>(qp + ks * 16) : 0u;
+            qn[ks][1] = hq < n_rep ? *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8) : 0u;
+        }
+    };
+    fetch_item(first_item);
     for (int item = first_item; item < n_items && ok; item += item_stride) {
         const int row = item / Hkv, kvh = item - row * Hkv;
-        const int n = g.s_len[row];
+        const int n = n_next;
         const int ntiles = (n + S_TP - 1) / S_TP;
-        // Q^T fragments (B operand): head = lane / 4, dims ks*16 + (lane%4)*2 (+8)
         uint32_t qb[KS][2];
-        {
-            const int hq = lane >> 2;
-            const __nv_bfloat16* qp = q + ((size_t)row * Hq + (size_t)kvh * n_rep + hq) * HD + (lane & 3) * 2;
 #pragma unroll
-            for (int ks = 0; ks < KS; ++ks) {
-                qb[ks][0] = hq < n_rep ? *reinterpret_cast<const uint32_t*>(qp + ks * 16) : 0u;
-                qb[ks][1] = hq < n_rep ? *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8) : 0u;
-            }
-        }
+        for (int ks = 0; ks < KS; ++ks) { qb[ks][0] = qn[ks][0]; qb[ks][1] = qn[ks][1]; }
+        fetch_item(item + item_stride);
         float o[DT][4];
 #pragma unroll
         for (int t = 0; t < DT; ++t) { o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f; }
@@ -511,36 +522,15 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
             obuf[(hh + 1) * HD + d + 8] = o[dt][3];
         }
         __syncwarp();
-        // merge with the prefix part and write: lane handles HD/32 consecutive dims of every head
+        // leave the suffix part as record number part.n_parts, next to the prefix records; attn_merge_kernel combines them
         constexpr int EPL = HD / 32;
+        const size_t base = (size_t)part.n_parts * part.stride + (size_t)row * Hq + (size_t)kvh * n_rep;
+        if (lane < n_rep) { part.m[base + lane] = s_ml[warp][lane]; part.l[base + lane] = s_ml[warp][8 + lane]; }
         for (int j = 0; j < n_rep; ++j) {
-            const size_t rh = (size_t)row * Hq + (size_t)kvh * n_rep + j;
-            const float ms = s_ml[warp][j], ls = s_ml[warp][8 + j];
-            float M = ms;
-            for (int pp = 0; pp < part.n_parts; ++pp) M = fmaxf(M, part.m[(size_t)pp * part.stride + rh]);
-            const float ws = exp2_safe(ms, M);
-            float denom = ls * ws;
-            float res[EPL];
-#pragma unroll
-            for (int e = 0; e < EPL; ++e) res[e] = obuf[j * HD + lane * EPL + e] * ws;
-            for (int pp = 0; pp < part.n_parts; ++pp) {          // fixed order: the result does not depend on CTA timing
-                const size_t ph = (size_t)pp * part.stride + rh;
-                const float wp = exp2_safe(part.m[ph], M);
-                if (wp > 0.f) {
-                    denom += part.l[ph] * wp;
-#pragma unroll
-                    for (int e = 0; e < EPL; ++e) res[e] += part.o[ph * HD + lane * EPL + e] * wp;
-                }
-            }
-            const float inv = denom > 0.f ? 1.f / denom : 0.f;
-#pragma unroll
-            for (int e = 0; e < EPL; ++e) res[e] *= inv;
-            __nv_bfloat16* dst = out + rh * HD + lane * EPL;
-            if (EPL == 4) {
-                *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(res[0], res[1]), pack_bf16(res[2], res[3]));
-            } else {
-                *reinterpret_cast<uint32_t*>(dst) = pack_bf16(res[0], res[1]);
-            }
+            float* dst = part.o + (base + j) * HD + lane * EPL;
+            const float* src = obuf + j * HD + lane * EPL;
+            if (EPL == 4) *reinterpret_cast<float4*>(dst) = *reinterpret_cast<const float4*>(src);
+            else *reinterpret_cast<float2*>(dst) = *reinterpret_cast<const float2*>(src);
         }
         __syncwarp();
     }
@@ -555,6 +545,52 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
         for (int i = 0; i < 2000; ++i) __nanosleep(1000);
     }
     __syncthreads();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Merge of the prefix records 0 .. n_parts-1 and the suffix record n_parts of every (row, query head) by their
+// log-sum-exp:  M = max m_i,  out = sum_i O_i 2^(m_i - M) / sum_i l_i 2^(m_i - M).  Records are added in index order.
+// One warp per (row, head); a lane owns HD/32 consecutive dims.
+// ---------------------------------------------------------------------------------------------
+template <int HD>
+__global__ void __launch_bounds__(256) attn_merge_kernel(const StepDesc* __restrict__ sd, int Hq, PrefixPartial part,
+                                                         __nv_bfloat16* __restrict__ out) {
+    constexpr int EPL = HD / 32;
+    const int lane = threadIdx.x & 31;
+    const size_t rh = (size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (rh >= (size_t)sd->n_rows * Hq) return;
+    const int n_rec = part.n_parts + 1;
+    float mi[MAX_PREFIX_PARTS + 1], li[MAX_PREFIX_PARTS + 1];
+    float M = -INFINITY;
+#pragma unroll
+    for (int i = 0; i <= MAX_PREFIX_PARTS; ++i) {
+        mi[i] = -INFINITY; li[i] = 0.f;
+        if (i < n_rec) { mi[i] = part.m[(size_t)i * part.stride + rh]; li[i] = part.l[(size_t)i * part.stride + rh]; }
+        M = fmaxf(M, mi[i]);
+    }
+    float acc[EPL];
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+    float denom = 0.f;
+#pragma unroll
+    for (int i = 0; i <= MAX_PREFIX_PARTS; ++i) {
+        const float w = exp2_safe(mi[i], M);
+        if (i < n_rec && w > 0.f) {
+            denom += li[i] * w;
+            const float* src = part.o + ((size_t)i * part.stride + rh) * HD + lane * EPL;
+            if (EPL == 4) {
+                const float4 v = *reinterpret_cast<const float4*>(src);
+                acc[0] += v.x * w; acc[1] += v.y * w; acc[2] += v.z * w; acc[3] += v.w * w;
+            } else {
+                const float2 v = *reinterpret_cast<const float2*>(src);
+                acc[0] += v.x * w; acc[1] += v.y * w;
+            }
+        }
+    }
+    const float inv = denom > 0.f ? 1.f / denom : 0.f;
+    __nv_bfloat16* dst = out + rh * HD + lane * EPL;
+    if (EPL == 4) *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc[0] * inv, acc[1] * inv), pack_bf16(acc[2] * inv, acc[3] * inv));
+    else *reinterpret_cast<uint32_t*>(dst) = pack_bf16(acc[0] * inv, acc[1] * inv);
 }
 
 }  // namespace am

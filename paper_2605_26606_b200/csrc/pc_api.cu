@@ -144,9 +144,9 @@ Carve carve(const pc_ctx* c, int max_rows, int max_prefill) {
     v.last_row = take(M * 4);
     // prefix part of the shared-prefix attention: (max, sum, unnormalised output) per (row, query head)
     const size_t R = (size_t)std::max(max_rows, 1);
-    v.part_m = take(pc::am::MAX_PREFIX_PARTS * R * d.n_q_heads * 4);
-    v.part_l = take(pc::am::MAX_PREFIX_PARTS * R * d.n_q_heads * 4);
-    v.part_o = take(pc::am::MAX_PREFIX_PARTS * R * d.n_q_heads * d.head_dim * 4);
+    v.part_m = take((pc::am::MAX_PREFIX_PARTS + 1) * R * d.n_q_heads * 4);
+    v.part_l = take((pc::am::MAX_PREFIX_PARTS + 1) * R * d.n_q_heads * 4);
+    v.part_o = take((pc::am::MAX_PREFIX_PARTS + 1) * R * d.n_q_heads * d.head_dim * 4);
     v.total = off;
     return v;
 }
@@ -287,9 +287,10 @@ int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, in
     const int sgrid = std::min(c->num_sms, (items + am::S_WARPS - 1) / am::S_WARPS);
     if (profile) cudaEventRecord(c->prof_start, st);
     am::attn_suffix_kernel<HD><<<sgrid, am::S_WARPS * 32, am::suffix_smem_bytes<HD>(), st>>>(
-        c->map_suffix_kv, sd, suffix_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, g, scale_log2, part, attn, c->err);
+        c->map_suffix_kv, sd, suffix_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, g, scale_log2, part, c->err);
     if (profile) cudaEventRecord(c->prof_stop, st);
-    count_launches(2);
+    am::attn_merge_kernel<HD><<<(M * d.n_q_heads + 7) / 8, 256, 0, st>>>(sd, d.n_q_heads, part, attn);
+    count_launches(3);
     return PC_OK;
 }
 
