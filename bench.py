@@ -144,6 +144,7 @@ def run_probe(args):
     weights = wl.gen_weights(w.model, seed=0)
     batch = wl.gen_batch(w)
     eng = RolloutEngine(w.model, weights, max_rows=P * G, max_prefill_tokens=int(batch.prompt_offsets[-1]))
+    eng.use_graphs = kv.get("graphs", "1") != "0"
     eng.load_batch(w, batch)
     eng.suffix_kv.zero_()
     eng.tokens.random_(0, w.model.vocab)

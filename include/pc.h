@@ -215,10 +215,14 @@ PC_API int pc_decode_run(pc_ctx* ctx, void* stream, int n_steps, const pc_step_d
  * Row r reads logits row logits_row[r] (NULL: row r), so all rollouts of a group can draw
  * their first token from their prompt's single prefill row.
  *   out_tokens  device int32; token of row r is stored at out_tokens[out_index[r]] (NULL: [r])
- *   out_top2_gap device [n_rows] float or NULL: largest minus second-largest perturbed score */
+ *   out_top2_gap device [n_rows] float or NULL: largest minus second-largest perturbed score
+ *   scratch     device, 16-byte aligned, scratch_bytes long, or NULL.  With few rows the vocabulary of a row is
+ *               scored by several blocks that leave 16-byte records here (n_rows * up to 32 records are used
+ *               when they fit); without scratch one block scores a whole row.  The result is the same. */
 PC_API int pc_sample(void* stream, int n_rows, int vocab, const float* logits, const int32_t* logits_row,
               float temperature, uint64_t seed, const int32_t* row_prompt, const int32_t* row_rollout,
-              const int32_t* row_step, int32_t* out_tokens, const int64_t* out_index, float* out_top2_gap);
+              const int32_t* row_step, int32_t* out_tokens, const int64_t* out_index, float* out_top2_gap,
+              void* scratch, size_t scratch_bytes);
 
 /* Binary reward of the synthetic workloads, standing in for the verifier R(q, o) in {0, 1} of
  * Section 3.3: reward[i] = 1 if tokens[last_index[i]] < threshold[i] else 0.  All device. */

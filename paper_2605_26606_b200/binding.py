@@ -88,7 +88,7 @@ def _lib():
         lib.pc_prefill_shared.argtypes = [p, p, i, p, p, i, i, p, i64, p, p]
         lib.pc_decode_step.argtypes = [p, p, i, p, p, p, p, p, p, i, p, i, p, p, i64, p, p, i64, p, C.POINTER(SampleParams)]
         lib.pc_decode_run.argtypes = [p, p, i, p, p, p, p, p, p, p, p, p, p, p, i64, p, p, i64, C.POINTER(SampleParams)]
-        lib.pc_sample.argtypes = [p, i, i, p, p, f, u64, p, p, p, p, p, p]
+        lib.pc_sample.argtypes = [p, i, i, p, p, f, u64, p, p, p, p, p, p, p, C.c_size_t]
         lib.pc_reward_last_token.argtypes = [p, i, p, p, p, p]
         lib.pc_group_stats.argtypes = [p, i, p, p, p, p, p, p, p]
         lib.pc_allocate.argtypes = [p, i, p, p, C.POINTER(AllocParams), p, p, p, p, p]
@@ -225,10 +225,11 @@ def pc_decode_run(ctx: Context, n_steps, steps_host, steps_dev, row_prompt, row_
 
 
 def pc_sample(n_rows, vocab, logits, logits_row, temperature, seed, row_prompt, row_rollout, row_step, out_tokens,
-              out_index=None, out_top2_gap=None) -> None:
+              out_index=None, out_top2_gap=None, scratch: Optional[torch.Tensor] = None) -> None:
     _check(_lib().pc_sample(_stream(), n_rows, vocab, _ptr(logits, torch.float32), _ptr(logits_row), temperature, seed,
                             _ptr(row_prompt), _ptr(row_rollout), _ptr(row_step), _ptr(out_tokens), _ptr(out_index),
-                            _ptr(out_top2_gap)), "pc_sample")
+                            _ptr(out_top2_gap), _ptr(scratch), scratch.numel() * scratch.element_size() if scratch is not None else 0),
+           "pc_sample")
 
 
 def pc_reward_last_token(n, tokens, last_index, threshold, reward) -> None:

@@ -79,8 +79,11 @@ struct PrefixPartial {
     float* o;               // [n_parts][stride * head_dim]
     int n_parts;
     size_t stride;          // rows capacity * Hq
+    int chunk_tiles;        // 0: one suffix record per (row, head); else the suffix is cut into ranges of >= chunk_tiles tiles
 };
 constexpr int MAX_PREFIX_PARTS = 8;
+constexpr int MAX_SUFFIX_CHUNKS = 8;
+constexpr int MAX_RECORDS = MAX_PREFIX_PARTS + MAX_SUFFIX_CHUNKS;
 
 // ---------------------------------------------------------------------------------------------
 // Group (shared-prefix / causal-prefill) kernel
@@ -320,6 +323,19 @@ template <int HD> constexpr int suffix_smem_bytes() {
     return S_WARPS * (S_STAGES * 2 * S_TP * HD * 2 + 8 * HD * 4) + 1024 + 256;
 }
 
+// With few rollouts there are about as many (rollout, KV head) streams as warps on the GPU, and one stream more than
+// warps doubles the kernel's time.  The suffix of a rollout is therefore cut into ranges of tiles ("chunks") that
+// are spread over the warps; every chunk leaves its own record.
+__device__ __forceinline__ int suffix_chunk_len(int ntiles, int chunk_tiles) {     // tiles per chunk of a row with ntiles tiles
+    return chunk_tiles <= 0 ? max(ntiles, 1) : max(chunk_tiles, (ntiles + MAX_SUFFIX_CHUNKS - 1) / MAX_SUFFIX_CHUNKS);
+}
+__device__ __forceinline__ int suffix_chunks(int n, int chunk_tiles) {             // records a row with n suffix slots leaves
+    const int ntiles = (n + S_TP - 1) / S_TP;
+    if (ntiles == 0) return 0;
+    const int ct = suffix_chunk_len(ntiles, chunk_tiles);
+    return (ntiles + ct - 1) / ct;
+}
+
 template <int HD>
 __global__ void __launch_bounds__(S_WARPS * 32, 1)
 attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __restrict__ sd, int64_t n_slots, int Hq, int Hkv,
@@ -347,23 +363,34 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
     }
     __syncthreads();
 
-    const int n_items = sd->n_rows * Hkv;
+    // work unit u = (item, chunk), item = (row, kv head); units of one item are consecutive, so they land on different warps
+    const int cpi = part.chunk_tiles > 0 ? MAX_SUFFIX_CHUNKS : 1;       // unit slots per item
+    const int n_items = sd->n_rows * Hkv * cpi;
     const int item_stride = gridDim.x * S_WARPS;
     const int first_item = blockIdx.x * S_WARPS + warp;
+    // tile range [t0, t1) of unit u for a row with n suffix slots; empty when the row has fewer chunks
+    auto unit_range = [&](int u, int n, int& t0, int& t1) {
+        const int ntiles = (n + S_TP - 1) / S_TP;
+        const int ct = suffix_chunk_len(ntiles, part.chunk_tiles);
+        t0 = min(ntiles, (u % cpi) * ct);
+        t1 = min(ntiles, t0 + ct);
+    };
 
     // producer cursor (tracked identically by every lane; lane 0 issues)
     int p_item = first_item, p_tile = 0, p_ntiles = 0;
     int64_t p_krow = 0, p_vrow = 0;
     auto p_load_item = [&]() {
         while (p_item < n_items) {
-            const int row = p_item / Hkv, kvh = p_item - row * Hkv;
-            const int n = g.s_len[row];
-            if (n > 0) {
-                p_ntiles = (n + S_TP - 1) / S_TP;
+            const int it = p_item / cpi;
+            const int row = it / Hkv, kvh = it - row * Hkv;
+            int t0, t1;
+            unit_range(p_item, g.s_len[row], t0, t1);
+            if (t1 > t0) {
+                p_ntiles = t1;
                 const int64_t st = g.s_start[row];
                 p_krow = (((int64_t)layer * 2 + 0) * Hkv + kvh) * n_slots + st;
                 p_vrow = (((int64_t)layer * 2 + 1) * Hkv + kvh) * n_slots + st;
-                p_tile = 0;
+                p_tile = t0;
                 return;
             }
             p_item += item_stride;
@@ -397,7 +424,8 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
     int n_next = 0;
     auto fetch_item = [&](int item) {
         if (item >= n_items) return;
-        const int row = item / Hkv, kvh = item - row * Hkv;
+        const int it = item / cpi;
+        const int row = it / Hkv, kvh = it - row * Hkv;
         n_next = g.s_len[row];
         const int hq = lane >> 2;
         const __nv_bfloat16* qp = q + ((size_t)row * Hq + (size_t)kvh * n_rep + hq) * HD + (lane & 3) * 2;
@@ -409,19 +437,22 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
     };
     fetch_item(first_item);
     for (int item = first_item; item < n_items && ok; item += item_stride) {
-        const int row = item / Hkv, kvh = item - row * Hkv;
+        const int it = item / cpi, chunk = item - it * cpi;
+        const int row = it / Hkv, kvh = it - row * Hkv;
         const int n = n_next;
-        const int ntiles = (n + S_TP - 1) / S_TP;
+        int t0, t1;
+        unit_range(item, n, t0, t1);
         uint32_t qb[KS][2];
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) { qb[ks][0] = qn[ks][0]; qb[ks][1] = qn[ks][1]; }
         fetch_item(item + item_stride);
+        if (t1 <= t0 && !(chunk == 0 && part.chunk_tiles <= 0)) continue;      // this row has fewer chunks: nothing to leave
         float o[DT][4];
 #pragma unroll
         for (int t = 0; t < DT; ++t) { o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f; }
         float mh[2] = {-INFINITY, -INFINITY}, lh[2] = {0.f, 0.f};      // heads (lane%4)*2 + {0, 1}
 
-        for (int tile = 0; tile < ntiles; ++tile) {
+        for (int tile = t0; tile < t1; ++tile) {
             const int stage = consumed % S_STAGES;
             const uint32_t phase = (uint32_t)(consumed / S_STAGES) & 1u;
             if (!mbar_wait(full0 + 8 * stage, phase, &s_abort)) { ok = false; break; }
@@ -522,9 +553,9 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
             obuf[(hh + 1) * HD + d + 8] = o[dt][3];
         }
         __syncwarp();
-        // leave the suffix part as record number part.n_parts, next to the prefix records; attn_merge_kernel combines them
+        // leave this chunk as record number part.n_parts + chunk, next to the prefix records; attn_merge_kernel combines them
         constexpr int EPL = HD / 32;
-        const size_t base = (size_t)part.n_parts * part.stride + (size_t)row * Hq + (size_t)kvh * n_rep;
+        const size_t base = (size_t)(part.n_parts + chunk) * part.stride + (size_t)row * Hq + (size_t)kvh * n_rep;
         if (lane < n_rep) { part.m[base + lane] = s_ml[warp][lane]; part.l[base + lane] = s_ml[warp][8 + lane]; }
         for (int j = 0; j < n_rep; ++j) {
             float* dst = part.o + (base + j) * HD + lane * EPL;
@@ -553,17 +584,20 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
 // One warp per (row, head); a lane owns HD/32 consecutive dims.
 // ---------------------------------------------------------------------------------------------
 template <int HD>
-__global__ void __launch_bounds__(256) attn_merge_kernel(const StepDesc* __restrict__ sd, int Hq, PrefixPartial part,
+__global__ void __launch_bounds__(256) attn_merge_kernel(const StepDesc* __restrict__ sd, int Hq, RowGeom g, PrefixPartial part,
                                                          __nv_bfloat16* __restrict__ out) {
     constexpr int EPL = HD / 32;
     const int lane = threadIdx.x & 31;
     const size_t rh = (size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (rh >= (size_t)sd->n_rows * Hq) return;
-    const int n_rec = part.n_parts + 1;
-    float mi[MAX_PREFIX_PARTS + 1], li[MAX_PREFIX_PARTS + 1];
+    const int row = (int)(rh / Hq);
+    // a row without suffix slots still has its (empty) record 0 when the suffix is not cut into chunks
+    const int n_sfx = part.chunk_tiles > 0 ? suffix_chunks(g.s_len[row], part.chunk_tiles) : 1;
+    const int n_rec = part.n_parts + n_sfx;
+    float mi[MAX_RECORDS], li[MAX_RECORDS];
     float M = -INFINITY;
 #pragma unroll
-    for (int i = 0; i <= MAX_PREFIX_PARTS; ++i) {
+    for (int i = 0; i < MAX_RECORDS; ++i) {
         mi[i] = -INFINITY; li[i] = 0.f;
         if (i < n_rec) { mi[i] = part.m[(size_t)i * part.stride + rh]; li[i] = part.l[(size_t)i * part.stride + rh]; }
         M = fmaxf(M, mi[i]);
@@ -573,7 +607,7 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const StepDesc* __restr
     for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
     float denom = 0.f;
 #pragma unroll
-    for (int i = 0; i <= MAX_PREFIX_PARTS; ++i) {
+    for (int i = 0; i < MAX_RECORDS; ++i) {
         const float w = exp2_safe(mi[i], M);
         if (i < n_rec && w > 0.f) {
             denom += li[i] * w;

@@ -47,7 +47,7 @@ constexpr int kMaxSplits = 8;
 
 struct Carve {
     size_t h, a, qkv, q, attn, act, logits, rope, pos, wslot, warena, p_start, p_len, s_start, s_len, token, last_row,
-        part_m, part_l, part_o, res_part, step_desc, step_counter, total;
+        part_m, part_l, part_o, res_part, step_desc, step_counter, sample_scratch, total;
 };
 
 // A captured decode step, replayable for every step that fits the same upper bounds and reads the same arrays.
@@ -128,6 +128,7 @@ Carve carve(const pc_ctx* c, int max_rows, int max_prefill) {
     v.res_part = take(split_rows * d.d_model * 4);
     v.step_desc = take(sizeof(pc::StepDesc));
     v.step_counter = take(4);
+    v.sample_scratch = take((size_t)std::max(max_rows, 1) * pc::SAMPLE_MAX_CHUNKS * sizeof(pc::Top2Rec));
     v.q = take(M * c->q_dim() * eb);
     v.attn = take(M * c->q_dim() * eb);
     v.act = take(M * (size_t)d.d_ff * eb);
@@ -144,9 +145,9 @@ Carve carve(const pc_ctx* c, int max_rows, int max_prefill) {
     v.last_row = take(M * 4);
     // prefix part of the shared-prefix attention: (max, sum, unnormalised output) per (row, query head)
     const size_t R = (size_t)std::max(max_rows, 1);
-    v.part_m = take((pc::am::MAX_PREFIX_PARTS + 1) * R * d.n_q_heads * 4);
-    v.part_l = take((pc::am::MAX_PREFIX_PARTS + 1) * R * d.n_q_heads * 4);
-    v.part_o = take((pc::am::MAX_PREFIX_PARTS + 1) * R * d.n_q_heads * d.head_dim * 4);
+    v.part_m = take(pc::am::MAX_RECORDS * R * d.n_q_heads * 4);
+    v.part_l = take(pc::am::MAX_RECORDS * R * d.n_q_heads * 4);
+    v.part_o = take(pc::am::MAX_RECORDS * R * d.n_q_heads * d.head_dim * 4);
     v.total = off;
     return v;
 }
@@ -271,7 +272,9 @@ int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, in
     const int base_ctas = std::max(1, q_tiles * d.n_kv_heads * plan.n_groups);
     const int n_parts = plan.prefill ? 1 : std::max(1, std::min(am::MAX_PREFIX_PARTS, c->num_sms / base_ctas));
     am::PrefixPartial part{reinterpret_cast<float*>(c->ws + c->cv.part_m), reinterpret_cast<float*>(c->ws + c->cv.part_l),
-                           reinterpret_cast<float*>(c->ws + c->cv.part_o), n_parts, (size_t)std::max(c->max_rows, 1) * d.n_q_heads};
+                           reinterpret_cast<float*>(c->ws + c->cv.part_o), n_parts, (size_t)std::max(c->max_rows, 1) * d.n_q_heads, 0};
+    // few (rollout, KV head) streams per warp: cut the suffixes into chunks of at least 4 tiles so that the load balances
+    if (M * d.n_kv_heads < 4 * c->num_sms * am::S_WARPS) part.chunk_tiles = 4;
     const dim3 ggrid(q_tiles * n_parts, d.n_kv_heads, plan.n_groups);
     if (plan.prefill) {
         am::attn_group_kernel<HD, true><<<ggrid, am::G_THREADS, am::group_smem_bytes<HD>(), st>>>(
@@ -283,13 +286,13 @@ int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, in
     am::attn_group_kernel<HD, false><<<ggrid, am::G_THREADS, am::group_smem_bytes<HD>(), st>>>(
         c->map_prompt_kv, sd, prompt_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, plan.group_row_start, g, scale_log2, part,
         attn, c->err);
-    const int items = M * d.n_kv_heads;
+    const int items = M * d.n_kv_heads * (part.chunk_tiles > 0 ? am::MAX_SUFFIX_CHUNKS : 1);
     const int sgrid = std::min(c->num_sms, (items + am::S_WARPS - 1) / am::S_WARPS);
     if (profile) cudaEventRecord(c->prof_start, st);
     am::attn_suffix_kernel<HD><<<sgrid, am::S_WARPS * 32, am::suffix_smem_bytes<HD>(), st>>>(
         c->map_suffix_kv, sd, suffix_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, g, scale_log2, part, c->err);
     if (profile) cudaEventRecord(c->prof_stop, st);
-    am::attn_merge_kernel<HD><<<(M * d.n_q_heads + 7) / 8, 256, 0, st>>>(sd, d.n_q_heads, part, attn);
+    am::attn_merge_kernel<HD><<<(M * d.n_q_heads + 7) / 8, 256, 0, st>>>(sd, d.n_q_heads, g, part, attn);
     count_launches(3);
     return PC_OK;
 }
@@ -658,10 +661,20 @@ int decode_launches(pc_ctx* ctx, cudaStream_t st, int m_bound, int groups_bound,
     rc = f32 ? run_lm_head<float>(ctx, st, m_bound, sd, nullptr, logits) : run_lm_head<__nv_bfloat16>(ctx, st, m_bound, sd, nullptr, logits);
     if (rc) return rc;
     if (a.sample) {
-        pc::sample_kernel<<<m_bound, 256, 0, st>>>(sd, ctx->d.vocab, logits, nullptr, a.temperature, (uint32_t)(a.seed & 0xffffffffu),
-                                                   (uint32_t)(a.seed >> 32), a.row_prompt, a.row_rollout, a.row_step, 1, a.tokens,
-                                                   a.row_tok_index, 1, nullptr);
-        count_launches(1);
+        const uint32_t k0 = (uint32_t)(a.seed & 0xffffffffu), k1 = (uint32_t)(a.seed >> 32);
+        const int chunks = pc::sample_chunks(m_bound, ctx->num_sms);
+        if (chunks == 1) {
+            pc::sample_kernel<<<m_bound, 256, 0, st>>>(sd, ctx->d.vocab, logits, nullptr, a.temperature, k0, k1, a.row_prompt,
+                                                       a.row_rollout, a.row_step, 1, a.tokens, a.row_tok_index, 1, nullptr);
+            count_launches(1);
+        } else {
+            pc::Top2Rec* scratch = reinterpret_cast<pc::Top2Rec*>(ctx->ws + ctx->cv.sample_scratch);
+            pc::sample_partial_kernel<<<dim3(m_bound, chunks), 256, 0, st>>>(sd, ctx->d.vocab, chunks, logits, nullptr, a.temperature,
+                                                                             k0, k1, a.row_prompt, a.row_rollout, a.row_step, 1, scratch);
+            pc::sample_reduce_kernel<<<(m_bound + 127) / 128, 128, 0, st>>>(sd, m_bound, chunks, scratch, a.tokens, a.row_tok_index, 1,
+                                                                            nullptr);
+            count_launches(2);
+        }
         PC_CUDA_CHECK_LAUNCH("sample");
     }
     return PC_OK;
@@ -773,15 +786,33 @@ int pc_decode_run(pc_ctx* ctx, void* stream, int n_steps, const pc_step_desc* st
 
 int pc_sample(void* stream, int n_rows, int vocab, const float* logits, const int32_t* logits_row, float temperature,
               uint64_t seed, const int32_t* row_prompt, const int32_t* row_rollout, const int32_t* row_step,
-              int32_t* out_tokens, const int64_t* out_index, float* out_top2_gap) {
+              int32_t* out_tokens, const int64_t* out_index, float* out_top2_gap, void* scratch, size_t scratch_bytes) {
     if (n_rows < 0 || vocab <= 0 || !(temperature > 0.f)) return PC_ERR_INVALID_ARG;
     if (n_rows == 0) return PC_OK;
     if (logits == nullptr || row_prompt == nullptr || row_rollout == nullptr || row_step == nullptr || out_tokens == nullptr)
         return PC_ERR_INVALID_ARG;
-    pc::sample_kernel<<<n_rows, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        nullptr, vocab, logits, logits_row, temperature, (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32), row_prompt, row_rollout,
-        row_step, 0, out_tokens, out_index, 0, out_top2_gap);
-    count_launches(1);
+    const uint32_t k0 = (uint32_t)(seed & 0xffffffffu), k1 = (uint32_t)(seed >> 32);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (scratch != nullptr && !aligned(scratch, 16)) return PC_ERR_ALIGNMENT;
+    int chunks = 1;
+    if (scratch != nullptr) {
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess)
+            chunks = pc::sample_chunks(n_rows, sms);
+        while (chunks > 1 && (size_t)n_rows * chunks * sizeof(pc::Top2Rec) > scratch_bytes) --chunks;    // use what fits
+    }
+    if (chunks == 1) {
+        pc::sample_kernel<<<n_rows, 256, 0, st>>>(nullptr, vocab, logits, logits_row, temperature, k0, k1, row_prompt, row_rollout,
+                                                  row_step, 0, out_tokens, out_index, 0, out_top2_gap);
+        count_launches(1);
+    } else {
+        pc::Top2Rec* rec = static_cast<pc::Top2Rec*>(scratch);
+        pc::sample_partial_kernel<<<dim3(n_rows, chunks), 256, 0, st>>>(nullptr, vocab, chunks, logits, logits_row, temperature, k0, k1,
+                                                                        row_prompt, row_rollout, row_step, 0, rec);
+        pc::sample_reduce_kernel<<<(n_rows + 127) / 128, 128, 0, st>>>(nullptr, n_rows, chunks, rec, out_tokens, out_index, 0,
+                                                                       out_top2_gap);
+        count_launches(2);
+    }
     PC_CUDA_CHECK_LAUNCH("sample");
     return PC_OK;
 }

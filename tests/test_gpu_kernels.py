@@ -36,6 +36,13 @@ def test_sample_matches_oracle(vocab, temperature):
     gap = torch.zeros(n, dtype=torch.float32, device="cuda")
     B.pc_sample(n, vocab, torch.from_numpy(logits).cuda(), None, temperature, seed, _i32(prompt), _i32(roll), _i32(step), out,
                 None, gap)
+    # the two-pass form (vocabulary of a row split over several blocks) must give the very same answer
+    out2 = torch.zeros(n, dtype=torch.int32, device="cuda")
+    gap2 = torch.zeros(n, dtype=torch.float32, device="cuda")
+    scratch = torch.empty(n * 32 * 16, dtype=torch.uint8, device="cuda")
+    B.pc_sample(n, vocab, torch.from_numpy(logits).cuda(), None, temperature, seed, _i32(prompt), _i32(roll), _i32(step), out2,
+                None, gap2, scratch)
+    assert torch.equal(out, out2) and torch.equal(gap, gap2)
     out, gap = out.cpu().numpy(), gap.cpu().numpy()
     for r in range(n):
         tok, g = osampler.sample(logits[r], temperature, seed, int(prompt[r]), int(roll[r]), int(step[r]))

@@ -51,10 +51,10 @@ def test_create_rejects_bad_arguments_on_the_host(lib):
 
 
 def test_entry_points_reject_bad_arguments_on_the_host(lib):
-    assert lib.pc_sample(None, -1, 8, None, None, 1.0, 0, None, None, None, None, None, None) == B.PC_ERR_INVALID_ARG
-    assert lib.pc_sample(None, 4, 8, None, None, 1.0, 0, None, None, None, None, None, None) == B.PC_ERR_INVALID_ARG
-    assert lib.pc_sample(None, 0, 8, None, None, 1.0, 0, None, None, None, None, None, None) == B.PC_OK
-    assert lib.pc_group_stats(None, 3, None, None, None, None, None, None, None) == B.PC_ERR_INVALID_ARG
+    assert lib.pc_sample(None, -1, 8, None, None, 1.0, 0, None, None, None, None, None, None, None, 0) == B.PC_ERR_INVALID_ARG
+    assert lib.pc_sample(None, 4, 8, None, None, 1.0, 0, None, None, None, None, None, None, None, 0) == B.PC_ERR_INVALID_ARG
+    assert lib.pc_sample(None, 0, 8, None, None, 1.0, 0, None, None, None, None, None, None, None, 0) == B.PC_OK
+    assert lib.pc_group_stats(None, 3, None, None, None, None, None, None, None, None, 0) == B.PC_ERR_INVALID_ARG
     assert lib.pc_group_stats(None, 0, None, None, None, None, None, None, None) == B.PC_OK
     assert lib.pc_grpo_advantage(None, 2, None, None, None, None, None) == B.PC_ERR_INVALID_ARG
     assert lib.pc_reward_last_token(None, 5, None, None, None, None) == B.PC_ERR_INVALID_ARG
