@@ -224,6 +224,23 @@ PC_API int pc_sample(void* stream, int n_rows, int vocab, const float* logits, c
               const int32_t* row_step, int32_t* out_tokens, const int64_t* out_index, float* out_top2_gap,
               void* scratch, size_t scratch_bytes);
 
+/* pc_sample for callers that cannot provide scratch memory.  The paper has no counterpart: this entry point exists for
+ * hosts of this library that must not allocate device memory at the moment they sample -- code running inside a
+ * stream-ordered region whose allocator is frozen, a plugin that is handed only its input and output buffers, a
+ * process whose memory pool is owned by another framework and already exhausted.  pc_sample needs caller-provided
+ * scratch to spread a small batch over the GPU; here the same two-pass sampler keeps its per-range records in an array
+ * that is part of the library image (2 MiB per GPU that loads the library, held until the process exits).
+ *   - at most 4096 rows per call; more is refused with PC_ERR_CAPACITY (pc_last_cuda_error gives the text).
+ *   - the first call on each device looks up the array's device address; make that first call outside any stream
+ *     capture, with the device that will run the kernels current.
+ *   - all calls on a device share the one array and it keeps the previous call's records.  Nothing needs clearing
+ *     (a call overwrites every record it later reads), but two calls that overlap on the GPU -- different streams,
+ *     or different host threads without ordering -- race on it: order them.
+ *   - no cudaMalloc, cudaFree or other allocating call is made.  Arguments and results exactly as pc_sample's. */
+PC_API int pc_sample_static(void* stream, int n_rows, int vocab, const float* logits, const int32_t* logits_row,
+                            float temperature, uint64_t seed, const int32_t* row_prompt, const int32_t* row_rollout,
+                            const int32_t* row_step, int32_t* out_tokens, const int64_t* out_index, float* out_top2_gap);
+
 /* Binary reward of the synthetic workloads, standing in for the verifier R(q, o) in {0, 1} of
  * Section 3.3: reward[i] = 1 if tokens[last_index[i]] < threshold[i] else 0.  All device. */
 PC_API int pc_reward_last_token(void* stream, int n, const int32_t* tokens, const int64_t* last_index,

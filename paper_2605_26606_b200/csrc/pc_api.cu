@@ -872,4 +872,66 @@ int pc_grpo_advantage(void* stream, int n_groups, const float* rewards, const in
     return PC_OK;
 }
 
+
+// ---------------------------------------------------------------------------------------------------------------
+// pc_sample_static: the two-pass sampler with its scratch inside the library image.
+// ---------------------------------------------------------------------------------------------------------------
+}  // extern "C"
+
+namespace {
+
+constexpr int kStaticSampleMaxRows = 4096;
+// One record per (row, vocabulary range).  The array lives in the device image of the library: every GPU that loads
+// libpc.so holds these 2 MiB until the process exits.  Its name is only a host-side handle here; kernels are given
+// the device address that cudaGetSymbolAddress returns.
+static __device__ __align__(256) unsigned char g_static_sample_scratch[(size_t)kStaticSampleMaxRows * pc::SAMPLE_MAX_CHUNKS *
+                                                                       sizeof(pc::Top2Rec)];
+
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {};      // device address of the array, per device ordinal
+int g_static_scratch_sms[kMaxDevices] = {};
+
+}  // namespace
+
+extern "C" {
+
+int pc_sample_static(void* stream, int n_rows, int vocab, const float* logits, const int32_t* logits_row, float temperature,
+                     uint64_t seed, const int32_t* row_prompt, const int32_t* row_rollout, const int32_t* row_step,
+                     int32_t* out_tokens, const int64_t* out_index, float* out_top2_gap) {
+    if (n_rows < 0 || vocab <= 0 || !(temperature > 0.f)) return PC_ERR_INVALID_ARG;
+    if (n_rows > kStaticSampleMaxRows) {
+        g_cuda_error = "pc_sample_static: n_rows exceeds the built-in scratch (4096 rows)";
+        return PC_ERR_CAPACITY;
+    }
+    if (n_rows == 0) return PC_OK;
+    if (logits == nullptr || row_prompt == nullptr || row_rollout == nullptr || row_step == nullptr || out_tokens == nullptr)
+        return PC_ERR_INVALID_ARG;
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (dev < 0 || dev >= kMaxDevices) return PC_ERR_UNSUPPORTED;
+    if (g_static_scratch_addr[dev] == nullptr) {
+        // first call on this device: resolve the array's device address (the device is current)
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_sample_scratch);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(static sampler scratch)");
+        int sms = 0;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+        g_static_scratch_sms[dev] = sms;
+        g_static_scratch_addr[dev] = p;
+    }
+    pc::Top2Rec* rec = static_cast<pc::Top2Rec*>(g_static_scratch_addr[dev]);
+    const int chunks = pc::sample_chunks(n_rows, g_static_scratch_sms[dev]);
+    const uint32_t k0 = (uint32_t)(seed & 0xffffffffu), k1 = (uint32_t)(seed >> 32);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // every record the second kernel reads is written by the first one in this same call: nothing has to start at zero
+    pc::sample_partial_kernel<<<dim3(n_rows, chunks), 256, 0, st>>>(nullptr, vocab, chunks, logits, logits_row, temperature, k0, k1,
+                                                                    row_prompt, row_rollout, row_step, 0, rec);
+    pc::sample_reduce_kernel<<<(n_rows + 127) / 128, 128, 0, st>>>(nullptr, n_rows, chunks, rec, out_tokens, out_index, 0, out_top2_gap);
+    count_launches(2);
+    PC_CUDA_CHECK_LAUNCH("sample (static scratch)");
+    return PC_OK;
+}
+
 }  // extern "C"
