@@ -24,7 +24,8 @@
  *    statistics are float; dot products accumulate in float.
  *  - KV arena layout (prompt arena and suffix arena alike):
  *        [n_layers][2 (0 = K after RoPE, 1 = V)][n_kv_heads][n_slots][head_dim]
- *    in the model's storage type; a "slot" holds one token position.  A prompt or a
+ *    in the model's storage type (bf16 models: K planes bfloat16, V planes IEEE half, both
+ *    2 bytes per element); a "slot" holds one token position.  A prompt or a
  *    rollout owns a contiguous range of slots given by its first slot (int64).
  *  - Index arrays are int32, slot numbers and token-buffer indices int64.
  *  - Device-side anomalies (an index outside its arena, a wait that ran out) set

@@ -23,6 +23,8 @@
 // transcendental.  Waits on mbarriers are bounded (see gemm_tc.cuh).
 #pragma once
 
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 #include "gemm_tc.cuh"
 #include "kernels_basic.cuh"
@@ -55,6 +57,17 @@ __device__ __forceinline__ void mma_bf16(float* c, uint32_t a0, uint32_t a1, uin
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// P V product with P and V in IEEE half (V is stored as half in the arenas, see qkv_post_kernel)
+__device__ __forceinline__ void mma_f16(float* c, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    const __half2 p = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&p);
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
@@ -98,7 +111,8 @@ template <int HD, bool FINAL>
 __global__ void __launch_bounds__(G_THREADS, 1)
 attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __restrict__ sd, int64_t n_slots, int Hq, int Hkv,
                   int layer, const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ group_row_start, RowGeom g,
-                  float scale_log2, PrefixPartial part, __nv_bfloat16* __restrict__ out, int32_t* err) {
+                  float scale_log2, PrefixPartial part, __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ out_lo,
+                  int32_t* err) {
     constexpr int KS = HD / 16;          // k-steps of Q K^T
     constexpr int NT = G_TK / 8;         // position n-tiles per stage
     constexpr int DT = HD / 8;           // dim n-tiles of the output
@@ -244,8 +258,8 @@ attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __
             float p[4];
 #pragma unroll
             for (int c = 0; c < 4; ++c) { p[c] = exp2_safe(s[nt][c], mrow[c >> 1]); lrow[c >> 1] += p[c]; }
-            pa[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p[0], p[1]);
-            pa[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p[2], p[3]);
+            pa[nt >> 1][(nt & 1) * 2 + 0] = pack_f16(p[0], p[1]);
+            pa[nt >> 1][(nt & 1) * 2 + 1] = pack_f16(p[2], p[3]);
         }
         // rows of V beyond the longest visible prefix of this CTA may be uninitialised memory: their P is 0, but
         // 0 * NaN would poison the sum, so positions >= max_len are never multiplied (k-steps past it are skipped)
@@ -268,8 +282,8 @@ attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __
                     const uint32_t m_hi = (p + 8 < valid_in_tile ? 0x0000ffffu : 0u) | (p + 9 < valid_in_tile ? 0xffff0000u : 0u);
                     b0 &= m_lo; b2 &= m_lo; b1 &= m_hi; b3 &= m_hi;
                 }
-                mma_bf16(o[2 * dp], pa[kk][0], pa[kk][1], pa[kk][2], pa[kk][3], b0, b1);
-                mma_bf16(o[2 * dp + 1], pa[kk][0], pa[kk][1], pa[kk][2], pa[kk][3], b2, b3);
+                mma_f16(o[2 * dp], pa[kk][0], pa[kk][1], pa[kk][2], pa[kk][3], b0, b1);
+                mma_f16(o[2 * dp + 1], pa[kk][0], pa[kk][1], pa[kk][2], pa[kk][3], b2, b3);
             }
         }
         __syncwarp();
@@ -295,8 +309,14 @@ attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __
         if (FINAL) {
             const float inv = lrow[i] > 0.f ? 1.f / lrow[i] : 0.f;
 #pragma unroll
-            for (int t = 0; t < DT; ++t)
-                *reinterpret_cast<uint32_t*>(out + rh * HD + t * 8 + (lane & 3) * 2) = pack_bf16(o[t][2 * i] * inv, o[t][2 * i + 1] * inv);
+            for (int t = 0; t < DT; ++t) {
+                const float y0 = o[t][2 * i] * inv, y1 = o[t][2 * i + 1] * inv;
+                const size_t at = rh * HD + t * 8 + (lane & 3) * 2;
+                *reinterpret_cast<uint32_t*>(out + at) = pack_bf16(y0, y1);
+                // rounding remainder, consumed as a second bf16 operand by the output projection
+                *reinterpret_cast<uint32_t*>(out_lo + at) = pack_bf16(y0 - __bfloat162float(__float2bfloat16_rn(y0)),
+                                                                      y1 - __bfloat162float(__float2bfloat16_rn(y1)));
+            }
         } else {
             const size_t ph = (size_t)my_part * part.stride + rh;
             if ((lane & 3) == 0) { part.m[ph] = mrow[i]; part.l[ph] = lrow[i]; }
@@ -506,8 +526,8 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
                 float p[4];
 #pragma unroll
                 for (int c = 0; c < 4; ++c) { p[c] = exp2_safe(s[mt][c], mh[c & 1]); lh[c & 1] += p[c]; }
-                const uint32_t b0 = movmatrix_t(pack_bf16(p[0], p[1]));
-                const uint32_t b1 = movmatrix_t(pack_bf16(p[2], p[3]));
+                const uint32_t b0 = movmatrix_t(pack_f16(p[0], p[1]));
+                const uint32_t b1 = movmatrix_t(pack_f16(p[2], p[3]));
                 const bool ragged = mt * 16 + 16 > valid;              // warp-uniform
 #pragma unroll
                 for (int dt = 0; dt < DT; ++dt) {
@@ -523,7 +543,7 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
                         const uint32_t m_hi = (pp + 8 < valid ? 0x0000ffffu : 0u) | (pp + 9 < valid ? 0xffff0000u : 0u);
                         a0 &= m_lo; a1 &= m_lo; a2 &= m_hi; a3 &= m_hi;
                     }
-                    mma_bf16(o[dt], a0, a1, a2, a3, b0, b1);
+                    mma_f16(o[dt], a0, a1, a2, a3, b0, b1);
                 }
             }
             ++consumed;
@@ -585,7 +605,7 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
 // ---------------------------------------------------------------------------------------------
 template <int HD>
 __global__ void __launch_bounds__(256) attn_merge_kernel(const StepDesc* __restrict__ sd, int Hq, RowGeom g, PrefixPartial part,
-                                                         __nv_bfloat16* __restrict__ out) {
+                                                         __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ out_lo) {
     constexpr int EPL = HD / 32;
     const int lane = threadIdx.x & 31;
     const size_t rh = (size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -622,9 +642,21 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const StepDesc* __restr
         }
     }
     const float inv = denom > 0.f ? 1.f / denom : 0.f;
+    float lo[EPL];
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) {
+        acc[e] *= inv;
+        lo[e] = acc[e] - __bfloat162float(__float2bfloat16_rn(acc[e]));     // rounding remainder: second operand of the O projection
+    }
     __nv_bfloat16* dst = out + rh * HD + lane * EPL;
-    if (EPL == 4) *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc[0] * inv, acc[1] * inv), pack_bf16(acc[2] * inv, acc[3] * inv));
-    else *reinterpret_cast<uint32_t*>(dst) = pack_bf16(acc[0] * inv, acc[1] * inv);
+    __nv_bfloat16* dst_lo = out_lo + rh * HD + lane * EPL;
+    if (EPL == 4) {
+        *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]));
+        *reinterpret_cast<uint2*>(dst_lo) = make_uint2(pack_bf16(lo[0], lo[1]), pack_bf16(lo[2], lo[3]));
+    } else {
+        *reinterpret_cast<uint32_t*>(dst) = pack_bf16(acc[0], acc[1]);
+        *reinterpret_cast<uint32_t*>(dst_lo) = pack_bf16(lo[0], lo[1]);
+    }
 }
 
 }  // namespace am

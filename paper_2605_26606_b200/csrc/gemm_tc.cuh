@@ -26,12 +26,16 @@ constexpr int UMMA_K = 16;
 constexpr int NUM_THREADS = 192;
 constexpr uint32_t WAIT_LIMIT = 1u << 24;
 
-__host__ __device__ constexpr int stage_bytes(int bn) { return (BM + bn) * BK * 2; }
-__host__ __device__ constexpr int num_stages(int bn) {
-    int s = (200 * 1024) / stage_bytes(bn);
+// dual: the A operand comes as two bf16 matrices (high part and rounding remainder) that are both multiplied with the
+// same weight tile, which removes the bf16 rounding of the activations from the product at the cost of a second MMA.
+__host__ __device__ constexpr int stage_bytes(int bn, bool dual) { return ((dual ? 2 : 1) * BM + bn) * BK * 2; }
+__host__ __device__ constexpr int num_stages(int bn, bool dual) {
+    int s = (200 * 1024) / stage_bytes(bn, dual);
     return s > 8 ? 8 : s;
 }
-__host__ __device__ constexpr int smem_bytes(int bn) { return num_stages(bn) * stage_bytes(bn) + 1024 /*align*/ + 256 /*barriers*/; }
+__host__ __device__ constexpr int smem_bytes(int bn, bool dual) {
+    return num_stages(bn, dual) * stage_bytes(bn, dual) + 1024 /*align*/ + 256 /*barriers*/;
+}
 
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -208,14 +212,16 @@ struct EpiSwiGLU {              // columns (2j, 2j+1) = (gate_j, up_j) -> out[ro
 // ---------------------------------------------------------------------------------------------
 // Kernel
 // ---------------------------------------------------------------------------------------------
-template <int BN, class Epi>
+template <int BN, bool DUAL, class Epi>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const StepDesc* __restrict__ sd,
-               int M, int N, int K, int splits, Epi epi, int32_t* err) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_a_lo,
+               const __grid_constant__ CUtensorMap map_w, const StepDesc* __restrict__ sd, int M, int N, int K, int splits, Epi epi,
+               int32_t* err) {
     if (sd != nullptr) M = sd->n_rows;          // live row count; the grid was sized for an upper bound
     epi.set_rows(M);
-    constexpr int STAGES = num_stages(BN);
-    constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
+    constexpr int STAGES = num_stages(BN, DUAL);
+    constexpr int A1_BYTES = BM * BK * 2;                    // one A tile
+    constexpr int A_BYTES = (DUAL ? 2 : 1) * A1_BYTES, B_BYTES = BN * BK * 2;
     constexpr uint32_t TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;
     extern __shared__ uint8_t smem_raw[];
     // tiles must start on a 1024-byte boundary for the 128-byte swizzle pattern
@@ -259,6 +265,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     const uint32_t sa = tiles_u32 + stage * (A_BYTES + B_BYTES), sb = sa + A_BYTES;
                     mbar_arrive_expect_tx(full0 + 8 * stage, A_BYTES + B_BYTES);
                     tma_load_2d(sa, &map_a, full0 + 8 * stage, kb * BK, m0);
+                    if (DUAL) tma_load_2d(sa + A1_BYTES, &map_a_lo, full0 + 8 * stage, kb * BK, m0);
                     tma_load_2d(sb, &map_w, full0 + 8 * stage, kb * BK, n0);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -286,6 +293,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     for (int kk = 0; kk < BK / UMMA_K; ++kk) {
                         // advancing 16 bf16 = 32 bytes inside the swizzle row: +2 in the (address >> 4) field
                         umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+                    }
+                    if (DUAL) {
+                        const uint64_t dl = make_smem_desc(sa + A1_BYTES);
+#pragma unroll
+                        for (int kk = 0; kk < BK / UMMA_K; ++kk) umma_bf16(d_tmem, dl + 2 * kk, db + 2 * kk, idesc, 1u);
                     }
                     umma_commit(empty0 + 8 * stage);          // frees the stage once these MMAs have read it
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -336,19 +348,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 }
 
 // Must run once per kernel instance before its first launch (raises the dynamic shared memory limit).
-template <int BN, class Epi>
+template <int BN, bool DUAL, class Epi>
 inline cudaError_t configure() {
-    return cudaFuncSetAttribute(gemm_tc_kernel<BN, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(BN));
+    return cudaFuncSetAttribute(gemm_tc_kernel<BN, DUAL, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(BN, DUAL));
 }
 
-// Host launcher.  map_w must have been encoded with box_rows = BN.
-template <int BN, class Epi>
-inline cudaError_t launch(cudaStream_t st, const CUtensorMap& map_a, const CUtensorMap& map_w, const StepDesc* sd, int M, int N,
-                          int K, int splits, Epi epi, int32_t* err, int num_sms) {
-    auto kern = gemm_tc_kernel<BN, Epi>;
+// Host launcher.  map_w must have been encoded with box_rows = BN; map_a_lo is ignored unless DUAL.
+template <int BN, bool DUAL, class Epi>
+inline cudaError_t launch(cudaStream_t st, const CUtensorMap& map_a, const CUtensorMap& map_a_lo, const CUtensorMap& map_w,
+                          const StepDesc* sd, int M, int N, int K, int splits, Epi epi, int32_t* err, int num_sms) {
+    auto kern = gemm_tc_kernel<BN, DUAL, Epi>;
     const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN) * splits;
     if (tiles == 0) return cudaSuccess;
-    kern<<<tiles < num_sms ? tiles : num_sms, NUM_THREADS, smem_bytes(BN), st>>>(map_a, map_w, sd, M, N, K, splits, epi, err);
+    kern<<<tiles < num_sms ? tiles : num_sms, NUM_THREADS, smem_bytes(BN, DUAL), st>>>(map_a, map_a_lo, map_w, sd, M, N, K, splits, epi, err);
     return cudaGetLastError();
 }
 

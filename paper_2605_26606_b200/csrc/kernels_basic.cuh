@@ -1,6 +1,8 @@
 // Row bookkeeping, embedding gather, RMSNorm, rotary tables, q/k/v post-processing, reward rule.
 #pragma once
 
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 
 namespace pc {
@@ -98,7 +100,8 @@ __global__ void rope_table_kernel(const StepDesc* __restrict__ sd, int half, dou
 // h[r, :] = E[token[r], :] (float residual stream); a[r, :] = RMSNorm(h[r, :]; gain) in storage type T.
 template <typename T>
 __global__ void embed_rmsnorm_kernel(const StepDesc* __restrict__ sd, int d, const int32_t* token, const T* __restrict__ embed,
-                                     const float* __restrict__ gain, float eps, float* __restrict__ h, T* __restrict__ a) {
+                                     const float* __restrict__ gain, float eps, float* __restrict__ h, T* __restrict__ a,
+                                     T* __restrict__ a_lo) {
     __shared__ float red[33];
     const int r = blockIdx.x;
     if (r >= sd->n_rows) return;
@@ -111,8 +114,11 @@ __global__ void embed_rmsnorm_kernel(const StepDesc* __restrict__ sd, int d, con
     }
     ss = block_sum(ss, red);
     const float rstd = rsqrtf(ss / (float)d + eps);
-    for (int i = threadIdx.x; i < d; i += blockDim.x)
-        a[(size_t)r * d + i] = from_f32<T>(h[(size_t)r * d + i] * rstd * gain[i]);
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        const float y = h[(size_t)r * d + i] * rstd * gain[i];
+        a[(size_t)r * d + i] = from_f32<T>(y);
+        if (a_lo != nullptr) a_lo[(size_t)r * d + i] = from_f32<T>(y - to_f32<T>(from_f32<T>(y)));
+    }
 }
 
 // K-slice sums left by a split GEMM: value(row, col) = sum over s < n of p[s * stride + row * ld + col], added in
@@ -133,12 +139,18 @@ template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16*
     *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
 }
 
+// Rounding remainder of a float4 after its conversion to bf16 (what a second, "low" bf16 operand carries).
+__device__ __forceinline__ float4 bf16_remainder(float4 v) {
+    return make_float4(v.x - __bfloat162float(__float2bfloat16_rn(v.x)), v.y - __bfloat162float(__float2bfloat16_rn(v.y)),
+                       v.z - __bfloat162float(__float2bfloat16_rn(v.z)), v.w - __bfloat162float(__float2bfloat16_rn(v.w)));
+}
+
 // One block of 256 threads per row; d is a multiple of 8 and at most 8192, so a thread keeps its <= 8 float4 of the
 // row in registers between the sum of squares and the scaling (one pass over global memory).
 template <typename T>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const StepDesc* __restrict__ sd, int d, float* __restrict__ h,
                                                       const int32_t* __restrict__ src, Partials pend, const float* __restrict__ gain,
-                                                      float eps, T* __restrict__ a) {
+                                                      float eps, T* __restrict__ a, T* __restrict__ a_lo) {
     __shared__ float red[33];
     const int r = blockIdx.x;
     if (sd != nullptr && r >= sd->n_rows) return;
@@ -170,8 +182,9 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const StepDesc* __restrict
         const int i = threadIdx.x + k * 256;
         if (i < n4) {
             const float4 gg = *reinterpret_cast<const float4*>(gain + 4 * i);
-            store4<T>(a + (size_t)r * d + 4 * i,
-                      make_float4(v[k].x * rstd * gg.x, v[k].y * rstd * gg.y, v[k].z * rstd * gg.z, v[k].w * rstd * gg.w));
+            const float4 y = make_float4(v[k].x * rstd * gg.x, v[k].y * rstd * gg.y, v[k].z * rstd * gg.z, v[k].w * rstd * gg.w);
+            store4<T>(a + (size_t)r * d + 4 * i, y);
+            if (a_lo != nullptr) store4<T>(a_lo + (size_t)r * d + 4 * i, bf16_remainder(y));
         }
     }
 }
@@ -228,6 +241,14 @@ __global__ void qkv_post_kernel(const StepDesc* __restrict__ sd, int Hq, int Hkv
     const int kvh = is_k ? head - Hq : head - Hq - Hkv;
     const int64_t plane = ((int64_t)layer * 2 + (is_k ? 0 : 1)) * Hkv + kvh;
     T* dst = reinterpret_cast<T*>(ar.base) + (plane * ar.n_slots + slot) * hd;
+    if (!is_k && sizeof(T) == 2) {
+        // 16-bit models keep V as IEEE half (same two bytes, three more mantissa bits than bfloat16): V is a linear map
+        // of a unit-RMS vector, far inside half's range, and its rounding is the largest single error source of the logits
+        __half* dv = reinterpret_cast<__half*>(dst);
+        dv[i] = __float2half_rn(x1);
+        dv[i + half] = __float2half_rn(x2);
+        return;
+    }
     dst[i] = from_f32<T>(x1);
     dst[i + half] = from_f32<T>(x2);
 }

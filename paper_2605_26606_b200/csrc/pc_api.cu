@@ -47,7 +47,7 @@ constexpr int kMaxSplits = 8;
 
 struct Carve {
     size_t h, a, qkv, q, attn, act, logits, rope, pos, wslot, warena, p_start, p_len, s_start, s_len, token, last_row,
-        part_m, part_l, part_o, res_part, step_desc, step_counter, sample_scratch, total;
+        part_m, part_l, part_o, res_part, step_desc, step_counter, sample_scratch, a_lo, attn_lo, total;
 };
 
 // A captured decode step, replayable for every step that fits the same upper bounds and reads the same arrays.
@@ -88,7 +88,7 @@ struct pc_ctx {
     std::vector<WMap> m_wqkv, m_wo, m_wgu, m_wdown;
     WMap m_lm;
     pc::Partials pend{nullptr, 0, 0, 0};     // residual K-slices produced by the last GEMM and not yet folded into h
-    CUtensorMap map_a, map_attn, map_act;
+    CUtensorMap map_a, map_attn, map_act, map_a_lo, map_attn_lo;
     int num_sms = 148;
     // TMA descriptors of the KV arenas, rebuilt when a call brings another arena
     const void* prompt_arena_ptr = nullptr; int64_t prompt_arena_slots = -1; CUtensorMap map_prompt_kv;
@@ -126,6 +126,8 @@ Carve carve(const pc_ctx* c, int max_rows, int max_prefill) {
     const size_t split_rows = std::min<size_t>(M, kSplitMaxRows) * kMaxSplits;      // rows x K-slices of a split GEMM
     v.qkv = take(std::max(M, split_rows) * c->n_qkv() * 4);
     v.res_part = take(split_rows * d.d_model * 4);
+    v.a_lo = take(M * d.d_model * eb);
+    v.attn_lo = take(M * c->q_dim() * eb);
     v.step_desc = take(sizeof(pc::StepDesc));
     v.step_counter = take(4);
     v.sample_scratch = take((size_t)std::max(max_rows, 1) * pc::SAMPLE_MAX_CHUNKS * sizeof(pc::Top2Rec));
@@ -193,10 +195,18 @@ GemmPlan plan_gemm(const pc_ctx* c, const WMap& w, int M, bool may_split) {
     return p;
 }
 
+// map_a_lo != nullptr: the activations come as a high bf16 part and its rounding remainder, both multiplied with the
+// weights (used for the projections whose input rounding would otherwise dominate the logit error).
 template <class Epi>
-int gemm_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, const CUtensorMap& map_a, const WMap& w, int M, GemmPlan p, Epi epi) {
-    cudaError_t e = p.wide ? pc::tc::launch<256>(st, map_a, w.wide, sd, M, w.N, w.K, p.splits, epi, c->err, c->num_sms)
-                           : pc::tc::launch<64>(st, map_a, w.narrow, sd, M, w.N, w.K, p.splits, epi, c->err, c->num_sms);
+int gemm_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, const CUtensorMap& map_a, const CUtensorMap* map_a_lo, const WMap& w,
+              int M, GemmPlan p, Epi epi) {
+    cudaError_t e;
+    if (map_a_lo != nullptr)
+        e = p.wide ? pc::tc::launch<256, true>(st, map_a, *map_a_lo, w.wide, sd, M, w.N, w.K, p.splits, epi, c->err, c->num_sms)
+                   : pc::tc::launch<64, true>(st, map_a, *map_a_lo, w.narrow, sd, M, w.N, w.K, p.splits, epi, c->err, c->num_sms);
+    else
+        e = p.wide ? pc::tc::launch<256, false>(st, map_a, map_a, w.wide, sd, M, w.N, w.K, p.splits, epi, c->err, c->num_sms)
+                   : pc::tc::launch<64, false>(st, map_a, map_a, w.narrow, sd, M, w.N, w.K, p.splits, epi, c->err, c->num_sms);
     if (e != cudaSuccess) return cuda_fail(e, "tensor-core gemm");
     return PC_OK;
 }
@@ -246,14 +256,18 @@ cudaError_t configure_attention() {
 }
 cudaError_t configure_kernels() {
     using namespace pc;
-    cudaError_t e = tc::configure<256, tc::EpiPartial>();
-    if (e == cudaSuccess) e = tc::configure<64, tc::EpiPartial>();
-    if (e == cudaSuccess) e = tc::configure<256, tc::EpiResidual>();
-    if (e == cudaSuccess) e = tc::configure<64, tc::EpiResidual>();
-    if (e == cudaSuccess) e = tc::configure<256, tc::EpiSwiGLU>();
-    if (e == cudaSuccess) e = tc::configure<64, tc::EpiSwiGLU>();
-    if (e == cudaSuccess) e = tc::configure<256, tc::EpiStoreF32>();
-    if (e == cudaSuccess) e = tc::configure<64, tc::EpiStoreF32>();
+    cudaError_t e = tc::configure<256, true, tc::EpiPartial>();
+    if (e == cudaSuccess) e = tc::configure<64, true, tc::EpiPartial>();
+    if (e == cudaSuccess) e = tc::configure<256, false, tc::EpiPartial>();
+    if (e == cudaSuccess) e = tc::configure<64, false, tc::EpiPartial>();
+    if (e == cudaSuccess) e = tc::configure<256, true, tc::EpiResidual>();
+    if (e == cudaSuccess) e = tc::configure<64, true, tc::EpiResidual>();
+    if (e == cudaSuccess) e = tc::configure<256, false, tc::EpiResidual>();
+    if (e == cudaSuccess) e = tc::configure<64, false, tc::EpiResidual>();
+    if (e == cudaSuccess) e = tc::configure<256, false, tc::EpiSwiGLU>();
+    if (e == cudaSuccess) e = tc::configure<64, false, tc::EpiSwiGLU>();
+    if (e == cudaSuccess) e = tc::configure<256, true, tc::EpiStoreF32>();
+    if (e == cudaSuccess) e = tc::configure<64, true, tc::EpiStoreF32>();
     if (e == cudaSuccess) e = configure_attention<128>();
     if (e == cudaSuccess) e = configure_attention<64>();
     return e;
@@ -262,6 +276,7 @@ cudaError_t configure_kernels() {
 template <int HD>
 int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, int layer, const AttnPlan& plan, pc::KvArena prompt_arena,
                    pc::KvArena suffix_arena, const __nv_bfloat16* q, __nv_bfloat16* attn, bool profile) {
+    __nv_bfloat16* attn_lo = reinterpret_cast<__nv_bfloat16*>(c->ws + c->cv.attn_lo);
     using namespace pc;
     const pc_model_desc& d = c->d;
     const RowGeom g = geom(c);
@@ -279,20 +294,20 @@ int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, in
     if (plan.prefill) {
         am::attn_group_kernel<HD, true><<<ggrid, am::G_THREADS, am::group_smem_bytes<HD>(), st>>>(
             c->map_prompt_kv, sd, prompt_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, plan.group_row_start, g, scale_log2,
-            part, attn, c->err);
+            part, attn, attn_lo, c->err);
         count_launches(1);
         return PC_OK;
     }
     am::attn_group_kernel<HD, false><<<ggrid, am::G_THREADS, am::group_smem_bytes<HD>(), st>>>(
         c->map_prompt_kv, sd, prompt_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, plan.group_row_start, g, scale_log2, part,
-        attn, c->err);
+        attn, attn_lo, c->err);
     const int items = M * d.n_kv_heads * (part.chunk_tiles > 0 ? am::MAX_SUFFIX_CHUNKS : 1);
     const int sgrid = std::min(c->num_sms, (items + am::S_WARPS - 1) / am::S_WARPS);
     if (profile) cudaEventRecord(c->prof_start, st);
     am::attn_suffix_kernel<HD><<<sgrid, am::S_WARPS * 32, am::suffix_smem_bytes<HD>(), st>>>(
         c->map_suffix_kv, sd, suffix_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, g, scale_log2, part, c->err);
     if (profile) cudaEventRecord(c->prof_stop, st);
-    am::attn_merge_kernel<HD><<<(M * d.n_q_heads + 7) / 8, 256, 0, st>>>(sd, d.n_q_heads, g, part, attn);
+    am::attn_merge_kernel<HD><<<(M * d.n_q_heads + 7) / 8, 256, 0, st>>>(sd, d.n_q_heads, g, part, attn, attn_lo);
     count_launches(3);
     return PC_OK;
 }
@@ -312,6 +327,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
     T* q = reinterpret_cast<T*>(w + c->cv.q);
     T* attn = reinterpret_cast<T*>(w + c->cv.attn);
     T* act = reinterpret_cast<T*>(w + c->cv.act);
+    T* a_lo = kF32 ? nullptr : reinterpret_cast<T*>(w + c->cv.a_lo);          // rounding remainders (bf16 models only)
     float2* rope = reinterpret_cast<float2*>(w + c->cv.rope);
     const RowGeom g = geom(c);
     const int half = d.head_dim / 2;
@@ -328,12 +344,12 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
 
     rope_table_kernel<<<(M * half + 255) / 256, 256, 0, st>>>(sd, half, (double)d.rope_theta, g.pos, rope);
     embed_rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, g.token, reinterpret_cast<const T*>(c->embed), c->attn_norm[0],
-                                               d.rms_eps, h, a);
+                                               d.rms_eps, h, a, a_lo);
     count_launches(2);
     PC_CUDA_CHECK_LAUNCH("embed_rmsnorm");
     for (int l = 0; l < d.n_layers; ++l) {
         if (l > 0) {
-            rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, h, nullptr, pend, c->attn_norm[l], d.rms_eps, a);
+            rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, h, nullptr, pend, c->attn_norm[l], d.rms_eps, a, a_lo);
             pend = none;
             count_launches(1);
         }
@@ -345,7 +361,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
         } else {
             const GemmPlan gp = plan_gemm(c, c->m_wqkv[l], M, true);
             qkv_parts.n = gp.splits;
-            if (int rc = gemm_bf16(c, st, sd, c->map_a, c->m_wqkv[l], M, gp, tc::EpiPartial{qkv, c->n_qkv(), qkv_parts.stride})) return rc;
+            if (int rc = gemm_bf16(c, st, sd, c->map_a, &c->map_a_lo, c->m_wqkv[l], M, gp, tc::EpiPartial{qkv, c->n_qkv(), qkv_parts.stride})) return rc;
         }
         qkv_post_kernel<T><<<dim3(M, d.n_q_heads + 2 * d.n_kv_heads), half, 0, st>>>(
             sd, d.n_q_heads, d.n_kv_heads, d.head_dim, l, qkv_parts, bias, d.qk_norm ? c->q_norm[l] : nullptr,
@@ -369,13 +385,13 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
             if (rc) return rc;
             const GemmPlan gp = plan_gemm(c, c->m_wo[l], M, true);
             if (gp.splits == 1) {
-                if (int rc2 = gemm_bf16(c, st, sd, c->map_attn, c->m_wo[l], M, gp, tc::EpiResidual{h, d.d_model})) return rc2;
+                if (int rc2 = gemm_bf16(c, st, sd, c->map_attn, &c->map_attn_lo, c->m_wo[l], M, gp, tc::EpiResidual{h, d.d_model})) return rc2;
             } else {
                 pend = Partials{res_part, gp.splits, (size_t)M * d.d_model, d.d_model};
-                if (int rc2 = gemm_bf16(c, st, sd, c->map_attn, c->m_wo[l], M, gp, tc::EpiPartial{res_part, d.d_model, pend.stride})) return rc2;
+                if (int rc2 = gemm_bf16(c, st, sd, c->map_attn, &c->map_attn_lo, c->m_wo[l], M, gp, tc::EpiPartial{res_part, d.d_model, pend.stride})) return rc2;
             }
         }
-        rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a);
+        rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a, nullptr);
         pend = none;
         count_launches(2);
         if constexpr (kF32) {
@@ -383,14 +399,14 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
                                 EpiSwiGLU<T>{act, d.d_ff});
             launch_gemm_simt<T>(st, sd, act, reinterpret_cast<const T*>(c->w_down[l]), M, d.d_model, d.d_ff, EpiResidual{h, d.d_model});
         } else {
-            if (int rc = gemm_bf16(c, st, sd, c->map_a, c->m_wgu[l], M, plan_gemm(c, c->m_wgu[l], M, false), tc::EpiSwiGLU{act, d.d_ff}))
+            if (int rc = gemm_bf16(c, st, sd, c->map_a, nullptr, c->m_wgu[l], M, plan_gemm(c, c->m_wgu[l], M, false), tc::EpiSwiGLU{act, d.d_ff}))
                 return rc;
             const GemmPlan gp = plan_gemm(c, c->m_wdown[l], M, true);
             if (gp.splits == 1) {
-                if (int rc = gemm_bf16(c, st, sd, c->map_act, c->m_wdown[l], M, gp, tc::EpiResidual{h, d.d_model})) return rc;
+                if (int rc = gemm_bf16(c, st, sd, c->map_act, nullptr, c->m_wdown[l], M, gp, tc::EpiResidual{h, d.d_model})) return rc;
             } else {
                 pend = Partials{res_part, gp.splits, (size_t)M * d.d_model, d.d_model};
-                if (int rc = gemm_bf16(c, st, sd, c->map_act, c->m_wdown[l], M, gp, tc::EpiPartial{res_part, d.d_model, pend.stride})) return rc;
+                if (int rc = gemm_bf16(c, st, sd, c->map_act, nullptr, c->m_wdown[l], M, gp, tc::EpiPartial{res_part, d.d_model, pend.stride})) return rc;
             }
         }
         count_launches(2);
@@ -407,13 +423,14 @@ int run_lm_head(pc_ctx* c, cudaStream_t st, int n, const pc::StepDesc* sd, const
     const pc_model_desc& d = c->d;
     float* h = reinterpret_cast<float*>(c->ws + c->cv.h);
     T* a = reinterpret_cast<T*>(c->ws + c->cv.a);
-    rmsnorm_kernel<T><<<n, 256, 0, st>>>(sd, d.d_model, h, src, c->pend, c->final_norm, d.rms_eps, a);
+    T* a_lo = std::is_same<T, float>::value ? nullptr : reinterpret_cast<T*>(c->ws + c->cv.a_lo);
+    rmsnorm_kernel<T><<<n, 256, 0, st>>>(sd, d.d_model, h, src, c->pend, c->final_norm, d.rms_eps, a, a_lo);
     c->pend = pc::Partials{nullptr, 0, 0, 0};
     if constexpr (std::is_same<T, float>::value) {
         const T* wlm = reinterpret_cast<const T*>(d.tied_embed ? c->embed : c->lm_head);
         launch_gemm_simt<T>(st, sd, a, wlm, n, d.vocab, d.d_model, EpiStoreF32{logits, d.vocab, nullptr});
     } else {
-        if (int rc = gemm_bf16(c, st, sd, c->map_a, c->m_lm, n, plan_gemm(c, c->m_lm, n, false), tc::EpiStoreF32{logits, d.vocab, nullptr}))
+        if (int rc = gemm_bf16(c, st, sd, c->map_a, &c->map_a_lo, c->m_lm, n, plan_gemm(c, c->m_lm, n, false), tc::EpiStoreF32{logits, d.vocab, nullptr}))
             return rc;
     }
     count_launches(2);
@@ -556,7 +573,9 @@ int pc_set_workspace(pc_ctx* ctx, void* dev_ws, size_t bytes, int max_rows, int 
         char* w = ctx->ws;
         if (!pc::make_bf16_map(&ctx->map_a, w + cv.a, cap, ctx->d.d_model, 128) ||
             !pc::make_bf16_map(&ctx->map_attn, w + cv.attn, cap, ctx->q_dim(), 128) ||
-            !pc::make_bf16_map(&ctx->map_act, w + cv.act, cap, ctx->d.d_ff, 128)) {
+            !pc::make_bf16_map(&ctx->map_act, w + cv.act, cap, ctx->d.d_ff, 128) ||
+            !pc::make_bf16_map(&ctx->map_a_lo, w + cv.a_lo, cap, ctx->d.d_model, 128) ||
+            !pc::make_bf16_map(&ctx->map_attn_lo, w + cv.attn_lo, cap, ctx->q_dim(), 128)) {
             ctx->ws = nullptr;
             g_cuda_error = "cuTensorMapEncodeTiled failed for an activation buffer";
             return PC_ERR_CUDA;

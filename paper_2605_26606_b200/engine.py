@@ -94,6 +94,7 @@ class RolloutEngine:
         self._arenas: Dict[str, Optional[torch.Tensor]] = {}
         self.profile_every = 0
         self.use_graphs = True
+        self.record_pilot_logits: Optional[dict] = None     # {decode step: None} -> filled during the pilot stage
         self.profile_layer = m.n_layers // 2
         self.profile_samples: List[tuple] = []      # (start event, stop event, rows, suffix slots read per row)
 
@@ -284,7 +285,7 @@ class RolloutEngine:
         b_t = P if b_t is None else b_t
         self.prefill()
         pp, rr = np.repeat(np.arange(P), k), np.tile(np.arange(k), P)
-        n_tok = self.run_stage(pp, rr)
+        n_tok = self.run_stage(pp, rr, record_logits=self.record_pilot_logits)
         pilot_count = torch.full((P,), k, dtype=torch.int32, device=self.device)
         B.pc_reward_last_token(P * G, self.tokens, self.last_index, self.thresholds, self.rewards)
         B.pc_group_stats(P, self.rewards, self.group_start, pilot_count, self.pilot_n, self.pilot_success, self.pilot_mean,
