@@ -346,13 +346,14 @@ template <int HD> constexpr int suffix_smem_bytes() {
 // With few rollouts there are about as many (rollout, KV head) streams as warps on the GPU, and one stream more than
 // warps doubles the kernel's time.  The suffix of a rollout is therefore cut into ranges of tiles ("chunks") that
 // are spread over the warps; every chunk leaves its own record.
-__device__ __forceinline__ int suffix_chunk_len(int ntiles, int chunk_tiles) {     // tiles per chunk of a row with ntiles tiles
-    return chunk_tiles <= 0 ? max(ntiles, 1) : max(chunk_tiles, (ntiles + MAX_SUFFIX_CHUNKS - 1) / MAX_SUFFIX_CHUNKS);
+// Tiles per chunk for a step whose longest suffix has max_slen slots: at least chunk_tiles, and large enough that no
+// row needs more than MAX_SUFFIX_CHUNKS chunks.  The same value serves every row of the step.
+__device__ __forceinline__ int suffix_chunk_len(int max_slen, int chunk_tiles) {
+    const int max_tiles = (max_slen + S_TP - 1) / S_TP;
+    return chunk_tiles <= 0 ? max(max_tiles, 1) : max(chunk_tiles, (max_tiles + MAX_SUFFIX_CHUNKS - 1) / MAX_SUFFIX_CHUNKS);
 }
-__device__ __forceinline__ int suffix_chunks(int n, int chunk_tiles) {             // records a row with n suffix slots leaves
+__device__ __forceinline__ int suffix_chunks(int n, int ct) {             // records a row with n suffix slots leaves
     const int ntiles = (n + S_TP - 1) / S_TP;
-    if (ntiles == 0) return 0;
-    const int ct = suffix_chunk_len(ntiles, chunk_tiles);
     return (ntiles + ct - 1) / ct;
 }
 
@@ -384,14 +385,15 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
     __syncthreads();
 
     // work unit u = (item, chunk), item = (row, kv head); units of one item are consecutive, so they land on different warps
-    const int cpi = part.chunk_tiles > 0 ? MAX_SUFFIX_CHUNKS : 1;       // unit slots per item
+    const int max_slen = *g.max_slen;
+    const int ct = suffix_chunk_len(max_slen, part.chunk_tiles);                                   // tiles per chunk
+    const int cpi = part.chunk_tiles > 0 ? max(1, suffix_chunks(max_slen, ct)) : 1;               // unit slots per item
     const int n_items = sd->n_rows * Hkv * cpi;
     const int item_stride = gridDim.x * S_WARPS;
     const int first_item = blockIdx.x * S_WARPS + warp;
     // tile range [t0, t1) of unit u for a row with n suffix slots; empty when the row has fewer chunks
     auto unit_range = [&](int u, int n, int& t0, int& t1) {
         const int ntiles = (n + S_TP - 1) / S_TP;
-        const int ct = suffix_chunk_len(ntiles, part.chunk_tiles);
         t0 = min(ntiles, (u % cpi) * ct);
         t1 = min(ntiles, t0 + ct);
     };
@@ -612,7 +614,7 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const StepDesc* __restr
     if (rh >= (size_t)sd->n_rows * Hq) return;
     const int row = (int)(rh / Hq);
     // a row without suffix slots still has its (empty) record 0 when the suffix is not cut into chunks
-    const int n_sfx = part.chunk_tiles > 0 ? suffix_chunks(g.s_len[row], part.chunk_tiles) : 1;
+    const int n_sfx = part.chunk_tiles > 0 ? suffix_chunks(g.s_len[row], suffix_chunk_len(*g.max_slen, part.chunk_tiles)) : 1;
     const int n_rec = part.n_parts + n_sfx;
     float mi[MAX_RECORDS], li[MAX_RECORDS];
     float M = -INFINITY;

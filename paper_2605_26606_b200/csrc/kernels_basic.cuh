@@ -17,14 +17,17 @@ struct RowGeom {
     int64_t* s_start;    // [M] first suffix-arena slot attended
     int32_t* s_len;      // [M] number of suffix-arena slots attended
     int32_t* token;      // [M] input token id
+    int32_t* max_slen;   // [1] largest s_len of the step (decode only)
 };
 
-__global__ void set_step_desc(StepDesc* sd, int n_rows, int n_groups, int max_group_rows) {
+__global__ void set_step_desc(StepDesc* sd, int n_rows, int n_groups, int max_group_rows, int32_t* max_slen) {
+    *max_slen = 0;
     sd->n_rows = n_rows; sd->n_groups = n_groups; sd->max_group_rows = max_group_rows; sd->reserved = 0;
     sd->row_off = 0; sd->group_off = 0;
 }
 // First node of a captured decode step: takes the next descriptor of the caller's schedule.
-__global__ void load_step_desc(const StepDesc* __restrict__ steps, int32_t* counter, StepDesc* sd) {
+__global__ void load_step_desc(const StepDesc* __restrict__ steps, int32_t* counter, StepDesc* sd, int32_t* max_slen) {
+    *max_slen = 0;
     const int i = *counter;
     *sd = steps[i];
     *counter = i + 1;
@@ -59,6 +62,7 @@ __global__ void prep_decode_rows(const StepDesc* __restrict__ sd, const int32_t*
     g.p_len[r] = ok ? Lp : 0;
     g.s_start[r] = ss;
     g.s_len[r] = ok ? step + 1 : 0;
+    if (ok) atomicMax(g.max_slen, step + 1);
 }
 
 // Prefill: packed token t of prompt p at position i attends prompt slots [start_p, start_p + i + 1).

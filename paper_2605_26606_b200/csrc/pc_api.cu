@@ -47,7 +47,7 @@ constexpr int kMaxSplits = 8;
 
 struct Carve {
     size_t h, a, qkv, q, attn, act, logits, rope, pos, wslot, warena, p_start, p_len, s_start, s_len, token, last_row,
-        part_m, part_l, part_o, res_part, step_desc, step_counter, sample_scratch, a_lo, attn_lo, total;
+        part_m, part_l, part_o, res_part, step_desc, step_counter, max_slen, sample_scratch, a_lo, attn_lo, total;
 };
 
 // A captured decode step, replayable for every step that fits the same upper bounds and reads the same arrays.
@@ -130,6 +130,7 @@ Carve carve(const pc_ctx* c, int max_rows, int max_prefill) {
     v.attn_lo = take(M * c->q_dim() * eb);
     v.step_desc = take(sizeof(pc::StepDesc));
     v.step_counter = take(4);
+    v.max_slen = take(4);
     v.sample_scratch = take((size_t)std::max(max_rows, 1) * pc::SAMPLE_MAX_CHUNKS * sizeof(pc::Top2Rec));
     v.q = take(M * c->q_dim() * eb);
     v.attn = take(M * c->q_dim() * eb);
@@ -165,6 +166,7 @@ pc::RowGeom geom(const pc_ctx* c) {
     g.s_start = reinterpret_cast<int64_t*>(w + c->cv.s_start);
     g.s_len = reinterpret_cast<int32_t*>(w + c->cv.s_len);
     g.token = reinterpret_cast<int32_t*>(w + c->cv.token);
+    g.max_slen = reinterpret_cast<int32_t*>(w + c->cv.max_slen);
     return g;
 }
 
@@ -599,7 +601,7 @@ int pc_prefill_shared(pc_ctx* ctx, void* stream, int n_prompts, const int32_t* p
     const pc::RowGeom g = geom(ctx);
     int32_t* last_row = reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.last_row);
     pc::StepDesc* sd = reinterpret_cast<pc::StepDesc*>(ctx->ws + ctx->cv.step_desc);
-    pc::set_step_desc<<<1, 1, 0, st>>>(sd, total_tokens, n_prompts, max_prompt_len);
+    pc::set_step_desc<<<1, 1, 0, st>>>(sd, total_tokens, n_prompts, max_prompt_len, g.max_slen);
     pc::prep_prefill_rows<<<n_prompts, 256, 0, st>>>(n_prompts, prompt_tokens, prompt_offsets, prompt_kv_start, prompt_slots,
                                                      ctx->d.vocab, g, last_row, ctx->err);
     count_launches(2);
@@ -721,7 +723,8 @@ int pc_decode_step(pc_ctx* ctx, void* stream, int n_rows, const int32_t* row_pro
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (ctx->d.dtype == PC_DTYPE_BF16)
         if (int rc = arena_maps(ctx, prompt_kv, prompt_slots, suffix_kv, suffix_slots)) return rc;
-    pc::set_step_desc<<<1, 1, 0, st>>>(reinterpret_cast<pc::StepDesc*>(ctx->ws + ctx->cv.step_desc), n_rows, n_groups, max_group_rows);
+    pc::set_step_desc<<<1, 1, 0, st>>>(reinterpret_cast<pc::StepDesc*>(ctx->ws + ctx->cv.step_desc), n_rows, n_groups, max_group_rows,
+                                       reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.max_slen));
     count_launches(1);
     return decode_launches(ctx, st, n_rows, n_groups, max_group_rows, a, logits_out);
 }
@@ -757,7 +760,8 @@ int pc_decode_run(pc_ctx* ctx, void* stream, int n_steps, const pc_step_desc* st
     if (e != cudaSuccess) return cuda_fail(e, "reset step counter");
     for (int s = 0; s < n_steps; ++s) {
         if (steps_host[s].n_rows == 0) {          // keep the device counter in step with the host loop
-            pc::load_step_desc<<<1, 1, 0, st>>>(reinterpret_cast<const pc::StepDesc*>(steps_dev), counter, sd);
+            pc::load_step_desc<<<1, 1, 0, st>>>(reinterpret_cast<const pc::StepDesc*>(steps_dev), counter, sd,
+                                                reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.max_slen));
             count_launches(1);
             continue;
         }
@@ -781,7 +785,8 @@ int pc_decode_run(pc_ctx* ctx, void* stream, int n_steps, const pc_step_desc* st
             cudaStream_t cs = ctx->capture_stream;
             e = cudaStreamBeginCapture(cs, cudaStreamCaptureModeThreadLocal);
             if (e != cudaSuccess) return cuda_fail(e, "begin graph capture");
-            pc::load_step_desc<<<1, 1, 0, cs>>>(reinterpret_cast<const pc::StepDesc*>(steps_dev), counter, sd);
+            pc::load_step_desc<<<1, 1, 0, cs>>>(reinterpret_cast<const pc::StepDesc*>(steps_dev), counter, sd,
+                                                reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.max_slen));
             count_launches(1);
             const int rc = decode_launches(ctx, cs, m_bound, groups_bound, group_rows_bound, a, nullptr);
             e = cudaStreamEndCapture(cs, &graph);
