@@ -150,3 +150,21 @@ def test_graph_replay_equals_step_by_step(model):
             if a["generated"][p, i]:
                 assert np.array_equal(a["tokens"][p][i], b["tokens"][p][i])
     assert np.array_equal(a["advantages"], b["advantages"])
+
+
+@pytest.mark.parametrize("base", [wl.QWEN3_8B, wl.QWEN3_14B], ids=lambda m: m.name)
+def test_qwen3_widths_two_layers_teacher_forced(base):
+    """The 8B / 14B layer shapes (d 4096 / 5120, 32/8 and 40/8 heads, QK-norm, untied head, theta 1e6) with two layers and a
+    reduced vocabulary, so that the oracle stays cheap: logits within 5e-2, tokens identical outside the 1e-1 gap."""
+    model = dataclasses.replace(base, name=base.name + "-2l", n_layers=2, vocab=8192)
+    w = dataclasses.replace(wl.WORKLOADS["config0"], model=model, n_prompts=2, prompt_len_lo=40, prompt_len_hi=90, group_size=5,
+                            n_pilot=5, max_new=6, cap_lo=2, cap_hi=6, data_seed=4, forced_explicit=None)
+    weights = wl.gen_weights(model, seed=3, threads=4)
+    batch = wl.gen_batch(w)
+    dec = Decoder(model, weights)
+    P, G = w.n_prompts, w.group_size
+    prompts, rollouts = np.repeat(np.arange(P), G), np.tile(np.arange(G), P)
+    ref = oracle_group_tokens(dec, w, batch, prompts, rollouts)
+    eng = RolloutEngine(model, weights, max_rows=P * G, max_prefill_tokens=int(batch.prompt_offsets[-1]))
+    worst, n_cmp, n_exempt = teacher_forced_compare(eng, w, batch, ref, prompts, rollouts, logit_tol=5e-2, gap_tol=1e-1)
+    assert n_cmp == int(batch.caps.sum())
