@@ -179,6 +179,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="config2", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--also-grpo", action="store_true",
+                    help="additionally time one step with k = G (all P*G rollouts concurrent, no filter) and report it as grpo_mode")
     ap.add_argument("--probe", default=None, metavar="rows=R,suffix=S,steps=N,prompt=L",
                     help="time N decode steps of R rollouts (16 groups) that already hold S suffix tokens, then exit")
     args = ap.parse_args()
@@ -313,6 +315,29 @@ def main():
     }
     if cpu_baseline is not None:
         line["cpu_baseline"] = cpu_baseline
+    if args.also_grpo and world == 1:
+        # every rollout of every group at once (what plain GRPO generates for the same prompts): same kernels, k = G
+        wg = dataclasses.replace(w, n_pilot=G)
+        del eng
+        torch.cuda.empty_cache()
+        eng2 = RolloutEngine(wg.model, weights, max_rows=P * G, max_prefill_tokens=total_prompt, device=dev)
+        eng2.load_batch(wg, batch)
+        eng2.run_device()                       # warm-up (graph capture, allocator)
+        torch.cuda.synchronize()
+        eng2.load_batch(wg, batch)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        _, n_tok = eng2.run_device()
+        e1.record()
+        torch.cuda.synchronize()
+        eng2.check_error_flag()
+        ms = e0.elapsed_time(e1)
+        cg = batch.caps.astype(np.float64)
+        b = (float(np.sum((cg - 1) * cg / 2.0)) + float(np.sum(cg - 1))) * kv_tok \
+            + float(sum((batch.caps[p].max() - 1) * batch.prompt_lens[p] for p in range(P))) * kv_tok \
+            + float(batch.caps.max() - 1) * m.weight_bytes_per_decode_step()
+        line["grpo_mode"] = {"rows": P * G, "tokens": n_tok, "ms_per_step": ms, "tokens_per_s": n_tok / (ms * 1e-3),
+                             "hbm_bytes_per_step": b, "hbm_frac_of_measured": b / (ms * 1e-3) / 1e9 / peak}
     print(json.dumps(line), flush=True)
 
 

@@ -60,6 +60,76 @@ __device__ __forceinline__ Top2 top2_warp_reduce(Top2 t) {
     return t;
 }
 
+// Scores the 4-id blocks b0, b0 + stride, ... < b1 of one row and folds them into t.
+//
+// Almost every candidate is rejected without evaluating its Gumbel noise: v can enter the thread's top two only if
+// logit_v / T + g_v > t.second, hence only if g_v > t.second - lmax (lmax >= every logit_v / T of the range), i.e. only if
+// 1 - u_v < 1 - exp(-exp(-(t.second - lmax))).  u_v is an affine function of the random word, so this is one integer
+// comparison per candidate against a bound that is refreshed whenever the thread's second-best score rises.  The bound
+// carries a slack far above the float error of its evaluation, and candidates that pass are scored exactly as before, so
+// the result is identical to scoring everything.
+__device__ __forceinline__ void scan_blocks(Top2& t, const float* __restrict__ lg, int vocab, int b_begin, int b_end,
+                                            float temperature, float lmax, uint32_t c1, uint32_t c2, uint32_t c3,
+                                            uint32_t k0, uint32_t k1) {
+    // The bound uses the largest second-best score of the warp: the final second-best is at least that, so a candidate
+    // below it can change neither the winner nor the gap.  Sharing it keeps a warp from entering the scoring branch
+    // for a lane or two on almost every draw.  Trip counts are warp-uniform (the shuffles need every lane).
+    uint32_t pass_below = 0xffffffffu;          // a candidate is scored iff (2^23 - (w >> 9)) < pass_below
+    float bound_for = -INFINITY;                // warp-wide score the bound was computed for
+    const int lane = threadIdx.x & 31;
+    for (int base = b_begin + (threadIdx.x - lane); base < b_end; base += blockDim.x) {
+        const float ws = warp_max(t.second);
+        if (ws > bound_for) {
+            bound_for = ws;
+            const float T = ws - lmax - 1e-3f * (1.f + fabsf(ws) + fabsf(lmax));     // conservative
+            // (1 - U0) * 2^23 with U0 = exp(-exp(-T)); expm1f keeps the relative accuracy when U0 is close to 1
+            const float d = -expm1f(-expf(-T)) * 8388608.f;
+            pass_below = d >= 8388608.f ? 0xffffffffu : (uint32_t)(d * 1.001f + 2.f);
+        }
+        const int b = base + lane;
+        if (b < b_end) {
+            const Philox4 w = philox4x32_10((uint32_t)b, c1, c2, c3, k0, k1);
+            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int v = b * 4 + i;
+                if (v < vocab && (8388608u - (ww[i] >> 9)) < pass_below)
+                    top2_push(t, lg[v] / temperature + gumbel_from_word(ww[i]), v);
+            }
+        }
+    }
+}
+
+// Largest logit / T over the blocks a thread block will scan (block-wide); `red` is 33 floats of shared memory.
+__device__ __forceinline__ float range_max(const float* __restrict__ lg, int v0, int v1, float temperature, float* red) {
+    float m = -INFINITY;
+    // 16-byte loads, four in flight per thread: a row is hundreds of KB and one scalar load per thread at a time would
+    // leave the pass bound by memory latency
+    int v = v0;
+    while (v < v1 && (reinterpret_cast<uintptr_t>(lg + v) & 15u) != 0) { if (threadIdx.x == 0) m = fmaxf(m, lg[v]); ++v; }
+    const int n4 = (v1 - v) >> 2;
+    const float4* p4 = reinterpret_cast<const float4*>(lg + v);
+    int i = threadIdx.x;
+    for (; i + 3 * (int)blockDim.x < n4; i += 4 * blockDim.x) {
+        const float4 a = p4[i], b = p4[i + blockDim.x], c = p4[i + 2 * blockDim.x], d = p4[i + 3 * blockDim.x];
+        m = fmaxf(m, fmaxf(fmaxf(fmaxf(a.x, a.y), fmaxf(a.z, a.w)), fmaxf(fmaxf(b.x, b.y), fmaxf(b.z, b.w))));
+        m = fmaxf(m, fmaxf(fmaxf(fmaxf(c.x, c.y), fmaxf(c.z, c.w)), fmaxf(fmaxf(d.x, d.y), fmaxf(d.z, d.w))));
+    }
+    for (; i < n4; i += blockDim.x) { const float4 a = p4[i]; m = fmaxf(m, fmaxf(fmaxf(a.x, a.y), fmaxf(a.z, a.w))); }
+    for (int t = v + 4 * n4 + threadIdx.x; t < v1; t += blockDim.x) m = fmaxf(m, lg[t]);
+    m = warp_max(m) / temperature;          // temperature > 0: the division is monotone
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) red[warp] = m;
+    __syncthreads();
+    if (warp == 0) {
+        float x = lane < (int)(blockDim.x >> 5) ? red[lane] : -INFINITY;
+        x = warp_max(x);
+        if (lane == 0) red[32] = x;
+    }
+    __syncthreads();
+    return red[32];
+}
+
 // One block per row.
 __global__ void __launch_bounds__(256) sample_kernel(const StepDesc* __restrict__ sd, int vocab, const float* __restrict__ logits,
                                                      const int32_t* __restrict__ logits_row, float temperature,
@@ -78,15 +148,9 @@ __global__ void __launch_bounds__(256) sample_kernel(const StepDesc* __restrict_
     const uint32_t c1 = (uint32_t)(row_step[ro] + step_offset), c2 = (uint32_t)row_rollout[ro], c3 = (uint32_t)row_prompt[ro];
     Top2 t{-INFINITY, -INFINITY, 0x7fffffff};
     const int n_blocks = (vocab + 3) >> 2;
-    for (int b = threadIdx.x; b < n_blocks; b += blockDim.x) {
-        const Philox4 w = philox4x32_10((uint32_t)b, c1, c2, c3, k0, k1);
-        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int v = b * 4 + i;
-            if (v < vocab) top2_push(t, lg[v] / temperature + gumbel_from_word(ww[i]), v);
-        }
-    }
+    __shared__ float red[33];
+    const float lmax = range_max(lg, 0, vocab, temperature, red);
+    scan_blocks(t, lg, vocab, 0, n_blocks, temperature, lmax, c1, c2, c3, k0, k1);
     t = top2_warp_reduce(t);
     __shared__ Top2 sh[8];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -126,15 +190,9 @@ __global__ void __launch_bounds__(256) sample_partial_kernel(const StepDesc* __r
     const int n_blocks = (vocab + 3) >> 2;
     const int per_chunk = (n_blocks + n_chunks - 1) / n_chunks;
     const int b_end = min(n_blocks, (chunk + 1) * per_chunk);
-    for (int b = chunk * per_chunk + threadIdx.x; b < b_end; b += blockDim.x) {
-        const Philox4 w = philox4x32_10((uint32_t)b, c1, c2, c3, k0, k1);
-        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int v = b * 4 + i;
-            if (v < vocab) top2_push(t, lg[v] / temperature + gumbel_from_word(ww[i]), v);
-        }
-    }
+    __shared__ float red[33];
+    const float lmax = range_max(lg, min(vocab, chunk * per_chunk * 4), min(vocab, b_end * 4), temperature, red);
+    scan_blocks(t, lg, vocab, chunk * per_chunk, b_end, temperature, lmax, c1, c2, c3, k0, k1);
     t = top2_warp_reduce(t);
     __shared__ Top2 sh[8];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
