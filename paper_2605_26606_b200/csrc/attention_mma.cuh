@@ -4,9 +4,9 @@
 // slots is fetched as head_dim/64 boxes of [TP rows x 64 columns] with the 128-byte swizzle, which makes
 // the ldmatrix reads below bank-conflict free.
 //
-//   attn_group_kernel   one CTA per (128 query rows of a group, KV head).  The query rows are all live
+//   attn_group_kernel   one CTA per (64 query rows of a group, KV head).  The query rows are all live
 //                       rollouts of the group times the query heads sharing the KV head, so the group's
-//                       prompt K/V is read once per 128 query rows instead of once per rollout
+//                       prompt K/V is read once per 64 query rows instead of once per rollout
 //                       (S = Q K^T and O = P V as m16n8k16 MMAs, online softmax in registers).  Every
 //                       query row carries its own number of visible prompt slots, which also makes this
 //                       the causal prefill kernel.  Decode: leaves (m, l, unnormalised O) per query row
@@ -101,14 +101,14 @@ constexpr int MAX_RECORDS = MAX_PREFIX_PARTS + MAX_SUFFIX_CHUNKS;
 // ---------------------------------------------------------------------------------------------
 // Group (shared-prefix / causal-prefill) kernel
 // ---------------------------------------------------------------------------------------------
-constexpr int G_THREADS = 256;      // 8 warps x 16 query rows
-constexpr int G_QROWS = 128;
+constexpr int G_THREADS = 128;      // 4 warps x 16 query rows; two such CTAs share an SM
+constexpr int G_QROWS = 64;
 constexpr int G_TK = 64;            // KV positions per stage
 constexpr int G_STAGES = 3;
 template <int HD> constexpr int group_smem_bytes() { return G_STAGES * 2 * G_TK * HD * 2 + 1024 + 128; }
 
 template <int HD, bool FINAL>
-__global__ void __launch_bounds__(G_THREADS, 1)
+__global__ void __launch_bounds__(G_THREADS, 2)
 attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __restrict__ sd, int64_t n_slots, int Hq, int Hkv,
                   int layer, const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ group_row_start, RowGeom g,
                   float scale_log2, PrefixPartial part, __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ out_lo,
