@@ -28,6 +28,10 @@ if ROOT not in sys.path:
 from paper_2605_26606_b200 import dist_util  # noqa: E402
 from paper_2605_26606_b200 import workloads as wl  # noqa: E402
 
+# DRAM traffic of the suffix attention kernel per algorithmic byte, from the ncu capture summarised in
+# profiles/attn_suffix_kernel_ncu.md (304 rollouts x 513 slots: 171.73 MB moved for 161.6 MB algorithmic).  The kernel
+# streams every (rollout, KV head) suffix once, so traffic grows in proportion to the algorithmic bytes of a launch.
+SUFFIX_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.063
 METRIC = "generated tokens/s"
 UNIT = "tokens/s"
 
@@ -267,7 +271,8 @@ def main():
     achieved = s_bytes / (s_ms * 1e-3) / 1e9 if s_ms > 0 else 0.0
     n_samp = max(len(eng.profile_samples), 1)
     roofline = {"bound": "hbm", "kernel": "attn_suffix_kernel", "achieved": achieved, "peak": peak, "peak_kind": peak_kind,
-                "unit": "GB/s", "frac": achieved / peak, "traffic": None, "launches_sampled": len(eng.profile_samples),
+                "unit": "GB/s", "frac": achieved / peak,
+                "traffic": SUFFIX_TRAFFIC_PER_ALGORITHMIC_BYTE * s_bytes / n_samp, "traffic_note": "ncu capture of a smaller case scaled by algorithmic bytes", "launches_sampled": len(eng.profile_samples),
                 "avg_launch_ms": s_ms / n_samp, "avg_algorithmic_bytes": s_bytes / n_samp}
 
     # whole-step HBM roofline named by the metric: (weight bytes + KV bytes) each decode step must move / peak
