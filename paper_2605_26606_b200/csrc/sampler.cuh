@@ -39,6 +39,12 @@ __device__ __forceinline__ void top2_push(Top2& t, float s, int v) {
     else if (s > t.second) t.second = s;
 }
 
+// Same fold when candidates arrive in arbitrary id order: equal scores keep the lowest id.
+__device__ __forceinline__ void top2_push_unordered(Top2& t, float s, int v) {
+    if (s > t.best || (s == t.best && v < t.idx)) { t.second = t.best; t.best = s; t.idx = v; }
+    else if (s > t.second) t.second = s;
+}
+
 __device__ __forceinline__ Top2 top2_merge(const Top2& a, const Top2& b) {
     Top2 o;
     const bool a_wins = a.best > b.best || (a.best == b.best && a.idx < b.idx);
@@ -68,15 +74,32 @@ __device__ __forceinline__ Top2 top2_warp_reduce(Top2 t) {
 // comparison per candidate against a bound that is refreshed whenever the thread's second-best score rises.  The bound
 // carries a slack far above the float error of its evaluation, and candidates that pass are scored exactly as before, so
 // the result is identical to scoring everything.
+constexpr int SAMPLE_QUEUE = 160;       // per-warp queue of candidates that passed the bound: 32 waiting + up to 128 new
+
 __device__ __forceinline__ void scan_blocks(Top2& t, const float* __restrict__ lg, int vocab, int b_begin, int b_end,
                                             float temperature, float lmax, uint32_t c1, uint32_t c2, uint32_t c3,
-                                            uint32_t k0, uint32_t k1) {
+                                            uint32_t k0, uint32_t k1, uint2* __restrict__ queue /*this warp's SAMPLE_QUEUE slots*/) {
     // The bound uses the largest second-best score of the warp: the final second-best is at least that, so a candidate
-    // below it can change neither the winner nor the gap.  Sharing it keeps a warp from entering the scoring branch
-    // for a lane or two on almost every draw.  Trip counts are warp-uniform (the shuffles need every lane).
+    // below it can change neither the winner nor the gap.  Candidates that pass are not scored where they are found (a
+    // lane or two would drag the whole warp through the logarithms on most draws) but parked in a warp-private queue
+    // and scored 32 at a time, one per lane.  Trip counts are warp-uniform (shuffles and ballots need every lane).
     uint32_t pass_below = 0xffffffffu;          // a candidate is scored iff (2^23 - (w >> 9)) < pass_below
     float bound_for = -INFINITY;                // warp-wide score the bound was computed for
     const int lane = threadIdx.x & 31;
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    int queued = 0;                             // warp-uniform
+    auto drain = [&](int keep) {                // scores queued candidates, 32 at a time, until at most `keep` remain
+        while (queued > keep) {
+            const int take = min(32, queued);
+            __syncwarp();
+            if (lane < take) {
+                const uint2 c = queue[queued - take + lane];
+                top2_push_unordered(t, lg[c.x] / temperature + gumbel_from_word(c.y), (int)c.x);
+            }
+            queued -= take;
+            __syncwarp();
+        }
+    };
     for (int base = b_begin + (threadIdx.x - lane); base < b_end; base += blockDim.x) {
         const float ws = warp_max(t.second);
         if (ws > bound_for) {
@@ -87,17 +110,20 @@ __device__ __forceinline__ void scan_blocks(Top2& t, const float* __restrict__ l
             pass_below = d >= 8388608.f ? 0xffffffffu : (uint32_t)(d * 1.001f + 2.f);
         }
         const int b = base + lane;
-        if (b < b_end) {
-            const Philox4 w = philox4x32_10((uint32_t)b, c1, c2, c3, k0, k1);
-            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+        Philox4 w{0, 0, 0, 0};
+        if (b < b_end) w = philox4x32_10((uint32_t)b, c1, c2, c3, k0, k1);
+        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int v = b * 4 + i;
-                if (v < vocab && (8388608u - (ww[i] >> 9)) < pass_below)
-                    top2_push(t, lg[v] / temperature + gumbel_from_word(ww[i]), v);
-            }
+        for (int i = 0; i < 4; ++i) {
+            const int v = b * 4 + i;
+            const bool pass = b < b_end && v < vocab && (8388608u - (ww[i] >> 9)) < pass_below;
+            const uint32_t m = __ballot_sync(0xffffffffu, pass);
+            if (pass) queue[queued + __popc(m & lt_mask)] = make_uint2((uint32_t)v, ww[i]);
+            queued += __popc(m);
         }
+        drain(31);
     }
+    drain(0);
 }
 
 // Largest logit / T over the blocks a thread block will scan (block-wide); `red` is 33 floats of shared memory.
@@ -149,8 +175,9 @@ __global__ void __launch_bounds__(256) sample_kernel(const StepDesc* __restrict_
     Top2 t{-INFINITY, -INFINITY, 0x7fffffff};
     const int n_blocks = (vocab + 3) >> 2;
     __shared__ float red[33];
+    __shared__ uint2 queue[8][SAMPLE_QUEUE];
     const float lmax = range_max(lg, 0, vocab, temperature, red);
-    scan_blocks(t, lg, vocab, 0, n_blocks, temperature, lmax, c1, c2, c3, k0, k1);
+    scan_blocks(t, lg, vocab, 0, n_blocks, temperature, lmax, c1, c2, c3, k0, k1, queue[threadIdx.x >> 5]);
     t = top2_warp_reduce(t);
     __shared__ Top2 sh[8];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -191,8 +218,9 @@ __global__ void __launch_bounds__(256) sample_partial_kernel(const StepDesc* __r
     const int per_chunk = (n_blocks + n_chunks - 1) / n_chunks;
     const int b_end = min(n_blocks, (chunk + 1) * per_chunk);
     __shared__ float red[33];
+    __shared__ uint2 queue[8][SAMPLE_QUEUE];
     const float lmax = range_max(lg, min(vocab, chunk * per_chunk * 4), min(vocab, b_end * 4), temperature, red);
-    scan_blocks(t, lg, vocab, chunk * per_chunk, b_end, temperature, lmax, c1, c2, c3, k0, k1);
+    scan_blocks(t, lg, vocab, chunk * per_chunk, b_end, temperature, lmax, c1, c2, c3, k0, k1, queue[threadIdx.x >> 5]);
     t = top2_warp_reduce(t);
     __shared__ Top2 sh[8];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
