@@ -225,6 +225,19 @@ PC_API int pc_sample(void* stream, int n_rows, int vocab, const float* logits, c
               const int32_t* row_step, int32_t* out_tokens, const int64_t* out_index, float* out_top2_gap,
               void* scratch, size_t scratch_bytes);
 
+/* Behaviour log-probability of drawn tokens, the denominator pi_theta_old(o_t | q, o_<t) of the token importance ratio
+ * (Eq. 2):  out = logits[token] / T - log sum_v exp(logits[v] / T).  Row r reads logits row logits_row[r] (NULL: r),
+ * its token is tokens[tok_index[r]] (NULL: tokens[r]) and the result goes to out_logprob[out_index[r]] (NULL: [r]).
+ * All pointers device. */
+PC_API int pc_token_logprob(void* stream, int n_rows, int vocab, const float* logits, const int32_t* logits_row,
+                            float temperature, const int32_t* tokens, const int64_t* tok_index, float* out_logprob,
+                            const int64_t* out_index);
+
+/* With a buffer set (device float, indexed exactly like the token buffer of pc_decode_step / pc_decode_run), every
+ * decode step that samples also stores the behaviour log-probability (Eq. 2) of the token it drew at
+ * logprobs[row_tok_index[r] + 1].  NULL switches it off (the default). */
+PC_API int pc_set_logprob_buffer(pc_ctx* ctx, float* logprobs);
+
 /* pc_sample for callers that cannot provide scratch memory.  The paper has no counterpart: this entry point exists for
  * hosts of this library that must not allocate device memory at the moment they sample -- code running inside a
  * stream-ordered region whose allocator is frozen, a plugin that is handed only its input and output buffers, a

@@ -23,7 +23,7 @@ PC_DTYPE_F32, PC_DTYPE_BF16 = 0, 1
 PC_STATUS_COMMIT, PC_STATUS_BUFFERED, PC_STATUS_DEFER_HARD, PC_STATUS_SKIP_EASY = 0, 1, 2, 3
 
 EXPORTS = ["pc_status_string", "pc_last_cuda_error", "pc_launch_count", "pc_profile_attention", "pc_create", "pc_destroy", "pc_workspace_bytes",
-           "pc_set_workspace", "pc_prefill_shared", "pc_decode_step", "pc_decode_run", "pc_sample", "pc_sample_static", "pc_reward_last_token",
+           "pc_set_workspace", "pc_prefill_shared", "pc_decode_step", "pc_decode_run", "pc_sample", "pc_sample_static", "pc_token_logprob", "pc_set_logprob_buffer", "pc_reward_last_token",
            "pc_group_stats", "pc_allocate", "pc_grpo_advantage"]
 
 
@@ -90,6 +90,8 @@ def _lib():
         lib.pc_decode_run.argtypes = [p, p, i, p, p, p, p, p, p, p, p, p, p, p, i64, p, p, i64, C.POINTER(SampleParams)]
         lib.pc_sample.argtypes = [p, i, i, p, p, f, u64, p, p, p, p, p, p, p, C.c_size_t]
         lib.pc_sample_static.argtypes = [p, i, i, p, p, f, u64, p, p, p, p, p, p]
+        lib.pc_token_logprob.argtypes = [p, i, i, p, p, f, p, p, p, p]
+        lib.pc_set_logprob_buffer.argtypes = [p, p]
         lib.pc_reward_last_token.argtypes = [p, i, p, p, p, p]
         lib.pc_group_stats.argtypes = [p, i, p, p, p, p, p, p, p]
         lib.pc_allocate.argtypes = [p, i, p, p, C.POINTER(AllocParams), p, p, p, p, p]
@@ -241,6 +243,17 @@ def pc_sample_static(n_rows, vocab, logits, logits_row, temperature, seed, row_p
     _check(_lib().pc_sample_static(_stream(), n_rows, vocab, _ptr(logits, torch.float32), _ptr(logits_row), temperature, seed,
                                    _ptr(row_prompt), _ptr(row_rollout), _ptr(row_step), _ptr(out_tokens), _ptr(out_index),
                                    _ptr(out_top2_gap)), "pc_sample_static")
+
+
+def pc_token_logprob(n_rows, vocab, logits, logits_row, temperature, tokens, tok_index, out_logprob, out_index=None) -> None:
+    _check(_lib().pc_token_logprob(_stream(), n_rows, vocab, _ptr(logits, torch.float32), _ptr(logits_row), temperature,
+                                   _ptr(tokens, torch.int32), _ptr(tok_index), _ptr(out_logprob, torch.float32), _ptr(out_index)),
+           "pc_token_logprob")
+
+
+def pc_set_logprob_buffer(ctx: Context, logprobs: Optional[torch.Tensor]) -> None:
+    _check(_lib().pc_set_logprob_buffer(ctx.handle, _ptr(logprobs)), "pc_set_logprob_buffer")
+    ctx._keep.append(logprobs)
 
 
 def pc_reward_last_token(n, tokens, last_index, threshold, reward) -> None:

@@ -96,6 +96,7 @@ struct pc_ctx {
     // one-shot profiling request (pc_profile_attention)
     int prof_layer = -1;
     cudaEvent_t prof_start = nullptr, prof_stop = nullptr;
+    float* logprobs = nullptr;       // pc_set_logprob_buffer
 
     std::vector<GraphEntry> graphs;
     cudaStream_t capture_stream = nullptr;      // decode steps are captured here (the caller's stream may be the default one)
@@ -468,6 +469,24 @@ const char* pc_last_cuda_error(void) { return g_cuda_error.c_str(); }
 
 uint64_t pc_launch_count(void) { return g_launches; }
 
+int pc_set_logprob_buffer(pc_ctx* ctx, float* logprobs) {
+    if (ctx == nullptr) return PC_ERR_INVALID_ARG;
+    ctx->logprobs = logprobs;
+    return PC_OK;
+}
+
+int pc_token_logprob(void* stream, int n_rows, int vocab, const float* logits, const int32_t* logits_row, float temperature,
+                     const int32_t* tokens, const int64_t* tok_index, float* out_logprob, const int64_t* out_index) {
+    if (n_rows < 0 || vocab <= 0 || !(temperature > 0.f)) return PC_ERR_INVALID_ARG;
+    if (n_rows == 0) return PC_OK;
+    if (logits == nullptr || tokens == nullptr || out_logprob == nullptr) return PC_ERR_INVALID_ARG;
+    pc::token_logprob_kernel<<<n_rows, 256, 0, static_cast<cudaStream_t>(stream)>>>(nullptr, vocab, logits, logits_row, temperature, tokens,
+                                                                                   tok_index, 0, out_logprob, out_index, 0);
+    count_launches(1);
+    PC_CUDA_CHECK_LAUNCH("token_logprob");
+    return PC_OK;
+}
+
 int pc_profile_attention(pc_ctx* ctx, int layer, void* event_start, void* event_stop) {
     if (ctx == nullptr || layer < 0 || layer >= ctx->d.n_layers || event_start == nullptr || event_stop == nullptr)
         return PC_ERR_INVALID_ARG;
@@ -631,6 +650,7 @@ struct DecodeArgs {
     int32_t* tokens; const int64_t* row_tok_index; const int32_t* group_row_start; const int32_t* prompt_len;
     const void* prompt_kv; int64_t prompt_slots; const int64_t* prompt_kv_start; void* suffix_kv; int64_t suffix_slots;
     float temperature; uint64_t seed; int sample;
+    float* logprobs;      // optional: behaviour log-probability of every sampled token (pc_set_logprob_buffer)
 };
 // Zero-filled first (padding included) so that two equal argument sets compare equal byte by byte.
 DecodeArgs make_decode_args(const int32_t* row_prompt, const int32_t* row_rollout, const int32_t* row_step, const int64_t* row_kv_start,
@@ -646,6 +666,7 @@ DecodeArgs make_decode_args(const int32_t* row_prompt, const int32_t* row_rollou
     a.temperature = sample ? sample->temperature : 1.f;
     a.seed = sample ? sample->seed : 0;
     a.sample = sample != nullptr;
+    a.logprobs = nullptr;
     return a;
 }
 static_assert(sizeof(DecodeArgs) <= sizeof(GraphKey::args), "graph key too small for the decode arguments");
@@ -696,6 +717,11 @@ int decode_launches(pc_ctx* ctx, cudaStream_t st, int m_bound, int groups_bound,
                                                                             nullptr);
             count_launches(2);
         }
+        if (a.logprobs != nullptr) {
+            pc::token_logprob_kernel<<<m_bound, 256, 0, st>>>(sd, ctx->d.vocab, logits, nullptr, a.temperature, a.tokens, a.row_tok_index,
+                                                              1, a.logprobs, a.row_tok_index, 1);
+            count_launches(1);
+        }
         PC_CUDA_CHECK_LAUNCH("sample");
     }
     return PC_OK;
@@ -713,9 +739,10 @@ int pc_decode_step(pc_ctx* ctx, void* stream, int n_rows, const int32_t* row_pro
     if (int rc = check_ready(ctx)) return rc;
     if (n_rows < 0 || n_groups < 0 || max_group_rows < 0) return PC_ERR_INVALID_ARG;
     if (n_rows == 0) return PC_OK;
-    const DecodeArgs a = make_decode_args(row_prompt, row_rollout, row_step, row_kv_start, tokens, row_tok_index, group_row_start,
+    DecodeArgs a = make_decode_args(row_prompt, row_rollout, row_step, row_kv_start, tokens, row_tok_index, group_row_start,
                                           prompt_len, prompt_kv, prompt_slots, prompt_kv_start, suffix_kv, suffix_slots, sample);
     if (int rc = check_decode_args(ctx, a)) return rc;
+    a.logprobs = ctx->logprobs;
     if (n_groups == 0 || max_group_rows == 0 || max_group_rows > n_rows || n_groups > n_rows) return PC_ERR_INVALID_ARG;
     if (logits_out == nullptr && sample == nullptr) return PC_ERR_INVALID_ARG;
     if (logits_out && !aligned(logits_out, 16)) return PC_ERR_ALIGNMENT;
@@ -739,9 +766,10 @@ int pc_decode_run(pc_ctx* ctx, void* stream, int n_steps, const pc_step_desc* st
     if (n_steps < 0) return PC_ERR_INVALID_ARG;
     if (n_steps == 0) return PC_OK;
     if (steps_host == nullptr || steps_dev == nullptr || sample == nullptr) return PC_ERR_INVALID_ARG;
-    const DecodeArgs a = make_decode_args(row_prompt, row_rollout, row_step, row_kv_start, tokens, row_tok_index, group_row_start,
+    DecodeArgs a = make_decode_args(row_prompt, row_rollout, row_step, row_kv_start, tokens, row_tok_index, group_row_start,
                                           prompt_len, prompt_kv, prompt_slots, prompt_kv_start, suffix_kv, suffix_slots, sample);
     if (int rc = check_decode_args(ctx, a)) return rc;
+    a.logprobs = ctx->logprobs;
     int groups_bound = 0, group_rows_bound = 0;
     for (int s = 0; s < n_steps; ++s) {
         const pc_step_desc& d = steps_host[s];

@@ -253,6 +253,33 @@ __global__ void sample_reduce_kernel(const StepDesc* __restrict__ sd, int n_rows
     if (out_gap) out_gap[r] = t.best - t.second;
 }
 
+// log softmax(logits / T)[token]: the behaviour log-probability of an already drawn token.  One block per row;
+// max and sum of exponentials are block reductions in a fixed shape, so the value does not depend on timing.
+__global__ void __launch_bounds__(256) token_logprob_kernel(const StepDesc* __restrict__ sd, int vocab, const float* __restrict__ logits,
+                                                            const int32_t* __restrict__ logits_row, float temperature,
+                                                            const int32_t* __restrict__ tokens, const int64_t* __restrict__ tok_index,
+                                                            int64_t tok_index_offset, float* __restrict__ out,
+                                                            const int64_t* __restrict__ out_index, int64_t out_index_offset) {
+    const int r = blockIdx.x;
+    int64_t ro = r;
+    if (sd != nullptr) {
+        if (r >= sd->n_rows) return;
+        ro += sd->row_off;
+    }
+    const float* lg = logits + (size_t)(logits_row ? logits_row[ro] : r) * vocab;
+    __shared__ float red[33];
+    const float mx = range_max(lg, 0, vocab, temperature, red);          // max of logits / T
+    const float inv_t = 1.f / temperature;
+    float s = 0.f;
+    for (int v = threadIdx.x; v < vocab; v += blockDim.x) s += expf(lg[v] * inv_t - mx);
+    s = block_sum(s, red);
+    if (threadIdx.x == 0) {
+        const int tok = tokens[tok_index ? tok_index[ro] + tok_index_offset : (int64_t)r];
+        const float lp = (tok >= 0 && tok < vocab) ? lg[tok] * inv_t - mx - logf(s) : -INFINITY;
+        out[out_index ? out_index[ro] + out_index_offset : (int64_t)r] = lp;
+    }
+}
+
 constexpr int SAMPLE_MAX_CHUNKS = 32;
 // Ranges per row so that about four blocks per SM are in flight; 1 means the one-pass kernel is the better choice.
 inline int sample_chunks(int n_rows, int num_sms) {

@@ -94,6 +94,7 @@ class RolloutEngine:
         self._arenas: Dict[str, Optional[torch.Tensor]] = {}
         self.profile_every = 0
         self.use_graphs = True
+        self.collect_logprobs = False       # also keep log pi(o_t) of every sampled token (Eq. 2's denominator)
         self.record_pilot_logits: Optional[dict] = None     # {decode step: None} -> filled during the pilot stage
         self.profile_layer = m.n_layers // 2
         self.profile_samples: List[tuple] = []      # (start event, stop event, rows, suffix slots read per row)
@@ -144,6 +145,8 @@ class RolloutEngine:
         self.suffix_kv = None
         self.suffix_kv = self.kv_arena(self.suffix_slots, "suffix")
         self.tokens = torch.full((P * G * wl.max_new,), -1, dtype=torch.int32, device=dev)
+        self.logprobs = torch.zeros(P * G * wl.max_new, dtype=torch.float32, device=dev) if self.collect_logprobs else None
+        B.pc_set_logprob_buffer(self.ctx, self.logprobs)
         self.last_logits = torch.empty((P, self.model.vocab), dtype=torch.float32, device=dev)
         self.rewards = torch.zeros(P * G, dtype=torch.float32, device=dev)
         self.adv = torch.zeros(P * G, dtype=torch.float32, device=dev)
@@ -222,6 +225,9 @@ class RolloutEngine:
         if not teacher_forced and step_range is None:
             B.pc_sample(n, self.model.vocab, self.last_logits, d_p, wl.temperature, wl.sample_seed, d_p, d_r, d_zero,
                         self.tokens, out_index=d_first)
+            if self.logprobs is not None:
+                B.pc_token_logprob(n, self.model.vocab, self.last_logits, d_p, wl.temperature, self.tokens, d_first, self.logprobs,
+                                   d_first)
         sch = self.build_schedule(prompts, rollouts)
         pr, rr, rs = sch.row_prompt.data_ptr(), sch.row_rollout.data_ptr(), sch.row_step.data_ptr()
         rk, rt, gs = sch.row_kv_start.data_ptr(), sch.row_tok_index.data_ptr(), sch.group_row_start.data_ptr()
@@ -319,4 +325,5 @@ class RolloutEngine:
                     pilot_var=h(self.pilot_var), status=status, extra=h(self.extra), evict=h(self.evict),
                     n_selected=int(self.n_selected.item()), total_rollouts=int(self.total_rollouts.item()),
                     union_n=h(self.union_n), union_success=h(self.union_success), union_mean=h(self.union_mean),
-                    union_var=h(self.union_var), advantages=h(self.adv).reshape(P, G))
+                    union_var=h(self.union_var), advantages=h(self.adv).reshape(P, G),
+                    logprobs=None if self.logprobs is None else h(self.logprobs).reshape(P, G, wl.max_new))

@@ -175,3 +175,22 @@ def test_philox_words_match_oracle_through_uniform_logits():
     for r in range(n):
         g = ophilox.gumbel_noise(V, seed, int(prompt[r]), int(roll[r]), int(step[r]))
         assert out[r] == int(np.argmax(g))
+
+
+def test_token_logprob_matches_oracle():
+    from oracle.logprob import token_logprob
+    rng = np.random.default_rng(8)
+    for vocab, T in ((7, 1.0), (4099, 0.7), (151936, 1.0)):
+        n = 9
+        logits = (rng.normal(size=(3, vocab)) * 4).astype(np.float32)
+        row = rng.integers(0, 3, n)
+        toks = rng.integers(0, vocab, n)
+        tok_buf = torch.from_numpy(np.stack([np.full(n, -7), toks], axis=1).reshape(-1).astype(np.int32)).cuda()
+        tok_idx = torch.arange(n, dtype=torch.int64, device="cuda") * 2 + 1
+        out = torch.full((n * 3,), 9.0, device="cuda")
+        out_idx = torch.arange(n, dtype=torch.int64, device="cuda") * 3 + 2
+        B.pc_token_logprob(n, vocab, torch.from_numpy(logits).cuda(), _i32(row), T, tok_buf, tok_idx, out, out_idx)
+        out = out.cpu().numpy().reshape(n, 3)
+        assert np.all(out[:, :2] == 9.0)
+        for r in range(n):
+            assert abs(out[r, 2] - token_logprob(logits[row[r]], int(toks[r]), T)) < 1e-4

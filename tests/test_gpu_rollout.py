@@ -168,3 +168,28 @@ def test_qwen3_widths_two_layers_teacher_forced(base):
     eng = RolloutEngine(model, weights, max_rows=P * G, max_prefill_tokens=int(batch.prompt_offsets[-1]))
     worst, n_cmp, n_exempt = teacher_forced_compare(eng, w, batch, ref, prompts, rollouts, logit_tol=5e-2, gap_tol=1e-1)
     assert n_cmp == int(batch.caps.sum())
+
+
+def test_behaviour_logprobs_along_free_running_rollouts():
+    """log pi(o_t) of every sampled token (Eq. 2's denominator), config 0: tokens are identical to the oracle's, so its
+    logits give the expected log-probabilities position by position."""
+    from oracle.logprob import token_logprob
+    w = dataclasses.replace(wl.WORKLOADS["config0"], forced_explicit=((0, 0.0), (1, 0.5), (2, 0.45), (3, 1.0)))
+    weights = wl.gen_weights(w.model, seed=0, threads=2, gain_jitter=0.1)
+    batch = wl.gen_batch(w)
+    dec = Decoder(w.model, weights)
+    eng = RolloutEngine(w.model, weights, max_rows=w.n_prompts * w.group_size, max_prefill_tokens=int(batch.prompt_offsets[-1]))
+    eng.collect_logprobs = True
+    out = eng.pilot_commit_step(w, batch)
+    assert np.any(out["status"] == ostats.COMMIT)
+    n_checked = 0
+    for p in range(w.n_prompts):
+        idx = [i for i in range(w.group_size) if out["generated"][p, i]]
+        ref = oracle_group_tokens(dec, w, batch, [p] * len(idx), idx)
+        for i in idx:
+            toks, logs = ref[(p, i)]
+            assert np.array_equal(toks, out["tokens"][p][i])
+            for s, t in enumerate(toks):
+                assert abs(out["logprobs"][p, i, s] - token_logprob(logs[s], int(t), w.temperature)) < 1e-4
+                n_checked += 1
+    assert n_checked == int(batch.caps[out["generated"]].sum())
