@@ -108,3 +108,13 @@ def sampling_cost(method: str, b_t: int, s: int, n_pilot: int, n_commit: int) ->
     if method == "pc":
         return b_g * n_pilot + b_t * n_commit
     raise ValueError(method)
+
+
+def dapo_filter(rewards: np.ndarray, start: np.ndarray, count: np.ndarray) -> np.ndarray:
+    """The baseline filter of Section 4.3 (DAPO): every prompt of the oversampled batch gets the full budget n and
+    prompts whose rewards are all correct or all incorrect are dropped.  Returns keep[g] in {0, 1}."""
+    keep = np.zeros(len(start), dtype=np.int32)
+    for g in range(len(start)):
+        r = np.asarray(rewards[start[g]:start[g] + count[g]], dtype=np.float64)
+        keep[g] = 1 if r.shape[0] > 0 and np.max(r) != np.min(r) else 0
+    return keep

@@ -1,0 +1,90 @@
+"""The multi-step bookkeeping of Algorithm 1: the oracle simulation against invariants and the paper's accounting, and the
+host controller against the oracle."""
+import numpy as np
+import pytest
+
+from oracle import controller as octl
+from oracle import stats as ostats
+from paper_2605_26606_b200.controller import PilotCommitController
+
+
+def _p_hat_table(n_prompts, n_steps, k, seed):
+    rng = np.random.default_rng(seed)
+    base = rng.beta(0.5, 0.5, size=n_prompts)
+    drift = np.minimum(1.0, base[None, :] + 0.02 * np.arange(n_steps)[:, None])      # prompts get easier over time
+    m = rng.binomial(k, drift)
+    return m / k
+
+
+def _simulate(seed, b_g=12, b_t=4, k=8, n_commit=8, d=2, n_prompts=60, n_epochs=3, pl=0.125, pu=0.75, ps=1.0):
+    table = _p_hat_table(n_prompts, 200, k, seed)
+    return table, octl.simulate(list(range(n_prompts)), n_epochs, b_g, b_t, k, n_commit, pl, pu, ps, d, lambda q, t: table[t, q])
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_oracle_simulation_invariants(seed):
+    b_g, b_t, k, nc, d = 12, 4, 8, 8, 2
+    table, log = _simulate(seed, b_g, b_t, k, nc, d)
+    solved_so_far, committed_all = set(), []
+    epoch_of_step, seen_in_epoch = {}, {}
+    for e in log:
+        t = e["step"]
+        assert len(e["selected"]) <= b_t
+        for q, born in e["selected"]:
+            assert 0 <= t - born <= d                                   # off-policy delay at most d (Section 3.4)
+            assert 0.125 <= table[born, q] <= 0.75                      # only pilot survivors commit
+        assert e["rollouts"] == len(e["batch"]) * k + len(e["selected"]) * nc       # Section 4.3
+        committed_all += [(q, born) for q, born in e["selected"]]
+        solved_so_far |= set(e["solved"])
+        assert all(table[t, q] >= 1.0 for q in e["solved"])
+    assert len(set(committed_all)) == len(committed_all)               # a buffered survivor is committed at most once
+    # a prompt solved in one epoch is never sampled in a later epoch (Section 3.4, "Evicting solved prompts")
+    first_solved = {}
+    for e in log:
+        for q in e["solved"]:
+            first_solved.setdefault(q, e["step"])
+    steps_per_epoch = (60 + b_g - 1) // b_g
+    for e in log:
+        for q in e["batch"]:
+            if q in first_solved and first_solved[q] < e["step"]:
+                assert False, "evicted prompt sampled again"
+    # whenever survivors are plentiful the batch is full: buffer carries the surplus to later steps
+    assert any(len(e["selected"]) == b_t and e["buffered"] > 0 for e in log)
+
+
+def test_full_buffer_reproduces_the_papers_rollouts_per_step():
+    # b_t = 128, b_g = 3 b_t, (n_pilot, n_commit) = (16, 48): 12,288 rollouts per step (Table 2) once enough prompts survive
+    log = octl.simulate(list(range(384 * 3)), 1, 384, 128, 16, 48, 0.125, 0.75, 1.0, 4, lambda q, t: 0.5)
+    assert [e["rollouts"] for e in log] == [12288] * 3
+    # d bounds the age of what stays buffered: with b_t = 1 and everything surviving, entries older than d are dropped
+    log = octl.simulate(list(range(40)), 1, 4, 1, 2, 2, 0.0, 1.0, 2.0, 2, lambda q, t: 0.5)
+    assert max(e["buffered"] for e in log) <= 2 * 4 and any(e["stale"] for e in log)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_host_controller_matches_the_oracle_simulation(seed):
+    b_g, b_t, k, nc, d, n_prompts, n_epochs = 12, 4, 8, 8, 2, 60, 3
+    table, log = _simulate(seed, b_g, b_t, k, nc, d, n_prompts, n_epochs)
+    ctl = PilotCommitController(k, nc, b_t, d)
+    dataset = list(range(n_prompts))
+    i = 0
+    for _ in range(n_epochs):
+        pool = ctl.sampling_pool(dataset)
+        for b0 in range(0, len(pool), b_g):
+            batch = pool[b0:b0 + b_g]
+            m = np.rint(table[ctl.t, batch] * k).astype(np.int64)
+            st, extra, ev, nsel, total = ostats.allocate(m, np.full(len(batch), k), 0.125, 0.75, 1.0, nc, len(batch))
+            plan = ctl.step(batch, st == ostats.COMMIT, ev)
+            e = log[i]; i += 1
+            assert plan.step == e["step"] and batch == e["batch"]
+            assert plan.committed == e["selected"] and sorted(plan.newly_evicted) == sorted(e["solved"])
+            assert plan.dropped_stale == e["stale"] and plan.buffered_after == e["buffered"]
+            assert plan.rollouts_sampled == e["rollouts"]
+    assert i == len(log)
+
+
+def test_controller_rejects_bad_arguments():
+    with pytest.raises(ValueError):
+        PilotCommitController(0, 1, 1, 1)
+    with pytest.raises(ValueError):
+        PilotCommitController(2, 2, 2, 2).step([1, 2], [1], [0, 0])

@@ -194,3 +194,23 @@ def test_token_logprob_matches_oracle():
         assert np.all(out[:, :2] == 9.0)
         for r in range(n):
             assert abs(out[r, 2] - token_logprob(logits[row[r]], int(toks[r]), T)) < 1e-4
+
+
+def test_dapo_and_grpo_modes_through_pc_allocate():
+    """DAPO's zero-variance filter (Section 4.3) = pc_allocate on full groups with thresholds 1/n, (n-1)/n and no commit."""
+    rng = np.random.default_rng(10)
+    for n in (2, 16, 64, 128):
+        P = 300
+        m = rng.integers(0, n + 1, size=P); m[:3] = [0, n, 1]
+        r = np.zeros((P, n))
+        for p in range(P):
+            r[p, rng.permutation(n)[:m[p]]] = 1.0
+        start, count = np.arange(P) * n, np.full(P, n)
+        cn, cm, _, var = _stats_gpu(r.reshape(-1), start, count)
+        assert np.array_equal(cm, m)
+        st, ex, ev, nsel, tot = _alloc_gpu(cm, cn, 1.0 / n, (n - 1.0) / n, 1.0, 0, P)
+        keep = ostats.dapo_filter(r.reshape(-1), start, count)
+        assert np.array_equal(st == B.PC_STATUS_COMMIT, keep == 1) and tot == P * n
+        assert np.array_equal(var > 0, keep == 1)
+        st, ex, ev, nsel, tot = _alloc_gpu(cm, cn, 0.0, 1.0, 2.0, 0, P)          # GRPO: nothing filtered
+        assert np.all(st == B.PC_STATUS_COMMIT) and nsel == P

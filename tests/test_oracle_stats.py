@@ -164,3 +164,24 @@ def test_statuses_partition_and_budget_conserved_random():
         assert np.sum(st == stats.BUFFERED) == kept - nsel
         assert total == P * k + extra.sum() and extra.sum() == nsel * nc
         assert set(np.unique(st)) <= {0, 1, 2, 3}
+
+
+def test_dapo_filter_is_the_pilot_filter_with_k_equal_n():
+    """Section 4.3: DAPO gives every prompt n rollouts and drops all-correct / all-incorrect groups.  That is the pilot
+    filter evaluated on the full group with thresholds 1/n and (n-1)/n and nothing left to commit."""
+    rng = np.random.default_rng(9)
+    for n in (2, 16, 64, 128):
+        P = 40
+        m = rng.integers(0, n + 1, size=P); m[:3] = [0, n, 1]
+        r = np.zeros((P, n)); 
+        for p in range(P):
+            r[p, :m[p]] = 1.0
+        keep = stats.dapo_filter(r.reshape(-1), np.arange(P) * n, np.full(P, n))
+        assert list(keep[:3]) == [0, 0, 1]
+        st, extra, ev, nsel, total = stats.allocate(m, np.full(P, n), 1.0 / n, (n - 1.0) / n, 1.0, n_commit=0, b_t=P)
+        assert np.array_equal(keep == 1, st == stats.COMMIT)
+        assert np.array_equal(st == stats.DEFER_HARD, m == 0) and np.array_equal(st == stats.SKIP_EASY, m == n)
+        assert total == P * n == stats.sampling_cost("dapo", P, 1, n, 0)       # b_g n rollouts generated
+    # GRPO: every prompt of the training batch gets n rollouts, none is filtered
+    st, *_ , total = stats.allocate(np.array([0, 3, 8]), np.full(3, 8), 0.0, 1.0, 2.0, 0, 3)
+    assert np.all(st == stats.COMMIT) and total == 24 == stats.sampling_cost("grpo", 3, 3, 8, 0)
