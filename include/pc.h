@@ -238,6 +238,14 @@ PC_API int pc_token_logprob(void* stream, int n_rows, int vocab, const float* lo
  * logprobs[row_tok_index[r] + 1].  NULL switches it off (the default). */
 PC_API int pc_set_logprob_buffer(pc_ctx* ctx, float* logprobs);
 
+/* Sampling keys of the prompts.  By default the decode steps key a draw by (seed, row_prompt, rollout, step), i.e. by a
+ * prompt's index in the arrays of the call.  When pilot rollouts of one sampling batch and commit rollouts of the
+ * previous batch's survivors share one decode batch (Section 3.4, "Binding pilot and commit"), a prompt's index in the
+ * combined arrays differs from the one it had when its pilot rollouts were drawn; prompt_key (device int32, one entry per
+ * prompt of the call, or NULL for the default) supplies the id to use in the key instead, so that a rollout's tokens do
+ * not depend on how batches are bound. */
+PC_API int pc_set_prompt_keys(pc_ctx* ctx, const int32_t* prompt_key);
+
 /* pc_sample for callers that cannot provide scratch memory.  The paper has no counterpart: this entry point exists for
  * hosts of this library that must not allocate device memory at the moment they sample -- code running inside a
  * stream-ordered region whose allocator is frozen, a plugin that is handed only its input and output buffers, a

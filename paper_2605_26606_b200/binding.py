@@ -23,7 +23,7 @@ PC_DTYPE_F32, PC_DTYPE_BF16 = 0, 1
 PC_STATUS_COMMIT, PC_STATUS_BUFFERED, PC_STATUS_DEFER_HARD, PC_STATUS_SKIP_EASY = 0, 1, 2, 3
 
 EXPORTS = ["pc_status_string", "pc_last_cuda_error", "pc_launch_count", "pc_profile_attention", "pc_create", "pc_destroy", "pc_workspace_bytes",
-           "pc_set_workspace", "pc_prefill_shared", "pc_decode_step", "pc_decode_run", "pc_sample", "pc_sample_static", "pc_token_logprob", "pc_set_logprob_buffer", "pc_reward_last_token",
+           "pc_set_workspace", "pc_prefill_shared", "pc_decode_step", "pc_decode_run", "pc_sample", "pc_sample_static", "pc_token_logprob", "pc_set_logprob_buffer", "pc_set_prompt_keys", "pc_reward_last_token",
            "pc_group_stats", "pc_allocate", "pc_grpo_advantage"]
 
 
@@ -92,6 +92,7 @@ def _lib():
         lib.pc_sample_static.argtypes = [p, i, i, p, p, f, u64, p, p, p, p, p, p]
         lib.pc_token_logprob.argtypes = [p, i, i, p, p, f, p, p, p, p]
         lib.pc_set_logprob_buffer.argtypes = [p, p]
+        lib.pc_set_prompt_keys.argtypes = [p, p]
         lib.pc_reward_last_token.argtypes = [p, i, p, p, p, p]
         lib.pc_group_stats.argtypes = [p, i, p, p, p, p, p, p, p]
         lib.pc_allocate.argtypes = [p, i, p, p, C.POINTER(AllocParams), p, p, p, p, p]
@@ -254,6 +255,11 @@ def pc_token_logprob(n_rows, vocab, logits, logits_row, temperature, tokens, tok
 def pc_set_logprob_buffer(ctx: Context, logprobs: Optional[torch.Tensor]) -> None:
     _check(_lib().pc_set_logprob_buffer(ctx.handle, _ptr(logprobs)), "pc_set_logprob_buffer")
     ctx._keep.append(logprobs)
+
+
+def pc_set_prompt_keys(ctx: Context, prompt_key: Optional[torch.Tensor]) -> None:
+    _check(_lib().pc_set_prompt_keys(ctx.handle, _ptr(prompt_key)), "pc_set_prompt_keys")
+    ctx._keep.append(prompt_key)
 
 
 def pc_reward_last_token(n, tokens, last_index, threshold, reward) -> None:

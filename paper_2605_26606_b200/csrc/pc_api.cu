@@ -97,6 +97,7 @@ struct pc_ctx {
     int prof_layer = -1;
     cudaEvent_t prof_start = nullptr, prof_stop = nullptr;
     float* logprobs = nullptr;       // pc_set_logprob_buffer
+    const int32_t* prompt_key = nullptr;    // pc_set_prompt_keys
 
     std::vector<GraphEntry> graphs;
     cudaStream_t capture_stream = nullptr;      // decode steps are captured here (the caller's stream may be the default one)
@@ -469,6 +470,12 @@ const char* pc_last_cuda_error(void) { return g_cuda_error.c_str(); }
 
 uint64_t pc_launch_count(void) { return g_launches; }
 
+int pc_set_prompt_keys(pc_ctx* ctx, const int32_t* prompt_key) {
+    if (ctx == nullptr) return PC_ERR_INVALID_ARG;
+    ctx->prompt_key = prompt_key;
+    return PC_OK;
+}
+
 int pc_set_logprob_buffer(pc_ctx* ctx, float* logprobs) {
     if (ctx == nullptr) return PC_ERR_INVALID_ARG;
     ctx->logprobs = logprobs;
@@ -651,6 +658,7 @@ struct DecodeArgs {
     const void* prompt_kv; int64_t prompt_slots; const int64_t* prompt_kv_start; void* suffix_kv; int64_t suffix_slots;
     float temperature; uint64_t seed; int sample;
     float* logprobs;      // optional: behaviour log-probability of every sampled token (pc_set_logprob_buffer)
+    const int32_t* prompt_key;   // optional: sampling-key id of every prompt (pc_set_prompt_keys)
 };
 // Zero-filled first (padding included) so that two equal argument sets compare equal byte by byte.
 DecodeArgs make_decode_args(const int32_t* row_prompt, const int32_t* row_rollout, const int32_t* row_step, const int64_t* row_kv_start,
@@ -667,6 +675,7 @@ DecodeArgs make_decode_args(const int32_t* row_prompt, const int32_t* row_rollou
     a.seed = sample ? sample->seed : 0;
     a.sample = sample != nullptr;
     a.logprobs = nullptr;
+    a.prompt_key = nullptr;
     return a;
 }
 static_assert(sizeof(DecodeArgs) <= sizeof(GraphKey::args), "graph key too small for the decode arguments");
@@ -707,12 +716,12 @@ int decode_launches(pc_ctx* ctx, cudaStream_t st, int m_bound, int groups_bound,
         const int chunks = pc::sample_chunks(m_bound, ctx->num_sms);
         if (chunks == 1) {
             pc::sample_kernel<<<m_bound, 256, 0, st>>>(sd, ctx->d.vocab, logits, nullptr, a.temperature, k0, k1, a.row_prompt,
-                                                       a.row_rollout, a.row_step, 1, a.tokens, a.row_tok_index, 1, nullptr);
+                                                       a.row_rollout, a.row_step, 1, a.tokens, a.row_tok_index, 1, nullptr, a.prompt_key);
             count_launches(1);
         } else {
             pc::Top2Rec* scratch = reinterpret_cast<pc::Top2Rec*>(ctx->ws + ctx->cv.sample_scratch);
             pc::sample_partial_kernel<<<dim3(m_bound, chunks), 256, 0, st>>>(sd, ctx->d.vocab, chunks, logits, nullptr, a.temperature,
-                                                                             k0, k1, a.row_prompt, a.row_rollout, a.row_step, 1, scratch);
+                                                                             k0, k1, a.row_prompt, a.row_rollout, a.row_step, 1, scratch, a.prompt_key);
             pc::sample_reduce_kernel<<<(m_bound + 127) / 128, 128, 0, st>>>(sd, m_bound, chunks, scratch, a.tokens, a.row_tok_index, 1,
                                                                             nullptr);
             count_launches(2);
@@ -743,6 +752,7 @@ int pc_decode_step(pc_ctx* ctx, void* stream, int n_rows, const int32_t* row_pro
                                           prompt_len, prompt_kv, prompt_slots, prompt_kv_start, suffix_kv, suffix_slots, sample);
     if (int rc = check_decode_args(ctx, a)) return rc;
     a.logprobs = ctx->logprobs;
+    a.prompt_key = ctx->prompt_key;
     if (n_groups == 0 || max_group_rows == 0 || max_group_rows > n_rows || n_groups > n_rows) return PC_ERR_INVALID_ARG;
     if (logits_out == nullptr && sample == nullptr) return PC_ERR_INVALID_ARG;
     if (logits_out && !aligned(logits_out, 16)) return PC_ERR_ALIGNMENT;
@@ -770,6 +780,7 @@ int pc_decode_run(pc_ctx* ctx, void* stream, int n_steps, const pc_step_desc* st
                                           prompt_len, prompt_kv, prompt_slots, prompt_kv_start, suffix_kv, suffix_slots, sample);
     if (int rc = check_decode_args(ctx, a)) return rc;
     a.logprobs = ctx->logprobs;
+    a.prompt_key = ctx->prompt_key;
     int groups_bound = 0, group_rows_bound = 0;
     for (int s = 0; s < n_steps; ++s) {
         const pc_step_desc& d = steps_host[s];
@@ -855,12 +866,12 @@ int pc_sample(void* stream, int n_rows, int vocab, const float* logits, const in
     }
     if (chunks == 1) {
         pc::sample_kernel<<<n_rows, 256, 0, st>>>(nullptr, vocab, logits, logits_row, temperature, k0, k1, row_prompt, row_rollout,
-                                                  row_step, 0, out_tokens, out_index, 0, out_top2_gap);
+                                                  row_step, 0, out_tokens, out_index, 0, out_top2_gap, nullptr);
         count_launches(1);
     } else {
         pc::Top2Rec* rec = static_cast<pc::Top2Rec*>(scratch);
         pc::sample_partial_kernel<<<dim3(n_rows, chunks), 256, 0, st>>>(nullptr, vocab, chunks, logits, logits_row, temperature, k0, k1,
-                                                                        row_prompt, row_rollout, row_step, 0, rec);
+                                                                        row_prompt, row_rollout, row_step, 0, rec, nullptr);
         pc::sample_reduce_kernel<<<(n_rows + 127) / 128, 128, 0, st>>>(nullptr, n_rows, chunks, rec, out_tokens, out_index, 0,
                                                                        out_top2_gap);
         count_launches(2);
@@ -979,7 +990,7 @@ int pc_sample_static(void* stream, int n_rows, int vocab, const float* logits, c
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // every record the second kernel reads is written by the first one in this same call: nothing has to start at zero
     pc::sample_partial_kernel<<<dim3(n_rows, chunks), 256, 0, st>>>(nullptr, vocab, chunks, logits, logits_row, temperature, k0, k1,
-                                                                    row_prompt, row_rollout, row_step, 0, rec);
+                                                                    row_prompt, row_rollout, row_step, 0, rec, nullptr);
     pc::sample_reduce_kernel<<<(n_rows + 127) / 128, 128, 0, st>>>(nullptr, n_rows, chunks, rec, out_tokens, out_index, 0, out_top2_gap);
     count_launches(2);
     PC_CUDA_CHECK_LAUNCH("sample (static scratch)");

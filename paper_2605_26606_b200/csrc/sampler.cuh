@@ -163,7 +163,7 @@ __global__ void __launch_bounds__(256) sample_kernel(const StepDesc* __restrict_
                                                      const int32_t* __restrict__ row_rollout, const int32_t* __restrict__ row_step,
                                                      int step_offset, int32_t* __restrict__ out_tokens,
                                                      const int64_t* __restrict__ out_index, int64_t out_index_offset,
-                                                     float* __restrict__ out_gap) {
+                                                     float* __restrict__ out_gap, const int32_t* __restrict__ prompt_key) {
     const int r = blockIdx.x;
     int64_t ro = r;                         // index into the caller's row arrays
     if (sd != nullptr) {
@@ -171,7 +171,8 @@ __global__ void __launch_bounds__(256) sample_kernel(const StepDesc* __restrict_
         ro += sd->row_off;
     }
     const float* lg = logits + (size_t)(logits_row ? logits_row[ro] : r) * vocab;
-    const uint32_t c1 = (uint32_t)(row_step[ro] + step_offset), c2 = (uint32_t)row_rollout[ro], c3 = (uint32_t)row_prompt[ro];
+    const uint32_t c1 = (uint32_t)(row_step[ro] + step_offset), c2 = (uint32_t)row_rollout[ro],
+                   c3 = (uint32_t)(prompt_key ? prompt_key[row_prompt[ro]] : row_prompt[ro]);    // key id of the prompt
     Top2 t{-INFINITY, -INFINITY, 0x7fffffff};
     const int n_blocks = (vocab + 3) >> 2;
     __shared__ float red[33];
@@ -204,7 +205,8 @@ __global__ void __launch_bounds__(256) sample_partial_kernel(const StepDesc* __r
                                                              const float* __restrict__ logits, const int32_t* __restrict__ logits_row,
                                                              float temperature, uint32_t k0, uint32_t k1,
                                                              const int32_t* __restrict__ row_prompt, const int32_t* __restrict__ row_rollout,
-                                                             const int32_t* __restrict__ row_step, int step_offset, Top2Rec* __restrict__ scratch) {
+                                                             const int32_t* __restrict__ row_step, int step_offset, Top2Rec* __restrict__ scratch,
+                                                             const int32_t* __restrict__ prompt_key) {
     const int r = blockIdx.x, chunk = blockIdx.y;
     int64_t ro = r;
     if (sd != nullptr) {
@@ -212,7 +214,8 @@ __global__ void __launch_bounds__(256) sample_partial_kernel(const StepDesc* __r
         ro += sd->row_off;
     }
     const float* lg = logits + (size_t)(logits_row ? logits_row[ro] : r) * vocab;
-    const uint32_t c1 = (uint32_t)(row_step[ro] + step_offset), c2 = (uint32_t)row_rollout[ro], c3 = (uint32_t)row_prompt[ro];
+    const uint32_t c1 = (uint32_t)(row_step[ro] + step_offset), c2 = (uint32_t)row_rollout[ro],
+                   c3 = (uint32_t)(prompt_key ? prompt_key[row_prompt[ro]] : row_prompt[ro]);    // key id of the prompt
     Top2 t{-INFINITY, -INFINITY, 0x7fffffff};
     const int n_blocks = (vocab + 3) >> 2;
     const int per_chunk = (n_blocks + n_chunks - 1) / n_chunks;

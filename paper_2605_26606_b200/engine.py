@@ -94,6 +94,7 @@ class RolloutEngine:
         self._arenas: Dict[str, Optional[torch.Tensor]] = {}
         self.profile_every = 0
         self.use_graphs = True
+        self.prompt_key_host: Optional[np.ndarray] = None    # sampling-key id per prompt (None: the prompt's index)
         self.collect_logprobs = False       # also keep log pi(o_t) of every sampled token (Eq. 2's denominator)
         self.record_pilot_logits: Optional[dict] = None     # {decode step: None} -> filled during the pilot stage
         self.profile_layer = m.n_layers // 2
@@ -147,6 +148,9 @@ class RolloutEngine:
         self.tokens = torch.full((P * G * wl.max_new,), -1, dtype=torch.int32, device=dev)
         self.logprobs = torch.zeros(P * G * wl.max_new, dtype=torch.float32, device=dev) if self.collect_logprobs else None
         B.pc_set_logprob_buffer(self.ctx, self.logprobs)
+        self.prompt_key_host = None
+        self.prompt_key_dev = None
+        B.pc_set_prompt_keys(self.ctx, None)
         self.last_logits = torch.empty((P, self.model.vocab), dtype=torch.float32, device=dev)
         self.rewards = torch.zeros(P * G, dtype=torch.float32, device=dev)
         self.adv = torch.zeros(P * G, dtype=torch.float32, device=dev)
@@ -219,11 +223,12 @@ class RolloutEngine:
         sp = B.SampleParams(wl.temperature, wl.sample_seed)
         d_p = torch.from_numpy(prompts.astype(np.int32)).to(dev)
         d_r = torch.from_numpy(rollouts.astype(np.int32)).to(dev)
+        d_key = d_p if self.prompt_key_host is None else torch.from_numpy(self.prompt_key_host[prompts].astype(np.int32)).to(dev)
         d_zero = torch.zeros(n, dtype=torch.int32, device=dev)
         rid = prompts.astype(np.int64) * wl.group_size + rollouts
         d_first = torch.from_numpy(rid * wl.max_new).to(dev)
         if not teacher_forced and step_range is None:
-            B.pc_sample(n, self.model.vocab, self.last_logits, d_p, wl.temperature, wl.sample_seed, d_p, d_r, d_zero,
+            B.pc_sample(n, self.model.vocab, self.last_logits, d_p, wl.temperature, wl.sample_seed, d_key, d_r, d_zero,
                         self.tokens, out_index=d_first)
             if self.logprobs is not None:
                 B.pc_token_logprob(n, self.model.vocab, self.last_logits, d_p, wl.temperature, self.tokens, d_first, self.logprobs,
@@ -308,6 +313,56 @@ class RolloutEngine:
                          self.union_var)
         B.pc_grpo_advantage(P, self.rewards, self.group_start, union_count, self.status, self.adv)
         return status, n_tok
+
+    def bound_pass(self, wl: Workload, batch_a: Batch, commit_a: np.ndarray, batch_b: Batch) -> dict:
+        """Section 3.4, "Binding pilot and commit": ONE inference pass that generates the commit rollouts (k .. G-1) of the
+        prompts `commit_a` of batch A together with the pilot rollouts (0 .. k-1) of the new batch B.
+
+        Must follow the pass that ran A's pilot rollouts on this engine: A's prompt KV and last-position logits are taken
+        over from it (the prompt is not evaluated again), B is prefilled.  Rollouts keep the sampling keys they would have
+        had in separate passes, so their tokens do not depend on the binding.
+        Returns {"a": {(p, i): tokens}, "b": {(p, i): tokens}} with the prompts' indices in their own batches."""
+        dev, G, k = self.device, wl.group_size, wl.n_pilot
+        commit_a = np.asarray(commit_a, dtype=np.int64)
+        nA, PB = len(commit_a), len(batch_b.prompt_lens)
+        old_kv, old_start, old_last = self.prompt_kv, self.batch.prompt_offsets[:-1].astype(np.int64), self.last_logits
+        lens = np.concatenate([batch_a.prompt_lens[commit_a], batch_b.prompt_lens]).astype(np.int32)
+        offsets = np.zeros(nA + PB + 1, dtype=np.int32)
+        offsets[1:] = np.cumsum(lens)
+        toks_a = [batch_a.prompt_tokens[batch_a.prompt_offsets[p]:batch_a.prompt_offsets[p + 1]] for p in commit_a]
+        comb = Batch(lens, offsets, np.concatenate(toks_a + [batch_b.prompt_tokens]).astype(np.int32),
+                     np.concatenate([batch_a.tau[commit_a], batch_b.tau]),
+                     np.concatenate([batch_a.reward_threshold[commit_a], batch_b.reward_threshold]).astype(np.int32),
+                     np.concatenate([batch_a.caps[commit_a], batch_b.caps]).astype(np.int32))
+        wl_c = dataclasses.replace(wl, n_prompts=nA + PB)
+        self._arenas["prompt"] = None                       # keep A's arena alive through old_kv while the new one is filled
+        self.load_batch(wl_c, comb)
+        for j, p in enumerate(commit_a):                    # A's prompt KV stays what its own pass computed
+            L, s_old, s_new = int(batch_a.prompt_lens[p]), int(old_start[p]), int(offsets[j])
+            self.prompt_kv[:, :, :, s_new:s_new + L] = old_kv[:, :, :, s_old:s_old + L]
+        self.last_logits[:nA] = old_last[torch.from_numpy(commit_a).to(dev)]
+        if PB:
+            off0 = int(offsets[nA])
+            offs_b = torch.from_numpy((offsets[nA:] - off0).astype(np.int32)).to(dev)
+            B.pc_prefill_shared(self.ctx, PB, self.prompt_tokens[off0:], offs_b, int(offsets[-1]) - off0,
+                                int(batch_b.prompt_lens.max()), self.prompt_kv, self.total_prompt_tokens,
+                                self.prompt_kv_start[nA:], self.last_logits[nA:])
+        self.prompt_key_host = np.concatenate([commit_a, np.arange(PB)]).astype(np.int32)
+        self.prompt_key_dev = torch.from_numpy(self.prompt_key_host).to(dev)
+        B.pc_set_prompt_keys(self.ctx, self.prompt_key_dev)
+        prompts = np.concatenate([np.repeat(np.arange(nA), G - k), np.repeat(nA + np.arange(PB), k)])
+        rollouts = np.concatenate([np.tile(np.arange(k, G), nA), np.tile(np.arange(k), PB)])
+        self.run_stage(prompts, rollouts)
+        self.check_error_flag()
+        toks = self.tokens.cpu().numpy().reshape(nA + PB, G, wl.max_new)
+        out = {"a": {}, "b": {}}
+        for j, p in enumerate(commit_a):
+            for i in range(k, G):
+                out["a"][(int(p), i)] = toks[j, i, :batch_a.caps[p, i]].copy()
+        for p in range(PB):
+            for i in range(k):
+                out["b"][(p, i)] = toks[nA + p, i, :batch_b.caps[p, i]].copy()
+        return out
 
     def collect(self, status: np.ndarray) -> dict:
         wl, P, G, k = self.wl, self.wl.n_prompts, self.wl.group_size, self.wl.n_pilot

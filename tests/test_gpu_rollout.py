@@ -193,3 +193,30 @@ def test_behaviour_logprobs_along_free_running_rollouts():
                 assert abs(out["logprobs"][p, i, s] - token_logprob(logs[s], int(t), w.temperature)) < 1e-4
                 n_checked += 1
     assert n_checked == int(batch.caps[out["generated"]].sum())
+
+
+def test_bound_pilot_and_commit_pass_gives_the_same_rollouts():
+    """Section 3.4 binding: commit rollouts of batch A's survivors and pilot rollouts of batch B in one decode batch are
+    token for token what separate passes produce (A's prompt KV is taken over, not recomputed)."""
+    w = dataclasses.replace(wl.WORKLOADS["config0"], n_prompts=4, prompt_len_lo=5, prompt_len_hi=40, cap_lo=3, cap_hi=16,
+                            forced_explicit=((0, 0.5), (1, 0.0), (2, 0.5), (3, 0.5)), data_seed=31)
+    wb = dataclasses.replace(w, data_seed=32, n_prompts=3, forced_explicit=None)
+    weights = wl.gen_weights(w.model, seed=0, threads=2)
+    batch_a, batch_b = wl.gen_batch(w), wl.gen_batch(wb)
+    P, G, k = w.n_prompts, w.group_size, w.n_pilot
+    eng = RolloutEngine(w.model, weights, max_rows=64, max_prefill_tokens=int(batch_a.prompt_offsets[-1] + batch_b.prompt_offsets[-1]))
+    # separate passes
+    full_a = eng.pilot_commit_step(w, batch_a)
+    commit_a = np.flatnonzero(full_a["status"] == ostats.COMMIT)
+    assert 0 < len(commit_a) < P
+    full_b = eng.pilot_commit_step(wb, batch_b)
+    # bound: A's pilot pass, then one pass with A's commit rows and B's pilot rows
+    eng.load_batch(w, batch_a)
+    eng.prefill()
+    eng.run_stage(np.repeat(np.arange(P), k), np.tile(np.arange(k), P))
+    bound = eng.bound_pass(w, batch_a, commit_a, batch_b)
+    assert len(bound["a"]) == len(commit_a) * (G - k) and len(bound["b"]) == wb.n_prompts * k
+    for (p, i), t in bound["a"].items():
+        assert np.array_equal(t, full_a["tokens"][p][i]), (p, i)
+    for (p, i), t in bound["b"].items():
+        assert np.array_equal(t, full_b["tokens"][p][i]), (p, i)
