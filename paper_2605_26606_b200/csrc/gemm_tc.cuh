@@ -6,8 +6,10 @@
 // epilogue, so the epilogue of tile i overlaps the main loop of tile i+1.  Tiles are ordered M-fastest:
 // CTAs running together share the same weight tile, which therefore leaves HBM once.
 //
-// Every output element accumulates its K products in the same order whatever M is, so a rollout's
-// activations do not depend on which other rollouts share its batch.
+// K may be cut into `splits` slices handled by different CTAs (small batches: otherwise a handful of CTAs would
+// stream the whole weight matrix); every slice leaves its own partial sum and the consuming kernel adds them in
+// slice order, so results are deterministic.  With DUAL the activations arrive as a bf16 value plus its bf16
+// rounding remainder and both are multiplied with the same weight tile.
 //
 // All waits on mbarriers are bounded; a wait that runs out raises DEV_ERR_WAIT_TIMEOUT in the caller's
 // error flag, every role leaves its loop, and the CTA frees its TMEM before it returns.
