@@ -289,7 +289,8 @@ int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, in
     // a group with few query rows keeps few CTAs busy: cut its prompt into ranges so that about one CTA per SM runs
     const int q_tiles = (plan.max_group_rows * n_rep + am::G_QROWS - 1) / am::G_QROWS;
     const int base_ctas = std::max(1, q_tiles * d.n_kv_heads * plan.n_groups);
-    const int n_parts = plan.prefill ? 1 : std::max(1, std::min(am::MAX_PREFIX_PARTS, c->num_sms / base_ctas));
+    // (two of these CTAs fit on an SM)
+    const int n_parts = plan.prefill ? 1 : std::max(1, std::min(am::MAX_PREFIX_PARTS, 2 * c->num_sms / base_ctas));
     am::PrefixPartial part{reinterpret_cast<float*>(c->ws + c->cv.part_m), reinterpret_cast<float*>(c->ws + c->cv.part_l),
                            reinterpret_cast<float*>(c->ws + c->cv.part_o), n_parts, (size_t)std::max(c->max_rows, 1) * d.n_q_heads, 0};
     // few (rollout, KV head) streams per warp: cut the suffixes into chunks of at least 4 tiles so that the load balances
