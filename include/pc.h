@@ -147,6 +147,14 @@ PC_API int pc_workspace_bytes(const pc_ctx* ctx, int max_rows, int max_prefill_t
 PC_API int pc_set_workspace(pc_ctx* ctx, void* dev_ws, size_t bytes, int max_rows, int max_prefill_tokens,
                      int32_t* dev_error_flag);
 
+/* Tuning aid: forces the tile width (64 or 256 output columns) and the number of K-slices of the bf16 tensor-core
+ * GEMMs instead of the built-in choice.  spec (host string) is a comma-separated list of name=WIDTHxSLICES with name
+ * in {qkv, o, gu, dn, lm} (QKV, output, gate/up, down projection, LM head), e.g. "dn=256x4,o=64x2"; names left out,
+ * NULL or "" keep the built-in choice.  The slice count is clamped to what the workspace holds for the step's row
+ * bound; gate/up and the LM head never split.  Results stay deterministic for a fixed plan.  Drops captured decode
+ * steps.  The paper has no counterpart. */
+PC_API int pc_set_gemm_plan(pc_ctx* ctx, const char* spec);
+
 /* Measurement aid: in the next pc_decode_step of this context, record the two CUDA events (cudaEvent_t,
  * created by the caller) around the attention kernel of `layer` that reads the rollouts' own suffix K/V
  * (for float32 models: the single attention kernel).  One-shot; the caller synchronises and reads the

@@ -42,7 +42,7 @@ int cuda_fail(cudaError_t e, const char* what) {
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-constexpr size_t kSplitMaxRows = 512;   // GEMMs over more rows are never split along K
+constexpr size_t kSplitMaxRows = 512;   // row count up to which the partial-sum buffers hold kMaxSplits K-slices; narrow tiles split only up to here
 constexpr int kMaxSplits = 8;
 
 struct Carve {
@@ -98,6 +98,10 @@ struct pc_ctx {
     cudaEvent_t prof_start = nullptr, prof_stop = nullptr;
     float* logprobs = nullptr;       // pc_set_logprob_buffer
     const int32_t* prompt_key = nullptr;    // pc_set_prompt_keys
+
+    // tile width / K-split forced through pc_set_gemm_plan (0 = built-in choice), indexed by GemmKind
+    int plan_bn[5] = {0, 0, 0, 0, 0}, plan_splits[5] = {0, 0, 0, 0, 0};
+    size_t split_capacity_rows = 0;          // rows x K-slices the partial-sum buffers hold
 
     std::vector<GraphEntry> graphs;
     cudaStream_t capture_stream = nullptr;      // decode steps are captured here (the caller's stream may be the default one)
@@ -186,16 +190,30 @@ struct GemmPlan {
     bool wide;
     int splits;
 };
-GemmPlan plan_gemm(const pc_ctx* c, const WMap& w, int M, bool may_split) {
+enum GemmKind { GEMM_QKV = 0, GEMM_O = 1, GEMM_GATE_UP = 2, GEMM_DOWN = 3, GEMM_LM_HEAD = 4 };
+GemmPlan plan_gemm(const pc_ctx* c, GemmKind kind, const WMap& w, int M, bool may_split) {
     const int tiles_m = (M + pc::tc::BM - 1) / pc::tc::BM;
+    const int k_blocks = w.K / pc::tc::BK;
+    // K-slices the partial-sum buffers can hold for M rows, and never fewer than 4 k-blocks per slice
+    const int max_splits = !may_split ? 1 : std::max(1, std::min(std::min((int)(c->split_capacity_rows / (size_t)std::max(M, 1)), kMaxSplits), k_blocks / 4));
     GemmPlan p{true, 1};
-    if (tiles_m * ((w.N + 255) / 256) >= c->num_sms / 2) return p;
+    if (c->plan_bn[kind] != 0) {
+        p.wide = c->plan_bn[kind] == 256;
+        p.splits = std::max(1, std::min(c->plan_splits[kind], max_splits));
+        return p;
+    }
+    const int tiles_wide = tiles_m * ((w.N + 255) / 256);
+    if (tiles_wide >= c->num_sms / 2) return p;
+    // Too few wide tiles to keep the SMs busy.  A wide tile moves half as many bytes from L2 into shared memory per
+    // flop as a narrow one, so from three row tiles on (and enough K per tile for that traffic to matter; crossover
+    // measured on the 1.5B shape at 128..896 rows) the wide tile stays and K is split until about every SM has a CTA.
+    if (may_split && tiles_m >= 3 && (long long)tiles_m * w.K >= 7680) {
+        p.splits = std::max(1, std::min(c->num_sms / tiles_wide, max_splits));
+        return p;
+    }
     p.wide = false;
     const int tiles = tiles_m * ((w.N + 63) / 64);
-    if (may_split && (size_t)M <= kSplitMaxRows) {
-        const int k_blocks = w.K / pc::tc::BK;
-        p.splits = std::max(1, std::min(std::min(c->num_sms / tiles, kMaxSplits), k_blocks / 4));
-    }
+    if ((size_t)M <= kSplitMaxRows) p.splits = std::max(1, std::min(c->num_sms / tiles, max_splits));
     return p;
 }
 
@@ -364,7 +382,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
             launch_gemm_simt<T>(st, sd, a, reinterpret_cast<const T*>(c->wqkv[l]), M, c->n_qkv(), d.d_model,
                                 EpiStoreF32{qkv, c->n_qkv(), nullptr});
         } else {
-            const GemmPlan gp = plan_gemm(c, c->m_wqkv[l], M, true);
+            const GemmPlan gp = plan_gemm(c, GEMM_QKV, c->m_wqkv[l], M, true);
             qkv_parts.n = gp.splits;
             if (int rc = gemm_bf16(c, st, sd, c->map_a, &c->map_a_lo, c->m_wqkv[l], M, gp, tc::EpiPartial{qkv, c->n_qkv(), qkv_parts.stride})) return rc;
         }
@@ -388,7 +406,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
                          ? attention_bf16<128>(c, st, sd, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer)
                          : attention_bf16<64>(c, st, sd, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer);
             if (rc) return rc;
-            const GemmPlan gp = plan_gemm(c, c->m_wo[l], M, true);
+            const GemmPlan gp = plan_gemm(c, GEMM_O, c->m_wo[l], M, true);
             if (gp.splits == 1) {
                 if (int rc2 = gemm_bf16(c, st, sd, c->map_attn, &c->map_attn_lo, c->m_wo[l], M, gp, tc::EpiResidual{h, d.d_model})) return rc2;
             } else {
@@ -404,9 +422,9 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
                                 EpiSwiGLU<T>{act, d.d_ff});
             launch_gemm_simt<T>(st, sd, act, reinterpret_cast<const T*>(c->w_down[l]), M, d.d_model, d.d_ff, EpiResidual{h, d.d_model});
         } else {
-            if (int rc = gemm_bf16(c, st, sd, c->map_a, nullptr, c->m_wgu[l], M, plan_gemm(c, c->m_wgu[l], M, false), tc::EpiSwiGLU{act, d.d_ff}))
+            if (int rc = gemm_bf16(c, st, sd, c->map_a, nullptr, c->m_wgu[l], M, plan_gemm(c, GEMM_GATE_UP, c->m_wgu[l], M, false), tc::EpiSwiGLU{act, d.d_ff}))
                 return rc;
-            const GemmPlan gp = plan_gemm(c, c->m_wdown[l], M, true);
+            const GemmPlan gp = plan_gemm(c, GEMM_DOWN, c->m_wdown[l], M, true);
             if (gp.splits == 1) {
                 if (int rc = gemm_bf16(c, st, sd, c->map_act, nullptr, c->m_wdown[l], M, gp, tc::EpiResidual{h, d.d_model})) return rc;
             } else {
@@ -435,7 +453,7 @@ int run_lm_head(pc_ctx* c, cudaStream_t st, int n, const pc::StepDesc* sd, const
         const T* wlm = reinterpret_cast<const T*>(d.tied_embed ? c->embed : c->lm_head);
         launch_gemm_simt<T>(st, sd, a, wlm, n, d.vocab, d.d_model, EpiStoreF32{logits, d.vocab, nullptr});
     } else {
-        if (int rc = gemm_bf16(c, st, sd, c->map_a, &c->map_a_lo, c->m_lm, n, plan_gemm(c, c->m_lm, n, false), tc::EpiStoreF32{logits, d.vocab, nullptr}))
+        if (int rc = gemm_bf16(c, st, sd, c->map_a, &c->map_a_lo, c->m_lm, n, plan_gemm(c, GEMM_LM_HEAD, c->m_lm, n, false), tc::EpiStoreF32{logits, d.vocab, nullptr}))
             return rc;
     }
     count_launches(2);
@@ -474,6 +492,32 @@ uint64_t pc_launch_count(void) { return g_launches; }
 int pc_set_prompt_keys(pc_ctx* ctx, const int32_t* prompt_key) {
     if (ctx == nullptr) return PC_ERR_INVALID_ARG;
     ctx->prompt_key = prompt_key;
+    return PC_OK;
+}
+
+int pc_set_gemm_plan(pc_ctx* ctx, const char* spec) {
+    if (ctx == nullptr) return PC_ERR_INVALID_ARG;
+    int bn[5] = {0, 0, 0, 0, 0}, sp[5] = {0, 0, 0, 0, 0};
+    static const char* const names[5] = {"qkv", "o", "gu", "dn", "lm"};
+    const char* p = spec ? spec : "";
+    while (*p) {
+        int kind = -1;
+        size_t len = 0;
+        for (int k = 0; k < 5; ++k) {
+            const size_t n = std::strlen(names[k]);
+            if (std::strncmp(p, names[k], n) == 0 && p[n] == '=') { kind = k; len = n + 1; }
+        }
+        if (kind < 0) return PC_ERR_INVALID_ARG;
+        int w = 0, s = 0, used = 0;
+        if (std::sscanf(p + len, "%dx%d%n", &w, &s, &used) != 2) return PC_ERR_INVALID_ARG;
+        if ((w != 64 && w != 256) || s < 1 || s > kMaxSplits) return PC_ERR_INVALID_ARG;
+        bn[kind] = w; sp[kind] = s;
+        p += len + used;
+        if (*p == ',') ++p;
+        else if (*p) return PC_ERR_INVALID_ARG;
+    }
+    for (int k = 0; k < 5; ++k) { ctx->plan_bn[k] = bn[k]; ctx->plan_splits[k] = sp[k]; }
+    ctx->drop_graphs();          // captured steps carry the old choice
     return PC_OK;
 }
 
@@ -594,6 +638,7 @@ int pc_set_workspace(pc_ctx* ctx, void* dev_ws, size_t bytes, int max_rows, int 
     ctx->max_prefill = max_prefill_tokens;
     ctx->err = dev_error_flag;
     ctx->cv = cv;
+    ctx->split_capacity_rows = std::min<size_t>((size_t)std::max(max_rows, max_prefill_tokens), kSplitMaxRows) * kMaxSplits;
     ctx->drop_graphs();
     if (ctx->d.dtype == PC_DTYPE_BF16) {
         cudaError_t ce = configure_kernels();
