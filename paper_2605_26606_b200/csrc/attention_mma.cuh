@@ -145,6 +145,35 @@ attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __
     }
     __syncthreads();
 
+    // Decode: the rows of a group share their prompt, so the visible prompt length is known from the group's first
+    // row and the first K/V tiles are requested before anything else is loaded.  Prefill: every row sees its own
+    // prefix; the longest one of the tile is found below.
+    const int64_t kv_start = g.p_start[row0];
+    const int64_t krow0 = (((int64_t)layer * 2 + 0) * Hkv + kvh) * n_slots + kv_start;
+    const int64_t vrow0 = (((int64_t)layer * 2 + 1) * Hkv + kvh) * n_slots + kv_start;
+    auto issue = [&](int tile, int stage) {
+        const uint32_t kb = tiles_u32 + stage * 2 * TILE_BYTES, vb = kb + TILE_BYTES;
+        mbar_arrive_expect_tx(full0 + 8 * stage, 2 * TILE_BYTES);
+#pragma unroll
+        for (int b = 0; b < HD / 64; ++b) {
+            tma_load_2d(kb + b * (G_TK * 128), &kv_map, full0 + 8 * stage, b * 64, (int)(krow0 + (int64_t)tile * G_TK));
+            tma_load_2d(vb + b * (G_TK * 128), &kv_map, full0 + 8 * stage, b * 64, (int)(vrow0 + (int64_t)tile * G_TK));
+        }
+    };
+    int max_len = 0, tile0 = 0, n_tiles = 0;
+    auto set_range = [&](int len) {
+        max_len = len;
+        const int n_tiles_all = (max_len + G_TK - 1) / G_TK;
+        const int tiles_per_part = (n_tiles_all + n_parts - 1) / n_parts;
+        tile0 = my_part * tiles_per_part;                                // this CTA covers tiles [tile0, tile0 + n_tiles)
+        n_tiles = max(0, min(n_tiles_all, tile0 + tiles_per_part) - tile0);
+    };
+    if (!FINAL) {
+        set_range(g.p_len[row0]);
+        if (threadIdx.x == 0)
+            for (int t = 0; t < G_STAGES && t < n_tiles; ++t) issue(tile0 + t, t);
+    }
+
     // this thread's two query rows: qr = q0 + warp*16 + lane/4 (+8); query row qr = (rollout row qr / n_rep, head qr % n_rep)
     int lim[2], grow[2], head[2];
 #pragma unroll
@@ -154,8 +183,9 @@ attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __
         grow[i] = valid ? row0 + qr / n_rep : -1;
         head[i] = kvh * n_rep + (valid ? qr % n_rep : 0);
         lim[i] = valid ? g.p_len[grow[i]] : 0;
+        if (!FINAL) lim[i] = min(lim[i], max_len);
     }
-    {
+    if (FINAL) {
         int mx = max(lim[0], lim[1]);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
@@ -177,27 +207,12 @@ attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __
             qa[ks][2 + i] = hi;      // a2, a3: dims + 8
         }
     }
-    __syncthreads();
-    const int max_len = s_maxlen;
-    const int n_tiles_all = (max_len + G_TK - 1) / G_TK;
-    const int tiles_per_part = (n_tiles_all + n_parts - 1) / n_parts;
-    const int tile0 = my_part * tiles_per_part;                          // this CTA covers tiles [tile0, tile0 + n_tiles)
-    const int n_tiles = max(0, min(n_tiles_all, tile0 + tiles_per_part) - tile0);
-    const int64_t kv_start = g.p_start[row0];
-    const int64_t krow0 = (((int64_t)layer * 2 + 0) * Hkv + kvh) * n_slots + kv_start;
-    const int64_t vrow0 = (((int64_t)layer * 2 + 1) * Hkv + kvh) * n_slots + kv_start;
-
-    auto issue = [&](int tile, int stage) {
-        const uint32_t kb = tiles_u32 + stage * 2 * TILE_BYTES, vb = kb + TILE_BYTES;
-        mbar_arrive_expect_tx(full0 + 8 * stage, 2 * TILE_BYTES);
-#pragma unroll
-        for (int b = 0; b < HD / 64; ++b) {
-            tma_load_2d(kb + b * (G_TK * 128), &kv_map, full0 + 8 * stage, b * 64, (int)(krow0 + (int64_t)tile * G_TK));
-            tma_load_2d(vb + b * (G_TK * 128), &kv_map, full0 + 8 * stage, b * 64, (int)(vrow0 + (int64_t)tile * G_TK));
-        }
-    };
-    if (threadIdx.x == 0)
-        for (int t = 0; t < G_STAGES && t < n_tiles; ++t) issue(tile0 + t, t);
+    if (FINAL) {
+        __syncthreads();
+        set_range(s_maxlen);
+        if (threadIdx.x == 0)
+            for (int t = 0; t < G_STAGES && t < n_tiles; ++t) issue(tile0 + t, t);
+    }
 
     float o[DT][4];
 #pragma unroll

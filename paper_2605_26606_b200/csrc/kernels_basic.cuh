@@ -129,10 +129,11 @@ __global__ void embed_rmsnorm_kernel(const StepDesc* __restrict__ sd, int d, con
 // the order s = 0, 1, ... so that the result does not depend on which CTA finished first.
 struct Partials {
     const float* p;
-    int n;              // 0: nothing pending
+    int n;              // 0: nothing pending; at most PARTIALS_MAX
     size_t stride;
     int ld;
 };
+constexpr int PARTIALS_MAX = 8;
 
 // Optional residual update followed by the norm:  h[row, :] += pending partial sums of row r;  a[r, :] = RMSNorm(h[row, :]; gain)
 // with row = src ? src[r] : r.  The partial sums are indexed by row, like h.
@@ -170,10 +171,16 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const StepDesc* __restrict
         if (i < n4) {
             v[k] = x[i];
             if (pend.n > 0) {
-                for (int s = 0; s < pend.n; ++s) {
-                    const float4 p = *reinterpret_cast<const float4*>(pend.p + (size_t)s * pend.stride + (size_t)row * pend.ld + 4 * i);
-                    v[k].x += p.x; v[k].y += p.y; v[k].z += p.z; v[k].w += p.w;
-                }
+                // all slices are requested before the first one is added (the adds stay in slice order): a loop that
+                // loads and adds one slice at a time pays the memory latency once per slice
+                float4 p[PARTIALS_MAX];
+#pragma unroll
+                for (int s = 0; s < PARTIALS_MAX; ++s)
+                    p[s] = s < pend.n ? *reinterpret_cast<const float4*>(pend.p + (size_t)s * pend.stride + (size_t)row * pend.ld + 4 * i)
+                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int s = 0; s < PARTIALS_MAX; ++s)
+                    if (s < pend.n) { v[k].x += p[s].x; v[k].y += p[s].y; v[k].z += p[s].z; v[k].w += p[s].w; }
                 x[i] = v[k];
             }
             ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
@@ -214,10 +221,17 @@ __global__ void qkv_post_kernel(const StepDesc* __restrict__ sd, int Hq, int Hkv
     qkv.stride = (size_t)sd->n_rows * qkv.ld;                           // slices are packed by the live row count
     const size_t col = (size_t)head * hd + i;
     float x1 = bias ? bias[col] : 0.f, x2 = bias ? bias[col + half] : 0.f;
-    for (int s = 0; s < qkv.n; ++s) {
-        const float* src = qkv.p + (size_t)s * qkv.stride + (size_t)r * qkv.ld + col;
-        x1 += src[0];
-        x2 += src[half];
+    {
+        float p1[PARTIALS_MAX], p2[PARTIALS_MAX];          // requested together, added in slice order
+#pragma unroll
+        for (int s = 0; s < PARTIALS_MAX; ++s) {
+            const float* src = qkv.p + (size_t)s * qkv.stride + (size_t)r * qkv.ld + col;
+            p1[s] = s < qkv.n ? src[0] : 0.f;
+            p2[s] = s < qkv.n ? src[half] : 0.f;
+        }
+#pragma unroll
+        for (int s = 0; s < PARTIALS_MAX; ++s)
+            if (s < qkv.n) { x1 += p1[s]; x2 += p2[s]; }
     }
     const bool is_q = head < Hq, is_k = !is_q && head < Hq + Hkv;
     if (is_q || is_k) {

@@ -43,7 +43,7 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 constexpr size_t kSplitMaxRows = 512;   // row count up to which the partial-sum buffers hold kMaxSplits K-slices; narrow tiles split only up to here
-constexpr int kMaxSplits = 8;
+constexpr int kMaxSplits = pc::PARTIALS_MAX;
 
 struct Carve {
     size_t h, a, qkv, q, attn, act, logits, rope, pos, wslot, warena, p_start, p_len, s_start, s_len, token, last_row,
