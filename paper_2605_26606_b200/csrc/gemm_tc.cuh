@@ -16,6 +16,7 @@
 #pragma once
 
 #include <cuda.h>
+#include <cuda_fp16.h>
 
 #include "common.cuh"
 
@@ -127,9 +128,10 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
     return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
-// Instruction descriptor: D = F32, A = B = BF16, both K-major, N >> 3 at bit 17, M >> 4 at bit 24.
-__host__ __device__ constexpr uint32_t make_idesc(int m, int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+// Instruction descriptor: D = F32, A and B both BF16 (format 1) or both IEEE half (format 0), both K-major,
+// N >> 3 at bit 17, M >> 4 at bit 24.
+__host__ __device__ constexpr uint32_t make_idesc(int m, int n, bool half_operands) {
+    return (1u << 4) | (half_operands ? 0u : ((1u << 7) | (1u << 10))) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -156,7 +158,7 @@ struct EpiStoreF32 {            // C = acc (+ bias)
 };
 struct EpiPartial {             // P[split][row][col] = acc   (raw K-slice sums; the consumer adds the slices in order)
     float* P; int ld; size_t split_stride;
-    __device__ __forceinline__ void set_rows(int m) { split_stride = (size_t)m * ld; }     // slices packed by live rows
+    __device__ __forceinline__ void set_rows(int m) { split_stride = (size_t)m * ld; }     // slices packed by the row bound
     __device__ __forceinline__ void operator()(int row, int col0, const float* v, int n_valid, int split) const {
         float* dst = P + (size_t)split * split_stride + (size_t)row * ld + col0;
         if (n_valid == 32 && (ld & 3) == 0) {
@@ -188,8 +190,8 @@ struct EpiResidual {            // H += acc
         }
     }
 };
-struct EpiSwiGLU {              // columns (2j, 2j+1) = (gate_j, up_j) -> out[row, j] = silu(gate) * up, bf16
-    __nv_bfloat16* out; int ld;
+struct EpiSwiGLU {              // columns (2j, 2j+1) = (gate_j, up_j) -> out[row, j] = silu(gate) * up, bf16 (or IEEE half)
+    __nv_bfloat16* out; int ld; int half_out;
     __device__ __forceinline__ void set_rows(int) {}
     __device__ __forceinline__ void operator()(int row, int col0, const float* v, int n_valid, int /*split*/) const {
         __nv_bfloat16* dst = out + (size_t)row * ld + (col0 >> 1);
@@ -198,15 +200,25 @@ struct EpiSwiGLU {              // columns (2j, 2j+1) = (gate_j, up_j) -> out[ro
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const float g0 = v[4 * i], u0 = v[4 * i + 1], g1 = v[4 * i + 2], u1 = v[4 * i + 3];
-                const __nv_bfloat162 p = __floats2bfloat162_rn(g0 / (1.f + expf(-g0)) * u0, g1 / (1.f + expf(-g1)) * u1);
-                w[i] = *reinterpret_cast<const uint32_t*>(&p);
+                const float y0 = g0 / (1.f + expf(-g0)) * u0, y1 = g1 / (1.f + expf(-g1)) * u1;
+                if (half_out) {
+                    const __half2 p = __floats2half2_rn(y0, y1);
+                    w[i] = *reinterpret_cast<const uint32_t*>(&p);
+                } else {
+                    const __nv_bfloat162 p = __floats2bfloat162_rn(y0, y1);
+                    w[i] = *reinterpret_cast<const uint32_t*>(&p);
+                }
             }
             *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
             *reinterpret_cast<uint4*>(dst + 8) = make_uint4(w[4], w[5], w[6], w[7]);
         } else {
 #pragma unroll
             for (int i = 0; i < 32; i += 2)
-                if (i + 1 < n_valid) dst[i >> 1] = __float2bfloat16_rn(v[i] / (1.f + expf(-v[i])) * v[i + 1]);
+                if (i + 1 < n_valid) {
+                    const float y = v[i] / (1.f + expf(-v[i])) * v[i + 1];
+                    if (half_out) reinterpret_cast<__half*>(dst)[i >> 1] = __float2half_rn(y);
+                    else dst[i >> 1] = __float2bfloat16_rn(y);
+                }
         }
     }
 };
@@ -218,8 +230,10 @@ template <int BN, bool DUAL, class Epi>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_a_lo,
                const __grid_constant__ CUtensorMap map_w, const StepDesc* __restrict__ sd, int M, int N, int K, int splits, Epi epi,
-               int32_t* err) {
-    if (sd != nullptr) M = sd->n_rows;          // live row count; the grid was sized for an upper bound
+               int32_t* err, int half_operands) {
+    // M is the row bound the grid, the tile order and the layout of partial sums were sized for; a captured step
+    // may hold fewer live rows (same number of row tiles: the bound is the live count rounded up to a tile), which
+    // only the epilogue needs to know, so the loads and MMAs never wait for the step descriptor.
     epi.set_rows(M);
     constexpr int STAGES = num_stages(BN, DUAL);
     constexpr int A1_BYTES = BM * BK * 2;                    // one A tile
@@ -277,7 +291,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else if (warp == 1) {
         if (lane == 0) {
             // ---------------- MMA issuer ----------------
-            constexpr uint32_t idesc = make_idesc(BM, BN);
+            const uint32_t idesc = make_idesc(BM, BN, half_operands != 0);
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
@@ -313,6 +327,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else {
         // ---------------- epilogue warps: TMEM -> registers -> global ----------------
         const int quarter = warp & 3;                  // a warp may only read its own 32 TMEM lanes
+        const int m_live = sd != nullptr ? min(M, sd->n_rows) : M;
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
@@ -325,7 +340,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (n0 + c >= N) break;                 // warp-uniform
                 float v[32];
                 tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + c, v);
-                if (row < M) epi(row, n0 + c, v, min(32, N - (n0 + c)), sp);
+                if (row < m_live) epi(row, n0 + c, v, min(32, N - (n0 + c)), sp);
             }
             tc_fence_before();
             __syncwarp();
@@ -358,11 +373,12 @@ inline cudaError_t configure() {
 // Host launcher.  map_w must have been encoded with box_rows = BN; map_a_lo is ignored unless DUAL.
 template <int BN, bool DUAL, class Epi>
 inline cudaError_t launch(cudaStream_t st, const CUtensorMap& map_a, const CUtensorMap& map_a_lo, const CUtensorMap& map_w,
-                          const StepDesc* sd, int M, int N, int K, int splits, Epi epi, int32_t* err, int num_sms) {
+                          const StepDesc* sd, int M, int N, int K, int splits, Epi epi, int32_t* err, int num_sms, bool half_operands = false) {
     auto kern = gemm_tc_kernel<BN, DUAL, Epi>;
     const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN) * splits;
     if (tiles == 0) return cudaSuccess;
-    kern<<<tiles < num_sms ? tiles : num_sms, NUM_THREADS, smem_bytes(BN, DUAL), st>>>(map_a, map_a_lo, map_w, sd, M, N, K, splits, epi, err);
+    kern<<<tiles < num_sms ? tiles : num_sms, NUM_THREADS, smem_bytes(BN, DUAL), st>>>(map_a, map_a_lo, map_w, sd, M, N, K, splits, epi, err,
+                                                                                       half_operands ? 1 : 0);
     return cudaGetLastError();
 }
 

@@ -155,32 +155,51 @@ __device__ __forceinline__ float4 bf16_remainder(float4 v) {
 template <typename T>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const StepDesc* __restrict__ sd, int d, float* __restrict__ h,
                                                       const int32_t* __restrict__ src, Partials pend, const float* __restrict__ gain,
-                                                      float eps, T* __restrict__ a, T* __restrict__ a_lo) {
+                                                      float eps, T* __restrict__ a, T* __restrict__ a_lo, int half_out) {
     __shared__ float red[33];
     const int r = blockIdx.x;
-    if (sd != nullptr && r >= sd->n_rows) return;
-    if (pend.n > 0 && sd != nullptr) pend.stride = (size_t)sd->n_rows * pend.ld;      // slices are packed by the live row count
+    // The grid covers the row bound of the step; rows past the live count are dropped only after this row's data has
+    // been requested (buffers hold the bound, so the reads are in range): the step descriptor, the row and its
+    // pending slices then arrive together instead of one memory latency after the other.
+    const int n_live = sd != nullptr ? sd->n_rows : gridDim.x;
     const int row = src ? src[r] : r;
     float4* x = reinterpret_cast<float4*>(h + (size_t)row * d);
     const int n4 = d >> 2;
     float4 v[8];
-    float ss = 0.f;
+    float4 p[2][PARTIALS_MAX];
+    float4 gg2[2];
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
         const int i = threadIdx.x + k * 256;
         if (i < n4) {
             v[k] = x[i];
+            if (k < 2) {
+                gg2[k] = *reinterpret_cast<const float4*>(gain + 4 * i);
+#pragma unroll
+                for (int s = 0; s < PARTIALS_MAX; ++s)
+                    p[k][s] = s < pend.n ? *reinterpret_cast<const float4*>(pend.p + (size_t)s * pend.stride + (size_t)row * pend.ld + 4 * i)
+                                         : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+    }
+    if (r >= n_live) return;
+    float ss = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int i = threadIdx.x + k * 256;
+        if (i < n4) {
             if (pend.n > 0) {
-                // all slices are requested before the first one is added (the adds stay in slice order): a loop that
-                // loads and adds one slice at a time pays the memory latency once per slice
-                float4 p[PARTIALS_MAX];
+                // the adds stay in slice order
+                if (k < 2) {
 #pragma unroll
-                for (int s = 0; s < PARTIALS_MAX; ++s)
-                    p[s] = s < pend.n ? *reinterpret_cast<const float4*>(pend.p + (size_t)s * pend.stride + (size_t)row * pend.ld + 4 * i)
-                                      : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                for (int s = 0; s < PARTIALS_MAX; ++s)
-                    if (s < pend.n) { v[k].x += p[s].x; v[k].y += p[s].y; v[k].z += p[s].z; v[k].w += p[s].w; }
+                    for (int s = 0; s < PARTIALS_MAX; ++s)
+                        if (s < pend.n) { v[k].x += p[k][s].x; v[k].y += p[k][s].y; v[k].z += p[k][s].z; v[k].w += p[k][s].w; }
+                } else {
+                    for (int s = 0; s < pend.n; ++s) {
+                        const float4 q = *reinterpret_cast<const float4*>(pend.p + (size_t)s * pend.stride + (size_t)row * pend.ld + 4 * i);
+                        v[k].x += q.x; v[k].y += q.y; v[k].z += q.z; v[k].w += q.w;
+                    }
+                }
                 x[i] = v[k];
             }
             ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
@@ -192,9 +211,15 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const StepDesc* __restrict
     for (int k = 0; k < 8; ++k) {
         const int i = threadIdx.x + k * 256;
         if (i < n4) {
-            const float4 gg = *reinterpret_cast<const float4*>(gain + 4 * i);
+            const float4 gg = k < 2 ? gg2[k] : *reinterpret_cast<const float4*>(gain + 4 * i);
             const float4 y = make_float4(v[k].x * rstd * gg.x, v[k].y * rstd * gg.y, v[k].z * rstd * gg.z, v[k].w * rstd * gg.w);
-            store4<T>(a + (size_t)r * d + 4 * i, y);
+            if (sizeof(T) == 2 && half_out) {          // IEEE half instead of bfloat16 (operand of a half-precision GEMM)
+                const __half2 lo = __floats2half2_rn(y.x, y.y), hi = __floats2half2_rn(y.z, y.w);
+                *reinterpret_cast<uint2*>(a + (size_t)r * d + 4 * i) =
+                    make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+            } else {
+                store4<T>(a + (size_t)r * d + 4 * i, y);
+            }
             if (a_lo != nullptr) store4<T>(a_lo + (size_t)r * d + 4 * i, bf16_remainder(y));
         }
     }
@@ -217,8 +242,11 @@ __global__ void qkv_post_kernel(const StepDesc* __restrict__ sd, int Hq, int Hkv
                                 T* __restrict__ q_out) {
     __shared__ float red[33];
     const int r = blockIdx.x, head = blockIdx.y, i = threadIdx.x, half = hd >> 1;
-    if (r >= sd->n_rows) return;
-    qkv.stride = (size_t)sd->n_rows * qkv.ld;                           // slices are packed by the live row count
+    // rows past the live count are dropped after the loads have been requested (buffers hold the step's row bound)
+    const int n_live = sd->n_rows;
+    const float2 cs = rope[(size_t)r * half + i];
+    const int64_t slot = g.wslot[r];
+    const int to_suffix = g.warena[r];
     const size_t col = (size_t)head * hd + i;
     float x1 = bias ? bias[col] : 0.f, x2 = bias ? bias[col + half] : 0.f;
     {
@@ -233,6 +261,7 @@ __global__ void qkv_post_kernel(const StepDesc* __restrict__ sd, int Hq, int Hkv
         for (int s = 0; s < PARTIALS_MAX; ++s)
             if (s < qkv.n) { x1 += p1[s]; x2 += p2[s]; }
     }
+    if (r >= n_live) return;
     const bool is_q = head < Hq, is_k = !is_q && head < Hq + Hkv;
     if (is_q || is_k) {
         const float* gain = is_q ? q_gain : k_gain;
@@ -242,7 +271,6 @@ __global__ void qkv_post_kernel(const StepDesc* __restrict__ sd, int Hq, int Hkv
             x1 = x1 * rstd * gain[i];
             x2 = x2 * rstd * gain[i + half];
         }
-        const float2 cs = rope[(size_t)r * half + i];
         const float y1 = x1 * cs.x - x2 * cs.y;
         const float y2 = x2 * cs.x + x1 * cs.y;
         x1 = y1; x2 = y2;
@@ -253,9 +281,8 @@ __global__ void qkv_post_kernel(const StepDesc* __restrict__ sd, int Hq, int Hkv
         dst[i + half] = from_f32<T>(x2);
         return;
     }
-    const int64_t slot = g.wslot[r];
     if (slot < 0) return;
-    const KvArena ar = g.warena[r] ? suffix_arena : prompt_arena;
+    const KvArena ar = to_suffix ? suffix_arena : prompt_arena;
     const int kvh = is_k ? head - Hq : head - Hq - Hkv;
     const int64_t plane = ((int64_t)layer * 2 + (is_k ? 0 : 1)) * Hkv + kvh;
     T* dst = reinterpret_cast<T*>(ar.base) + (plane * ar.n_slots + slot) * hd;

@@ -221,14 +221,14 @@ GemmPlan plan_gemm(const pc_ctx* c, GemmKind kind, const WMap& w, int M, bool ma
 // weights (used for the projections whose input rounding would otherwise dominate the logit error).
 template <class Epi>
 int gemm_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, const CUtensorMap& map_a, const CUtensorMap* map_a_lo, const WMap& w,
-              int M, GemmPlan p, Epi epi) {
+              int M, GemmPlan p, Epi epi, bool half_operands = false) {
     cudaError_t e;
     if (map_a_lo != nullptr)
         e = p.wide ? pc::tc::launch<256, true>(st, map_a, *map_a_lo, w.wide, sd, M, w.N, w.K, p.splits, epi, c->err, c->num_sms)
                    : pc::tc::launch<64, true>(st, map_a, *map_a_lo, w.narrow, sd, M, w.N, w.K, p.splits, epi, c->err, c->num_sms);
     else
-        e = p.wide ? pc::tc::launch<256, false>(st, map_a, map_a, w.wide, sd, M, w.N, w.K, p.splits, epi, c->err, c->num_sms)
-                   : pc::tc::launch<64, false>(st, map_a, map_a, w.narrow, sd, M, w.N, w.K, p.splits, epi, c->err, c->num_sms);
+        e = p.wide ? pc::tc::launch<256, false>(st, map_a, map_a, w.wide, sd, M, w.N, w.K, p.splits, epi, c->err, c->num_sms, half_operands)
+                   : pc::tc::launch<64, false>(st, map_a, map_a, w.narrow, sd, M, w.N, w.K, p.splits, epi, c->err, c->num_sms, half_operands);
     if (e != cudaSuccess) return cuda_fail(e, "tensor-core gemm");
     return PC_OK;
 }
@@ -364,6 +364,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
     float* res_part = reinterpret_cast<float*>(w + c->cv.res_part);
     const Partials none{nullptr, 0, 0, 0};
     Partials pend = none;
+    const bool mlp_half = !kF32 && d.mlp_half != 0;      // MLP operands (weights and both activations) in IEEE half
 
     rope_table_kernel<<<(M * half + 255) / 256, 256, 0, st>>>(sd, half, (double)d.rope_theta, g.pos, rope);
     embed_rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, g.token, reinterpret_cast<const T*>(c->embed), c->attn_norm[0],
@@ -372,7 +373,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
     PC_CUDA_CHECK_LAUNCH("embed_rmsnorm");
     for (int l = 0; l < d.n_layers; ++l) {
         if (l > 0) {
-            rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, h, nullptr, pend, c->attn_norm[l], d.rms_eps, a, a_lo);
+            rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, h, nullptr, pend, c->attn_norm[l], d.rms_eps, a, a_lo, 0);
             pend = none;
             count_launches(1);
         }
@@ -414,7 +415,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
                 if (int rc2 = gemm_bf16(c, st, sd, c->map_attn, &c->map_attn_lo, c->m_wo[l], M, gp, tc::EpiPartial{res_part, d.d_model, pend.stride})) return rc2;
             }
         }
-        rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a, nullptr);
+        rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a, nullptr, mlp_half ? 1 : 0);
         pend = none;
         count_launches(2);
         if constexpr (kF32) {
@@ -422,14 +423,14 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
                                 EpiSwiGLU<T>{act, d.d_ff});
             launch_gemm_simt<T>(st, sd, act, reinterpret_cast<const T*>(c->w_down[l]), M, d.d_model, d.d_ff, EpiResidual{h, d.d_model});
         } else {
-            if (int rc = gemm_bf16(c, st, sd, c->map_a, nullptr, c->m_wgu[l], M, plan_gemm(c, GEMM_GATE_UP, c->m_wgu[l], M, false), tc::EpiSwiGLU{act, d.d_ff}))
+            if (int rc = gemm_bf16(c, st, sd, c->map_a, nullptr, c->m_wgu[l], M, plan_gemm(c, GEMM_GATE_UP, c->m_wgu[l], M, false), tc::EpiSwiGLU{act, d.d_ff, mlp_half ? 1 : 0}, mlp_half))
                 return rc;
             const GemmPlan gp = plan_gemm(c, GEMM_DOWN, c->m_wdown[l], M, true);
             if (gp.splits == 1) {
-                if (int rc = gemm_bf16(c, st, sd, c->map_act, nullptr, c->m_wdown[l], M, gp, tc::EpiResidual{h, d.d_model})) return rc;
+                if (int rc = gemm_bf16(c, st, sd, c->map_act, nullptr, c->m_wdown[l], M, gp, tc::EpiResidual{h, d.d_model}, mlp_half)) return rc;
             } else {
                 pend = Partials{res_part, gp.splits, (size_t)M * d.d_model, d.d_model};
-                if (int rc = gemm_bf16(c, st, sd, c->map_act, nullptr, c->m_wdown[l], M, gp, tc::EpiPartial{res_part, d.d_model, pend.stride})) return rc;
+                if (int rc = gemm_bf16(c, st, sd, c->map_act, nullptr, c->m_wdown[l], M, gp, tc::EpiPartial{res_part, d.d_model, pend.stride}, mlp_half)) return rc;
             }
         }
         count_launches(2);
@@ -447,7 +448,7 @@ int run_lm_head(pc_ctx* c, cudaStream_t st, int n, const pc::StepDesc* sd, const
     float* h = reinterpret_cast<float*>(c->ws + c->cv.h);
     T* a = reinterpret_cast<T*>(c->ws + c->cv.a);
     T* a_lo = std::is_same<T, float>::value ? nullptr : reinterpret_cast<T*>(c->ws + c->cv.a_lo);
-    rmsnorm_kernel<T><<<n, 256, 0, st>>>(sd, d.d_model, h, src, c->pend, c->final_norm, d.rms_eps, a, a_lo);
+    rmsnorm_kernel<T><<<n, 256, 0, st>>>(sd, d.d_model, h, src, c->pend, c->final_norm, d.rms_eps, a, a_lo, 0);
     c->pend = pc::Partials{nullptr, 0, 0, 0};
     if constexpr (std::is_same<T, float>::value) {
         const T* wlm = reinterpret_cast<const T*>(d.tied_embed ? c->embed : c->lm_head);
@@ -553,6 +554,7 @@ int pc_create(const pc_model_desc* desc, const pc_weights* wts, pc_ctx** out) {
     *out = nullptr;
     const pc_model_desc& d = *desc;
     if (d.dtype != PC_DTYPE_F32 && d.dtype != PC_DTYPE_BF16) return PC_ERR_INVALID_ARG;
+    if (d.mlp_half != 0 && (d.mlp_half != 1 || d.dtype != PC_DTYPE_BF16)) return PC_ERR_INVALID_ARG;
     if (d.n_layers <= 0 || d.d_model <= 0 || d.n_q_heads <= 0 || d.n_kv_heads <= 0 || d.d_ff <= 0 || d.vocab <= 0 ||
         !(d.rms_eps >= 0.f) || !(d.rope_theta > 0.f))
         return PC_ERR_INVALID_ARG;

@@ -20,9 +20,14 @@ from . import binding as B
 from .workloads import DTYPE_BF16, DTYPE_F32, Batch, ModelShape, Weights, Workload
 
 
-def _dev_matrix(w: Weights, names: List[str], model: ModelShape, device, interleave: bool = False) -> torch.Tensor:
-    """Concatenates (or row-interleaves) matrices and uploads them in the model's storage type."""
-    if model.dtype == DTYPE_BF16:
+def _dev_matrix(w: Weights, names: List[str], model: ModelShape, device, interleave: bool = False, half: bool = False) -> torch.Tensor:
+    """Concatenates (or row-interleaves) matrices and uploads them in the model's storage type.
+
+    half: a bf16 model's matrix is uploaded as IEEE half instead (same two bytes; a storage-format conversion of the
+    bfloat16 value, exact unless the value is below 2^-14 in magnitude)."""
+    if model.dtype == DTYPE_BF16 and half:
+        parts = [torch.from_numpy((w.bits(n).astype(np.uint32) << 16).view(np.float32).astype(np.float16).view(np.int16)) for n in names]
+    elif model.dtype == DTYPE_BF16:
         parts = [torch.from_numpy(w.bits(n).view(np.int16)) for n in names]
     else:
         parts = [torch.from_numpy(w[n]) for n in names]
@@ -60,8 +65,12 @@ class StageSchedule:
 
 
 class RolloutEngine:
-    def __init__(self, model: ModelShape, weights: Weights, max_rows: int, max_prefill_tokens: int, device="cuda:0"):
+    def __init__(self, model: ModelShape, weights: Weights, max_rows: int, max_prefill_tokens: int, device="cuda:0",
+                 mlp_half: Optional[bool] = None):
+        """mlp_half: hand the MLP matrices of a bf16 model to the library as IEEE half (pc_model_desc.mlp_half); default
+        on for bf16 models: the synthetic weights N(0, 0.02) and the unit-scale MLP activations sit well inside half's range."""
         self.model = model
+        self.mlp_half = (model.dtype == DTYPE_BF16) if mlp_half is None else bool(mlp_half)
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
         m, dev = model, self.device
@@ -78,10 +87,11 @@ class RolloutEngine:
         self.q_norm = [f32(f"layers.{l}.q_norm") for l in L] if m.qk_norm else None
         self.k_norm = [f32(f"layers.{l}.k_norm") for l in L] if m.qk_norm else None
         self.wo = [_dev_matrix(weights, [f"layers.{l}.wo"], m, dev) for l in L]
-        self.w_gate_up = [_dev_matrix(weights, [f"layers.{l}.w_gate", f"layers.{l}.w_up"], m, dev, interleave=True) for l in L]
-        self.w_down = [_dev_matrix(weights, [f"layers.{l}.w_down"], m, dev) for l in L]
+        self.w_gate_up = [_dev_matrix(weights, [f"layers.{l}.w_gate", f"layers.{l}.w_up"], m, dev, interleave=True, half=self.mlp_half)
+                          for l in L]
+        self.w_down = [_dev_matrix(weights, [f"layers.{l}.w_down"], m, dev, half=self.mlp_half) for l in L]
         desc = B.ModelDesc(m.n_layers, m.d_model, m.n_q_heads, m.n_kv_heads, m.head_dim, m.d_ff, m.vocab, m.rms_eps,
-                           m.rope_theta, m.dtype, int(m.tied_embed), int(m.qk_norm), int(m.qkv_bias))
+                           m.rope_theta, m.dtype, int(m.tied_embed), int(m.qk_norm), int(m.qkv_bias), int(self.mlp_half))
         self.ctx = B.pc_create(desc, self.embed, self.lm_head, self.final_norm, self.attn_norm, self.wqkv, self.bqkv,
                                self.q_norm, self.k_norm, self.wo, self.mlp_norm, self.w_gate_up, self.w_down)
         self.max_rows, self.max_prefill = max_rows, max_prefill_tokens
