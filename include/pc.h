@@ -80,12 +80,16 @@ typedef struct pc_model_desc {
     int32_t tied_embed;  /* 1: the LM head is the embedding matrix                         */
     int32_t qk_norm;     /* 1: per-head RMSNorm of q and k over head_dim, before RoPE      */
     int32_t qkv_bias;    /* 1: q/k/v projections have a bias                               */
-    int32_t mlp_half;    /* bf16 models only.  1: w_gate_up and w_down are IEEE half (binary16)
-                          * instead of bfloat16 and the MLP's two activation operands are rounded
-                          * to half: three more mantissa bits at the same bytes and flops.  A
-                          * bfloat16 weight converts to half exactly unless it is below 2^-14 in
-                          * magnitude (then to within 2^-25); the caller answers for weights and
-                          * activations of the MLP staying inside half's range (|x| < 65504).     */
+    int32_t half_gemm;   /* bf16 models only.  1: every matrix that feeds a GEMM (wqkv, wo, w_gate_up,
+                          * w_down, lm_head) is IEEE half (binary16) instead of bfloat16 and the
+                          * activation operands of those GEMMs are rounded to half: three more
+                          * mantissa bits at the same bytes and flops, which takes the place of the
+                          * second bf16 operand (value + rounding remainder) the bfloat16 path needs
+                          * for QKV, output projection and LM head.  lm_head must then be given even
+                          * when tied_embed = 1 (a half copy of the embedding, which itself stays
+                          * bfloat16 for the token lookup).  A bfloat16 weight converts to half exactly
+                          * unless it is below 2^-14 in magnitude (then to within 2^-25); the caller
+                          * answers for weights and GEMM inputs staying inside half's range.           */
 } pc_model_desc;
 
 /* Device pointers to the weights.  The per-layer members are HOST arrays of n_layers
@@ -98,7 +102,8 @@ typedef struct pc_model_desc {
  *   q_norm, k_norm [head_dim] float, or NULL arrays when qk_norm = 0
  *   wo         [d_model, Hq * head_dim]
  *   w_gate_up  [2 * d_ff, d_model]   INTERLEAVED: row 2j = gate row j, row 2j+1 = up row j
- *   w_down     [d_model, d_ff]       (both IEEE half when mlp_half = 1)
+ *   w_down     [d_model, d_ff]
+ *   With half_gemm = 1 wqkv, wo, w_gate_up, w_down and lm_head are IEEE half; embed stays bfloat16.
  */
 typedef struct pc_weights {
     const void* embed;

@@ -30,7 +30,7 @@ EXPORTS = ["pc_status_string", "pc_last_cuda_error", "pc_launch_count", "pc_prof
 class ModelDesc(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ff", "vocab")] + \
                [("rms_eps", C.c_float), ("rope_theta", C.c_float)] + \
-               [(n, C.c_int32) for n in ("dtype", "tied_embed", "qk_norm", "qkv_bias", "mlp_half")]
+               [(n, C.c_int32) for n in ("dtype", "tied_embed", "qk_norm", "qkv_bias", "half_gemm")]
 
 
 class WeightsDesc(C.Structure):

@@ -327,10 +327,14 @@ attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __
             for (int t = 0; t < DT; ++t) {
                 const float y0 = o[t][2 * i] * inv, y1 = o[t][2 * i + 1] * inv;
                 const size_t at = rh * HD + t * 8 + (lane & 3) * 2;
-                *reinterpret_cast<uint32_t*>(out + at) = pack_bf16(y0, y1);
-                // rounding remainder, consumed as a second bf16 operand by the output projection
-                *reinterpret_cast<uint32_t*>(out_lo + at) = pack_bf16(y0 - __bfloat162float(__float2bfloat16_rn(y0)),
-                                                                      y1 - __bfloat162float(__float2bfloat16_rn(y1)));
+                if (out_lo == nullptr) {         // the output projection takes IEEE half operands
+                    *reinterpret_cast<uint32_t*>(out + at) = pack_f16(y0, y1);
+                } else {
+                    *reinterpret_cast<uint32_t*>(out + at) = pack_bf16(y0, y1);
+                    // rounding remainder, consumed as a second bf16 operand by the output projection
+                    *reinterpret_cast<uint32_t*>(out_lo + at) = pack_bf16(y0 - __bfloat162float(__float2bfloat16_rn(y0)),
+                                                                          y1 - __bfloat162float(__float2bfloat16_rn(y1)));
+                }
             }
         } else {
             const size_t ph = (size_t)my_part * part.stride + rh;
@@ -666,6 +670,11 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const StepDesc* __restr
         lo[e] = acc[e] - __bfloat162float(__float2bfloat16_rn(acc[e]));     // rounding remainder: second operand of the O projection
     }
     __nv_bfloat16* dst = out + rh * HD + lane * EPL;
+    if (out_lo == nullptr) {                 // the output projection takes IEEE half operands: no remainder needed
+        if (EPL == 4) *reinterpret_cast<uint2*>(dst) = make_uint2(pack_f16(acc[0], acc[1]), pack_f16(acc[2], acc[3]));
+        else *reinterpret_cast<uint32_t*>(dst) = pack_f16(acc[0], acc[1]);
+        return;
+    }
     __nv_bfloat16* dst_lo = out_lo + rh * HD + lane * EPL;
     if (EPL == 4) {
         *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc[0], acc[1]), pack_bf16(acc[2], acc[3]));

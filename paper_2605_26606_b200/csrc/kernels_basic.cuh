@@ -105,7 +105,7 @@ __global__ void rope_table_kernel(const StepDesc* __restrict__ sd, int half, dou
 template <typename T>
 __global__ void embed_rmsnorm_kernel(const StepDesc* __restrict__ sd, int d, const int32_t* token, const T* __restrict__ embed,
                                      const float* __restrict__ gain, float eps, float* __restrict__ h, T* __restrict__ a,
-                                     T* __restrict__ a_lo) {
+                                     T* __restrict__ a_lo, int half_out) {
     __shared__ float red[33];
     const int r = blockIdx.x;
     if (r >= sd->n_rows) return;
@@ -120,7 +120,8 @@ __global__ void embed_rmsnorm_kernel(const StepDesc* __restrict__ sd, int d, con
     const float rstd = rsqrtf(ss / (float)d + eps);
     for (int i = threadIdx.x; i < d; i += blockDim.x) {
         const float y = h[(size_t)r * d + i] * rstd * gain[i];
-        a[(size_t)r * d + i] = from_f32<T>(y);
+        if (sizeof(T) == 2 && half_out) reinterpret_cast<__half*>(a)[(size_t)r * d + i] = __float2half_rn(y);
+        else a[(size_t)r * d + i] = from_f32<T>(y);
         if (a_lo != nullptr) a_lo[(size_t)r * d + i] = from_f32<T>(y - to_f32<T>(from_f32<T>(y)));
     }
 }

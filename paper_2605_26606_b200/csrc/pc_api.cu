@@ -290,6 +290,8 @@ cudaError_t configure_kernels() {
     if (e == cudaSuccess) e = tc::configure<64, false, tc::EpiSwiGLU>();
     if (e == cudaSuccess) e = tc::configure<256, true, tc::EpiStoreF32>();
     if (e == cudaSuccess) e = tc::configure<64, true, tc::EpiStoreF32>();
+    if (e == cudaSuccess) e = tc::configure<256, false, tc::EpiStoreF32>();
+    if (e == cudaSuccess) e = tc::configure<64, false, tc::EpiStoreF32>();
     if (e == cudaSuccess) e = configure_attention<128>();
     if (e == cudaSuccess) e = configure_attention<64>();
     return e;
@@ -298,9 +300,10 @@ cudaError_t configure_kernels() {
 template <int HD>
 int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, int layer, const AttnPlan& plan, pc::KvArena prompt_arena,
                    pc::KvArena suffix_arena, const __nv_bfloat16* q, __nv_bfloat16* attn, bool profile) {
-    __nv_bfloat16* attn_lo = reinterpret_cast<__nv_bfloat16*>(c->ws + c->cv.attn_lo);
     using namespace pc;
     const pc_model_desc& d = c->d;
+    // half_gemm: the attention output is written once, as IEEE half; else as bf16 plus its bf16 rounding remainder
+    __nv_bfloat16* attn_lo = d.half_gemm ? nullptr : reinterpret_cast<__nv_bfloat16*>(c->ws + c->cv.attn_lo);
     const RowGeom g = geom(c);
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)d.head_dim);
     const int n_rep = d.n_q_heads / d.n_kv_heads;
@@ -350,7 +353,8 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
     T* q = reinterpret_cast<T*>(w + c->cv.q);
     T* attn = reinterpret_cast<T*>(w + c->cv.attn);
     T* act = reinterpret_cast<T*>(w + c->cv.act);
-    T* a_lo = kF32 ? nullptr : reinterpret_cast<T*>(w + c->cv.a_lo);          // rounding remainders (bf16 models only)
+    const bool half_gemm = !kF32 && d.half_gemm != 0;      // every GEMM operand in IEEE half
+    T* a_lo = kF32 || half_gemm ? nullptr : reinterpret_cast<T*>(w + c->cv.a_lo);          // rounding remainders (bf16 operands only)
     float2* rope = reinterpret_cast<float2*>(w + c->cv.rope);
     const RowGeom g = geom(c);
     const int half = d.head_dim / 2;
@@ -364,16 +368,15 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
     float* res_part = reinterpret_cast<float*>(w + c->cv.res_part);
     const Partials none{nullptr, 0, 0, 0};
     Partials pend = none;
-    const bool mlp_half = !kF32 && d.mlp_half != 0;      // MLP operands (weights and both activations) in IEEE half
 
     rope_table_kernel<<<(M * half + 255) / 256, 256, 0, st>>>(sd, half, (double)d.rope_theta, g.pos, rope);
     embed_rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, g.token, reinterpret_cast<const T*>(c->embed), c->attn_norm[0],
-                                               d.rms_eps, h, a, a_lo);
+                                               d.rms_eps, h, a, a_lo, half_gemm ? 1 : 0);
     count_launches(2);
     PC_CUDA_CHECK_LAUNCH("embed_rmsnorm");
     for (int l = 0; l < d.n_layers; ++l) {
         if (l > 0) {
-            rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, h, nullptr, pend, c->attn_norm[l], d.rms_eps, a, a_lo, 0);
+            rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, h, nullptr, pend, c->attn_norm[l], d.rms_eps, a, a_lo, half_gemm ? 1 : 0);
             pend = none;
             count_launches(1);
         }
@@ -385,7 +388,9 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
         } else {
             const GemmPlan gp = plan_gemm(c, GEMM_QKV, c->m_wqkv[l], M, true);
             qkv_parts.n = gp.splits;
-            if (int rc = gemm_bf16(c, st, sd, c->map_a, &c->map_a_lo, c->m_wqkv[l], M, gp, tc::EpiPartial{qkv, c->n_qkv(), qkv_parts.stride})) return rc;
+            if (int rc = gemm_bf16(c, st, sd, c->map_a, half_gemm ? nullptr : &c->map_a_lo, c->m_wqkv[l], M, gp,
+                                   tc::EpiPartial{qkv, c->n_qkv(), qkv_parts.stride}, half_gemm))
+                return rc;
         }
         qkv_post_kernel<T><<<dim3(M, d.n_q_heads + 2 * d.n_kv_heads), half, 0, st>>>(
             sd, d.n_q_heads, d.n_kv_heads, d.head_dim, l, qkv_parts, bias, d.qk_norm ? c->q_norm[l] : nullptr,
@@ -409,13 +414,17 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
             if (rc) return rc;
             const GemmPlan gp = plan_gemm(c, GEMM_O, c->m_wo[l], M, true);
             if (gp.splits == 1) {
-                if (int rc2 = gemm_bf16(c, st, sd, c->map_attn, &c->map_attn_lo, c->m_wo[l], M, gp, tc::EpiResidual{h, d.d_model})) return rc2;
+                if (int rc2 = gemm_bf16(c, st, sd, c->map_attn, half_gemm ? nullptr : &c->map_attn_lo, c->m_wo[l], M, gp,
+                                        tc::EpiResidual{h, d.d_model}, half_gemm))
+                    return rc2;
             } else {
                 pend = Partials{res_part, gp.splits, (size_t)M * d.d_model, d.d_model};
-                if (int rc2 = gemm_bf16(c, st, sd, c->map_attn, &c->map_attn_lo, c->m_wo[l], M, gp, tc::EpiPartial{res_part, d.d_model, pend.stride})) return rc2;
+                if (int rc2 = gemm_bf16(c, st, sd, c->map_attn, half_gemm ? nullptr : &c->map_attn_lo, c->m_wo[l], M, gp,
+                                        tc::EpiPartial{res_part, d.d_model, pend.stride}, half_gemm))
+                    return rc2;
             }
         }
-        rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a, nullptr, mlp_half ? 1 : 0);
+        rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a, nullptr, half_gemm ? 1 : 0);
         pend = none;
         count_launches(2);
         if constexpr (kF32) {
@@ -423,14 +432,14 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
                                 EpiSwiGLU<T>{act, d.d_ff});
             launch_gemm_simt<T>(st, sd, act, reinterpret_cast<const T*>(c->w_down[l]), M, d.d_model, d.d_ff, EpiResidual{h, d.d_model});
         } else {
-            if (int rc = gemm_bf16(c, st, sd, c->map_a, nullptr, c->m_wgu[l], M, plan_gemm(c, GEMM_GATE_UP, c->m_wgu[l], M, false), tc::EpiSwiGLU{act, d.d_ff, mlp_half ? 1 : 0}, mlp_half))
+            if (int rc = gemm_bf16(c, st, sd, c->map_a, nullptr, c->m_wgu[l], M, plan_gemm(c, GEMM_GATE_UP, c->m_wgu[l], M, false), tc::EpiSwiGLU{act, d.d_ff, half_gemm ? 1 : 0}, half_gemm))
                 return rc;
             const GemmPlan gp = plan_gemm(c, GEMM_DOWN, c->m_wdown[l], M, true);
             if (gp.splits == 1) {
-                if (int rc = gemm_bf16(c, st, sd, c->map_act, nullptr, c->m_wdown[l], M, gp, tc::EpiResidual{h, d.d_model}, mlp_half)) return rc;
+                if (int rc = gemm_bf16(c, st, sd, c->map_act, nullptr, c->m_wdown[l], M, gp, tc::EpiResidual{h, d.d_model}, half_gemm)) return rc;
             } else {
                 pend = Partials{res_part, gp.splits, (size_t)M * d.d_model, d.d_model};
-                if (int rc = gemm_bf16(c, st, sd, c->map_act, nullptr, c->m_wdown[l], M, gp, tc::EpiPartial{res_part, d.d_model, pend.stride}, mlp_half)) return rc;
+                if (int rc = gemm_bf16(c, st, sd, c->map_act, nullptr, c->m_wdown[l], M, gp, tc::EpiPartial{res_part, d.d_model, pend.stride}, half_gemm)) return rc;
             }
         }
         count_launches(2);
@@ -447,14 +456,16 @@ int run_lm_head(pc_ctx* c, cudaStream_t st, int n, const pc::StepDesc* sd, const
     const pc_model_desc& d = c->d;
     float* h = reinterpret_cast<float*>(c->ws + c->cv.h);
     T* a = reinterpret_cast<T*>(c->ws + c->cv.a);
-    T* a_lo = std::is_same<T, float>::value ? nullptr : reinterpret_cast<T*>(c->ws + c->cv.a_lo);
-    rmsnorm_kernel<T><<<n, 256, 0, st>>>(sd, d.d_model, h, src, c->pend, c->final_norm, d.rms_eps, a, a_lo, 0);
+    const bool half_gemm = !std::is_same<T, float>::value && d.half_gemm != 0;
+    T* a_lo = std::is_same<T, float>::value || half_gemm ? nullptr : reinterpret_cast<T*>(c->ws + c->cv.a_lo);
+    rmsnorm_kernel<T><<<n, 256, 0, st>>>(sd, d.d_model, h, src, c->pend, c->final_norm, d.rms_eps, a, a_lo, half_gemm ? 1 : 0);
     c->pend = pc::Partials{nullptr, 0, 0, 0};
     if constexpr (std::is_same<T, float>::value) {
         const T* wlm = reinterpret_cast<const T*>(d.tied_embed ? c->embed : c->lm_head);
         launch_gemm_simt<T>(st, sd, a, wlm, n, d.vocab, d.d_model, EpiStoreF32{logits, d.vocab, nullptr});
     } else {
-        if (int rc = gemm_bf16(c, st, sd, c->map_a, &c->map_a_lo, c->m_lm, n, plan_gemm(c, GEMM_LM_HEAD, c->m_lm, n, false), tc::EpiStoreF32{logits, d.vocab, nullptr}))
+        if (int rc = gemm_bf16(c, st, sd, c->map_a, half_gemm ? nullptr : &c->map_a_lo, c->m_lm, n, plan_gemm(c, GEMM_LM_HEAD, c->m_lm, n, false),
+                               tc::EpiStoreF32{logits, d.vocab, nullptr}, half_gemm))
             return rc;
     }
     count_launches(2);
@@ -554,7 +565,7 @@ int pc_create(const pc_model_desc* desc, const pc_weights* wts, pc_ctx** out) {
     *out = nullptr;
     const pc_model_desc& d = *desc;
     if (d.dtype != PC_DTYPE_F32 && d.dtype != PC_DTYPE_BF16) return PC_ERR_INVALID_ARG;
-    if (d.mlp_half != 0 && (d.mlp_half != 1 || d.dtype != PC_DTYPE_BF16)) return PC_ERR_INVALID_ARG;
+    if (d.half_gemm != 0 && (d.half_gemm != 1 || d.dtype != PC_DTYPE_BF16)) return PC_ERR_INVALID_ARG;
     if (d.n_layers <= 0 || d.d_model <= 0 || d.n_q_heads <= 0 || d.n_kv_heads <= 0 || d.d_ff <= 0 || d.vocab <= 0 ||
         !(d.rms_eps >= 0.f) || !(d.rope_theta > 0.f))
         return PC_ERR_INVALID_ARG;
@@ -562,7 +573,7 @@ int pc_create(const pc_model_desc* desc, const pc_weights* wts, pc_ctx** out) {
     if (d.n_q_heads % d.n_kv_heads != 0 || d.n_q_heads / d.n_kv_heads > pc::ATTN_MAX_REP) return PC_ERR_SHAPE;
     if (d.d_model % 8 != 0 || d.d_ff % 8 != 0 || d.d_model > 8192) return PC_ERR_SHAPE;
     if (d.dtype == PC_DTYPE_BF16 && (d.d_model % 64 != 0 || d.d_ff % 64 != 0)) return PC_ERR_SHAPE;
-    if (wts->embed == nullptr || wts->final_norm == nullptr || (!d.tied_embed && wts->lm_head == nullptr)) return PC_ERR_INVALID_ARG;
+    if (wts->embed == nullptr || wts->final_norm == nullptr || ((!d.tied_embed || d.half_gemm) && wts->lm_head == nullptr)) return PC_ERR_INVALID_ARG;
     if (wts->attn_norm == nullptr || wts->wqkv == nullptr || wts->wo == nullptr || wts->mlp_norm == nullptr ||
         wts->w_gate_up == nullptr || wts->w_down == nullptr)
         return PC_ERR_INVALID_ARG;
@@ -609,7 +620,7 @@ int pc_create(const pc_model_desc* desc, const pc_weights* wts, pc_ctx** out) {
             ok = make_wmap(&c->m_wqkv[l], c->wqkv[l], c->n_qkv(), d.d_model) && make_wmap(&c->m_wo[l], c->wo[l], d.d_model, c->q_dim()) &&
                  make_wmap(&c->m_wgu[l], c->w_gate_up[l], 2 * d.d_ff, d.d_model) && make_wmap(&c->m_wdown[l], c->w_down[l], d.d_model, d.d_ff);
         }
-        ok = ok && make_wmap(&c->m_lm, d.tied_embed ? c->embed : c->lm_head, d.vocab, d.d_model);
+        ok = ok && make_wmap(&c->m_lm, d.tied_embed && !d.half_gemm ? c->embed : c->lm_head, d.vocab, d.d_model);
         if (!ok) {
             delete c;
             g_cuda_error = "cuTensorMapEncodeTiled failed for a weight matrix";

@@ -66,32 +66,34 @@ class StageSchedule:
 
 class RolloutEngine:
     def __init__(self, model: ModelShape, weights: Weights, max_rows: int, max_prefill_tokens: int, device="cuda:0",
-                 mlp_half: Optional[bool] = None):
-        """mlp_half: hand the MLP matrices of a bf16 model to the library as IEEE half (pc_model_desc.mlp_half); default
-        on for bf16 models: the synthetic weights N(0, 0.02) and the unit-scale MLP activations sit well inside half's range."""
+                 half_gemm: Optional[bool] = None):
+        """half_gemm: hand the GEMM matrices of a bf16 model to the library as IEEE half (pc_model_desc.half_gemm); default
+        on for bf16 models: the synthetic weights N(0, 0.02) and the unit-scale GEMM inputs sit well inside half's range."""
         self.model = model
-        self.mlp_half = (model.dtype == DTYPE_BF16) if mlp_half is None else bool(mlp_half)
+        self.half_gemm = (model.dtype == DTYPE_BF16) if half_gemm is None else bool(half_gemm)
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
         m, dev = model, self.device
         f32 = lambda n: torch.from_numpy(np.ascontiguousarray(weights[n], dtype=np.float32)).to(dev)
         L = range(m.n_layers)
         self.embed = _dev_matrix(weights, ["embed"], m, dev)
-        self.lm_head = None if m.tied_embed else _dev_matrix(weights, ["lm_head"], m, dev)
+        hg = self.half_gemm
+        lm_name = "embed" if m.tied_embed else "lm_head"
+        self.lm_head = None if (m.tied_embed and not hg) else _dev_matrix(weights, [lm_name], m, dev, half=hg)
         self.final_norm = f32("final_norm")
         self.attn_norm = [f32(f"layers.{l}.attn_norm") for l in L]
         self.mlp_norm = [f32(f"layers.{l}.mlp_norm") for l in L]
-        self.wqkv = [_dev_matrix(weights, [f"layers.{l}.wq", f"layers.{l}.wk", f"layers.{l}.wv"], m, dev) for l in L]
+        self.wqkv = [_dev_matrix(weights, [f"layers.{l}.wq", f"layers.{l}.wk", f"layers.{l}.wv"], m, dev, half=hg) for l in L]
         self.bqkv = [torch.cat([f32(f"layers.{l}.bq"), f32(f"layers.{l}.bk"), f32(f"layers.{l}.bv")]) for l in L] \
             if m.qkv_bias else None
         self.q_norm = [f32(f"layers.{l}.q_norm") for l in L] if m.qk_norm else None
         self.k_norm = [f32(f"layers.{l}.k_norm") for l in L] if m.qk_norm else None
-        self.wo = [_dev_matrix(weights, [f"layers.{l}.wo"], m, dev) for l in L]
-        self.w_gate_up = [_dev_matrix(weights, [f"layers.{l}.w_gate", f"layers.{l}.w_up"], m, dev, interleave=True, half=self.mlp_half)
+        self.wo = [_dev_matrix(weights, [f"layers.{l}.wo"], m, dev, half=hg) for l in L]
+        self.w_gate_up = [_dev_matrix(weights, [f"layers.{l}.w_gate", f"layers.{l}.w_up"], m, dev, interleave=True, half=self.half_gemm)
                           for l in L]
-        self.w_down = [_dev_matrix(weights, [f"layers.{l}.w_down"], m, dev, half=self.mlp_half) for l in L]
+        self.w_down = [_dev_matrix(weights, [f"layers.{l}.w_down"], m, dev, half=self.half_gemm) for l in L]
         desc = B.ModelDesc(m.n_layers, m.d_model, m.n_q_heads, m.n_kv_heads, m.head_dim, m.d_ff, m.vocab, m.rms_eps,
-                           m.rope_theta, m.dtype, int(m.tied_embed), int(m.qk_norm), int(m.qkv_bias), int(self.mlp_half))
+                           m.rope_theta, m.dtype, int(m.tied_embed), int(m.qk_norm), int(m.qkv_bias), int(self.half_gemm))
         self.ctx = B.pc_create(desc, self.embed, self.lm_head, self.final_norm, self.attn_norm, self.wqkv, self.bqkv,
                                self.q_norm, self.k_norm, self.wo, self.mlp_norm, self.w_gate_up, self.w_down)
         self.max_rows, self.max_prefill = max_rows, max_prefill_tokens

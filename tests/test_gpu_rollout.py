@@ -78,9 +78,11 @@ def test_config0_teacher_forced_logits_within_1e_4():
     assert n_cmp == P * G * 16 and n_exempt <= 2
 
 
+@pytest.mark.parametrize("half_gemm", [True, False], ids=["half-operands", "bf16-operands"])
 @pytest.mark.parametrize("model", [wl.TINY_BF16, wl.SMALL_BF16, wl.SMALL_QKNORM_BF16], ids=lambda m: m.name)
-def test_small_bf16_models_teacher_forced(model):
-    """bf16 storage: logits within 5e-2; sampled token identical wherever the oracle's top-two gap exceeds 1e-1."""
+def test_small_bf16_models_teacher_forced(model, half_gemm):
+    """bf16 storage: logits within 5e-2; sampled token identical wherever the oracle's top-two gap exceeds 1e-1.
+    Both operand modes of the GEMMs: IEEE half (the engine's default) and bfloat16 value + rounding remainder."""
     w = dataclasses.replace(wl.WORKLOADS["config0"], model=model, n_prompts=3, prompt_len_lo=5, prompt_len_hi=70,
                             group_size=6, n_pilot=2, max_new=12, cap_lo=3, cap_hi=12, data_seed=11,
                             forced_explicit=None)
@@ -90,7 +92,7 @@ def test_small_bf16_models_teacher_forced(model):
     P, G = w.n_prompts, w.group_size
     prompts, rollouts = np.repeat(np.arange(P), G), np.tile(np.arange(G), P)
     ref = oracle_group_tokens(dec, w, batch, prompts, rollouts)
-    eng = RolloutEngine(model, weights, max_rows=P * G, max_prefill_tokens=int(batch.prompt_offsets[-1]))
+    eng = RolloutEngine(model, weights, max_rows=P * G, max_prefill_tokens=int(batch.prompt_offsets[-1]), half_gemm=half_gemm)
     worst, n_cmp, n_exempt = teacher_forced_compare(eng, w, batch, ref, prompts, rollouts, logit_tol=5e-2, gap_tol=1e-1)
     assert n_cmp == int(batch.caps.sum())
 

@@ -47,6 +47,8 @@ def test_create_rejects_bad_arguments_on_the_host(lib):
     assert lib.pc_create(C.byref(_desc(n_q_heads=3, n_kv_heads=2)), C.byref(w), C.byref(out)) == B.PC_ERR_SHAPE
     assert lib.pc_create(C.byref(_desc(dtype=7)), C.byref(w), C.byref(out)) == B.PC_ERR_INVALID_ARG
     assert lib.pc_create(C.byref(_desc()), C.byref(w), C.byref(out)) == B.PC_ERR_INVALID_ARG      # null weight pointers
+    assert lib.pc_create(C.byref(_desc(half_gemm=1)), C.byref(w), C.byref(out)) == B.PC_ERR_INVALID_ARG   # half operands need a bf16 model
+    assert lib.pc_create(C.byref(_desc(dtype=1, half_gemm=2)), C.byref(w), C.byref(out)) == B.PC_ERR_INVALID_ARG
     assert out.value is None
 
 
