@@ -29,9 +29,9 @@ from paper_2605_26606_b200 import dist_util  # noqa: E402
 from paper_2605_26606_b200 import workloads as wl  # noqa: E402
 
 # DRAM traffic of the suffix attention kernel per algorithmic byte, from the ncu capture summarised in
-# profiles/attn_suffix_kernel_ncu.md (304 rollouts x 513 slots: 171.73 MB moved for 161.6 MB algorithmic).  The kernel
+# profiles/attn_suffix_kernel_ncu.md (304 rollouts x 513 slots: 168.98 MB moved for 161.6 MB algorithmic).  The kernel
 # streams every (rollout, KV head) suffix once, so traffic grows in proportion to the algorithmic bytes of a launch.
-SUFFIX_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.063
+SUFFIX_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.046
 METRIC = "generated tokens/s"
 UNIT = "tokens/s"
 
