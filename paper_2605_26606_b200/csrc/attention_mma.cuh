@@ -92,7 +92,8 @@ struct PrefixPartial {
     float* o;               // [n_parts][stride * head_dim]
     int n_parts;
     size_t stride;          // rows capacity * Hq
-    int chunk_tiles;        // 0: one suffix record per (row, head); else the suffix is cut into ranges of >= chunk_tiles tiles
+    int n_kv_heads;
+    int n_suffix_warps;     // warps of the suffix kernel's grid: how suffixes are cut into ranges is planned for this many
 };
 constexpr int MAX_PREFIX_PARTS = 8;
 constexpr int MAX_SUFFIX_CHUNKS = 8;
@@ -364,12 +365,23 @@ template <int HD> constexpr int suffix_smem_bytes() {
 
 // With few rollouts there are about as many (rollout, KV head) streams as warps on the GPU, and one stream more than
 // warps doubles the kernel's time.  The suffix of a rollout is therefore cut into ranges of tiles ("chunks") that
-// are spread over the warps; every chunk leaves its own record.
-// Tiles per chunk for a step whose longest suffix has max_slen slots: at least chunk_tiles, and large enough that no
-// row needs more than MAX_SUFFIX_CHUNKS chunks.  The same value serves every row of the step.
-__device__ __forceinline__ int suffix_chunk_len(int max_slen, int chunk_tiles) {
-    const int max_tiles = (max_slen + S_TP - 1) / S_TP;
-    return chunk_tiles <= 0 ? max(max_tiles, 1) : max(chunk_tiles, (max_tiles + MAX_SUFFIX_CHUNKS - 1) / MAX_SUFFIX_CHUNKS);
+// are spread over the warps; every chunk leaves its own record.  Tiles per chunk (ct) and chunk slots per (row, KV
+// head) item (cpi) for a step whose longest suffix has max_slen slots: among 1..MAX_SUFFIX_CHUNKS chunks per item, the
+// choice that minimises (units the busiest warp gets) x (tiles per unit + 2), the + 2 standing for the fixed cost of a
+// unit (length lookup, first TMA round trip, record) in tile times.  The same value serves every row of the step, and
+// the merge kernel recomputes it from the same inputs.
+struct SuffixPlan { int ct, cpi; };
+__device__ __forceinline__ SuffixPlan suffix_plan(int max_slen, int n_items, int n_warps) {
+    const int ntiles = max(1, (max_slen + S_TP - 1) / S_TP);
+    SuffixPlan best{ntiles, 1};
+    long long best_cost = -1;
+    for (int c = 1; c <= MAX_SUFFIX_CHUNKS; ++c) {
+        const int ct = (ntiles + c - 1) / c;
+        const int cc = (ntiles + ct - 1) / ct;
+        const long long cost = (long long)((n_items * cc + n_warps - 1) / max(n_warps, 1)) * (ct + 2);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = SuffixPlan{ct, cc}; }
+    }
+    return best;
 }
 __device__ __forceinline__ int suffix_chunks(int n, int ct) {             // records a row with n suffix slots leaves
     const int ntiles = (n + S_TP - 1) / S_TP;
@@ -405,8 +417,8 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
 
     // work unit u = (item, chunk), item = (row, kv head); units of one item are consecutive, so they land on different warps
     const int max_slen = *g.max_slen;
-    const int ct = suffix_chunk_len(max_slen, part.chunk_tiles);                                   // tiles per chunk
-    const int cpi = part.chunk_tiles > 0 ? max(1, suffix_chunks(max_slen, ct)) : 1;               // unit slots per item
+    const SuffixPlan sp = suffix_plan(max_slen, sd->n_rows * Hkv, part.n_suffix_warps);
+    const int ct = sp.ct, cpi = sp.cpi;                                                            // tiles per chunk, unit slots per item
     const int n_items = sd->n_rows * Hkv * cpi;
     const int item_stride = gridDim.x * S_WARPS;
     const int first_item = blockIdx.x * S_WARPS + warp;
@@ -487,7 +499,7 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) { qb[ks][0] = qn[ks][0]; qb[ks][1] = qn[ks][1]; }
         fetch_item(item + item_stride);
-        if (t1 <= t0 && !(chunk == 0 && part.chunk_tiles <= 0)) continue;      // this row has fewer chunks: nothing to leave
+        if (t1 <= t0) continue;      // this row has fewer chunks: nothing to leave
         float o[DT][4];
 #pragma unroll
         for (int t = 0; t < DT; ++t) { o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f; }
@@ -632,8 +644,7 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const StepDesc* __restr
     const size_t rh = (size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (rh >= (size_t)sd->n_rows * Hq) return;
     const int row = (int)(rh / Hq);
-    // a row without suffix slots still has its (empty) record 0 when the suffix is not cut into chunks
-    const int n_sfx = part.chunk_tiles > 0 ? suffix_chunks(g.s_len[row], suffix_chunk_len(*g.max_slen, part.chunk_tiles)) : 1;
+    const int n_sfx = suffix_chunks(g.s_len[row], suffix_plan(*g.max_slen, sd->n_rows * (part.n_kv_heads), part.n_suffix_warps).ct);
     const int n_rec = part.n_parts + n_sfx;
     float mi[MAX_RECORDS], li[MAX_RECORDS];
     float M = -INFINITY;

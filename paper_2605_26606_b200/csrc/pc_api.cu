@@ -312,10 +312,13 @@ int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, in
     const int base_ctas = std::max(1, q_tiles * d.n_kv_heads * plan.n_groups);
     // (two of these CTAs fit on an SM)
     const int n_parts = plan.prefill ? 1 : std::max(1, std::min(am::MAX_PREFIX_PARTS, 2 * c->num_sms / base_ctas));
+    // the suffix kernel takes one warp per (rollout, KV head, range of the suffix); how the suffixes are cut into ranges
+    // is decided on the device for the warps of this grid (the longest suffix of the step is only known there)
+    const int items = M * d.n_kv_heads * am::MAX_SUFFIX_CHUNKS;
+    const int sgrid = std::min(c->num_sms, (items + am::S_WARPS - 1) / am::S_WARPS);
     am::PrefixPartial part{reinterpret_cast<float*>(c->ws + c->cv.part_m), reinterpret_cast<float*>(c->ws + c->cv.part_l),
-                           reinterpret_cast<float*>(c->ws + c->cv.part_o), n_parts, (size_t)std::max(c->max_rows, 1) * d.n_q_heads, 0};
-    // few (rollout, KV head) streams per warp: cut the suffixes into chunks of at least 4 tiles so that the load balances
-    if (M * d.n_kv_heads < 4 * c->num_sms * am::S_WARPS) part.chunk_tiles = 4;
+                           reinterpret_cast<float*>(c->ws + c->cv.part_o), n_parts, (size_t)std::max(c->max_rows, 1) * d.n_q_heads,
+                           d.n_kv_heads, sgrid * am::S_WARPS};
     const dim3 ggrid(q_tiles * n_parts, d.n_kv_heads, plan.n_groups);
     if (plan.prefill) {
         am::attn_group_kernel<HD, true><<<ggrid, am::G_THREADS, am::group_smem_bytes<HD>(), st>>>(
@@ -327,8 +330,6 @@ int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, in
     am::attn_group_kernel<HD, false><<<ggrid, am::G_THREADS, am::group_smem_bytes<HD>(), st>>>(
         c->map_prompt_kv, sd, prompt_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, plan.group_row_start, g, scale_log2, part,
         attn, attn_lo, c->err);
-    const int items = M * d.n_kv_heads * (part.chunk_tiles > 0 ? am::MAX_SUFFIX_CHUNKS : 1);
-    const int sgrid = std::min(c->num_sms, (items + am::S_WARPS - 1) / am::S_WARPS);
     if (profile) cudaEventRecord(c->prof_start, st);
     am::attn_suffix_kernel<HD><<<sgrid, am::S_WARPS * 32, am::suffix_smem_bytes<HD>(), st>>>(
         c->map_suffix_kv, sd, suffix_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, g, scale_log2, part, c->err);
