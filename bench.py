@@ -183,6 +183,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="config2", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--also-bound", action="store_true",
+                    help="additionally time one bound pass (Section 3.4): the commit rollouts of the timed batch's survivors and the "
+                         "pilot rollouts of a second batch in one decode batch; reported as bound_pass")
+    ap.add_argument("--also-logprobs", action="store_true",
+                    help="additionally time one step that also keeps the behaviour log-probability of every sampled token (Eq. 2's "
+                         "denominator); reported as with_logprobs")
     ap.add_argument("--also-grpo", action="store_true",
                     help="additionally time one step with k = G (all P*G rollouts concurrent, no filter) and report it as grpo_mode")
     ap.add_argument("--probe", default=None, metavar="rows=R,suffix=S,steps=N,prompt=L",
@@ -320,6 +326,37 @@ def main():
     }
     if cpu_baseline is not None:
         line["cpu_baseline"] = cpu_baseline
+    if args.also_logprobs and world == 1:
+        eng.profile_every = 0
+        eng.collect_logprobs = True
+        one_step(False)                                       # buffers and graphs of this mode
+        n_tok, d_ms, _, _ = one_step(True)
+        eng.collect_logprobs = False
+        line["with_logprobs"] = {"tokens": n_tok, "ms_per_step": d_ms, "tokens_per_s": n_tok / (d_ms * 1e-3),
+                                 "step_time_ratio": d_ms / (t_ms / max(args.steps, 1))}
+    if args.also_bound and world == 1:
+        # steady state of Section 3.4: batch A's pilot pass has just run on this engine (the timed step leaves A's prompt KV,
+        # last-position logits and statuses in place); one pass then generates A's commit rollouts and B's pilot rollouts
+        eng.profile_every = 0
+        wb = dataclasses.replace(w, data_seed=w.data_seed + 1000)
+        batch_b = wl.gen_batch(wb)
+        commit_a = np.flatnonzero(status == B.PC_STATUS_COMMIT)
+        times = []
+        for rep in range(2):                                   # first repetition: graphs and allocator
+            eng.load_batch(w, batch)
+            eng.run_device()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            out_b = eng.bound_pass(w, batch, commit_a, batch_b)
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        n_tok_b = int(sum(len(t) for t in out_b["a"].values()) + sum(len(t) for t in out_b["b"].values()))
+        rows_b = len(commit_a) * (G - k) + P * k
+        line["bound_pass"] = {"rows": rows_b, "commit_prompts_of_previous_batch": int(len(commit_a)), "pilot_prompts": P, "tokens": n_tok_b,
+                              "ms_per_pass": times[-1], "tokens_per_s": n_tok_b / (times[-1] * 1e-3),
+                              "note": "prefill of the new batch, decode of both row sets and the read-back of the tokens included"}
     if args.also_grpo and world == 1:
         # every rollout of every group at once (what plain GRPO generates for the same prompts): same kernels, k = G
         wg = dataclasses.replace(w, n_pilot=G)
