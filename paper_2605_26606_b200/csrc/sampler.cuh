@@ -274,7 +274,24 @@ __global__ void __launch_bounds__(256) token_logprob_kernel(const StepDesc* __re
     const float mx = range_max(lg, 0, vocab, temperature, red);          // max of logits / T
     const float inv_t = 1.f / temperature;
     float s = 0.f;
-    for (int v = threadIdx.x; v < vocab; v += blockDim.x) s += expf(lg[v] * inv_t - mx);
+    {
+        // 16-byte loads, four in flight per thread (one scalar load at a time leaves the pass bound by memory latency);
+        // every thread adds its elements in a fixed order, so the sum does not depend on timing
+        int v = 0;
+        while (v < vocab && (reinterpret_cast<uintptr_t>(lg + v) & 15u) != 0) { if (threadIdx.x == 0) s += expf(lg[v] * inv_t - mx); ++v; }
+        const int n4 = (vocab - v) >> 2;
+        const float4* p4 = reinterpret_cast<const float4*>(lg + v);
+        auto add4 = [&](const float4 a) {
+            s += expf(a.x * inv_t - mx); s += expf(a.y * inv_t - mx); s += expf(a.z * inv_t - mx); s += expf(a.w * inv_t - mx);
+        };
+        int i = threadIdx.x;
+        for (; i + 3 * (int)blockDim.x < n4; i += 4 * blockDim.x) {
+            const float4 a = p4[i], b = p4[i + blockDim.x], c = p4[i + 2 * blockDim.x], d = p4[i + 3 * blockDim.x];
+            add4(a); add4(b); add4(c); add4(d);
+        }
+        for (; i < n4; i += blockDim.x) add4(p4[i]);
+        for (int t = v + 4 * n4 + threadIdx.x; t < vocab; t += blockDim.x) s += expf(lg[t] * inv_t - mx);
+    }
     s = block_sum(s, red);
     if (threadIdx.x == 0) {
         const int tok = tokens[tok_index ? tok_index[ro] + tok_index_offset : (int64_t)r];
