@@ -97,6 +97,29 @@ def test_small_bf16_models_teacher_forced(model, half_gemm):
     assert n_cmp == int(batch.caps.sum())
 
 
+@pytest.mark.parametrize("spec", ["qkv=256x2,o=256x3,dn=256x4,gu=64x1,lm=64x1", "qkv=64x1,o=64x1,dn=64x8,gu=256x1,lm=256x1"])
+def test_forced_gemm_plans_stay_within_tolerance(spec):
+    """pc_set_gemm_plan: tile width and K-split change the order of the float additions, nothing else; a bad spec is refused."""
+    from paper_2605_26606_b200 import binding as B
+    model = wl.SMALL_BF16
+    w = dataclasses.replace(wl.WORKLOADS["config0"], model=model, n_prompts=3, prompt_len_lo=5, prompt_len_hi=70,
+                            group_size=6, n_pilot=2, max_new=12, cap_lo=3, cap_hi=12, data_seed=11, forced_explicit=None)
+    weights = wl.gen_weights(model, seed=1, threads=2, gain_jitter=0.1)
+    batch = wl.gen_batch(w)
+    dec = Decoder(model, weights)
+    P, G = w.n_prompts, w.group_size
+    prompts, rollouts = np.repeat(np.arange(P), G), np.tile(np.arange(G), P)
+    ref = oracle_group_tokens(dec, w, batch, prompts, rollouts)
+    eng = RolloutEngine(model, weights, max_rows=P * G, max_prefill_tokens=int(batch.prompt_offsets[-1]))
+    B.pc_set_gemm_plan(eng.ctx, spec)
+    worst, n_cmp, _ = teacher_forced_compare(eng, w, batch, ref, prompts, rollouts, logit_tol=5e-2, gap_tol=1e-1)
+    assert n_cmp == int(batch.caps.sum())
+    for bad in ("qkv=128x1", "zz=64x1", "dn=64x0", "dn=64"):
+        with pytest.raises(B.PcError):
+            B.pc_set_gemm_plan(eng.ctx, bad)
+    B.pc_set_gemm_plan(eng.ctx, None)
+
+
 def test_run_twice_is_deterministic_and_batch_invariant():
     """Same inputs give bit-identical tokens; a rollout's tokens do not depend on its batch mates."""
     w = dataclasses.replace(wl.WORKLOADS["config0"], model=wl.TINY_BF16, n_pilot=8)
