@@ -308,9 +308,11 @@ def main():
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": t_ms / max(args.steps, 1), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16" if m.dtype == wl.DTYPE_BF16 else "f32", "data": "synthetic",
+        "dtype": ("f16" if eng.half_gemm else "bf16") if m.dtype == wl.DTYPE_BF16 else "f32", "data": "synthetic",
         "config": {"workload": w.name, "model": m.name, "prompts": P, "group_size": G, "n_pilot": k, "max_new": w.max_new,
-                   "mode": "pilot-commit", "committed_prompts": int((status == B.PC_STATUS_COMMIT).sum()),
+                   "mode": "pilot-commit",
+                   "arithmetic": "16-bit storage (bf16 model); GEMM operands IEEE half, K / q / embedding bfloat16, float32 accumulation"
+                                 if m.dtype == wl.DTYPE_BF16 and eng.half_gemm else "model storage type, float32 accumulation", "committed_prompts": int((status == B.PC_STATUS_COMMIT).sum()),
                    "rollouts_generated": n_roll, "rollouts_per_s": n_roll * world / (t_ms * 1e-3 / max(args.steps, 1)),
                    "l2": "inputs larger than L2 (3.1 GB of weights and tens of GB of KV per step); no flush",
                    "parallelism": f"replicas x{world}, one sampling batch per GPU"},
