@@ -642,18 +642,38 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const StepDesc* __restr
     constexpr int EPL = HD / 32;
     const int lane = threadIdx.x & 31;
     const size_t rh = (size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (rh >= (size_t)sd->n_rows * Hq) return;
+    // The grid covers the row bound; the row's suffix length is requested together with the step descriptor (buffers
+    // hold the bound), and every record of the (row, head) -- (m, l) and its output slice -- is requested before the
+    // first one is used, so the kernel pays two memory round trips instead of four.  Records are added in index order.
     const int row = (int)(rh / Hq);
-    const int n_sfx = suffix_chunks(g.s_len[row], suffix_plan(*g.max_slen, sd->n_rows * (part.n_kv_heads), part.n_suffix_warps).ct);
+    const int row_in = min(row, (int)(part.stride / (size_t)Hq) - 1);          // the last block may reach past the row bound
+    const int n_live = sd->n_rows, slen = g.s_len[row_in], max_slen = *g.max_slen;
+    if (rh >= (size_t)n_live * Hq) return;
+    const int n_sfx = suffix_chunks(slen, suffix_plan(max_slen, n_live * part.n_kv_heads, part.n_suffix_warps).ct);
     const int n_rec = part.n_parts + n_sfx;
     float mi[MAX_RECORDS], li[MAX_RECORDS];
-    float M = -INFINITY;
+    float ov[MAX_RECORDS][EPL];
 #pragma unroll
     for (int i = 0; i < MAX_RECORDS; ++i) {
         mi[i] = -INFINITY; li[i] = 0.f;
-        if (i < n_rec) { mi[i] = part.m[(size_t)i * part.stride + rh]; li[i] = part.l[(size_t)i * part.stride + rh]; }
-        M = fmaxf(M, mi[i]);
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) ov[i][e] = 0.f;
+        if (i < n_rec) {
+            mi[i] = part.m[(size_t)i * part.stride + rh];
+            li[i] = part.l[(size_t)i * part.stride + rh];
+            const float* src = part.o + ((size_t)i * part.stride + rh) * HD + lane * EPL;
+            if (EPL == 4) {
+                const float4 v = *reinterpret_cast<const float4*>(src);
+                ov[i][0] = v.x; ov[i][1] = v.y; ov[i][2] = v.z; ov[i][3] = v.w;
+            } else {
+                const float2 v = *reinterpret_cast<const float2*>(src);
+                ov[i][0] = v.x; ov[i][1] = v.y;
+            }
+        }
     }
+    float M = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < MAX_RECORDS; ++i) M = fmaxf(M, mi[i]);
     float acc[EPL];
 #pragma unroll
     for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
@@ -661,16 +681,10 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const StepDesc* __restr
 #pragma unroll
     for (int i = 0; i < MAX_RECORDS; ++i) {
         const float w = exp2_safe(mi[i], M);
-        if (i < n_rec && w > 0.f) {
+        if (i < n_rec && w > 0.f) {          // a record with m = -inf was left by an empty range: its output slice is not defined
             denom += li[i] * w;
-            const float* src = part.o + ((size_t)i * part.stride + rh) * HD + lane * EPL;
-            if (EPL == 4) {
-                const float4 v = *reinterpret_cast<const float4*>(src);
-                acc[0] += v.x * w; acc[1] += v.y * w; acc[2] += v.z * w; acc[3] += v.w * w;
-            } else {
-                const float2 v = *reinterpret_cast<const float2*>(src);
-                acc[0] += v.x * w; acc[1] += v.y * w;
-            }
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) acc[e] += ov[i][e] * w;
         }
     }
     const float inv = denom > 0.f ? 1.f / denom : 0.f;
