@@ -115,8 +115,9 @@ class Decoder:
         return rmsnorm(h, self.W("final_norm"), self.m.rms_eps) @ self.lm_head().T
 
     # -- mode 1: the definition ----------------------------------------------------------
-    def forward_full(self, tokens: np.ndarray, return_kv: bool = False, last_only: bool = False):
-        """Causal forward over one whole sequence.  Returns logits [T, V] (or [1, V] with last_only).
+    def forward_full(self, tokens: np.ndarray, return_kv: bool = False, last_only: bool = False, positions=None):
+        """Causal forward over one whole sequence.  Returns logits [T, V] (or [1, V] with last_only, or one row per
+        entry of `positions`: the LM head is then applied to those positions only).
 
         With return_kv also returns [(K_l, V_l)] with K_l, V_l of shape [T, Hkv, hd] (K after RoPE).
         """
@@ -143,6 +144,8 @@ class Decoder:
             h = h + self.mlp(l, h)
         if last_only:
             h = h[-1:, :]
+        elif positions is not None:
+            h = h[np.asarray(positions, dtype=np.int64), :]
         logits = self.logits_from_hidden(h)
         return (logits, kv) if return_kv else logits
 

@@ -109,6 +109,8 @@ class RolloutEngine:
         self.prompt_key_host: Optional[np.ndarray] = None    # sampling-key id per prompt (None: the prompt's index)
         self.collect_logprobs = False       # also keep log pi(o_t) of every sampled token (Eq. 2's denominator)
         self.record_pilot_logits: Optional[dict] = None     # {decode step: None} -> filled during the pilot stage
+        self.record_commit_logits: Optional[dict] = None    # the same for the commit stage
+        self.record_rows: Optional[set] = None              # keep only the logits rows of these (prompt, rollout) pairs
         self.profile_layer = m.n_layers // 2
         self.profile_samples: List[tuple] = []      # (start event, stop event, rows, suffix slots read per row)
 
@@ -265,6 +267,10 @@ class RolloutEngine:
                              int(sch.groups_per_step[s]), gs + 4 * go, int(sch.max_group_rows[s]), self.prompt_len,
                              self.prompt_kv, self.total_prompt_tokens, self.prompt_kv_start, self.suffix_kv,
                              self.suffix_slots, logits_out, None if teacher_forced else sp)
+            if logits_out is not None and self.record_rows is not None:
+                _, rec_p, rec_r = record_logits[s]
+                keep = np.flatnonzero([(int(a), int(b)) in self.record_rows for a, b in zip(rec_p, rec_r)])
+                record_logits[s] = (logits_out[torch.from_numpy(keep).to(dev)].clone(), rec_p[keep], rec_r[keep])
 
         def profiled(s):
             return bool(self.profile_every) and s % self.profile_every == self.profile_every // 2
@@ -318,7 +324,8 @@ class RolloutEngine:
         status = self.status.cpu().numpy()            # the commit stage's row set depends on it
         commit = np.flatnonzero(status == B.PC_STATUS_COMMIT)
         if G > k and commit.size:
-            n_tok += self.run_stage(np.repeat(commit, G - k), np.tile(np.arange(k, G), commit.size))
+            n_tok += self.run_stage(np.repeat(commit, G - k), np.tile(np.arange(k, G), commit.size),
+                                    record_logits=self.record_commit_logits)
         B.pc_reward_last_token(P * G, self.tokens, self.last_index, self.thresholds, self.rewards)
         union_count = torch.from_numpy(np.where(status == B.PC_STATUS_COMMIT, G, k).astype(np.int32)).to(self.device)
         B.pc_group_stats(P, self.rewards, self.group_start, union_count, self.union_n, self.union_success, self.union_mean,
@@ -364,7 +371,7 @@ class RolloutEngine:
         B.pc_set_prompt_keys(self.ctx, self.prompt_key_dev)
         prompts = np.concatenate([np.repeat(np.arange(nA), G - k), np.repeat(nA + np.arange(PB), k)])
         rollouts = np.concatenate([np.tile(np.arange(k, G), nA), np.tile(np.arange(k), PB)])
-        self.run_stage(prompts, rollouts)
+        self.run_stage(prompts, rollouts, record_logits=self.record_pilot_logits)
         self.check_error_flag()
         toks = self.tokens.cpu().numpy().reshape(nA + PB, G, wl.max_new)
         out = {"a": {}, "b": {}}
