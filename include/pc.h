@@ -166,6 +166,15 @@ PC_API int pc_set_workspace(pc_ctx* ctx, void* dev_ws, size_t bytes, int max_row
  * steps.  The paper has no counterpart. */
 PC_API int pc_set_gemm_plan(pc_ctx* ctx, const char* spec);
 
+/* How the decode steps of a bf16 model with half_gemm = 1 are issued.  mode 1: everything between two
+ * attention calls of a step -- output projection, residual + RMSNorm, gate/up + SwiGLU, down projection, residual +
+ * RMSNorm, QKV projection of the next layer and its bias / QK-norm / RoPE / KV append; embedding before the first
+ * layer, LM head after the last -- runs as phases of ONE persistent cooperative kernel with grid-wide barriers, the
+ * weight tiles of the next GEMM being requested across the barriers.  mode 0 (the default): one kernel per operation.  Both modes
+ * run the same arithmetic in the same order and give identical results; models of other types always use mode 0.
+ * Drops captured decode steps.  The paper has no counterpart. */
+PC_API int pc_set_decode_mode(pc_ctx* ctx, int mode);
+
 /* Measurement aid: in the next pc_decode_step of this context, record the two CUDA events (cudaEvent_t,
  * created by the caller) around the attention kernel of `layer` that reads the rollouts' own suffix K/V
  * (for float32 models: the single attention kernel).  One-shot; the caller synchronises and reads the

@@ -637,16 +637,14 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
 // One warp per (row, head); a lane owns HD/32 consecutive dims.
 // ---------------------------------------------------------------------------------------------
 template <int HD>
-__global__ void __launch_bounds__(256) attn_merge_kernel(const StepDesc* __restrict__ sd, int Hq, RowGeom g, PrefixPartial part,
-                                                         __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ out_lo) {
+__device__ __forceinline__ void merge_item_warp(int lane, size_t rh, const StepDesc* __restrict__ sd, int Hq, const RowGeom& g,
+                                                const PrefixPartial& part, __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ out_lo) {
     constexpr int EPL = HD / 32;
-    const int lane = threadIdx.x & 31;
-    const size_t rh = (size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    // The grid covers the row bound; the row's suffix length is requested together with the step descriptor (buffers
-    // hold the bound), and every record of the (row, head) -- (m, l) and its output slice -- is requested before the
-    // first one is used, so the kernel pays two memory round trips instead of four.  Records are added in index order.
+    // The row's suffix length is requested together with the step descriptor, and every record of the (row, head) --
+    // (m, l) and its output slice -- is requested before the first one is used, so an item pays two memory round trips
+    // instead of four.  Records are added in index order.
     const int row = (int)(rh / Hq);
-    const int row_in = min(row, (int)(part.stride / (size_t)Hq) - 1);          // the last block may reach past the row bound
+    const int row_in = min(row, (int)(part.stride / (size_t)Hq) - 1);          // callers may reach past the row bound
     const int n_live = sd->n_rows, slen = g.s_len[row_in], max_slen = *g.max_slen;
     if (rh >= (size_t)n_live * Hq) return;
     const int n_sfx = suffix_chunks(slen, suffix_plan(max_slen, n_live * part.n_kv_heads, part.n_suffix_warps).ct);
@@ -708,6 +706,13 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const StepDesc* __restr
         *reinterpret_cast<uint32_t*>(dst) = pack_bf16(acc[0], acc[1]);
         *reinterpret_cast<uint32_t*>(dst_lo) = pack_bf16(lo[0], lo[1]);
     }
+}
+
+// Stand-alone form: the grid covers the row bound of the step.
+template <int HD>
+__global__ void __launch_bounds__(256) attn_merge_kernel(const StepDesc* __restrict__ sd, int Hq, RowGeom g, PrefixPartial part,
+                                                         __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ out_lo) {
+    merge_item_warp<HD>(threadIdx.x & 31, (size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), sd, Hq, g, part, out, out_lo);
 }
 
 }  // namespace am

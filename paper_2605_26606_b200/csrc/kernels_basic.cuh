@@ -20,13 +20,20 @@ struct RowGeom {
     int32_t* max_slen;   // [1] largest s_len of the step (decode only)
 };
 
-__global__ void set_step_desc(StepDesc* sd, int n_rows, int n_groups, int max_group_rows, int32_t* max_slen) {
+// Both step-descriptor kernels also zero the grid-barrier words of the persistent decode kernel (bar, n_bar words;
+// launched with STEP_DESC_THREADS threads).
+constexpr int STEP_DESC_THREADS = 128;
+__global__ void set_step_desc(StepDesc* sd, int n_rows, int n_groups, int max_group_rows, int32_t* max_slen, int32_t* bar, int n_bar) {
+    for (int i = threadIdx.x; i < n_bar; i += blockDim.x) bar[i] = 0;
+    if (threadIdx.x != 0) return;
     *max_slen = 0;
     sd->n_rows = n_rows; sd->n_groups = n_groups; sd->max_group_rows = max_group_rows; sd->reserved = 0;
     sd->row_off = 0; sd->group_off = 0;
 }
 // First node of a captured decode step: takes the next descriptor of the caller's schedule.
-__global__ void load_step_desc(const StepDesc* __restrict__ steps, int32_t* counter, StepDesc* sd, int32_t* max_slen) {
+__global__ void load_step_desc(const StepDesc* __restrict__ steps, int32_t* counter, StepDesc* sd, int32_t* max_slen, int32_t* bar, int n_bar) {
+    for (int i = threadIdx.x; i < n_bar; i += blockDim.x) bar[i] = 0;
+    if (threadIdx.x != 0) return;
     *max_slen = 0;
     const int i = *counter;
     *sd = steps[i];
@@ -101,31 +108,6 @@ __global__ void rope_table_kernel(const StepDesc* __restrict__ sd, int half, dou
     table[idx] = make_float2((float)c, (float)s);
 }
 
-// h[r, :] = E[token[r], :] (float residual stream); a[r, :] = RMSNorm(h[r, :]; gain) in storage type T.
-template <typename T>
-__global__ void embed_rmsnorm_kernel(const StepDesc* __restrict__ sd, int d, const int32_t* token, const T* __restrict__ embed,
-                                     const float* __restrict__ gain, float eps, float* __restrict__ h, T* __restrict__ a,
-                                     T* __restrict__ a_lo, int half_out) {
-    __shared__ float red[33];
-    const int r = blockIdx.x;
-    if (r >= sd->n_rows) return;
-    const T* e = embed + (size_t)token[r] * d;
-    float ss = 0.f;
-    for (int i = threadIdx.x; i < d; i += blockDim.x) {
-        const float v = to_f32<T>(e[i]);
-        h[(size_t)r * d + i] = v;
-        ss += v * v;
-    }
-    ss = block_sum(ss, red);
-    const float rstd = rsqrtf(ss / (float)d + eps);
-    for (int i = threadIdx.x; i < d; i += blockDim.x) {
-        const float y = h[(size_t)r * d + i] * rstd * gain[i];
-        if (sizeof(T) == 2 && half_out) reinterpret_cast<__half*>(a)[(size_t)r * d + i] = __float2half_rn(y);
-        else a[(size_t)r * d + i] = from_f32<T>(y);
-        if (a_lo != nullptr) a_lo[(size_t)r * d + i] = from_f32<T>(y - to_f32<T>(from_f32<T>(y)));
-    }
-}
-
 // K-slice sums left by a split GEMM: value(row, col) = sum over s < n of p[s * stride + row * ld + col], added in
 // the order s = 0, 1, ... so that the result does not depend on which CTA finished first.
 struct Partials {
@@ -136,8 +118,6 @@ struct Partials {
 };
 constexpr int PARTIALS_MAX = 8;
 
-// Optional residual update followed by the norm:  h[row, :] += pending partial sums of row r;  a[r, :] = RMSNorm(h[row, :]; gain)
-// with row = src ? src[r] : r.  The partial sums are indexed by row, like h.
 template <typename T> __device__ __forceinline__ void store4(T* p, float4 v);
 template <> __device__ __forceinline__ void store4<float>(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
 template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16* p, float4 v) {
@@ -151,79 +131,129 @@ __device__ __forceinline__ float4 bf16_remainder(float4 v) {
                        v.z - __bfloat162float(__float2bfloat16_rn(v.z)), v.w - __bfloat162float(__float2bfloat16_rn(v.w)));
 }
 
-// One block of 256 threads per row; d is a multiple of 8 and at most 8192, so a thread keeps its <= 8 float4 of the
-// row in registers between the sum of squares and the scaling (one pass over global memory).
+// The row-wise operations below are written for ONE WARP per row (or per (row, head)), so that the stand-alone kernels
+// and the phases of the persistent decode kernel (decode_chain.cuh) run the very same arithmetic in the same order.
+
 template <typename T>
-__global__ void __launch_bounds__(256) rmsnorm_kernel(const StepDesc* __restrict__ sd, int d, float* __restrict__ h,
-                                                      const int32_t* __restrict__ src, Partials pend, const float* __restrict__ gain,
-                                                      float eps, T* __restrict__ a, T* __restrict__ a_lo, int half_out) {
-    __shared__ float red[33];
-    const int r = blockIdx.x;
-    // The grid covers the row bound of the step; rows past the live count are dropped only after this row's data has
-    // been requested (buffers hold the bound, so the reads are in range): the step descriptor, the row and its
-    // pending slices then arrive together instead of one memory latency after the other.
-    const int n_live = sd != nullptr ? sd->n_rows : gridDim.x;
-    const int row = src ? src[r] : r;
-    float4* x = reinterpret_cast<float4*>(h + (size_t)row * d);
+__device__ __forceinline__ void store_norm_out(T* __restrict__ a_row, T* __restrict__ a_lo_row, int i4, float4 y, int half_out) {
+    if (sizeof(T) == 2 && half_out) {          // IEEE half instead of bfloat16 (operand of a half-precision GEMM)
+        const __half2 lo = __floats2half2_rn(y.x, y.y), hi = __floats2half2_rn(y.z, y.w);
+        *reinterpret_cast<uint2*>(a_row + 4 * i4) =
+            make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+    } else {
+        store4<T>(a_row + 4 * i4, y);
+    }
+    if (a_lo_row != nullptr) store4<T>(a_lo_row + 4 * i4, bf16_remainder(y));
+}
+
+// Residual update followed by the norm, one warp per row:
+//   h_row[:] += pending K-slice sums (pend_row = their row offset, in slice order);  a_row[:] = RMSNorm(h_row; gain).
+// d is a multiple of 8.  Rows of up to NORM_REG4 * 128 elements stay in registers between the sum of squares and
+// the scaling (one pass over memory, every load of the row and of its slices requested before the first use);
+// longer rows are read twice.
+constexpr int NORM_REG4 = 12;
+template <typename T>
+__device__ __forceinline__ void norm_row_warp(int lane, int d, float* __restrict__ h_row, Partials pend, size_t pend_row,
+                                              const float* __restrict__ gain, float eps, T* __restrict__ a_row,
+                                              T* __restrict__ a_lo_row, int half_out) {
     const int n4 = d >> 2;
-    float4 v[8];
-    float4 p[2][PARTIALS_MAX];
-    float4 gg2[2];
+    float4* x = reinterpret_cast<float4*>(h_row);
+    float ss = 0.f;
+    if (n4 <= NORM_REG4 * 32) {
+        float4 v[NORM_REG4], gg[NORM_REG4];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-        const int i = threadIdx.x + k * 256;
-        if (i < n4) {
-            v[k] = x[i];
-            if (k < 2) {
-                gg2[k] = *reinterpret_cast<const float4*>(gain + 4 * i);
-#pragma unroll
-                for (int s = 0; s < PARTIALS_MAX; ++s)
-                    p[k][s] = s < pend.n ? *reinterpret_cast<const float4*>(pend.p + (size_t)s * pend.stride + (size_t)row * pend.ld + 4 * i)
-                                         : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int k = 0; k < NORM_REG4; ++k) {
+            const int i = lane + 32 * k;
+            if (i < n4) {
+                v[k] = x[i];
+                gg[k] = *reinterpret_cast<const float4*>(gain + 4 * i);
             }
         }
-    }
-    if (r >= n_live) return;
-    float ss = 0.f;
+        if (pend.n > 0) {
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-        const int i = threadIdx.x + k * 256;
-        if (i < n4) {
-            if (pend.n > 0) {
-                // the adds stay in slice order
-                if (k < 2) {
+            for (int k = 0; k < NORM_REG4; ++k) {
+                const int i = lane + 32 * k;
+                if (i < n4) {
+                    float4 p[PARTIALS_MAX];
 #pragma unroll
                     for (int s = 0; s < PARTIALS_MAX; ++s)
-                        if (s < pend.n) { v[k].x += p[k][s].x; v[k].y += p[k][s].y; v[k].z += p[k][s].z; v[k].w += p[k][s].w; }
-                } else {
-                    for (int s = 0; s < pend.n; ++s) {
-                        const float4 q = *reinterpret_cast<const float4*>(pend.p + (size_t)s * pend.stride + (size_t)row * pend.ld + 4 * i);
-                        v[k].x += q.x; v[k].y += q.y; v[k].z += q.z; v[k].w += q.w;
-                    }
-                }
-                x[i] = v[k];
-            }
-            ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
-        }
-    }
-    ss = block_sum(ss, red);
-    const float rstd = rsqrtf(ss / (float)d + eps);
+                        if (s < pend.n) p[s] = *reinterpret_cast<const float4*>(pend.p + (size_t)s * pend.stride + pend_row + 4 * i);
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-        const int i = threadIdx.x + k * 256;
-        if (i < n4) {
-            const float4 gg = k < 2 ? gg2[k] : *reinterpret_cast<const float4*>(gain + 4 * i);
-            const float4 y = make_float4(v[k].x * rstd * gg.x, v[k].y * rstd * gg.y, v[k].z * rstd * gg.z, v[k].w * rstd * gg.w);
-            if (sizeof(T) == 2 && half_out) {          // IEEE half instead of bfloat16 (operand of a half-precision GEMM)
-                const __half2 lo = __floats2half2_rn(y.x, y.y), hi = __floats2half2_rn(y.z, y.w);
-                *reinterpret_cast<uint2*>(a + (size_t)r * d + 4 * i) =
-                    make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
-            } else {
-                store4<T>(a + (size_t)r * d + 4 * i, y);
+                    for (int s = 0; s < PARTIALS_MAX; ++s)          // the adds stay in slice order
+                        if (s < pend.n) { v[k].x += p[s].x; v[k].y += p[s].y; v[k].z += p[s].z; v[k].w += p[s].w; }
+                    x[i] = v[k];
+                }
             }
-            if (a_lo != nullptr) store4<T>(a_lo + (size_t)r * d + 4 * i, bf16_remainder(y));
         }
+#pragma unroll
+        for (int k = 0; k < NORM_REG4; ++k)
+            if (lane + 32 * k < n4) ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
+        ss = warp_sum(ss);
+        const float rstd = rsqrtf(ss / (float)d + eps);
+#pragma unroll
+        for (int k = 0; k < NORM_REG4; ++k) {
+            const int i = lane + 32 * k;
+            if (i < n4)
+                store_norm_out<T>(a_row, a_lo_row, i,
+                                  make_float4(v[k].x * rstd * gg[k].x, v[k].y * rstd * gg[k].y, v[k].z * rstd * gg[k].z, v[k].w * rstd * gg[k].w),
+                                  half_out);
+        }
+        return;
     }
+    for (int i = lane; i < n4; i += 32) {
+        float4 v = x[i];
+        if (pend.n > 0) {
+            for (int s = 0; s < pend.n; ++s) {
+                const float4 q = *reinterpret_cast<const float4*>(pend.p + (size_t)s * pend.stride + pend_row + 4 * i);
+                v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
+            }
+            x[i] = v;
+        }
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+    ss = warp_sum(ss);
+    const float rstd = rsqrtf(ss / (float)d + eps);
+    for (int i = lane; i < n4; i += 32) {
+        const float4 v = x[i], gg = *reinterpret_cast<const float4*>(gain + 4 * i);     // this lane's own writes
+        store_norm_out<T>(a_row, a_lo_row, i, make_float4(v.x * rstd * gg.x, v.y * rstd * gg.y, v.z * rstd * gg.z, v.w * rstd * gg.w), half_out);
+    }
+}
+
+// h_row[:] = E[token, :] as float (the residual stream), one warp per row; d is a multiple of 8.
+template <typename T>
+__device__ __forceinline__ void embed_row_warp(int lane, int d, const T* __restrict__ e_row, float* __restrict__ h_row) {
+    for (int i = lane; i < (d >> 2); i += 32) {
+        float v[4];
+        VecLoad<T, 4>::load(e_row + 4 * i, v);
+        reinterpret_cast<float4*>(h_row)[i] = make_float4(v[0], v[1], v[2], v[3]);
+    }
+}
+
+constexpr int ROW_WARPS = 8;         // rows per block of the stand-alone row-wise kernels
+
+// h[r, :] = E[token[r], :] (float residual stream); a[r, :] = RMSNorm(h[r, :]; gain) in storage type T.
+template <typename T>
+__global__ void __launch_bounds__(ROW_WARPS * 32) embed_rmsnorm_kernel(const StepDesc* __restrict__ sd, int d, const int32_t* token,
+                                                                        const T* __restrict__ embed, const float* __restrict__ gain, float eps,
+                                                                        float* __restrict__ h, T* __restrict__ a, T* __restrict__ a_lo, int half_out) {
+    const int r = blockIdx.x * ROW_WARPS + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (r >= sd->n_rows) return;
+    embed_row_warp<T>(lane, d, embed + (size_t)token[r] * d, h + (size_t)r * d);
+    norm_row_warp<T>(lane, d, h + (size_t)r * d, Partials{nullptr, 0, 0, 0}, 0, gain, eps, a + (size_t)r * d,
+                     a_lo ? a_lo + (size_t)r * d : nullptr, half_out);
+}
+
+// Optional residual update followed by the norm:  h[row, :] += pending partial sums of row;  a[r, :] = RMSNorm(h[row, :]; gain)
+// with row = src ? src[r] : r.  The partial sums are indexed by row, like h.  n_rows bounds r when there is no step descriptor.
+template <typename T>
+__global__ void __launch_bounds__(ROW_WARPS * 32) rmsnorm_kernel(const StepDesc* __restrict__ sd, int n_rows, int d, float* __restrict__ h,
+                                                                  const int32_t* __restrict__ src, Partials pend, const float* __restrict__ gain,
+                                                                  float eps, T* __restrict__ a, T* __restrict__ a_lo, int half_out) {
+    const int r = blockIdx.x * ROW_WARPS + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (r >= (sd != nullptr ? sd->n_rows : n_rows)) return;
+    const int row = src ? src[r] : r;
+    norm_row_warp<T>(lane, d, h + (size_t)row * d, pend, (size_t)row * pend.ld, gain, eps, a + (size_t)r * d,
+                     a_lo ? a_lo + (size_t)r * d : nullptr, half_out);
 }
 
 struct KvArena {
@@ -231,72 +261,123 @@ struct KvArena {
     int64_t n_slots;
 };
 
-// One block per (row, head of the fused q|k|v projection); thread i handles the rotary pair (i, i + hd/2).
-// The projection arrives as K-slice partial sums (one slice when the GEMM was not split); the bias is added here.
-// q heads: optional RMSNorm over head_dim, RoPE, stored to q_out [M, Hq*hd] as T.
-// k heads: optional RMSNorm, RoPE, stored to the row's KV slot.  v heads: stored to the row's KV slot.
+// Everything the q/k/v post-processing needs besides the item index.
 template <typename T>
-__global__ void qkv_post_kernel(const StepDesc* __restrict__ sd, int Hq, int Hkv, int hd, int layer, Partials qkv,
-                                const float* __restrict__ bias,
-                                const float* __restrict__ q_gain, const float* __restrict__ k_gain, float eps,
-                                const float2* __restrict__ rope, RowGeom g, KvArena prompt_arena, KvArena suffix_arena,
-                                T* __restrict__ q_out) {
-    __shared__ float red[33];
-    const int r = blockIdx.x, head = blockIdx.y, i = threadIdx.x, half = hd >> 1;
-    // rows past the live count are dropped after the loads have been requested (buffers hold the step's row bound)
-    const int n_live = sd->n_rows;
-    const float2 cs = rope[(size_t)r * half + i];
-    const int64_t slot = g.wslot[r];
-    const int to_suffix = g.warena[r];
-    const size_t col = (size_t)head * hd + i;
-    float x1 = bias ? bias[col] : 0.f, x2 = bias ? bias[col + half] : 0.f;
-    {
-        float p1[PARTIALS_MAX], p2[PARTIALS_MAX];          // requested together, added in slice order
+struct QkvPostArgs {
+    int Hq, Hkv, hd, layer;
+    Partials qkv;                 // the projection as K-slice partial sums (one slice when the GEMM was not split)
+    const float* bias;            // or nullptr
+    const float* q_gain;          // per-head RMSNorm gains, or nullptr
+    const float* k_gain;
+    float eps;
+    const float2* rope;           // [rows, hd/2] (cos, sin)
+    RowGeom g;
+    KvArena prompt_arena, suffix_arena;
+    T* q_out;                     // [rows, Hq * hd]
+};
+
+// One warp per (row, head of the fused q|k|v projection); lane i handles the rotary pairs (i, i + hd/2) and, for
+// head_dim 128, (i + 32, i + 32 + hd/2).  The bias is added here.
+// q heads: optional RMSNorm over head_dim, RoPE, stored to q_out as T.
+// k heads: optional RMSNorm, RoPE, stored to the row's KV slot.  v heads: stored to the row's KV slot.
+// NB items are processed together so that their loads are all in flight before the first one is used.
+template <typename T, int NB>
+__device__ __forceinline__ void qkv_post_items_warp(int lane, const QkvPostArgs<T>& A, const int* rows, const int* heads, int n_items) {
+    const int half = A.hd >> 1, npair = half > 32 ? 2 : 1;
+    float x1[NB][2], x2[NB][2];
+    float2 cs[NB][2];
+    int64_t slot[NB];
+    int to_suffix[NB];
 #pragma unroll
-        for (int s = 0; s < PARTIALS_MAX; ++s) {
-            const float* src = qkv.p + (size_t)s * qkv.stride + (size_t)r * qkv.ld + col;
-            p1[s] = s < qkv.n ? src[0] : 0.f;
-            p2[s] = s < qkv.n ? src[half] : 0.f;
+    for (int b = 0; b < NB; ++b) {
+        if (b >= n_items) continue;
+        const int r = rows[b], head = heads[b];
+        slot[b] = A.g.wslot[r];
+        to_suffix[b] = A.g.warena[r];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            if (j >= npair) continue;
+            const int i = lane + 32 * j;
+            const size_t col = (size_t)head * A.hd + i;
+            cs[b][j] = A.rope[(size_t)r * half + i];
+            float p1[PARTIALS_MAX], p2[PARTIALS_MAX];          // requested together, added in slice order
+#pragma unroll
+            for (int s = 0; s < PARTIALS_MAX; ++s) {
+                const float* src = A.qkv.p + (size_t)s * A.qkv.stride + (size_t)r * A.qkv.ld + col;
+                p1[s] = s < A.qkv.n ? src[0] : 0.f;
+                p2[s] = s < A.qkv.n ? src[half] : 0.f;
+            }
+            float a1 = A.bias ? A.bias[col] : 0.f, a2 = A.bias ? A.bias[col + half] : 0.f;
+#pragma unroll
+            for (int s = 0; s < PARTIALS_MAX; ++s)
+                if (s < A.qkv.n) { a1 += p1[s]; a2 += p2[s]; }
+            x1[b][j] = a1; x2[b][j] = a2;
+        }
+    }
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+        if (b >= n_items) continue;
+        const int r = rows[b], head = heads[b];
+        const bool is_q = head < A.Hq, is_k = !is_q && head < A.Hq + A.Hkv;
+        if (is_q || is_k) {
+            const float* gain = is_q ? A.q_gain : A.k_gain;
+            if (gain != nullptr) {
+                float ss = 0.f;
+#pragma unroll
+                for (int j = 0; j < 2; ++j)
+                    if (j < npair) ss += x1[b][j] * x1[b][j] + x2[b][j] * x2[b][j];
+                ss = warp_sum(ss);
+                const float rstd = rsqrtf(ss / (float)A.hd + A.eps);
+#pragma unroll
+                for (int j = 0; j < 2; ++j)
+                    if (j < npair) {
+                        x1[b][j] = x1[b][j] * rstd * gain[lane + 32 * j];
+                        x2[b][j] = x2[b][j] * rstd * gain[lane + 32 * j + half];
+                    }
+            }
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+                if (j < npair) {
+                    const float y1 = x1[b][j] * cs[b][j].x - x2[b][j] * cs[b][j].y;
+                    const float y2 = x2[b][j] * cs[b][j].x + x1[b][j] * cs[b][j].y;
+                    x1[b][j] = y1; x2[b][j] = y2;
+                }
+        }
+        if (is_q) {
+            T* dst = A.q_out + (size_t)r * A.Hq * A.hd + (size_t)head * A.hd;
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+                if (j < npair) { dst[lane + 32 * j] = from_f32<T>(x1[b][j]); dst[lane + 32 * j + half] = from_f32<T>(x2[b][j]); }
+            continue;
+        }
+        if (slot[b] < 0) continue;
+        const KvArena ar = to_suffix[b] ? A.suffix_arena : A.prompt_arena;
+        const int kvh = is_k ? head - A.Hq : head - A.Hq - A.Hkv;
+        const int64_t plane = ((int64_t)A.layer * 2 + (is_k ? 0 : 1)) * A.Hkv + kvh;
+        T* dst = reinterpret_cast<T*>(ar.base) + (plane * ar.n_slots + slot[b]) * A.hd;
+        if (!is_k && sizeof(T) == 2) {
+            // 16-bit models keep V as IEEE half (same two bytes, three more mantissa bits than bfloat16): V is a linear map
+            // of a unit-RMS vector, far inside half's range, and its rounding is the largest single error source of the logits
+            __half* dv = reinterpret_cast<__half*>(dst);
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+                if (j < npair) { dv[lane + 32 * j] = __float2half_rn(x1[b][j]); dv[lane + 32 * j + half] = __float2half_rn(x2[b][j]); }
+            continue;
         }
 #pragma unroll
-        for (int s = 0; s < PARTIALS_MAX; ++s)
-            if (s < qkv.n) { x1 += p1[s]; x2 += p2[s]; }
+        for (int j = 0; j < 2; ++j)
+            if (j < npair) { dst[lane + 32 * j] = from_f32<T>(x1[b][j]); dst[lane + 32 * j + half] = from_f32<T>(x2[b][j]); }
     }
-    if (r >= n_live) return;
-    const bool is_q = head < Hq, is_k = !is_q && head < Hq + Hkv;
-    if (is_q || is_k) {
-        const float* gain = is_q ? q_gain : k_gain;
-        if (gain != nullptr) {
-            const float ss = block_sum(x1 * x1 + x2 * x2, red);
-            const float rstd = rsqrtf(ss / (float)hd + eps);
-            x1 = x1 * rstd * gain[i];
-            x2 = x2 * rstd * gain[i + half];
-        }
-        const float y1 = x1 * cs.x - x2 * cs.y;
-        const float y2 = x2 * cs.x + x1 * cs.y;
-        x1 = y1; x2 = y2;
-    }
-    if (is_q) {
-        T* dst = q_out + (size_t)r * Hq * hd + (size_t)head * hd;
-        dst[i] = from_f32<T>(x1);
-        dst[i + half] = from_f32<T>(x2);
-        return;
-    }
-    if (slot < 0) return;
-    const KvArena ar = to_suffix ? suffix_arena : prompt_arena;
-    const int kvh = is_k ? head - Hq : head - Hq - Hkv;
-    const int64_t plane = ((int64_t)layer * 2 + (is_k ? 0 : 1)) * Hkv + kvh;
-    T* dst = reinterpret_cast<T*>(ar.base) + (plane * ar.n_slots + slot) * hd;
-    if (!is_k && sizeof(T) == 2) {
-        // 16-bit models keep V as IEEE half (same two bytes, three more mantissa bits than bfloat16): V is a linear map
-        // of a unit-RMS vector, far inside half's range, and its rounding is the largest single error source of the logits
-        __half* dv = reinterpret_cast<__half*>(dst);
-        dv[i] = __float2half_rn(x1);
-        dv[i + half] = __float2half_rn(x2);
-        return;
-    }
-    dst[i] = from_f32<T>(x1);
-    dst[i + half] = from_f32<T>(x2);
+}
+
+// Stand-alone form: one warp per (row, head), ROW_WARPS items per block, item = row * n_heads + head.
+template <typename T>
+__global__ void __launch_bounds__(ROW_WARPS * 32) qkv_post_kernel(const StepDesc* __restrict__ sd, QkvPostArgs<T> A) {
+    const int n_heads = A.Hq + 2 * A.Hkv;
+    const int item = blockIdx.x * ROW_WARPS + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (item >= sd->n_rows * n_heads) return;
+    const int row = item / n_heads, head = item - row * n_heads;
+    qkv_post_items_warp<T, 1>(lane, A, &row, &head, 1);
 }
 
 __global__ void reward_last_token_kernel(int n, const int32_t* tokens, const int64_t* last_index,

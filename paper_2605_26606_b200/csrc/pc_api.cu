@@ -5,6 +5,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -15,6 +16,7 @@
 #include "attention_mma.cuh"
 #include "attention_simt.cuh"
 #include "common.cuh"
+#include "decode_chain.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "kernels_basic.cuh"
@@ -25,8 +27,12 @@
 namespace {
 
 thread_local std::string g_cuda_error;
-unsigned long long g_launches = 0;     // kernels launched by this library since it was loaded
-inline void count_launches(int n) { g_launches += (unsigned long long)n; }
+std::atomic<unsigned long long> g_launches{0};     // kernels launched by this library since it was loaded (all contexts, all threads)
+thread_local long long g_capture_launches = -1;    // >= 0 while this thread captures a decode step: launches recorded, not run
+inline void count_launches(int n) {
+    if (g_capture_launches >= 0) g_capture_launches += n;
+    else g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed);
+}
 
 int cuda_fail(cudaError_t e, const char* what) {
     g_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
@@ -47,7 +53,8 @@ constexpr int kMaxSplits = pc::PARTIALS_MAX;
 
 struct Carve {
     size_t h, a, qkv, q, attn, act, logits, rope, pos, wslot, warena, p_start, p_len, s_start, s_len, token, last_row,
-        part_m, part_l, part_o, res_part, step_desc, step_counter, max_slen, sample_scratch, a_lo, attn_lo, total;
+        part_m, part_l, part_o, res_part, step_desc, step_counter, max_slen, sample_scratch, a_lo, attn_lo, chain_layers, chain_glob,
+        chain_bar, total;
 };
 
 // A captured decode step, replayable for every step that fits the same upper bounds and reads the same arrays.
@@ -64,7 +71,7 @@ struct GraphEntry {
 
 // TMA descriptors of one bf16 weight matrix [N, K], one per tile width the GEMM may pick.
 struct WMap {
-    CUtensorMap wide, narrow;   // boxes of 256 and 64 rows
+    CUtensorMap wide, narrow, mid;   // boxes of 256, 64 and 128 rows
     int N = 0, K = 0;
 };
 
@@ -103,6 +110,9 @@ struct pc_ctx {
     int plan_bn[5] = {0, 0, 0, 0, 0}, plan_splits[5] = {0, 0, 0, 0, 0};
     size_t split_capacity_rows = 0;          // rows x K-slices the partial-sum buffers hold
 
+    int decode_mode = 0;                     // 1: persistent chain kernel between attention calls (half-operand bf16 models); 0: one kernel per operation
+    bool chain_ready = false;                // tables uploaded by pc_set_workspace
+
     std::vector<GraphEntry> graphs;
     cudaStream_t capture_stream = nullptr;      // decode steps are captured here (the caller's stream may be the default one)
     void drop_graphs() {
@@ -121,6 +131,8 @@ struct pc_ctx {
 
 namespace {
 
+inline size_t chain_bar_words(int n_layers) { return (size_t)(n_layers + 1) * pc::chain::BAR_WORDS_PER_SEG; }
+
 Carve carve(const pc_ctx* c, int max_rows, int max_prefill) {
     const pc_model_desc& d = c->d;
     const size_t M = (size_t)std::max(max_rows, max_prefill), eb = c->eb();
@@ -134,6 +146,9 @@ Carve carve(const pc_ctx* c, int max_rows, int max_prefill) {
     v.res_part = take(split_rows * d.d_model * 4);
     v.a_lo = take(M * d.d_model * eb);
     v.attn_lo = take(M * c->q_dim() * eb);
+    v.chain_layers = take((size_t)d.n_layers * sizeof(pc::chain::LayerTab));
+    v.chain_glob = take(sizeof(pc::chain::GlobalTab));
+    v.chain_bar = take(chain_bar_words(d.n_layers) * 4);
     v.step_desc = take(sizeof(pc::StepDesc));
     v.step_counter = take(4);
     v.max_slen = take(4);
@@ -179,7 +194,8 @@ pc::RowGeom geom(const pc_ctx* c) {
 bool make_wmap(WMap* w, const void* base, int N, int K) {
     w->N = N;
     w->K = K;
-    return pc::make_bf16_map(&w->wide, base, N, K, 256) && pc::make_bf16_map(&w->narrow, base, N, K, 64);
+    return pc::make_bf16_map(&w->wide, base, N, K, 256) && pc::make_bf16_map(&w->narrow, base, N, K, 64) &&
+           pc::make_bf16_map(&w->mid, base, N, K, 128);
 }
 
 // Tile width and K-split of a bf16 GEMM over M rows.  Large batches take 128 x 256 tiles.  Small batches would
@@ -371,13 +387,14 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
     Partials pend = none;
 
     rope_table_kernel<<<(M * half + 255) / 256, 256, 0, st>>>(sd, half, (double)d.rope_theta, g.pos, rope);
-    embed_rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, g.token, reinterpret_cast<const T*>(c->embed), c->attn_norm[0],
+    const int row_blocks = (M + ROW_WARPS - 1) / ROW_WARPS;
+    embed_rmsnorm_kernel<T><<<row_blocks, ROW_WARPS * 32, 0, st>>>(sd, d.d_model, g.token, reinterpret_cast<const T*>(c->embed), c->attn_norm[0],
                                                d.rms_eps, h, a, a_lo, half_gemm ? 1 : 0);
     count_launches(2);
     PC_CUDA_CHECK_LAUNCH("embed_rmsnorm");
     for (int l = 0; l < d.n_layers; ++l) {
         if (l > 0) {
-            rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, h, nullptr, pend, c->attn_norm[l], d.rms_eps, a, a_lo, half_gemm ? 1 : 0);
+            rmsnorm_kernel<T><<<row_blocks, ROW_WARPS * 32, 0, st>>>(sd, M, d.d_model, h, nullptr, pend, c->attn_norm[l], d.rms_eps, a, a_lo, half_gemm ? 1 : 0);
             pend = none;
             count_launches(1);
         }
@@ -393,9 +410,10 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
                                    tc::EpiPartial{qkv, c->n_qkv(), qkv_parts.stride}, half_gemm))
                 return rc;
         }
-        qkv_post_kernel<T><<<dim3(M, d.n_q_heads + 2 * d.n_kv_heads), half, 0, st>>>(
-            sd, d.n_q_heads, d.n_kv_heads, d.head_dim, l, qkv_parts, bias, d.qk_norm ? c->q_norm[l] : nullptr,
-            d.qk_norm ? c->k_norm[l] : nullptr, d.rms_eps, rope, g, prompt_arena, suffix_arena, q);
+        const int post_items = M * (d.n_q_heads + 2 * d.n_kv_heads);
+        qkv_post_kernel<T><<<(post_items + ROW_WARPS - 1) / ROW_WARPS, ROW_WARPS * 32, 0, st>>>(
+            sd, QkvPostArgs<T>{d.n_q_heads, d.n_kv_heads, d.head_dim, l, qkv_parts, bias, d.qk_norm ? c->q_norm[l] : nullptr,
+                               d.qk_norm ? c->k_norm[l] : nullptr, d.rms_eps, rope, g, prompt_arena, suffix_arena, q});
         count_launches(2);
         if constexpr (kF32) {
             if (l == prof_layer) cudaEventRecord(c->prof_start, st);
@@ -425,7 +443,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
                     return rc2;
             }
         }
-        rmsnorm_kernel<T><<<M, 256, 0, st>>>(sd, d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a, nullptr, half_gemm ? 1 : 0);
+        rmsnorm_kernel<T><<<row_blocks, ROW_WARPS * 32, 0, st>>>(sd, M, d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a, nullptr, half_gemm ? 1 : 0);
         pend = none;
         count_launches(2);
         if constexpr (kF32) {
@@ -459,7 +477,7 @@ int run_lm_head(pc_ctx* c, cudaStream_t st, int n, const pc::StepDesc* sd, const
     T* a = reinterpret_cast<T*>(c->ws + c->cv.a);
     const bool half_gemm = !std::is_same<T, float>::value && d.half_gemm != 0;
     T* a_lo = std::is_same<T, float>::value || half_gemm ? nullptr : reinterpret_cast<T*>(c->ws + c->cv.a_lo);
-    rmsnorm_kernel<T><<<n, 256, 0, st>>>(sd, d.d_model, h, src, c->pend, c->final_norm, d.rms_eps, a, a_lo, half_gemm ? 1 : 0);
+    rmsnorm_kernel<T><<<(n + ROW_WARPS - 1) / ROW_WARPS, ROW_WARPS * 32, 0, st>>>(sd, n, d.d_model, h, src, c->pend, c->final_norm, d.rms_eps, a, a_lo, half_gemm ? 1 : 0);
     c->pend = pc::Partials{nullptr, 0, 0, 0};
     if constexpr (std::is_same<T, float>::value) {
         const T* wlm = reinterpret_cast<const T*>(d.tied_embed ? c->embed : c->lm_head);
@@ -500,7 +518,7 @@ const char* pc_status_string(int status) {
 
 const char* pc_last_cuda_error(void) { return g_cuda_error.c_str(); }
 
-uint64_t pc_launch_count(void) { return g_launches; }
+uint64_t pc_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 int pc_set_prompt_keys(pc_ctx* ctx, const int32_t* prompt_key) {
     if (ctx == nullptr) return PC_ERR_INVALID_ARG;
@@ -531,6 +549,13 @@ int pc_set_gemm_plan(pc_ctx* ctx, const char* spec) {
     }
     for (int k = 0; k < 5; ++k) { ctx->plan_bn[k] = bn[k]; ctx->plan_splits[k] = sp[k]; }
     ctx->drop_graphs();          // captured steps carry the old choice
+    return PC_OK;
+}
+
+int pc_set_decode_mode(pc_ctx* ctx, int mode) {
+    if (ctx == nullptr || (mode != 0 && mode != 1)) return PC_ERR_INVALID_ARG;
+    if (mode != ctx->decode_mode) ctx->drop_graphs();          // captured steps carry the old choice
+    ctx->decode_mode = mode;
     return PC_OK;
 }
 
@@ -668,6 +693,33 @@ int pc_set_workspace(pc_ctx* ctx, void* dev_ws, size_t bytes, int max_rows, int 
             g_cuda_error = "cuTensorMapEncodeTiled failed for an activation buffer";
             return PC_ERR_CUDA;
         }
+        ctx->chain_ready = false;
+        if (ctx->d.half_gemm) {
+            // constants of the persistent decode kernel: per-layer weight descriptors and gain / bias pointers
+            const pc_model_desc& d = ctx->d;
+            std::vector<pc::chain::LayerTab> tabs((size_t)d.n_layers);
+            auto put3 = [](CUtensorMap* dst, const WMap& m) { dst[0] = m.narrow; dst[1] = m.mid; dst[2] = m.wide; };
+            for (int l = 0; l < d.n_layers; ++l) {
+                pc::chain::LayerTab& t = tabs[(size_t)l];
+                std::memset(&t, 0, sizeof(t));
+                put3(t.wqkv, ctx->m_wqkv[l]); put3(t.wo, ctx->m_wo[l]); put3(t.wgu, ctx->m_wgu[l]); put3(t.wdown, ctx->m_wdown[l]);
+                t.attn_norm = ctx->attn_norm[l]; t.mlp_norm = ctx->mlp_norm[l];
+                t.bqkv = d.qkv_bias ? ctx->bqkv[l] : nullptr;
+                t.q_norm = d.qk_norm ? ctx->q_norm[l] : nullptr;
+                t.k_norm = d.qk_norm ? ctx->k_norm[l] : nullptr;
+            }
+            pc::chain::GlobalTab gt;
+            std::memset(&gt, 0, sizeof(gt));
+            gt.a = ctx->map_a; gt.attn = ctx->map_attn; gt.act = ctx->map_act;
+            put3(gt.lm, ctx->m_lm);
+            gt.final_norm = ctx->final_norm;
+            ce = cudaMemcpy(w + cv.chain_layers, tabs.data(), tabs.size() * sizeof(pc::chain::LayerTab), cudaMemcpyHostToDevice);
+            if (ce == cudaSuccess) ce = cudaMemcpy(w + cv.chain_glob, &gt, sizeof(gt), cudaMemcpyHostToDevice);
+            if (ce == cudaSuccess)
+                ce = cudaFuncSetAttribute(pc::chain::decode_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pc::chain::SMEM_BYTES);
+            if (ce != cudaSuccess) { ctx->ws = nullptr; return cuda_fail(ce, "tables of the persistent decode kernel"); }
+            ctx->chain_ready = true;
+        }
     }
     return PC_OK;
 }
@@ -687,7 +739,7 @@ int pc_prefill_shared(pc_ctx* ctx, void* stream, int n_prompts, const int32_t* p
     const pc::RowGeom g = geom(ctx);
     int32_t* last_row = reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.last_row);
     pc::StepDesc* sd = reinterpret_cast<pc::StepDesc*>(ctx->ws + ctx->cv.step_desc);
-    pc::set_step_desc<<<1, 1, 0, st>>>(sd, total_tokens, n_prompts, max_prompt_len, g.max_slen);
+    pc::set_step_desc<<<1, pc::STEP_DESC_THREADS, 0, st>>>(sd, total_tokens, n_prompts, max_prompt_len, g.max_slen, nullptr, 0);
     pc::prep_prefill_rows<<<n_prompts, 256, 0, st>>>(n_prompts, prompt_tokens, prompt_offsets, prompt_kv_start, prompt_slots,
                                                      ctx->d.vocab, g, last_row, ctx->err);
     count_launches(2);
@@ -752,6 +804,91 @@ int check_decode_args(const pc_ctx* ctx, const DecodeArgs& a) {
     return PC_OK;
 }
 
+// One segment of the persistent decode kernel (decode_chain.cuh) over the rows described by *sd.
+int launch_chain(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, int seg, pc::KvArena prompt_arena, pc::KvArena suffix_arena,
+                 const pc::am::PrefixPartial& part, float* logits) {
+    using namespace pc;
+    const pc_model_desc& d = c->d;
+    char* w = c->ws;
+    chain::ChainParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.sd = sd; p.M = M; p.seg = seg; p.with_merge = 0;
+    p.n_layers = d.n_layers; p.d_model = d.d_model; p.n_qkv = c->n_qkv(); p.q_dim = c->q_dim(); p.d_ff = d.d_ff; p.vocab = d.vocab;
+    p.Hq = d.n_q_heads; p.Hkv = d.n_kv_heads; p.hd = d.head_dim; p.eps = d.rms_eps;
+    const WMap* maps[5] = {&c->m_wqkv[0], &c->m_wo[0], &c->m_wgu[0], &c->m_wdown[0], &c->m_lm};
+    const bool may_split[5] = {true, true, false, true, false};
+    for (int k = 0; k < 5; ++k) {
+        const GemmPlan gp = plan_gemm(c, (GemmKind)k, *maps[k], M, may_split[k]);
+        p.bn[k] = gp.wide ? 256 : 64;
+        p.splits[k] = gp.splits;
+    }
+    auto pick = [](const WMap& m, int bn) -> const CUtensorMap& { return bn == 256 ? m.wide : (bn == 128 ? m.mid : m.narrow); };
+    const int l_here = seg < 0 ? 0 : seg;
+    p.maps[chain::MAP_A] = c->map_a; p.maps[chain::MAP_ATTN] = c->map_attn; p.maps[chain::MAP_ACT] = c->map_act;
+    p.maps[chain::MAP_WO] = pick(c->m_wo[l_here], p.bn[GEMM_O]);
+    p.maps[chain::MAP_WGU] = pick(c->m_wgu[l_here], p.bn[GEMM_GATE_UP]);
+    p.maps[chain::MAP_WDOWN] = pick(c->m_wdown[l_here], p.bn[GEMM_DOWN]);
+    p.maps[chain::MAP_WNEXT] = seg == d.n_layers - 1 ? pick(c->m_lm, p.bn[GEMM_LM_HEAD]) : pick(c->m_wqkv[seg + 1], p.bn[GEMM_QKV]);
+    p.layers = reinterpret_cast<const chain::LayerTab*>(w + c->cv.chain_layers);
+    p.glob = reinterpret_cast<const chain::GlobalTab*>(w + c->cv.chain_glob);
+    p.embed = c->embed;
+    p.h = reinterpret_cast<float*>(w + c->cv.h);
+    p.a = reinterpret_cast<__nv_bfloat16*>(w + c->cv.a);
+    p.qkv = reinterpret_cast<float*>(w + c->cv.qkv);
+    p.res_part = reinterpret_cast<float*>(w + c->cv.res_part);
+    p.q = reinterpret_cast<__nv_bfloat16*>(w + c->cv.q);
+    p.attn = reinterpret_cast<__nv_bfloat16*>(w + c->cv.attn);
+    p.act = reinterpret_cast<__nv_bfloat16*>(w + c->cv.act);
+    p.logits = logits;
+    p.rope = reinterpret_cast<const float2*>(w + c->cv.rope);
+    p.g = geom(c);
+    p.prompt_arena = prompt_arena; p.suffix_arena = suffix_arena;
+    p.part = part;
+    p.bar = reinterpret_cast<int32_t*>(w + c->cv.chain_bar);
+    p.err = c->err;
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)c->num_sms); cfg.blockDim = dim3(chain::THREADS); cfg.dynamicSmemBytes = chain::SMEM_BYTES; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeCooperative;       // every CTA must be resident: they wait for one another
+    at[0].val.cooperative = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, chain::decode_chain_kernel, p);
+    if (e != cudaSuccess) return cuda_fail(e, "persistent decode kernel");
+    count_launches(1);
+    return PC_OK;
+}
+
+// The decoder layers and the LM head of a decode step with the persistent kernel between the attention calls.
+int run_decode_chained(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::KvArena prompt_arena, pc::KvArena suffix_arena,
+                       const AttnPlan& plan, float* logits) {
+    using namespace pc;
+    const pc_model_desc& d = c->d;
+    char* w = c->ws;
+    const RowGeom g = geom(c);
+    const int half = d.head_dim / 2;
+    int prof_layer = c->prof_layer;
+    c->prof_layer = -1;                               // one-shot (a captured step never carries the events)
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    cudaStreamIsCapturing(st, &cap);
+    if (cap != cudaStreamCaptureStatusNone) prof_layer = -1;
+    rope_table_kernel<<<(M * half + 255) / 256, 256, 0, st>>>(sd, half, (double)d.rope_theta, g.pos, reinterpret_cast<float2*>(w + c->cv.rope));
+    count_launches(1);
+    PC_CUDA_CHECK_LAUNCH("rope table");
+    const am::PrefixPartial none{nullptr, nullptr, nullptr, 0, 0, 0, 0};
+    if (int rc = launch_chain(c, st, M, sd, -1, prompt_arena, suffix_arena, none, logits)) return rc;
+    const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(w + c->cv.q);
+    __nv_bfloat16* attn = reinterpret_cast<__nv_bfloat16*>(w + c->cv.attn);
+    for (int l = 0; l < d.n_layers; ++l) {
+        int rc = d.head_dim == 128 ? attention_bf16<128>(c, st, sd, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer)
+                                   : attention_bf16<64>(c, st, sd, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer);
+        if (rc) return rc;
+        if ((rc = launch_chain(c, st, M, sd, l, prompt_arena, suffix_arena, none, logits))) return rc;
+    }
+    PC_CUDA_CHECK_LAUNCH("chained decode step");
+    return PC_OK;
+}
+
 // The kernels of one decode step.  Grids and GEMM plans are sized for (m_bound rows, groups_bound groups of at most
 // group_rows_bound rows); the live counts and the offsets into the caller's row arrays are in the step descriptor.
 int decode_launches(pc_ctx* ctx, cudaStream_t st, int m_bound, int groups_bound, int group_rows_bound, const DecodeArgs& a,
@@ -766,11 +903,17 @@ int decode_launches(pc_ctx* ctx, cudaStream_t st, int m_bound, int groups_bound,
     const pc::KvArena pa{const_cast<void*>(a.prompt_kv), a.prompt_slots}, sa{a.suffix_kv, a.suffix_slots};
     const bool f32 = ctx->d.dtype == PC_DTYPE_F32;
     const AttnPlan plan{false, groups_bound, a.group_row_start, group_rows_bound};
-    int rc = f32 ? run_layers<float>(ctx, st, m_bound, sd, pa, sa, plan) : run_layers<__nv_bfloat16>(ctx, st, m_bound, sd, pa, sa, plan);
-    if (rc) return rc;
     float* logits = logits_out ? logits_out : reinterpret_cast<float*>(ctx->ws + ctx->cv.logits);
-    rc = f32 ? run_lm_head<float>(ctx, st, m_bound, sd, nullptr, logits) : run_lm_head<__nv_bfloat16>(ctx, st, m_bound, sd, nullptr, logits);
-    if (rc) return rc;
+    int rc;
+    if (!f32 && ctx->decode_mode == 1 && ctx->chain_ready) {
+        rc = run_decode_chained(ctx, st, m_bound, sd, pa, sa, plan, logits);
+        if (rc) return rc;
+    } else {
+        rc = f32 ? run_layers<float>(ctx, st, m_bound, sd, pa, sa, plan) : run_layers<__nv_bfloat16>(ctx, st, m_bound, sd, pa, sa, plan);
+        if (rc) return rc;
+        rc = f32 ? run_lm_head<float>(ctx, st, m_bound, sd, nullptr, logits) : run_lm_head<__nv_bfloat16>(ctx, st, m_bound, sd, nullptr, logits);
+        if (rc) return rc;
+    }
     if (a.sample) {
         const uint32_t k0 = (uint32_t)(a.seed & 0xffffffffu), k1 = (uint32_t)(a.seed >> 32);
         const int chunks = pc::sample_chunks(m_bound, ctx->num_sms);
@@ -820,8 +963,10 @@ int pc_decode_step(pc_ctx* ctx, void* stream, int n_rows, const int32_t* row_pro
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (ctx->d.dtype == PC_DTYPE_BF16)
         if (int rc = arena_maps(ctx, prompt_kv, prompt_slots, suffix_kv, suffix_slots)) return rc;
-    pc::set_step_desc<<<1, 1, 0, st>>>(reinterpret_cast<pc::StepDesc*>(ctx->ws + ctx->cv.step_desc), n_rows, n_groups, max_group_rows,
-                                       reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.max_slen));
+    pc::set_step_desc<<<1, pc::STEP_DESC_THREADS, 0, st>>>(reinterpret_cast<pc::StepDesc*>(ctx->ws + ctx->cv.step_desc), n_rows, n_groups,
+                                                           max_group_rows, reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.max_slen),
+                                                           reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.chain_bar),
+                                                           (int)chain_bar_words(ctx->d.n_layers));
     count_launches(1);
     return decode_launches(ctx, st, n_rows, n_groups, max_group_rows, a, logits_out);
 }
@@ -859,8 +1004,8 @@ int pc_decode_run(pc_ctx* ctx, void* stream, int n_steps, const pc_step_desc* st
     if (e != cudaSuccess) return cuda_fail(e, "reset step counter");
     for (int s = 0; s < n_steps; ++s) {
         if (steps_host[s].n_rows == 0) {          // keep the device counter in step with the host loop
-            pc::load_step_desc<<<1, 1, 0, st>>>(reinterpret_cast<const pc::StepDesc*>(steps_dev), counter, sd,
-                                                reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.max_slen));
+            pc::load_step_desc<<<1, pc::STEP_DESC_THREADS, 0, st>>>(reinterpret_cast<const pc::StepDesc*>(steps_dev), counter, sd,
+                                                                    reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.max_slen), nullptr, 0);
             count_launches(1);
             continue;
         }
@@ -875,7 +1020,6 @@ int pc_decode_run(pc_ctx* ctx, void* stream, int n_steps, const pc_step_desc* st
             if (std::memcmp(&ent.key, &key, sizeof(key)) == 0) { exec = ent.exec; break; }
         if (exec == nullptr) {
             if (ctx->graphs.size() >= 64) ctx->drop_graphs();
-            const unsigned long long launches_before = g_launches;
             cudaGraph_t graph = nullptr;
             if (ctx->capture_stream == nullptr) {
                 e = cudaStreamCreateWithFlags(&ctx->capture_stream, cudaStreamNonBlocking);
@@ -884,19 +1028,23 @@ int pc_decode_run(pc_ctx* ctx, void* stream, int n_steps, const pc_step_desc* st
             cudaStream_t cs = ctx->capture_stream;
             e = cudaStreamBeginCapture(cs, cudaStreamCaptureModeThreadLocal);
             if (e != cudaSuccess) return cuda_fail(e, "begin graph capture");
-            pc::load_step_desc<<<1, 1, 0, cs>>>(reinterpret_cast<const pc::StepDesc*>(steps_dev), counter, sd,
-                                                reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.max_slen));
+            g_capture_launches = 0;                // launches are recorded into the graph, not run
+            pc::load_step_desc<<<1, pc::STEP_DESC_THREADS, 0, cs>>>(reinterpret_cast<const pc::StepDesc*>(steps_dev), counter, sd,
+                                                                    reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.max_slen),
+                                                                    reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.chain_bar),
+                                                                    (int)chain_bar_words(ctx->d.n_layers));
             count_launches(1);
             const int rc = decode_launches(ctx, cs, m_bound, groups_bound, group_rows_bound, a, nullptr);
             e = cudaStreamEndCapture(cs, &graph);
+            const int captured = (int)g_capture_launches;
+            g_capture_launches = -1;
             if (rc != PC_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
             if (e != cudaSuccess) return cuda_fail(e, "end graph capture");
             e = cudaGraphInstantiate(&exec, graph, 0);
             cudaGraphDestroy(graph);
             if (e != cudaSuccess) return cuda_fail(e, "graph instantiate");
             GraphEntry ent;
-            ent.key = key; ent.exec = exec; ent.launches = (int)(g_launches - launches_before);
-            g_launches = launches_before;         // capturing launched nothing
+            ent.key = key; ent.exec = exec; ent.launches = captured;
             ctx->graphs.push_back(ent);
         }
         e = cudaGraphLaunch(exec, st);

@@ -334,3 +334,35 @@ def test_bound_pass_bf16_logits_against_full_recompute():
                 assert int(toks[s + 1]) == tok_o, (key_prompt, i, s, gap)
             n_cmp += 1
     assert n_cmp > 50 and worst <= 5e-2, (n_cmp, worst)
+
+
+@pytest.mark.parametrize("model", [wl.SMALL_BF16, wl.SMALL_QKNORM_BF16, wl.TINY_BF16], ids=lambda m: m.name)
+def test_persistent_decode_kernel_equals_one_kernel_per_operation(model):
+    """pc_set_decode_mode: the persistent kernel (phases separated by grid barriers) runs the arithmetic of the separate
+    kernels in the same order, so a free-running Pilot-Commit step gives identical tokens and identical recorded logits; a
+    missed barrier or a stale tile would show up as a difference."""
+    from paper_2605_26606_b200 import binding as B
+    w = dataclasses.replace(wl.WORKLOADS["config0"], model=model, n_prompts=5, prompt_len_lo=3, prompt_len_hi=90, group_size=40,
+                            n_pilot=8, max_new=40, cap_lo=1, cap_hi=40, data_seed=21,
+                            forced_explicit=((0, 0.5), (1, 0.5), (2, 0.5), (3, 0.0), (4, 0.5)))
+    weights = wl.gen_weights(model, seed=0, threads=2, gain_jitter=0.1)
+    batch = wl.gen_batch(w)
+    eng = RolloutEngine(model, weights, max_rows=200, max_prefill_tokens=int(batch.prompt_offsets[-1]))
+    outs, logits = [], []
+    for mode in (0, 1, 1):
+        B.pc_set_decode_mode(eng.ctx, mode)
+        eng.record_pilot_logits = {s: None for s in (0, 5, 17)}
+        outs.append(eng.pilot_commit_step(w, batch))
+        logits.append({s: v[0].clone() for s, v in eng.record_pilot_logits.items()})
+    eng.record_pilot_logits = None
+    a = outs[0]
+    assert np.any(a["status"] == ostats.COMMIT)
+    for b, lg in zip(outs[1:], logits[1:]):
+        assert np.array_equal(a["status"], b["status"])
+        for p in range(w.n_prompts):
+            for i in range(w.group_size):
+                if a["generated"][p, i]:
+                    assert np.array_equal(a["tokens"][p][i], b["tokens"][p][i]), (p, i)
+        for s in lg:
+            assert torch.equal(lg[s], logits[0][s]), s
+        assert np.array_equal(a["advantages"], b["advantages"])
