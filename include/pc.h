@@ -175,6 +175,14 @@ PC_API int pc_set_gemm_plan(pc_ctx* ctx, const char* spec);
  * Drops captured decode steps.  The paper has no counterpart. */
 PC_API int pc_set_decode_mode(pc_ctx* ctx, int mode);
 
+/* Tracing aid for mode 1: with a buffer set (device int64, at least pc_chain_trace_words(ctx) words, zeroed by the
+ * caller), the first four CTAs of every launch of the persistent kernel store SM clock stamps of their roles per phase:
+ * trace[segment + 1][phase][cta][16], events 0..11 = workers begin / barrier passed / done, producer begin / barrier
+ * passed / done, first operand tile arrived / MMAs issued, first accumulator ready / epilogues done, kernel begin / end
+ * (the last two in phase 0).  NULL switches it off (the default).  Drops captured decode steps.  No counterpart in the paper. */
+PC_API int pc_set_chain_trace(pc_ctx* ctx, int64_t* trace, size_t n_words);
+PC_API size_t pc_chain_trace_words(const pc_ctx* ctx);
+
 /* Measurement aid: in the next pc_decode_step of this context, record the two CUDA events (cudaEvent_t,
  * created by the caller) around the attention kernel of `layer` that reads the rollouts' own suffix K/V
  * (for float32 models: the single attention kernel).  One-shot; the caller synchronises and reads the

@@ -636,39 +636,35 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
 // log-sum-exp:  M = max m_i,  out = sum_i O_i 2^(m_i - M) / sum_i l_i 2^(m_i - M).  Records are added in index order.
 // One warp per (row, head); a lane owns HD/32 consecutive dims.
 // ---------------------------------------------------------------------------------------------
+// rh = row * Hq + head (the caller keeps it below n_live * Hq).  ct = tiles per suffix chunk of this step (suffix_plan);
+// n_load = how many records to request: every record index the step can have produced (part.n_parts + chunk slots per
+// item), so that the loads do not wait for the row's suffix length; records past the row's own count are ignored.
 template <int HD>
-__device__ __forceinline__ void merge_item_warp(int lane, size_t rh, const StepDesc* __restrict__ sd, int Hq, const RowGeom& g,
-                                                const PrefixPartial& part, __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ out_lo) {
+__device__ __forceinline__ void merge_item_warp(int lane, size_t rh, int Hq, const RowGeom& g, const PrefixPartial& part, int ct, int n_load,
+                                                __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ out_lo) {
     constexpr int EPL = HD / 32;
-    // The row's suffix length is requested together with the step descriptor, and every record of the (row, head) --
-    // (m, l) and its output slice -- is requested before the first one is used, so an item pays two memory round trips
-    // instead of four.  Records are added in index order.
     const int row = (int)(rh / Hq);
-    const int row_in = min(row, (int)(part.stride / (size_t)Hq) - 1);          // callers may reach past the row bound
-    const int n_live = sd->n_rows, slen = g.s_len[row_in], max_slen = *g.max_slen;
-    if (rh >= (size_t)n_live * Hq) return;
-    const int n_sfx = suffix_chunks(slen, suffix_plan(max_slen, n_live * part.n_kv_heads, part.n_suffix_warps).ct);
-    const int n_rec = part.n_parts + n_sfx;
+    const int slen = g.s_len[row];
     float mi[MAX_RECORDS], li[MAX_RECORDS];
     float ov[MAX_RECORDS][EPL];
 #pragma unroll
     for (int i = 0; i < MAX_RECORDS; ++i) {
-        mi[i] = -INFINITY; li[i] = 0.f;
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) ov[i][e] = 0.f;
-        if (i < n_rec) {
-            mi[i] = part.m[(size_t)i * part.stride + rh];
-            li[i] = part.l[(size_t)i * part.stride + rh];
-            const float* src = part.o + ((size_t)i * part.stride + rh) * HD + lane * EPL;
-            if (EPL == 4) {
-                const float4 v = *reinterpret_cast<const float4*>(src);
-                ov[i][0] = v.x; ov[i][1] = v.y; ov[i][2] = v.z; ov[i][3] = v.w;
-            } else {
-                const float2 v = *reinterpret_cast<const float2*>(src);
-                ov[i][0] = v.x; ov[i][1] = v.y;
-            }
+        const bool ld = i < n_load;
+        mi[i] = ld ? part.m[(size_t)i * part.stride + rh] : -INFINITY;
+        li[i] = ld ? part.l[(size_t)i * part.stride + rh] : 0.f;
+        const float* src = part.o + ((size_t)i * part.stride + rh) * HD + lane * EPL;
+        if (EPL == 4) {
+            const float4 v = ld ? *reinterpret_cast<const float4*>(src) : make_float4(0.f, 0.f, 0.f, 0.f);
+            ov[i][0] = v.x; ov[i][1] = v.y; ov[i][2] = v.z; ov[i][3] = v.w;
+        } else {
+            const float2 v = ld ? *reinterpret_cast<const float2*>(src) : make_float2(0.f, 0.f);
+            ov[i][0] = v.x; ov[i][1] = v.y;
         }
     }
+    const int n_rec = part.n_parts + suffix_chunks(slen, ct);
+#pragma unroll
+    for (int i = 0; i < MAX_RECORDS; ++i)
+        if (i >= n_rec) mi[i] = -INFINITY;           // not a record of this row (stale memory)
     float M = -INFINITY;
 #pragma unroll
     for (int i = 0; i < MAX_RECORDS; ++i) M = fmaxf(M, mi[i]);
@@ -712,7 +708,11 @@ __device__ __forceinline__ void merge_item_warp(int lane, size_t rh, const StepD
 template <int HD>
 __global__ void __launch_bounds__(256) attn_merge_kernel(const StepDesc* __restrict__ sd, int Hq, RowGeom g, PrefixPartial part,
                                                          __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ out_lo) {
-    merge_item_warp<HD>(threadIdx.x & 31, (size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), sd, Hq, g, part, out, out_lo);
+    const size_t rh = (size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int n_live = sd->n_rows;
+    if (rh >= (size_t)n_live * Hq) return;
+    const SuffixPlan sp = suffix_plan(*g.max_slen, n_live * part.n_kv_heads, part.n_suffix_warps);
+    merge_item_warp<HD>(threadIdx.x & 31, rh, Hq, g, part, sp.ct, part.n_parts + sp.cpi, out, out_lo);
 }
 
 }  // namespace am

@@ -46,13 +46,13 @@ using tc::tma_load_2d;
 constexpr int THREADS = 256;
 constexpr int WORKER_WARP0 = 2, N_WORKER_WARPS = 6;
 constexpr int A_BYTES = BM * BK * 2;
-constexpr int SLOT_BYTES = 48 * 1024;            // activation tile (16 KB) + weight tile of up to 256 rows (32 KB)
-constexpr int SLOTS = 4;
+constexpr int RING_BYTES = 192 * 1024;           // operand ring: slots of (activation tile 16 KB + widest weight tile of the launch)
+constexpr int MAX_SLOTS = 8;
 constexpr int ACC_COLS = 256;                    // TMEM columns per accumulator (two accumulators)
 constexpr uint32_t TMEM_COLS = 512;
 constexpr int MAX_PHASES = 10;
 constexpr int BAR_WORDS_PER_SEG = 16;
-constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int SMEM_BYTES = RING_BYTES + 1024 /*align*/ + 512 /*barriers, flags*/;
 constexpr uint32_t GRID_WAIT_LIMIT = 1u << 22;
 
 enum Phase : int { PH_END = 0, PH_EMBED, PH_MERGE, PH_O, PH_NORM_MLP, PH_GU, PH_DOWN, PH_NORM_NEXT, PH_QKV, PH_POST, PH_LM };
@@ -87,6 +87,7 @@ struct ChainParams {
     int n_layers, d_model, n_qkv, q_dim, d_ff, vocab, Hq, Hkv, hd;
     float eps;
     int bn[5], splits[5];        // tile width and K-slices per GEMM kind
+    int slot_bytes, slots;       // operand ring of this launch: 16 KB + 128 B x the widest tile, RING_BYTES / slot_bytes slots
     const LayerTab* layers;
     const GlobalTab* glob;
     const void* embed;
@@ -104,7 +105,15 @@ struct ChainParams {
     am::PrefixPartial part;
     int32_t* bar;                // BAR_WORDS_PER_SEG words per segment, zero when the step starts
     int32_t* err;
+    long long* trace;            // optional: SM clock stamps of the first TRACE_CTAS CTAs, [segment][phase][cta][TRACE_EVENTS]
 };
+constexpr int TRACE_CTAS = 4, TRACE_EVENTS = 16;
+enum TraceEvent : int { TR_W_BEGIN = 0, TR_W_WAITED, TR_W_DONE, TR_P_BEGIN, TR_P_BARRIER, TR_P_DONE, TR_M_FIRST_FULL, TR_M_DONE,
+                        TR_E_FIRST_FULL, TR_E_DONE, TR_KERNEL_BEGIN, TR_KERNEL_END };
+__device__ __forceinline__ void stamp(const ChainParams& p, int j, int ev) {
+    if (p.trace != nullptr && blockIdx.x < TRACE_CTAS)
+        p.trace[((size_t)((p.seg + 1) * MAX_PHASES + j) * TRACE_CTAS + blockIdx.x) * TRACE_EVENTS + ev] = clock64();
+}
 
 __device__ __forceinline__ bool is_gemm(int ph) { return ph == PH_O || ph == PH_GU || ph == PH_DOWN || ph == PH_QKV || ph == PH_LM; }
 
@@ -198,22 +207,28 @@ __device__ __forceinline__ bool grid_wait_relayed(const int32_t* bar, int target
 __global__ void __launch_bounds__(THREADS, 1) decode_chain_kernel(const __grid_constant__ ChainParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + SLOTS * SLOT_BYTES);
-    // bars: full[SLOTS], empty[SLOTS], tmem_full[2], tmem_empty[2]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * SLOTS + 4);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + RING_BYTES);
+    // bars: full[MAX_SLOTS], empty[MAX_SLOTS], tmem_full[2], tmem_empty[2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * MAX_SLOTS + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int* s_arrive = reinterpret_cast<int*>(tmem_slot + 2);          // [MAX_PHASES]
     volatile int* s_relay = reinterpret_cast<volatile int*>(s_arrive + MAX_PHASES);       // [MAX_PHASES]
+    int* s_norm_cnt = s_arrive + 2 * MAX_PHASES;                    // [MAX_PHASES]
+    volatile float* s_norm_red = reinterpret_cast<volatile float*>(s_norm_cnt + MAX_PHASES);     // [MAX_PHASES][8]
+    const int SLOTS = p.slots, SLOT_BYTES = p.slot_bytes;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * SLOTS, tfull0 = empty0 + 8 * SLOTS, tempty0 = tfull0 + 16;
+    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * MAX_SLOTS, tfull0 = empty0 + 8 * MAX_SLOTS, tempty0 = tfull0 + 16;
     const uint32_t tiles_u32 = smem_u32(tiles);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < SLOTS; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        for (int s = 0; s < MAX_SLOTS; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(tfull0 + 8 * b, 1); mbar_init(tempty0 + 8 * b, 4); }
         *abort_flag = 0;
-        for (int j = 0; j < MAX_PHASES; ++j) { s_arrive[j] = 0; s_relay[j] = 0; }
+        for (int j = 0; j < MAX_PHASES; ++j) {
+            s_arrive[j] = 0; s_relay[j] = 0; s_norm_cnt[j] = 0;
+            for (int g = 0; g < 8; ++g) s_norm_red[j * 8 + g] = 0.f;
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -223,6 +238,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_chain_kernel(const __grid_c
     tc::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    if (threadIdx.x == 0) stamp(p, 0, TR_KERNEL_BEGIN);
     const int M = p.M, tiles_m = (M + BM - 1) / BM;
     int32_t* bar = p.bar + (p.seg + 1) * BAR_WORDS_PER_SEG;
     const int n_cta = gridDim.x;
@@ -244,44 +260,51 @@ __global__ void __launch_bounds__(THREADS, 1) decode_chain_kernel(const __grid_c
                 // k-blocks of this CTA in this phase, in order: (tile, kb).  The weight tile of a k-block is requested as
                 // soon as its slot is free; the activation tile follows once the previous phase is complete everywhere,
                 // so up to SLOTS weight tiles are already on their way when the barrier opens.
-                bool a_ready = j == 0;          // a first phase reads what earlier launches wrote
-                int tb = blockIdx.x, kbb = 0;                       // cursor of the weight loads
-                uint32_t slot_b = slot, phase_b = phase;
-                int ahead = 0;                                      // weight loads issued whose activation load is pending
-                auto tile_geom = [&](int t, int& m0, int& n0, int& kb0, int& kb1) {
-                    const int sp = (t / tiles_m) % gd.splits;
-                    m0 = (t % tiles_m) * BM; n0 = (t / (tiles_m * gd.splits)) * gd.BN;
-                    kb0 = sp * kbt / gd.splits; kb1 = (sp + 1) * kbt / gd.splits;
+                stamp(p, j, TR_P_BEGIN);
+                struct Cursor { int t, kb, kb1, m0, n0; };
+                auto seek = [&](Cursor& c) {                        // geometry of tile c.t (a few integer divisions: once per tile)
+                    if (c.t >= n_tiles) return;
+                    const int sp = (c.t / tiles_m) % gd.splits;
+                    c.m0 = (c.t % tiles_m) * BM; c.n0 = (c.t / (tiles_m * gd.splits)) * gd.BN;
+                    c.kb = sp * kbt / gd.splits; c.kb1 = (sp + 1) * kbt / gd.splits;
                 };
-                int ta = blockIdx.x, kba = 0;                       // cursor of the activation loads
-                while (ok && ta < n_tiles) {
-                    // weight loads: run ahead while slots are free (all the way when the activations are ready)
-                    while (ok && tb < n_tiles && ahead < SLOTS) {
-                        int m0, n0, kb0, kb1;
-                        tile_geom(tb, m0, n0, kb0, kb1);
+                auto advance = [&](Cursor& c) { if (++c.kb == c.kb1) { c.t += n_cta; seek(c); } };
+                Cursor cb{(int)blockIdx.x, 0, 0, 0, 0};
+                seek(cb);
+                if (j > 0 && cb.t < n_tiles) {
+                    // the phase reads what the previous phase wrote: weight tiles first, as many as there are slots
+                    Cursor ca = cb;
+                    uint32_t slot_b = slot, phase_b = phase;
+                    int ahead = 0;
+                    while (cb.t < n_tiles && ahead < SLOTS) {
                         if (!mbar_wait(empty0 + 8 * slot_b, phase_b ^ 1u, abort_flag)) { ok = false; break; }
                         mbar_arrive_expect_tx(full0 + 8 * slot_b, stage_tx);
-                        tma_load_2d(tiles_u32 + slot_b * SLOT_BYTES + A_BYTES, map_w, full0 + 8 * slot_b, (kb0 + kbb) * BK, n0);
+                        tma_load_2d(tiles_u32 + slot_b * SLOT_BYTES + A_BYTES, map_w, full0 + 8 * slot_b, cb.kb * BK, cb.n0);
                         ++ahead;
-                        if (++slot_b == SLOTS) { slot_b = 0; phase_b ^= 1u; }
-                        if (kb0 + ++kbb == kb1) { kbb = 0; tb += n_cta; }
-                        if (a_ready) break;                         // steady state: one weight load, then its activation load
+                        if (++slot_b == (uint32_t)SLOTS) { slot_b = 0; phase_b ^= 1u; }
+                        advance(cb);
                     }
                     if (!ok) break;
-                    if (!a_ready) {
-                        if (!grid_wait(bar + (j - 1), n_cta, abort_flag)) { ok = false; break; }
-                        asm volatile("fence.proxy.async;" ::: "memory");             // other CTAs' stores before this thread's TMA reads
-                        a_ready = true;
-                    }
-                    while (ahead > 0) {
-                        int m0, n0, kb0, kb1;
-                        tile_geom(ta, m0, n0, kb0, kb1);
-                        tma_load_2d(tiles_u32 + slot * SLOT_BYTES, map_a, full0 + 8 * slot, (kb0 + kba) * BK, m0);
-                        --ahead;
-                        if (++slot == SLOTS) { slot = 0; phase ^= 1u; }
-                        if (kb0 + ++kba == kb1) { kba = 0; ta += n_cta; }
+                    if (!grid_wait(bar + (j - 1), n_cta, abort_flag)) { ok = false; break; }
+                    asm volatile("fence.proxy.async;" ::: "memory");             // other CTAs' stores before this thread's TMA reads
+                    stamp(p, j, TR_P_BARRIER);
+                    for (; ahead > 0; --ahead) {
+                        tma_load_2d(tiles_u32 + slot * SLOT_BYTES, map_a, full0 + 8 * slot, ca.kb * BK, ca.m0);
+                        if (++slot == (uint32_t)SLOTS) { slot = 0; phase ^= 1u; }
+                        advance(ca);
                     }
                 }
+                while (cb.t < n_tiles) {
+                    if (!mbar_wait(empty0 + 8 * slot, phase ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t sa = tiles_u32 + slot * SLOT_BYTES;
+                    mbar_arrive_expect_tx(full0 + 8 * slot, stage_tx);
+                    tma_load_2d(sa + A_BYTES, map_w, full0 + 8 * slot, cb.kb * BK, cb.n0);
+                    tma_load_2d(sa, map_a, full0 + 8 * slot, cb.kb * BK, cb.m0);
+                    if (++slot == (uint32_t)SLOTS) { slot = 0; phase ^= 1u; }
+                    advance(cb);
+                }
+                if (!ok) break;
+                stamp(p, j, TR_P_DONE);
             }
             if (!ok) { *abort_flag = 1; set_error(p.err, DEV_ERR_WAIT_TIMEOUT); }
         }
@@ -297,6 +320,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_chain_kernel(const __grid_c
                 const GemmDesc gd = gemm_desc(p, ph);
                 const int tiles_n = (gd.N + gd.BN - 1) / gd.BN, n_tiles = tiles_m * tiles_n * gd.splits, kbt = gd.K / BK;
                 const uint32_t idesc = tc::make_idesc(BM, gd.BN, true);
+                bool first = true;
                 for (int t = blockIdx.x; t < n_tiles && ok; t += n_cta) {
                     if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                     tc::tc_fence_after();
@@ -305,6 +329,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_chain_kernel(const __grid_c
                     const int k_blocks = (sp + 1) * kbt / gd.splits - sp * kbt / gd.splits;
                     for (int kb = 0; kb < k_blocks; ++kb) {
                         if (!mbar_wait(full0 + 8 * slot, phase, abort_flag)) { ok = false; break; }
+                        if (first) { stamp(p, j, TR_M_FIRST_FULL); first = false; }
                         tc::tc_fence_after();
                         const uint32_t sa = tiles_u32 + slot * SLOT_BYTES, sb = sa + A_BYTES;
                         const uint64_t da = tc::make_smem_desc(sa), db = tc::make_smem_desc(sb);
@@ -312,12 +337,13 @@ __global__ void __launch_bounds__(THREADS, 1) decode_chain_kernel(const __grid_c
                         for (int kk = 0; kk < BK / tc::UMMA_K; ++kk)
                             tc::umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
                         tc::umma_commit(empty0 + 8 * slot);
-                        if (++slot == SLOTS) { slot = 0; phase ^= 1u; }
+                        if (++slot == (uint32_t)SLOTS) { slot = 0; phase ^= 1u; }
                     }
                     if (!ok) break;
                     tc::umma_commit(tfull0 + 8 * acc);
                     if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
                 }
+                stamp(p, j, TR_M_DONE);
             }
             if (!ok) { *abort_flag = 1; set_error(p.err, DEV_ERR_WAIT_TIMEOUT); }
         }
@@ -333,6 +359,8 @@ __global__ void __launch_bounds__(THREADS, 1) decode_chain_kernel(const __grid_c
             if (ph == PH_END) break;
             const int l_here = p.seg < 0 ? 0 : p.seg;
             const bool last_layer = p.seg == p.n_layers - 1;
+            const bool tracer = lane == 0 && warp == (is_gemm(ph) ? 4 : WORKER_WARP0);
+            if (tracer) stamp(p, j, TR_W_BEGIN);
             if (is_gemm(ph)) {
                 if (warp >= 4) {
                     const GemmDesc gd = gemm_desc(p, ph);
@@ -350,6 +378,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_chain_kernel(const __grid_c
                     for (int t = blockIdx.x; t < n_tiles && ok; t += n_cta) {
                         const int m0 = (t % tiles_m) * BM, sp = (t / tiles_m) % gd.splits, n0 = (t / (tiles_m * gd.splits)) * gd.BN;
                         if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
+                        if (tracer && t == (int)blockIdx.x) stamp(p, j, TR_E_FIRST_FULL);
                         tc::tc_fence_after();
                         const int row = m0 + quarter * 32 + lane;
 #pragma unroll 1
@@ -379,6 +408,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_chain_kernel(const __grid_c
                     good = __shfl_sync(0xffffffffu, good, 0);
                     if (!good) { ok = false; break; }
                 }
+                if (tracer) stamp(p, j, TR_W_WAITED);
                 if (ph == PH_EMBED || ph == PH_NORM_MLP || ph == PH_NORM_NEXT) {
                     Partials pend{nullptr, 0, 0, 0};
                     const float* gain;
@@ -390,13 +420,38 @@ __global__ void __launch_bounds__(THREADS, 1) decode_chain_kernel(const __grid_c
                         gain = last_layer ? p.glob->final_norm : p.layers[l_here + 1].attn_norm;
                         if (p.splits[GK_DOWN] > 1) pend = Partials{p.res_part, p.splits[GK_DOWN], (size_t)M * p.d_model, p.d_model};
                     }
-                    for (int r = gw; r < m_live; r += n_gw) {
-                        float* h_row = p.h + (size_t)r * p.d_model;
-                        if (ph == PH_EMBED)
-                            embed_row_warp<__nv_bfloat16>(lane, p.d_model,
-                                                          reinterpret_cast<const __nv_bfloat16*>(p.embed) + (size_t)p.g.token[r] * p.d_model, h_row);
-                        norm_row_warp<__nv_bfloat16>(lane, p.d_model, h_row, pend, (size_t)r * p.d_model, gain, p.eps,
-                                                     p.a + (size_t)r * p.d_model, nullptr, 1);
+                    if (m_live <= n_cta && norm_row_fits_cta(p.d_model)) {
+                        // few rows: one row per CTA, its segments spread over the worker warps (one memory round trip per row)
+                        const int r = blockIdx.x, w = warp - WORKER_WARP0;
+                        if (r < m_live) {
+                            float* h_row = p.h + (size_t)r * p.d_model;
+                            if (ph == PH_EMBED) {
+                                const __nv_bfloat16* e_row = reinterpret_cast<const __nv_bfloat16*>(p.embed) + (size_t)p.g.token[r] * p.d_model;
+#pragma unroll
+                                for (int kk = 0; kk < NORM_SEG_REG4; ++kk) {
+                                    const int i = lane + 32 * (w + NORM_SEGS * kk);
+                                    if (i < (p.d_model >> 2)) {
+                                        float v[4];
+                                        VecLoad<__nv_bfloat16, 4>::load(e_row + 4 * i, v);
+                                        reinterpret_cast<float4*>(h_row)[i] = make_float4(v[0], v[1], v[2], v[3]);
+                                    }
+                                }
+                            }
+                            if (!norm_row_cta<__nv_bfloat16>(w, lane, p.d_model, h_row, pend, (size_t)r * p.d_model, gain, p.eps,
+                                                             p.a + (size_t)r * p.d_model, 1, s_norm_red + j * 8, s_norm_cnt + j)) {
+                                ok = false;
+                                break;
+                            }
+                        }
+                    } else {
+                        for (int r = gw; r < m_live; r += n_gw) {
+                            float* h_row = p.h + (size_t)r * p.d_model;
+                            if (ph == PH_EMBED)
+                                embed_row_warp<__nv_bfloat16>(lane, p.d_model,
+                                                              reinterpret_cast<const __nv_bfloat16*>(p.embed) + (size_t)p.g.token[r] * p.d_model, h_row);
+                            norm_row_warp<__nv_bfloat16>(lane, p.d_model, h_row, pend, (size_t)r * p.d_model, gain, p.eps,
+                                                         p.a + (size_t)r * p.d_model, nullptr, 1);
+                        }
                     }
                 } else if (ph == PH_POST) {
                     const int layer = p.seg + 1;
@@ -416,17 +471,24 @@ __global__ void __launch_bounds__(THREADS, 1) decode_chain_kernel(const __grid_c
                             rows[b] = it / n_heads;
                             heads[b] = it - rows[b] * n_heads;
                         }
-                        qkv_post_items_warp<__nv_bfloat16, 4>(lane, A, rows, heads, nb);
+                        // straight-line code per batch size: the loads of all items are in flight together
+                        if (nb == 4) qkv_post_items_warp<__nv_bfloat16, 4>(lane, A, rows, heads, 4);
+                        else if (nb == 3) qkv_post_items_warp<__nv_bfloat16, 3>(lane, A, rows, heads, 3);
+                        else if (nb == 2) qkv_post_items_warp<__nv_bfloat16, 2>(lane, A, rows, heads, 2);
+                        else qkv_post_items_warp<__nv_bfloat16, 1>(lane, A, rows, heads, 1);
                     }
                 } else if (ph == PH_MERGE) {
                     const int items = m_live * p.Hq;
+                    const am::SuffixPlan sp = am::suffix_plan(*p.g.max_slen, p.sd->n_rows * p.part.n_kv_heads, p.part.n_suffix_warps);
+                    const int n_load = p.part.n_parts + sp.cpi;
                     for (int it = gw; it < items; it += n_gw) {
-                        if (p.hd == 128) am::merge_item_warp<128>(lane, it, p.sd, p.Hq, p.g, p.part, p.attn, nullptr);
-                        else am::merge_item_warp<64>(lane, it, p.sd, p.Hq, p.g, p.part, p.attn, nullptr);
+                        if (p.hd == 128) am::merge_item_warp<128>(lane, it, p.Hq, p.g, p.part, sp.ct, n_load, p.attn, nullptr);
+                        else am::merge_item_warp<64>(lane, it, p.Hq, p.g, p.part, sp.ct, n_load, p.attn, nullptr);
                     }
                 }
             }
             // this warp's part of phase j is done: the CTA's last worker warp signals the grid barrier
+            if (tracer) stamp(p, j, TR_W_DONE);
             __threadfence();
             __syncwarp();
             if (lane == 0) {
@@ -442,6 +504,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_chain_kernel(const __grid_c
 
     tc::tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) stamp(p, 0, TR_KERNEL_END);
     if (*abort_flag) {
         // give copies that may still be in flight time to land before the shared memory is released
         for (int i = 0; i < 2000; ++i) __nanosleep(1000);

@@ -146,50 +146,62 @@ __device__ __forceinline__ void store_norm_out(T* __restrict__ a_row, T* __restr
     if (a_lo_row != nullptr) store4<T>(a_lo_row + 4 * i4, bf16_remainder(y));
 }
 
-// Residual update followed by the norm, one warp per row:
+// Residual update followed by the norm:
 //   h_row[:] += pending K-slice sums (pend_row = their row offset, in slice order);  a_row[:] = RMSNorm(h_row; gain).
-// d is a multiple of 8.  Rows of up to NORM_REG4 * 128 elements stay in registers between the sum of squares and
-// the scaling (one pass over memory, every load of the row and of its slices requested before the first use);
-// longer rows are read twice.
-constexpr int NORM_REG4 = 12;
+// d is a multiple of 8.  The row is cut into NORM_SEGS interleaved segments (the 128-element block b belongs to segment
+// b mod NORM_SEGS); a segment's sum of squares is the warp sum of its lanes' partial sums (blocks in increasing order) and
+// the row's sum adds the segments in order.  That fixes the arithmetic whether one warp walks all segments
+// (norm_row_warp) or NORM_SEGS warps of a CTA take one segment each (the persistent decode kernel at small batches).
+constexpr int NORM_SEGS = 6;
+constexpr int NORM_REG4 = 12;            // blocks of a row one warp keeps in registers (d <= 1536)
+
+// One 128-element block of the row: loads value, gain and every pending slice (straight-line, all requested before the
+// first add waits), returns the updated value.
+__device__ __forceinline__ float4 norm_block_load(const float4* __restrict__ x, int i, const Partials& pend, size_t pend_row) {
+    float4 v = x[i];
+    float4 q[PARTIALS_MAX];
+#pragma unroll
+    for (int s = 0; s < PARTIALS_MAX; ++s)
+        q[s] = s < pend.n ? *reinterpret_cast<const float4*>(pend.p + (size_t)s * pend.stride + pend_row + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int s = 0; s < PARTIALS_MAX; ++s)          // the adds stay in slice order
+        if (s < pend.n) { v.x += q[s].x; v.y += q[s].y; v.z += q[s].z; v.w += q[s].w; }
+    return v;
+}
+// Explicitly rounded operations: the compiler must not contract them differently in the two forms of the row norm.
+__device__ __forceinline__ float sq4(float4 v) {
+    return __fmaf_rn(v.w, v.w, __fmaf_rn(v.z, v.z, __fmaf_rn(v.y, v.y, __fmul_rn(v.x, v.x))));
+}
+
 template <typename T>
 __device__ __forceinline__ void norm_row_warp(int lane, int d, float* __restrict__ h_row, Partials pend, size_t pend_row,
                                               const float* __restrict__ gain, float eps, T* __restrict__ a_row,
                                               T* __restrict__ a_lo_row, int half_out) {
     const int n4 = d >> 2;
     float4* x = reinterpret_cast<float4*>(h_row);
-    float ss = 0.f;
+    float seg[NORM_SEGS];
+#pragma unroll
+    for (int g = 0; g < NORM_SEGS; ++g) seg[g] = 0.f;
     if (n4 <= NORM_REG4 * 32) {
         float4 v[NORM_REG4], gg[NORM_REG4];
 #pragma unroll
         for (int k = 0; k < NORM_REG4; ++k) {
             const int i = lane + 32 * k;
             if (i < n4) {
-                v[k] = x[i];
                 gg[k] = *reinterpret_cast<const float4*>(gain + 4 * i);
+                v[k] = norm_block_load(x, i, pend, pend_row);
+                seg[k % NORM_SEGS] = __fadd_rn(seg[k % NORM_SEGS], sq4(v[k]));
             }
         }
         if (pend.n > 0) {
 #pragma unroll
-            for (int k = 0; k < NORM_REG4; ++k) {
-                const int i = lane + 32 * k;
-                if (i < n4) {
-                    float4 p[PARTIALS_MAX];
-#pragma unroll
-                    for (int s = 0; s < PARTIALS_MAX; ++s)
-                        if (s < pend.n) p[s] = *reinterpret_cast<const float4*>(pend.p + (size_t)s * pend.stride + pend_row + 4 * i);
-#pragma unroll
-                    for (int s = 0; s < PARTIALS_MAX; ++s)          // the adds stay in slice order
-                        if (s < pend.n) { v[k].x += p[s].x; v[k].y += p[s].y; v[k].z += p[s].z; v[k].w += p[s].w; }
-                    x[i] = v[k];
-                }
-            }
+            for (int k = 0; k < NORM_REG4; ++k)
+                if (lane + 32 * k < n4) x[lane + 32 * k] = v[k];
         }
+        float ss = 0.f;
 #pragma unroll
-        for (int k = 0; k < NORM_REG4; ++k)
-            if (lane + 32 * k < n4) ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
-        ss = warp_sum(ss);
-        const float rstd = rsqrtf(ss / (float)d + eps);
+        for (int g = 0; g < NORM_SEGS; ++g) ss = __fadd_rn(ss, warp_sum(seg[g]));
+        const float rstd = rsqrtf(__fadd_rn(__fdiv_rn(ss, (float)d), eps));
 #pragma unroll
         for (int k = 0; k < NORM_REG4; ++k) {
             const int i = lane + 32 * k;
@@ -200,23 +212,84 @@ __device__ __forceinline__ void norm_row_warp(int lane, int d, float* __restrict
         }
         return;
     }
-    for (int i = lane; i < n4; i += 32) {
-        float4 v = x[i];
-        if (pend.n > 0) {
-            for (int s = 0; s < pend.n; ++s) {
-                const float4 q = *reinterpret_cast<const float4*>(pend.p + (size_t)s * pend.stride + pend_row + 4 * i);
-                v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
+    const int nk = (n4 + 31) >> 5;
+#pragma unroll
+    for (int g = 0; g < NORM_SEGS; ++g) {
+        for (int k = g; k < nk; k += NORM_SEGS) {
+            const int i = lane + 32 * k;
+            if (i < n4) {
+                const float4 v = norm_block_load(x, i, pend, pend_row);
+                if (pend.n > 0) x[i] = v;
+                seg[g] = __fadd_rn(seg[g], sq4(v));
             }
-            x[i] = v;
         }
-        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
     }
-    ss = warp_sum(ss);
-    const float rstd = rsqrtf(ss / (float)d + eps);
+    float ss = 0.f;
+#pragma unroll
+    for (int g = 0; g < NORM_SEGS; ++g) ss = __fadd_rn(ss, warp_sum(seg[g]));
+    const float rstd = rsqrtf(__fadd_rn(__fdiv_rn(ss, (float)d), eps));
     for (int i = lane; i < n4; i += 32) {
         const float4 v = x[i], gg = *reinterpret_cast<const float4*>(gain + 4 * i);     // this lane's own writes
         store_norm_out<T>(a_row, a_lo_row, i, make_float4(v.x * rstd * gg.x, v.y * rstd * gg.y, v.z * rstd * gg.z, v.w * rstd * gg.w), half_out);
     }
+}
+
+// The same row handled by NORM_SEGS warps of one CTA, warp w taking segment w.  The segment sums are exchanged through
+// shared memory: red[NORM_SEGS] floats and one counter, both used once (zero before); the wait on the counter is
+// bounded and returns false when it ran out.  Rows whose segments do not fit NORM_SEG_REG4 blocks per warp are not
+// handled here (the caller falls back to one warp per row).
+constexpr int NORM_SEG_REG4 = 2;
+__device__ __forceinline__ bool norm_row_fits_cta(int d) { return ((d >> 2) + 31) / 32 <= NORM_SEGS * NORM_SEG_REG4; }
+template <typename T>
+__device__ __forceinline__ bool norm_row_cta(int w, int lane, int d, float* __restrict__ h_row, Partials pend, size_t pend_row,
+                                             const float* __restrict__ gain, float eps, T* __restrict__ a_row, int half_out,
+                                             volatile float* red, int* counter) {
+    const int n4 = d >> 2;
+    float4* x = reinterpret_cast<float4*>(h_row);
+    float4 v[NORM_SEG_REG4], gg[NORM_SEG_REG4];
+    float part = 0.f;
+#pragma unroll
+    for (int kk = 0; kk < NORM_SEG_REG4; ++kk) {
+        const int i = lane + 32 * (w + NORM_SEGS * kk);
+        if (i < n4) {
+            gg[kk] = *reinterpret_cast<const float4*>(gain + 4 * i);
+            v[kk] = norm_block_load(x, i, pend, pend_row);
+            part = __fadd_rn(part, sq4(v[kk]));
+        }
+    }
+    if (pend.n > 0) {
+#pragma unroll
+        for (int kk = 0; kk < NORM_SEG_REG4; ++kk) {
+            const int i = lane + 32 * (w + NORM_SEGS * kk);
+            if (i < n4) x[i] = v[kk];
+        }
+    }
+    part = warp_sum(part);
+    if (lane == 0) {
+        red[w] = part;
+        __threadfence_block();
+        atomicAdd(counter, 1);
+    }
+    bool ok = false;
+    for (uint32_t it = 0; it < (1u << 22); ++it) {
+        if (*reinterpret_cast<volatile int*>(counter) >= NORM_SEGS) { ok = true; break; }
+        __nanosleep(20);
+    }
+    __threadfence_block();
+    if (!ok) return false;
+    float ss = 0.f;
+#pragma unroll
+    for (int g = 0; g < NORM_SEGS; ++g) ss = __fadd_rn(ss, red[g]);
+    const float rstd = rsqrtf(__fadd_rn(__fdiv_rn(ss, (float)d), eps));
+#pragma unroll
+    for (int kk = 0; kk < NORM_SEG_REG4; ++kk) {
+        const int i = lane + 32 * (w + NORM_SEGS * kk);
+        if (i < n4)
+            store_norm_out<T>(a_row, static_cast<T*>(nullptr), i,
+                              make_float4(v[kk].x * rstd * gg[kk].x, v[kk].y * rstd * gg[kk].y, v[kk].z * rstd * gg[kk].z, v[kk].w * rstd * gg[kk].w),
+                              half_out);
+    }
+    return true;
 }
 
 // h_row[:] = E[token, :] as float (the residual stream), one warp per row; d is a multiple of 8.
@@ -280,7 +353,8 @@ struct QkvPostArgs {
 // head_dim 128, (i + 32, i + 32 + hd/2).  The bias is added here.
 // q heads: optional RMSNorm over head_dim, RoPE, stored to q_out as T.
 // k heads: optional RMSNorm, RoPE, stored to the row's KV slot.  v heads: stored to the row's KV slot.
-// NB items are processed together so that their loads are all in flight before the first one is used.
+// NB items are processed together so that their loads are all in flight before the first one is used (callers pass
+// n_items = NB: the code is then straight-line).
 template <typename T, int NB>
 __device__ __forceinline__ void qkv_post_items_warp(int lane, const QkvPostArgs<T>& A, const int* rows, const int* heads, int n_items) {
     const int half = A.hd >> 1, npair = half > 32 ? 2 : 1;

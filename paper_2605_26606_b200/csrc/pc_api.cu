@@ -112,6 +112,7 @@ struct pc_ctx {
 
     int decode_mode = 0;                     // 1: persistent chain kernel between attention calls (half-operand bf16 models); 0: one kernel per operation
     bool chain_ready = false;                // tables uploaded by pc_set_workspace
+    long long* chain_trace = nullptr;        // pc_set_chain_trace
 
     std::vector<GraphEntry> graphs;
     cudaStream_t capture_stream = nullptr;      // decode steps are captured here (the caller's stream may be the default one)
@@ -313,9 +314,11 @@ cudaError_t configure_kernels() {
     return e;
 }
 
+// part_out != nullptr: the records are left unmerged and described there (the caller merges them).
 template <int HD>
 int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, int layer, const AttnPlan& plan, pc::KvArena prompt_arena,
-                   pc::KvArena suffix_arena, const __nv_bfloat16* q, __nv_bfloat16* attn, bool profile) {
+                   pc::KvArena suffix_arena, const __nv_bfloat16* q, __nv_bfloat16* attn, bool profile,
+                   pc::am::PrefixPartial* part_out = nullptr) {
     using namespace pc;
     const pc_model_desc& d = c->d;
     // half_gemm: the attention output is written once, as IEEE half; else as bf16 plus its bf16 rounding remainder
@@ -350,6 +353,11 @@ int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, in
     am::attn_suffix_kernel<HD><<<sgrid, am::S_WARPS * 32, am::suffix_smem_bytes<HD>(), st>>>(
         c->map_suffix_kv, sd, suffix_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, g, scale_log2, part, c->err);
     if (profile) cudaEventRecord(c->prof_stop, st);
+    if (part_out != nullptr) {
+        *part_out = part;
+        count_launches(2);
+        return PC_OK;
+    }
     am::attn_merge_kernel<HD><<<(M * d.n_q_heads + 7) / 8, 256, 0, st>>>(sd, d.n_q_heads, g, part, attn, attn_lo);
     count_launches(3);
     return PC_OK;
@@ -557,6 +565,19 @@ int pc_set_decode_mode(pc_ctx* ctx, int mode) {
     if (mode != ctx->decode_mode) ctx->drop_graphs();          // captured steps carry the old choice
     ctx->decode_mode = mode;
     return PC_OK;
+}
+
+int pc_set_chain_trace(pc_ctx* ctx, int64_t* trace, size_t n_words) {
+    if (ctx == nullptr) return PC_ERR_INVALID_ARG;
+    if (trace != nullptr && n_words < pc_chain_trace_words(ctx)) return PC_ERR_CAPACITY;
+    ctx->chain_trace = reinterpret_cast<long long*>(trace);
+    ctx->drop_graphs();
+    return PC_OK;
+}
+
+size_t pc_chain_trace_words(const pc_ctx* ctx) {
+    if (ctx == nullptr) return 0;
+    return (size_t)(ctx->d.n_layers + 1) * pc::chain::MAX_PHASES * pc::chain::TRACE_CTAS * pc::chain::TRACE_EVENTS;
 }
 
 int pc_set_logprob_buffer(pc_ctx* ctx, float* logprobs) {
@@ -806,22 +827,27 @@ int check_decode_args(const pc_ctx* ctx, const DecodeArgs& a) {
 
 // One segment of the persistent decode kernel (decode_chain.cuh) over the rows described by *sd.
 int launch_chain(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, int seg, pc::KvArena prompt_arena, pc::KvArena suffix_arena,
-                 const pc::am::PrefixPartial& part, float* logits) {
+                 const pc::am::PrefixPartial* part, float* logits) {
     using namespace pc;
     const pc_model_desc& d = c->d;
     char* w = c->ws;
     chain::ChainParams p;
     std::memset(&p, 0, sizeof(p));
-    p.sd = sd; p.M = M; p.seg = seg; p.with_merge = 0;
+    p.sd = sd; p.M = M; p.seg = seg; p.with_merge = part != nullptr ? 1 : 0;
     p.n_layers = d.n_layers; p.d_model = d.d_model; p.n_qkv = c->n_qkv(); p.q_dim = c->q_dim(); p.d_ff = d.d_ff; p.vocab = d.vocab;
     p.Hq = d.n_q_heads; p.Hkv = d.n_kv_heads; p.hd = d.head_dim; p.eps = d.rms_eps;
     const WMap* maps[5] = {&c->m_wqkv[0], &c->m_wo[0], &c->m_wgu[0], &c->m_wdown[0], &c->m_lm};
     const bool may_split[5] = {true, true, false, true, false};
+    int bn_max = 64;
     for (int k = 0; k < 5; ++k) {
         const GemmPlan gp = plan_gemm(c, (GemmKind)k, *maps[k], M, may_split[k]);
         p.bn[k] = gp.wide ? 256 : 64;
         p.splits[k] = gp.splits;
+        const bool used = k == GEMM_LM_HEAD ? seg == d.n_layers - 1 : (k == GEMM_QKV ? seg != d.n_layers - 1 : seg >= 0);
+        if (used) bn_max = std::max(bn_max, p.bn[k]);
     }
+    p.slot_bytes = chain::A_BYTES + bn_max * pc::tc::BK * 2;
+    p.slots = std::min(chain::MAX_SLOTS, chain::RING_BYTES / p.slot_bytes);
     auto pick = [](const WMap& m, int bn) -> const CUtensorMap& { return bn == 256 ? m.wide : (bn == 128 ? m.mid : m.narrow); };
     const int l_here = seg < 0 ? 0 : seg;
     p.maps[chain::MAP_A] = c->map_a; p.maps[chain::MAP_ATTN] = c->map_attn; p.maps[chain::MAP_ACT] = c->map_act;
@@ -843,9 +869,10 @@ int launch_chain(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, int 
     p.rope = reinterpret_cast<const float2*>(w + c->cv.rope);
     p.g = geom(c);
     p.prompt_arena = prompt_arena; p.suffix_arena = suffix_arena;
-    p.part = part;
+    if (part != nullptr) p.part = *part;
     p.bar = reinterpret_cast<int32_t*>(w + c->cv.chain_bar);
     p.err = c->err;
+    p.trace = c->chain_trace;
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)c->num_sms); cfg.blockDim = dim3(chain::THREADS); cfg.dynamicSmemBytes = chain::SMEM_BYTES; cfg.stream = st;
@@ -875,15 +902,15 @@ int run_decode_chained(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd
     rope_table_kernel<<<(M * half + 255) / 256, 256, 0, st>>>(sd, half, (double)d.rope_theta, g.pos, reinterpret_cast<float2*>(w + c->cv.rope));
     count_launches(1);
     PC_CUDA_CHECK_LAUNCH("rope table");
-    const am::PrefixPartial none{nullptr, nullptr, nullptr, 0, 0, 0, 0};
-    if (int rc = launch_chain(c, st, M, sd, -1, prompt_arena, suffix_arena, none, logits)) return rc;
+    if (int rc = launch_chain(c, st, M, sd, -1, prompt_arena, suffix_arena, nullptr, logits)) return rc;
     const __nv_bfloat16* q = reinterpret_cast<const __nv_bfloat16*>(w + c->cv.q);
     __nv_bfloat16* attn = reinterpret_cast<__nv_bfloat16*>(w + c->cv.attn);
     for (int l = 0; l < d.n_layers; ++l) {
-        int rc = d.head_dim == 128 ? attention_bf16<128>(c, st, sd, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer)
-                                   : attention_bf16<64>(c, st, sd, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer);
+        am::PrefixPartial part;
+        int rc = d.head_dim == 128 ? attention_bf16<128>(c, st, sd, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer, &part)
+                                   : attention_bf16<64>(c, st, sd, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer, &part);
         if (rc) return rc;
-        if ((rc = launch_chain(c, st, M, sd, l, prompt_arena, suffix_arena, none, logits))) return rc;
+        if ((rc = launch_chain(c, st, M, sd, l, prompt_arena, suffix_arena, &part, logits))) return rc;
     }
     PC_CUDA_CHECK_LAUNCH("chained decode step");
     return PC_OK;
