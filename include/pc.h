@@ -16,7 +16,11 @@
  *    (bad arguments, shapes, alignment, capacity) are returned before anything is
  *    launched.  Nothing here synchronises the stream: work is asynchronous.
  *  - The caller owns all device memory: weights, KV arenas, workspace, inputs,
- *    outputs.  The library never allocates or frees device memory.
+ *    outputs.  The library calls no device allocator.  Two entry points use driver
+ *    resources of their own, stated there: pc_set_workspace copies small tables into
+ *    the workspace with a synchronous cudaMemcpy, and pc_decode_run creates one CUDA
+ *    stream per context and instantiates CUDA graphs (which the driver backs with
+ *    memory of its own); both are released by pc_destroy.
  *  - "device" / "host" in a comment says where a pointer must point.
  *  - Matrices are row-major [out_features, in_features] in the model's storage type
  *    (dtype): float (PC_DTYPE_F32) or bfloat16 (PC_DTYPE_BF16).  Norm gains and
@@ -28,9 +32,14 @@
  *    2 bytes per element); a "slot" holds one token position.  A prompt or a
  *    rollout owns a contiguous range of slots given by its first slot (int64).
  *  - Index arrays are int32, slot numbers and token-buffer indices int64.
- *  - Device-side anomalies (an index outside its arena, a wait that ran out) set
- *    *dev_error_flag (see pc_set_workspace) to a non-zero code and skip the access;
- *    no kernel traps.
+ *  - Device-side anomalies set *dev_error_flag (see pc_set_workspace) to a non-zero
+ *    code and skip the access; no kernel traps.  What is checked: KV slot ranges
+ *    against their arenas, token ids against the vocabulary, every bounded wait, and
+ *    -- once the caller has stated the sizes with pc_set_index_bounds -- row_prompt
+ *    against the per-prompt arrays and row_tok_index against the token buffer (a row
+ *    that fails is switched off for the step).  Other index arrays (row_kv_start,
+ *    group_row_start, logits_row, out_index of pc_sample) are the caller's
+ *    responsibility.
  */
 #ifndef PC_H_
 #define PC_H_
@@ -138,8 +147,11 @@ PC_API const char* pc_status_string(int status);
 /* Text of the last CUDA error seen by this thread inside the library (host pointer, static storage). */
 PC_API const char* pc_last_cuda_error(void);
 
-/* Number of kernels this library has launched since it was loaded (host counter, all contexts). */
+/* Number of kernels this library has launched since it was loaded (host counter, all contexts and
+ * host threads; updated atomically). */
 PC_API uint64_t pc_launch_count(void);
+/* Number of decode steps this context has captured and instantiated as CUDA graphs so far (see pc_decode_run). */
+PC_API uint64_t pc_capture_count(const pc_ctx* ctx);
 
 /* Builds a context: copies the description and the pointer tables (host memory only)
  * and, for bf16 models, encodes the TMA descriptors of the weight matrices.  Needs a
@@ -165,6 +177,11 @@ PC_API int pc_set_workspace(pc_ctx* ctx, void* dev_ws, size_t bytes, int max_row
  * bound; gate/up and the LM head never split.  Results stay deterministic for a fixed plan.  Drops captured decode
  * steps.  The paper has no counterpart. */
 PC_API int pc_set_gemm_plan(pc_ctx* ctx, const char* spec);
+
+/* Sizes of the caller's per-prompt arrays (prompt_len, prompt_kv_start, prompt keys) and of the token buffer, so that
+ * the decode steps can check row_prompt and row_tok_index against them (see "Device-side anomalies" above).  0 = not
+ * stated, not checked (the default). */
+PC_API int pc_set_index_bounds(pc_ctx* ctx, int n_prompts, int64_t n_tokens);
 
 /* How the decode steps of a bf16 model with half_gemm = 1 are issued.  mode 1: everything between two
  * attention calls of a step -- output projection, residual + RMSNorm, gate/up + SwiGLU, down projection, residual +
@@ -235,8 +252,12 @@ typedef struct pc_step_desc {
 /* n_steps consecutive decode steps (each exactly a pc_decode_step with sampling and no logits output) over a
  * schedule that already lives on the device: the row_* arrays and group_row_start hold every step's entries back to
  * back and step s uses the slices named by steps[s].  steps_host and steps_dev are the same n_steps descriptors in
- * host and in device memory.  The kernels of a step are captured once per batch-size class into a CUDA graph and
- * replayed, so the host issues one launch per step; the stream must not be capturing.  Steps with n_rows = 0 are
+ * host and in device memory.  The kernels of a step are captured once per shape class (rows rounded up to 128, groups
+ * to a power of two, largest group to a query-tile boundary; per pair of KV arenas) into a CUDA graph and replayed, so
+ * the host issues one launch per step; the caller's arrays and sampling parameters are read through a device-resident
+ * argument block, so a new schedule, token buffer or seed needs no new capture.  The first call creates a CUDA stream
+ * owned by the context (captures run there) and every capture instantiates a graph; pc_destroy, pc_set_workspace,
+ * pc_set_gemm_plan and pc_set_decode_mode release them.  The stream must not be capturing.  Steps with n_rows = 0 are
  * skipped.  All other arguments as in pc_decode_step. */
 PC_API int pc_decode_run(pc_ctx* ctx, void* stream, int n_steps, const pc_step_desc* steps_host, const pc_step_desc* steps_dev,
                          const int32_t* row_prompt, const int32_t* row_rollout, const int32_t* row_step,

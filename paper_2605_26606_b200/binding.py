@@ -22,7 +22,7 @@ PC_ERR_UNSUPPORTED, PC_ERR_CUDA, PC_ERR_NO_WORKSPACE = 5, 6, 7
 PC_DTYPE_F32, PC_DTYPE_BF16 = 0, 1
 PC_STATUS_COMMIT, PC_STATUS_BUFFERED, PC_STATUS_DEFER_HARD, PC_STATUS_SKIP_EASY = 0, 1, 2, 3
 
-EXPORTS = ["pc_status_string", "pc_last_cuda_error", "pc_launch_count", "pc_profile_attention", "pc_set_gemm_plan", "pc_set_decode_mode", "pc_set_chain_trace", "pc_chain_trace_words", "pc_create", "pc_destroy", "pc_workspace_bytes",
+EXPORTS = ["pc_status_string", "pc_last_cuda_error", "pc_launch_count", "pc_profile_attention", "pc_set_gemm_plan", "pc_set_decode_mode", "pc_set_chain_trace", "pc_chain_trace_words", "pc_capture_count", "pc_set_index_bounds", "pc_create", "pc_destroy", "pc_workspace_bytes",
            "pc_set_workspace", "pc_prefill_shared", "pc_decode_step", "pc_decode_run", "pc_sample", "pc_sample_static", "pc_token_logprob", "pc_set_logprob_buffer", "pc_set_prompt_keys", "pc_reward_last_token",
            "pc_group_stats", "pc_allocate", "pc_grpo_advantage"]
 
@@ -81,6 +81,9 @@ def _lib():
         lib.pc_profile_attention.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         lib.pc_set_gemm_plan.argtypes = [C.c_void_p, C.c_char_p]
         lib.pc_set_decode_mode.argtypes = [C.c_void_p, C.c_int]
+        lib.pc_capture_count.argtypes = [C.c_void_p]
+        lib.pc_capture_count.restype = C.c_uint64
+        lib.pc_set_index_bounds.argtypes = [C.c_void_p, C.c_int, C.c_int64]
         lib.pc_set_chain_trace.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
         lib.pc_chain_trace_words.argtypes = [C.c_void_p]
         lib.pc_chain_trace_words.restype = C.c_size_t
@@ -103,7 +106,7 @@ def _lib():
         lib.pc_allocate.argtypes = [p, i, p, p, C.POINTER(AllocParams), p, p, p, p, p]
         lib.pc_grpo_advantage.argtypes = [p, i, p, p, p, p, p]
         for name in EXPORTS[3:]:
-            if name not in ("pc_destroy", "pc_chain_trace_words"):
+            if name not in ("pc_destroy", "pc_chain_trace_words", "pc_capture_count"):
                 getattr(lib, name).restype = C.c_int
         _LIB = lib
     return _LIB
@@ -151,6 +154,14 @@ def pc_set_gemm_plan(ctx: "Context", spec: Optional[str]) -> None:
 
 def pc_set_decode_mode(ctx: "Context", mode: int) -> None:
     _check(_lib().pc_set_decode_mode(ctx.handle, mode), "pc_set_decode_mode")
+
+
+def pc_capture_count(ctx: "Context") -> int:
+    return int(_lib().pc_capture_count(ctx.handle))
+
+
+def pc_set_index_bounds(ctx: "Context", n_prompts: int, n_tokens: int) -> None:
+    _check(_lib().pc_set_index_bounds(ctx.handle, n_prompts, n_tokens), "pc_set_index_bounds")
 
 
 def pc_chain_trace_words(ctx: "Context") -> int:

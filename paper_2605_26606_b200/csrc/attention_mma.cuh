@@ -120,7 +120,7 @@ attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __
     constexpr int TILE_BYTES = G_TK * HD * 2;
     const int grp = blockIdx.z, kvh = blockIdx.y;
     if (grp >= sd->n_groups) return;
-    group_row_start += sd->group_off;
+    // group_row_start holds this pass's groups from entry 0 on (decode: the copy prep_decode_rows leaves in the workspace)
     const int row0 = group_row_start[grp], n_rows = group_row_start[grp + 1] - row0;
     const int n_rep = Hq / Hkv;
     const int n_parts = FINAL ? 1 : part.n_parts;

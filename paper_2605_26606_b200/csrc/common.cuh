@@ -27,6 +27,37 @@ struct StepDesc {
     int64_t group_off;        // offset of this step's group_row_start entries
 };
 
+// The caller's arrays of a decode call, kept in device memory (part of the workspace) and rewritten, in stream order, by
+// every pc_decode_step / pc_decode_run: captured decode steps read the pointers here, so a CUDA graph does not depend on
+// where a stage's schedule happens to live.
+struct DecodeArgsDev {
+    const StepDesc* steps;            // pc_decode_run: the schedule (the device counter indexes it)
+    const int32_t* row_prompt;
+    const int32_t* row_rollout;
+    const int32_t* row_step;
+    const int64_t* row_kv_start;
+    int32_t* tokens;
+    const int64_t* row_tok_index;
+    const int32_t* group_row_start;
+    const int32_t* prompt_len;
+    const int64_t* prompt_kv_start;
+    float* logprobs;                  // or nullptr
+    const int32_t* prompt_key;        // or nullptr
+    float temperature;
+    uint32_t k0, k1;                  // sampling seed
+    int32_t n_prompts;                // entries of prompt_len / prompt_kv_start / prompt_key (0: unknown, not checked)
+    int64_t n_tokens;                 // length of the token buffer (0: unknown, not checked)
+};
+
+// Per-row sampling keys and output positions of a decode step, compacted into the workspace by prep_decode_rows.
+struct RowKeys {
+    int32_t* key_prompt;     // [M] prompt id of the sampling key
+    int32_t* rollout;        // [M]
+    int32_t* step_key;       // [M] step counter of the key: suffix tokens cached + 1
+    int64_t* out_index;      // [M] where the drawn token goes in the token buffer
+    int32_t* group_start;    // [groups + 1] first row of every group of the step
+};
+
 __device__ __forceinline__ void set_error(int32_t* flag, int32_t code) {
     if (flag != nullptr) atomicCAS(flag, 0, code);
 }

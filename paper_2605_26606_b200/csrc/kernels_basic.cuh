@@ -31,33 +31,41 @@ __global__ void set_step_desc(StepDesc* sd, int n_rows, int n_groups, int max_gr
     sd->row_off = 0; sd->group_off = 0;
 }
 // First node of a captured decode step: takes the next descriptor of the caller's schedule.
-__global__ void load_step_desc(const StepDesc* __restrict__ steps, int32_t* counter, StepDesc* sd, int32_t* max_slen, int32_t* bar, int n_bar) {
+__global__ void load_step_desc(const DecodeArgsDev* __restrict__ da, int32_t* counter, StepDesc* sd, int32_t* max_slen, int32_t* bar, int n_bar) {
     for (int i = threadIdx.x; i < n_bar; i += blockDim.x) bar[i] = 0;
     if (threadIdx.x != 0) return;
     *max_slen = 0;
     const int i = *counter;
-    *sd = steps[i];
+    *sd = da->steps[i];
     *counter = i + 1;
 }
 
 // Decode: row r of prompt p with `step` suffix tokens cached attends prompt slots [start_p, start_p + Lp)
 // and suffix slots [kv_start_r, kv_start_r + step + 1); its own K/V goes to suffix slot kv_start_r + step.
-__global__ void prep_decode_rows(const StepDesc* __restrict__ sd, const int32_t* row_prompt, const int32_t* row_step,
-                                 const int64_t* row_kv_start, const int32_t* tokens, const int64_t* row_tok_index,
-                                 const int32_t* prompt_len, const int64_t* prompt_kv_start, int64_t prompt_slots,
-                                 int64_t suffix_slots, int vocab, RowGeom g, int32_t* err) {
+// Also compacts the row's sampling key, the position of its next token and the step's group boundaries into the
+// workspace.  A row whose indices do not fit their arrays is switched off (no KV access, token 0) and flagged.
+__global__ void prep_decode_rows(const StepDesc* __restrict__ sd, const DecodeArgsDev* __restrict__ da, int64_t prompt_slots,
+                                 int64_t suffix_slots, int vocab, RowGeom g, RowKeys keys, int32_t* err) {
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
-    if (r >= sd->n_rows) return;
+    const int n_rows = sd->n_rows;
+    if (r <= sd->n_groups) keys.group_start[r] = da->group_row_start[sd->group_off + r];
+    if (r >= n_rows) return;
     const int64_t ro = sd->row_off + r;
-    const int p = row_prompt[ro];
-    const int step = row_step[ro];
-    const int Lp = prompt_len[p];
-    const int64_t ps = prompt_kv_start[p];
-    const int64_t ss = row_kv_start[ro];
-    int tok = tokens[row_tok_index[ro]];
+    int p = da->row_prompt[ro];
+    const int step = da->row_step[ro];
+    const int64_t ti = da->row_tok_index[ro];
     bool ok = true;
+    if (p < 0 || (da->n_prompts > 0 && p >= da->n_prompts) || ti < 0 || (da->n_tokens > 0 && ti + 1 >= da->n_tokens)) {
+        set_error(err, DEV_ERR_GROUP_RANGE);
+        ok = false;
+        p = 0;
+    }
+    const int Lp = ok ? da->prompt_len[p] : 0;
+    const int64_t ps = ok ? da->prompt_kv_start[p] : 0;
+    const int64_t ss = da->row_kv_start[ro];
+    int tok = ok ? da->tokens[ti] : 0;
     if (tok < 0 || tok >= vocab) { set_error(err, DEV_ERR_TOKEN_RANGE); tok = 0; }
-    if (ps < 0 || Lp < 0 || ps + Lp > prompt_slots || ss < 0 || step < 0 || ss + step + 1 > suffix_slots) {
+    if (ok && (ps < 0 || Lp < 0 || ps + Lp > prompt_slots || ss < 0 || step < 0 || ss + step + 1 > suffix_slots)) {
         set_error(err, DEV_ERR_SLOT_RANGE);
         ok = false;
     }
@@ -69,6 +77,10 @@ __global__ void prep_decode_rows(const StepDesc* __restrict__ sd, const int32_t*
     g.p_len[r] = ok ? Lp : 0;
     g.s_start[r] = ss;
     g.s_len[r] = ok ? step + 1 : 0;
+    keys.key_prompt[r] = ok && da->prompt_key ? da->prompt_key[p] : p;
+    keys.rollout[r] = da->row_rollout[ro];
+    keys.step_key[r] = step + 1;
+    keys.out_index[r] = ok ? ti + 1 : -1;            // -1: nothing is stored for this row
     if (ok) atomicMax(g.max_slen, step + 1);
 }
 
@@ -457,7 +469,9 @@ __global__ void __launch_bounds__(ROW_WARPS * 32) qkv_post_kernel(const StepDesc
 __global__ void reward_last_token_kernel(int n, const int32_t* tokens, const int64_t* last_index,
                                          const int32_t* threshold, float* reward) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < n) reward[i] = tokens[last_index[i]] < threshold[i] ? 1.f : 0.f;
+    if (i >= n) return;
+    const int tok = tokens[last_index[i]];
+    reward[i] = tok >= 0 && tok < threshold[i] ? 1.f : 0.f;        // a cell that was never generated (-1) earns nothing
 }
 
 }  // namespace pc

@@ -54,14 +54,16 @@ constexpr int kMaxSplits = pc::PARTIALS_MAX;
 struct Carve {
     size_t h, a, qkv, q, attn, act, logits, rope, pos, wslot, warena, p_start, p_len, s_start, s_len, token, last_row,
         part_m, part_l, part_o, res_part, step_desc, step_counter, max_slen, sample_scratch, a_lo, attn_lo, chain_layers, chain_glob,
-        chain_bar, total;
+        chain_bar, dargs, key_prompt, key_rollout, key_step, out_index, group_start, total;
 };
 
-// A captured decode step, replayable for every step that fits the same upper bounds and reads the same arrays.
+// A captured decode step, replayable for every step that fits the same upper bounds on the same KV arenas.  The
+// caller's row arrays, token buffer and sampling parameters are not part of the key: the captured kernels read them
+// from the device-resident argument block (DecodeArgsDev) that every call rewrites.
 struct GraphKey {
-    int m_bound, groups_bound, group_rows_bound, pad;
-    const void* steps_dev;
-    unsigned char args[160];
+    int m_bound, groups_bound, group_rows_bound, sample, logprobs, decode_mode;
+    const void* prompt_kv; int64_t prompt_slots;
+    const void* suffix_kv; int64_t suffix_slots;
 };
 struct GraphEntry {
     GraphKey key;
@@ -113,6 +115,9 @@ struct pc_ctx {
     int decode_mode = 0;                     // 1: persistent chain kernel between attention calls (half-operand bf16 models); 0: one kernel per operation
     bool chain_ready = false;                // tables uploaded by pc_set_workspace
     long long* chain_trace = nullptr;        // pc_set_chain_trace
+    unsigned long long captures = 0;         // decode steps captured and instantiated so far (pc_capture_count)
+    int32_t n_prompts_hint = 0;              // pc_set_index_bounds: sizes of the caller's per-prompt arrays and token buffer (0: unknown)
+    int64_t n_tokens_hint = 0;
 
     std::vector<GraphEntry> graphs;
     cudaStream_t capture_stream = nullptr;      // decode steps are captured here (the caller's stream may be the default one)
@@ -168,6 +173,12 @@ Carve carve(const pc_ctx* c, int max_rows, int max_prefill) {
     v.s_len = take(M * 4);
     v.token = take(M * 4);
     v.last_row = take(M * 4);
+    v.dargs = take(sizeof(pc::DecodeArgsDev));
+    v.key_prompt = take(M * 4);
+    v.key_rollout = take(M * 4);
+    v.key_step = take(M * 4);
+    v.out_index = take(M * 8);
+    v.group_start = take((M + 1) * 4);
     // prefix part of the shared-prefix attention: (max, sum, unnormalised output) per (row, query head)
     const size_t R = (size_t)std::max(max_rows, 1);
     v.part_m = take(pc::am::MAX_RECORDS * R * d.n_q_heads * 4);
@@ -580,6 +591,15 @@ size_t pc_chain_trace_words(const pc_ctx* ctx) {
     return (size_t)(ctx->d.n_layers + 1) * pc::chain::MAX_PHASES * pc::chain::TRACE_CTAS * pc::chain::TRACE_EVENTS;
 }
 
+uint64_t pc_capture_count(const pc_ctx* ctx) { return ctx ? ctx->captures : 0; }
+
+int pc_set_index_bounds(pc_ctx* ctx, int n_prompts, int64_t n_tokens) {
+    if (ctx == nullptr || n_prompts < 0 || n_tokens < 0) return PC_ERR_INVALID_ARG;
+    ctx->n_prompts_hint = n_prompts;
+    ctx->n_tokens_hint = n_tokens;
+    return PC_OK;
+}
+
 int pc_set_logprob_buffer(pc_ctx* ctx, float* logprobs) {
     if (ctx == nullptr) return PC_ERR_INVALID_ARG;
     ctx->logprobs = logprobs;
@@ -592,7 +612,7 @@ int pc_token_logprob(void* stream, int n_rows, int vocab, const float* logits, c
     if (n_rows == 0) return PC_OK;
     if (logits == nullptr || tokens == nullptr || out_logprob == nullptr) return PC_ERR_INVALID_ARG;
     pc::token_logprob_kernel<<<n_rows, 256, 0, static_cast<cudaStream_t>(stream)>>>(nullptr, vocab, logits, logits_row, temperature, tokens,
-                                                                                   tok_index, 0, out_logprob, out_index, 0);
+                                                                                   tok_index, 0, out_logprob, out_index, 0, nullptr);
     count_launches(1);
     PC_CUDA_CHECK_LAUNCH("token_logprob");
     return PC_OK;
@@ -811,7 +831,41 @@ DecodeArgs make_decode_args(const int32_t* row_prompt, const int32_t* row_rollou
     a.prompt_key = nullptr;
     return a;
 }
-static_assert(sizeof(DecodeArgs) <= sizeof(GraphKey::args), "graph key too small for the decode arguments");
+
+pc::RowKeys row_keys(const pc_ctx* c) {
+    char* w = c->ws;
+    return pc::RowKeys{reinterpret_cast<int32_t*>(w + c->cv.key_prompt), reinterpret_cast<int32_t*>(w + c->cv.key_rollout),
+                       reinterpret_cast<int32_t*>(w + c->cv.key_step), reinterpret_cast<int64_t*>(w + c->cv.out_index),
+                       reinterpret_cast<int32_t*>(w + c->cv.group_start)};
+}
+
+// Upper bounds of a step's group geometry, rounded up to classes so that steps of similar shape share a captured graph
+// and a step-by-step call picks the same attention plan as a captured one: the number of groups to the next power of
+// two, the largest group to the most rows that need the same number of query tiles (neither beyond the row bound).
+void canonical_group_bounds(const pc_ctx* c, int n_groups, int max_group_rows, int row_bound, int* groups_bound, int* group_rows_bound) {
+    int gb = 1;
+    while (gb < n_groups) gb <<= 1;
+    *groups_bound = std::min(gb, std::max(row_bound, 1));
+    const int n_rep = c->d.n_q_heads / c->d.n_kv_heads;
+    const int q_tiles = (std::max(max_group_rows, 1) * n_rep + pc::am::G_QROWS - 1) / pc::am::G_QROWS;
+    *group_rows_bound = std::min(q_tiles * pc::am::G_QROWS / n_rep, std::max(row_bound, 1));
+}
+
+// Rewrites the device-resident argument block (stream-ordered: work already queued keeps the values it was issued with).
+int upload_decode_args(pc_ctx* ctx, cudaStream_t st, const DecodeArgs& a, const pc_step_desc* steps_dev) {
+    pc::DecodeArgsDev d;
+    std::memset(&d, 0, sizeof(d));
+    d.steps = reinterpret_cast<const pc::StepDesc*>(steps_dev);
+    d.row_prompt = a.row_prompt; d.row_rollout = a.row_rollout; d.row_step = a.row_step; d.row_kv_start = a.row_kv_start;
+    d.tokens = a.tokens; d.row_tok_index = a.row_tok_index; d.group_row_start = a.group_row_start; d.prompt_len = a.prompt_len;
+    d.prompt_kv_start = a.prompt_kv_start; d.logprobs = a.logprobs; d.prompt_key = a.prompt_key;
+    d.temperature = a.temperature;
+    d.k0 = (uint32_t)(a.seed & 0xffffffffu); d.k1 = (uint32_t)(a.seed >> 32);
+    d.n_prompts = ctx->n_prompts_hint; d.n_tokens = ctx->n_tokens_hint;
+    const cudaError_t e = cudaMemcpyAsync(ctx->ws + ctx->cv.dargs, &d, sizeof(d), cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(e, "decode argument block");
+    return PC_OK;
+}
 
 int check_decode_args(const pc_ctx* ctx, const DecodeArgs& a) {
     if (a.row_prompt == nullptr || a.row_rollout == nullptr || a.row_step == nullptr || a.row_kv_start == nullptr ||
@@ -921,15 +975,15 @@ int run_decode_chained(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd
 int decode_launches(pc_ctx* ctx, cudaStream_t st, int m_bound, int groups_bound, int group_rows_bound, const DecodeArgs& a,
                     float* logits_out) {
     const pc::RowGeom g = geom(ctx);
+    const pc::RowKeys keys = row_keys(ctx);
     const pc::StepDesc* sd = reinterpret_cast<const pc::StepDesc*>(ctx->ws + ctx->cv.step_desc);
-    pc::prep_decode_rows<<<(m_bound + 127) / 128, 128, 0, st>>>(sd, a.row_prompt, a.row_step, a.row_kv_start, a.tokens,
-                                                                a.row_tok_index, a.prompt_len, a.prompt_kv_start, a.prompt_slots,
-                                                                a.suffix_slots, ctx->d.vocab, g, ctx->err);
+    const pc::DecodeArgsDev* da = reinterpret_cast<const pc::DecodeArgsDev*>(ctx->ws + ctx->cv.dargs);
+    pc::prep_decode_rows<<<(m_bound + 128) / 128, 128, 0, st>>>(sd, da, a.prompt_slots, a.suffix_slots, ctx->d.vocab, g, keys, ctx->err);
     count_launches(1);
     PC_CUDA_CHECK_LAUNCH("prep_decode_rows");
     const pc::KvArena pa{const_cast<void*>(a.prompt_kv), a.prompt_slots}, sa{a.suffix_kv, a.suffix_slots};
     const bool f32 = ctx->d.dtype == PC_DTYPE_F32;
-    const AttnPlan plan{false, groups_bound, a.group_row_start, group_rows_bound};
+    const AttnPlan plan{false, groups_bound, keys.group_start, group_rows_bound};
     float* logits = logits_out ? logits_out : reinterpret_cast<float*>(ctx->ws + ctx->cv.logits);
     int rc;
     if (!f32 && ctx->decode_mode == 1 && ctx->chain_ready) {
@@ -942,23 +996,23 @@ int decode_launches(pc_ctx* ctx, cudaStream_t st, int m_bound, int groups_bound,
         if (rc) return rc;
     }
     if (a.sample) {
-        const uint32_t k0 = (uint32_t)(a.seed & 0xffffffffu), k1 = (uint32_t)(a.seed >> 32);
+        // keys, output positions, token buffer, temperature and seed come from the workspace copies / the argument block
         const int chunks = pc::sample_chunks(m_bound, ctx->num_sms);
         if (chunks == 1) {
-            pc::sample_kernel<<<m_bound, 256, 0, st>>>(sd, ctx->d.vocab, logits, nullptr, a.temperature, k0, k1, a.row_prompt,
-                                                       a.row_rollout, a.row_step, 1, a.tokens, a.row_tok_index, 1, nullptr, a.prompt_key);
+            pc::sample_kernel<<<m_bound, 256, 0, st>>>(sd, ctx->d.vocab, logits, nullptr, 1.f, 0u, 0u, keys.key_prompt, keys.rollout,
+                                                       keys.step_key, 0, nullptr, keys.out_index, 0, nullptr, nullptr, da);
             count_launches(1);
         } else {
             pc::Top2Rec* scratch = reinterpret_cast<pc::Top2Rec*>(ctx->ws + ctx->cv.sample_scratch);
-            pc::sample_partial_kernel<<<dim3(m_bound, chunks), 256, 0, st>>>(sd, ctx->d.vocab, chunks, logits, nullptr, a.temperature,
-                                                                             k0, k1, a.row_prompt, a.row_rollout, a.row_step, 1, scratch, a.prompt_key);
-            pc::sample_reduce_kernel<<<(m_bound + 127) / 128, 128, 0, st>>>(sd, m_bound, chunks, scratch, a.tokens, a.row_tok_index, 1,
-                                                                            nullptr);
+            pc::sample_partial_kernel<<<dim3(m_bound, chunks), 256, 0, st>>>(sd, ctx->d.vocab, chunks, logits, nullptr, 1.f, 0u, 0u,
+                                                                             keys.key_prompt, keys.rollout, keys.step_key, 0, scratch, nullptr, da);
+            pc::sample_reduce_kernel<<<(m_bound + 127) / 128, 128, 0, st>>>(sd, m_bound, chunks, scratch, nullptr, keys.out_index, 0,
+                                                                            nullptr, da);
             count_launches(2);
         }
         if (a.logprobs != nullptr) {
-            pc::token_logprob_kernel<<<m_bound, 256, 0, st>>>(sd, ctx->d.vocab, logits, nullptr, a.temperature, a.tokens, a.row_tok_index,
-                                                              1, a.logprobs, a.row_tok_index, 1);
+            pc::token_logprob_kernel<<<m_bound, 256, 0, st>>>(sd, ctx->d.vocab, logits, nullptr, 1.f, nullptr, keys.out_index, 0, nullptr,
+                                                              keys.out_index, 0, da);
             count_launches(1);
         }
         PC_CUDA_CHECK_LAUNCH("sample");
@@ -990,12 +1044,15 @@ int pc_decode_step(pc_ctx* ctx, void* stream, int n_rows, const int32_t* row_pro
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (ctx->d.dtype == PC_DTYPE_BF16)
         if (int rc = arena_maps(ctx, prompt_kv, prompt_slots, suffix_kv, suffix_slots)) return rc;
+    if (int rc = upload_decode_args(ctx, st, a, nullptr)) return rc;
     pc::set_step_desc<<<1, pc::STEP_DESC_THREADS, 0, st>>>(reinterpret_cast<pc::StepDesc*>(ctx->ws + ctx->cv.step_desc), n_rows, n_groups,
                                                            max_group_rows, reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.max_slen),
                                                            reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.chain_bar),
                                                            (int)chain_bar_words(ctx->d.n_layers));
     count_launches(1);
-    return decode_launches(ctx, st, n_rows, n_groups, max_group_rows, a, logits_out);
+    int groups_bound, group_rows_bound;
+    canonical_group_bounds(ctx, n_groups, max_group_rows, n_rows, &groups_bound, &group_rows_bound);
+    return decode_launches(ctx, st, n_rows, groups_bound, group_rows_bound, a, logits_out);
 }
 
 int pc_decode_run(pc_ctx* ctx, void* stream, int n_steps, const pc_step_desc* steps_host, const pc_step_desc* steps_dev,
@@ -1013,35 +1070,36 @@ int pc_decode_run(pc_ctx* ctx, void* stream, int n_steps, const pc_step_desc* st
     if (int rc = check_decode_args(ctx, a)) return rc;
     a.logprobs = ctx->logprobs;
     a.prompt_key = ctx->prompt_key;
-    int groups_bound = 0, group_rows_bound = 0;
     for (int s = 0; s < n_steps; ++s) {
         const pc_step_desc& d = steps_host[s];
         if (d.n_rows < 0 || d.n_rows > ctx->max_rows || d.n_groups < 0 || d.n_groups > d.n_rows || d.max_group_rows < 0 ||
             d.max_group_rows > d.n_rows || d.row_offset < 0 || d.group_offset < 0 || (d.n_rows > 0 && (d.n_groups == 0 || d.max_group_rows == 0)))
             return d.n_rows > ctx->max_rows ? PC_ERR_CAPACITY : PC_ERR_INVALID_ARG;
-        groups_bound = std::max(groups_bound, d.n_groups);
-        group_rows_bound = std::max(group_rows_bound, d.max_group_rows);
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (ctx->d.dtype == PC_DTYPE_BF16)
         if (int rc = arena_maps(ctx, prompt_kv, prompt_slots, suffix_kv, suffix_slots)) return rc;
     int32_t* counter = reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.step_counter);
     pc::StepDesc* sd = reinterpret_cast<pc::StepDesc*>(ctx->ws + ctx->cv.step_desc);
+    if (int rc = upload_decode_args(ctx, st, a, steps_dev)) return rc;
+    const pc::DecodeArgsDev* da = reinterpret_cast<const pc::DecodeArgsDev*>(ctx->ws + ctx->cv.dargs);
     cudaError_t e = cudaMemsetAsync(counter, 0, sizeof(int32_t), st);
     if (e != cudaSuccess) return cuda_fail(e, "reset step counter");
     for (int s = 0; s < n_steps; ++s) {
         if (steps_host[s].n_rows == 0) {          // keep the device counter in step with the host loop
-            pc::load_step_desc<<<1, pc::STEP_DESC_THREADS, 0, st>>>(reinterpret_cast<const pc::StepDesc*>(steps_dev), counter, sd,
-                                                                    reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.max_slen), nullptr, 0);
+            pc::load_step_desc<<<1, pc::STEP_DESC_THREADS, 0, st>>>(da, counter, sd, reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.max_slen),
+                                                                    nullptr, 0);
             count_launches(1);
             continue;
         }
         const int m_bound = std::min(ctx->max_rows, (steps_host[s].n_rows + 127) / 128 * 128);
-        GraphKey key{};
+        int groups_bound, group_rows_bound;
+        canonical_group_bounds(ctx, steps_host[s].n_groups, steps_host[s].max_group_rows, m_bound, &groups_bound, &group_rows_bound);
+        GraphKey key;
         std::memset(&key, 0, sizeof(key));
         key.m_bound = m_bound; key.groups_bound = groups_bound; key.group_rows_bound = group_rows_bound;
-        key.steps_dev = steps_dev;
-        std::memcpy(key.args, &a, sizeof(a));
+        key.sample = a.sample; key.logprobs = a.logprobs != nullptr; key.decode_mode = ctx->decode_mode;
+        key.prompt_kv = a.prompt_kv; key.prompt_slots = a.prompt_slots; key.suffix_kv = a.suffix_kv; key.suffix_slots = a.suffix_slots;
         cudaGraphExec_t exec = nullptr;
         for (auto& ent : ctx->graphs)
             if (std::memcmp(&ent.key, &key, sizeof(key)) == 0) { exec = ent.exec; break; }
@@ -1056,7 +1114,7 @@ int pc_decode_run(pc_ctx* ctx, void* stream, int n_steps, const pc_step_desc* st
             e = cudaStreamBeginCapture(cs, cudaStreamCaptureModeThreadLocal);
             if (e != cudaSuccess) return cuda_fail(e, "begin graph capture");
             g_capture_launches = 0;                // launches are recorded into the graph, not run
-            pc::load_step_desc<<<1, pc::STEP_DESC_THREADS, 0, cs>>>(reinterpret_cast<const pc::StepDesc*>(steps_dev), counter, sd,
+            pc::load_step_desc<<<1, pc::STEP_DESC_THREADS, 0, cs>>>(da, counter, sd,
                                                                     reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.max_slen),
                                                                     reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.chain_bar),
                                                                     (int)chain_bar_words(ctx->d.n_layers));
@@ -1072,6 +1130,7 @@ int pc_decode_run(pc_ctx* ctx, void* stream, int n_steps, const pc_step_desc* st
             if (e != cudaSuccess) return cuda_fail(e, "graph instantiate");
             GraphEntry ent;
             ent.key = key; ent.exec = exec; ent.launches = captured;
+            ++ctx->captures;
             ctx->graphs.push_back(ent);
         }
         e = cudaGraphLaunch(exec, st);
@@ -1101,14 +1160,14 @@ int pc_sample(void* stream, int n_rows, int vocab, const float* logits, const in
     }
     if (chunks == 1) {
         pc::sample_kernel<<<n_rows, 256, 0, st>>>(nullptr, vocab, logits, logits_row, temperature, k0, k1, row_prompt, row_rollout,
-                                                  row_step, 0, out_tokens, out_index, 0, out_top2_gap, nullptr);
+                                                  row_step, 0, out_tokens, out_index, 0, out_top2_gap, nullptr, nullptr);
         count_launches(1);
     } else {
         pc::Top2Rec* rec = static_cast<pc::Top2Rec*>(scratch);
         pc::sample_partial_kernel<<<dim3(n_rows, chunks), 256, 0, st>>>(nullptr, vocab, chunks, logits, logits_row, temperature, k0, k1,
-                                                                        row_prompt, row_rollout, row_step, 0, rec, nullptr);
+                                                                        row_prompt, row_rollout, row_step, 0, rec, nullptr, nullptr);
         pc::sample_reduce_kernel<<<(n_rows + 127) / 128, 128, 0, st>>>(nullptr, n_rows, chunks, rec, out_tokens, out_index, 0,
-                                                                       out_top2_gap);
+                                                                       out_top2_gap, nullptr);
         count_launches(2);
     }
     PC_CUDA_CHECK_LAUNCH("sample");
@@ -1225,8 +1284,8 @@ int pc_sample_static(void* stream, int n_rows, int vocab, const float* logits, c
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // every record the second kernel reads is written by the first one in this same call: nothing has to start at zero
     pc::sample_partial_kernel<<<dim3(n_rows, chunks), 256, 0, st>>>(nullptr, vocab, chunks, logits, logits_row, temperature, k0, k1,
-                                                                    row_prompt, row_rollout, row_step, 0, rec, nullptr);
-    pc::sample_reduce_kernel<<<(n_rows + 127) / 128, 128, 0, st>>>(nullptr, n_rows, chunks, rec, out_tokens, out_index, 0, out_top2_gap);
+                                                                    row_prompt, row_rollout, row_step, 0, rec, nullptr, nullptr);
+    pc::sample_reduce_kernel<<<(n_rows + 127) / 128, 128, 0, st>>>(nullptr, n_rows, chunks, rec, out_tokens, out_index, 0, out_top2_gap, nullptr);
     count_launches(2);
     PC_CUDA_CHECK_LAUNCH("sample (static scratch)");
     return PC_OK;

@@ -163,12 +163,13 @@ __global__ void __launch_bounds__(256) sample_kernel(const StepDesc* __restrict_
                                                      const int32_t* __restrict__ row_rollout, const int32_t* __restrict__ row_step,
                                                      int step_offset, int32_t* __restrict__ out_tokens,
                                                      const int64_t* __restrict__ out_index, int64_t out_index_offset,
-                                                     float* __restrict__ out_gap, const int32_t* __restrict__ prompt_key) {
+                                                     float* __restrict__ out_gap, const int32_t* __restrict__ prompt_key,
+                                                     const DecodeArgsDev* __restrict__ da) {
     const int r = blockIdx.x;
-    int64_t ro = r;                         // index into the caller's row arrays
-    if (sd != nullptr) {
-        if (r >= sd->n_rows) return;
-        ro += sd->row_off;
+    const int64_t ro = r;                   // index into the row arrays
+    if (sd != nullptr && r >= sd->n_rows) return;
+    if (da != nullptr) {                    // decode step: token buffer, temperature and seed from the device-resident arguments
+        out_tokens = da->tokens; temperature = da->temperature; k0 = da->k0; k1 = da->k1;
     }
     const float* lg = logits + (size_t)(logits_row ? logits_row[ro] : r) * vocab;
     const uint32_t c1 = (uint32_t)(row_step[ro] + step_offset), c2 = (uint32_t)row_rollout[ro],
@@ -188,7 +189,8 @@ __global__ void __launch_bounds__(256) sample_kernel(const StepDesc* __restrict_
         Top2 u = lane < (int)(blockDim.x >> 5) ? sh[lane] : Top2{-INFINITY, -INFINITY, 0x7fffffff};
         u = top2_warp_reduce(u);
         if (lane == 0) {
-            out_tokens[out_index ? out_index[ro] + out_index_offset : (int64_t)r] = u.idx;
+            const int64_t at = out_index ? out_index[ro] + out_index_offset : (int64_t)r;
+            if (at >= 0) out_tokens[at] = u.idx;
             if (out_gap) out_gap[r] = u.best - u.second;
         }
     }
@@ -206,13 +208,11 @@ __global__ void __launch_bounds__(256) sample_partial_kernel(const StepDesc* __r
                                                              float temperature, uint32_t k0, uint32_t k1,
                                                              const int32_t* __restrict__ row_prompt, const int32_t* __restrict__ row_rollout,
                                                              const int32_t* __restrict__ row_step, int step_offset, Top2Rec* __restrict__ scratch,
-                                                             const int32_t* __restrict__ prompt_key) {
+                                                             const int32_t* __restrict__ prompt_key, const DecodeArgsDev* __restrict__ da) {
     const int r = blockIdx.x, chunk = blockIdx.y;
-    int64_t ro = r;
-    if (sd != nullptr) {
-        if (r >= sd->n_rows) return;
-        ro += sd->row_off;
-    }
+    const int64_t ro = r;
+    if (sd != nullptr && r >= sd->n_rows) return;
+    if (da != nullptr) { temperature = da->temperature; k0 = da->k0; k1 = da->k1; }
     const float* lg = logits + (size_t)(logits_row ? logits_row[ro] : r) * vocab;
     const uint32_t c1 = (uint32_t)(row_step[ro] + step_offset), c2 = (uint32_t)row_rollout[ro],
                    c3 = (uint32_t)(prompt_key ? prompt_key[row_prompt[ro]] : row_prompt[ro]);    // key id of the prompt
@@ -238,21 +238,18 @@ __global__ void __launch_bounds__(256) sample_partial_kernel(const StepDesc* __r
 
 __global__ void sample_reduce_kernel(const StepDesc* __restrict__ sd, int n_rows, int n_chunks, const Top2Rec* __restrict__ scratch,
                                      int32_t* __restrict__ out_tokens, const int64_t* __restrict__ out_index,
-                                     int64_t out_index_offset, float* __restrict__ out_gap) {
+                                     int64_t out_index_offset, float* __restrict__ out_gap, const DecodeArgsDev* __restrict__ da) {
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
-    int64_t ro = r;
-    if (sd != nullptr) {
-        if (r >= sd->n_rows) return;
-        ro += sd->row_off;
-    } else if (r >= n_rows) {
-        return;
-    }
+    const int64_t ro = r;
+    if (r >= (sd != nullptr ? sd->n_rows : n_rows)) return;
+    if (da != nullptr) out_tokens = da->tokens;
     Top2 t{-INFINITY, -INFINITY, 0x7fffffff};
     for (int c = 0; c < n_chunks; ++c) {
         const Top2Rec x = scratch[(size_t)r * n_chunks + c];
         t = top2_merge(t, Top2{x.best, x.second, x.idx});
     }
-    out_tokens[out_index ? out_index[ro] + out_index_offset : (int64_t)r] = t.idx;
+    const int64_t at = out_index ? out_index[ro] + out_index_offset : (int64_t)r;
+    if (at >= 0) out_tokens[at] = t.idx;
     if (out_gap) out_gap[r] = t.best - t.second;
 }
 
@@ -262,13 +259,12 @@ __global__ void __launch_bounds__(256) token_logprob_kernel(const StepDesc* __re
                                                             const int32_t* __restrict__ logits_row, float temperature,
                                                             const int32_t* __restrict__ tokens, const int64_t* __restrict__ tok_index,
                                                             int64_t tok_index_offset, float* __restrict__ out,
-                                                            const int64_t* __restrict__ out_index, int64_t out_index_offset) {
+                                                            const int64_t* __restrict__ out_index, int64_t out_index_offset,
+                                                            const DecodeArgsDev* __restrict__ da) {
     const int r = blockIdx.x;
-    int64_t ro = r;
-    if (sd != nullptr) {
-        if (r >= sd->n_rows) return;
-        ro += sd->row_off;
-    }
+    const int64_t ro = r;
+    if (sd != nullptr && r >= sd->n_rows) return;
+    if (da != nullptr) { tokens = da->tokens; out = da->logprobs; temperature = da->temperature; }
     const float* lg = logits + (size_t)(logits_row ? logits_row[ro] : r) * vocab;
     __shared__ float red[33];
     const float mx = range_max(lg, 0, vocab, temperature, red);          // max of logits / T
@@ -294,7 +290,9 @@ __global__ void __launch_bounds__(256) token_logprob_kernel(const StepDesc* __re
     }
     s = block_sum(s, red);
     if (threadIdx.x == 0) {
-        const int tok = tokens[tok_index ? tok_index[ro] + tok_index_offset : (int64_t)r];
+        const int64_t ti = tok_index ? tok_index[ro] + tok_index_offset : (int64_t)r;
+        if (ti < 0) return;
+        const int tok = tokens[ti];
         const float lp = (tok >= 0 && tok < vocab) ? lg[tok] * inv_t - mx - logf(s) : -INFINITY;
         out[out_index ? out_index[ro] + out_index_offset : (int64_t)r] = lp;
     }

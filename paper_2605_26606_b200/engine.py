@@ -162,6 +162,7 @@ class RolloutEngine:
         self.tokens = torch.full((P * G * wl.max_new,), -1, dtype=torch.int32, device=dev)
         self.logprobs = torch.zeros(P * G * wl.max_new, dtype=torch.float32, device=dev) if self.collect_logprobs else None
         B.pc_set_logprob_buffer(self.ctx, self.logprobs)
+        B.pc_set_index_bounds(self.ctx, P, P * G * wl.max_new)
         self.prompt_key_host = None
         self.prompt_key_dev = None
         B.pc_set_prompt_keys(self.ctx, None)

@@ -366,3 +366,42 @@ def test_persistent_decode_kernel_equals_one_kernel_per_operation(model):
         for s in lg:
             assert torch.equal(lg[s], logits[0][s]), s
         assert np.array_equal(a["advantages"], b["advantages"])
+
+
+def test_new_schedules_and_token_buffers_reuse_the_captured_steps():
+    """pc_decode_run keys its captured steps on shapes and arenas only: running the same step again (fresh schedule tensors, a
+    fresh token buffer, another sampling seed) captures nothing new, and a bad row index is caught on the device."""
+    from paper_2605_26606_b200 import binding as B
+    w = dataclasses.replace(wl.WORKLOADS["config0"], model=wl.SMALL_BF16, n_prompts=5, prompt_len_lo=3, prompt_len_hi=50, group_size=9,
+                            n_pilot=3, max_new=40, cap_lo=1, cap_hi=40, data_seed=21,
+                            forced_explicit=((0, 0.5), (1, 0.5), (2, 0.5), (3, 0.0), (4, 0.5)))
+    weights = wl.gen_weights(w.model, seed=0, threads=2)
+    batch = wl.gen_batch(w)
+    eng = RolloutEngine(w.model, weights, max_rows=45, max_prefill_tokens=int(batch.prompt_offsets[-1]))
+    a = eng.pilot_commit_step(w, batch)
+    n1 = B.pc_capture_count(eng.ctx)
+    assert n1 > 0
+    keep = [eng.tokens, eng._keep_schedule]              # keep the old buffers alive so that the allocator hands out new addresses
+    b = eng.pilot_commit_step(w, batch)
+    assert B.pc_capture_count(eng.ctx) == n1
+    for p in range(w.n_prompts):
+        for i in range(w.group_size):
+            if a["generated"][p, i]:
+                assert np.array_equal(a["tokens"][p][i], b["tokens"][p][i])
+    c = eng.pilot_commit_step(dataclasses.replace(w, sample_seed=77), batch)
+    assert B.pc_capture_count(eng.ctx) == n1
+    assert any(not np.array_equal(a["tokens"][p][0], c["tokens"][p][0]) for p in range(w.n_prompts))
+    del keep
+    # a row that names a prompt outside the per-prompt arrays is switched off and flagged instead of read
+    eng.load_batch(w, batch)
+    eng.prefill()
+    sch_prompts = np.array([1], dtype=np.int64)
+    longest = np.argsort(-batch.caps[1])[:2]                          # two rollouts of prompt 1 with several decode steps
+    assert batch.caps[1, longest[1]] > 2
+    eng.run_stage(sch_prompts, longest[:1])                           # a valid one-row stage first
+    eng.check_error_flag()
+    B.pc_set_index_bounds(eng.ctx, w.n_prompts, 8)                   # token buffer "of 8 cells": every row_tok_index is beyond it
+    eng.use_graphs = False
+    eng.run_stage(sch_prompts, longest[1:])
+    assert int(eng.err_flag.item()) == 4                             # DEV_ERR_GROUP_RANGE
+    eng.err_flag.zero_()
