@@ -97,8 +97,9 @@ typedef struct pc_model_desc {
                           * for QKV, output projection and LM head.  lm_head must then be given even
                           * when tied_embed = 1 (a half copy of the embedding, which itself stays
                           * bfloat16 for the token lookup).  A bfloat16 weight converts to half exactly
-                          * unless it is below 2^-14 in magnitude (then to within 2^-25); the caller
-                          * answers for weights and GEMM inputs staying inside half's range.           */
+                          * unless it is below 2^-14 in magnitude (then to within 2^-25).  Activations
+                          * and V values that do not fit half (|x| > 65504, or NaN) are stored saturated
+                          * (NaN as 0) and reported as code 5 in *dev_error_flag.                        */
 } pc_model_desc;
 
 /* Device pointers to the weights.  The per-layer members are HOST arrays of n_layers
@@ -177,6 +178,11 @@ PC_API int pc_set_workspace(pc_ctx* ctx, void* dev_ws, size_t bytes, int max_row
  * bound; gate/up and the LM head never split.  Results stay deterministic for a fixed plan.  Drops captured decode
  * steps.  The paper has no counterpart. */
 PC_API int pc_set_gemm_plan(pc_ctx* ctx, const char* spec);
+
+/* Self-test of the bounded waits every kernel here uses on its mbarriers: launches one warp that waits, for at most
+ * spin_limit polls (1 .. 2^20), on a barrier nothing arrives at; the wait gives up, stores DEV_ERR_WAIT_TIMEOUT (3) in
+ * *dev_error_flag (device int32) and the kernel returns normally, so the context stays usable.  No counterpart in the paper. */
+PC_API int pc_selftest_wait_timeout(void* stream, uint32_t spin_limit, int32_t* dev_error_flag);
 
 /* Sizes of the caller's per-prompt arrays (prompt_len, prompt_kv_start, prompt keys) and of the token buffer, so that
  * the decode steps can check row_prompt and row_tok_index against them (see "Device-side anomalies" above).  0 = not

@@ -22,7 +22,7 @@ PC_ERR_UNSUPPORTED, PC_ERR_CUDA, PC_ERR_NO_WORKSPACE = 5, 6, 7
 PC_DTYPE_F32, PC_DTYPE_BF16 = 0, 1
 PC_STATUS_COMMIT, PC_STATUS_BUFFERED, PC_STATUS_DEFER_HARD, PC_STATUS_SKIP_EASY = 0, 1, 2, 3
 
-EXPORTS = ["pc_status_string", "pc_last_cuda_error", "pc_launch_count", "pc_profile_attention", "pc_set_gemm_plan", "pc_set_decode_mode", "pc_set_chain_trace", "pc_chain_trace_words", "pc_capture_count", "pc_set_index_bounds", "pc_create", "pc_destroy", "pc_workspace_bytes",
+EXPORTS = ["pc_status_string", "pc_last_cuda_error", "pc_launch_count", "pc_profile_attention", "pc_set_gemm_plan", "pc_set_decode_mode", "pc_set_chain_trace", "pc_chain_trace_words", "pc_capture_count", "pc_set_index_bounds", "pc_selftest_wait_timeout", "pc_create", "pc_destroy", "pc_workspace_bytes",
            "pc_set_workspace", "pc_prefill_shared", "pc_decode_step", "pc_decode_run", "pc_sample", "pc_sample_static", "pc_token_logprob", "pc_set_logprob_buffer", "pc_set_prompt_keys", "pc_reward_last_token",
            "pc_group_stats", "pc_allocate", "pc_grpo_advantage"]
 
@@ -84,6 +84,7 @@ def _lib():
         lib.pc_capture_count.argtypes = [C.c_void_p]
         lib.pc_capture_count.restype = C.c_uint64
         lib.pc_set_index_bounds.argtypes = [C.c_void_p, C.c_int, C.c_int64]
+        lib.pc_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p]
         lib.pc_set_chain_trace.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
         lib.pc_chain_trace_words.argtypes = [C.c_void_p]
         lib.pc_chain_trace_words.restype = C.c_size_t
@@ -162,6 +163,10 @@ def pc_capture_count(ctx: "Context") -> int:
 
 def pc_set_index_bounds(ctx: "Context", n_prompts: int, n_tokens: int) -> None:
     _check(_lib().pc_set_index_bounds(ctx.handle, n_prompts, n_tokens), "pc_set_index_bounds")
+
+
+def pc_selftest_wait_timeout(spin_limit: int, err_flag: torch.Tensor) -> None:
+    _check(_lib().pc_selftest_wait_timeout(_stream(), spin_limit, _ptr(err_flag, torch.int32)), "pc_selftest_wait_timeout")
 
 
 def pc_chain_trace_words(ctx: "Context") -> int:

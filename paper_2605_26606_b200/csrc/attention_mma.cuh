@@ -69,6 +69,10 @@ __device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
     const __half2 p = __floats2half2_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&p);
 }
+// The same for values that leave the kernel as a GEMM operand: out-of-range values are saturated and reported.
+__device__ __forceinline__ uint32_t pack_f16_guard(float lo, float hi, int32_t* err) {
+    return pack_f16(half_guard(lo, err), half_guard(hi, err));
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&p);
@@ -329,7 +333,7 @@ attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __
                 const float y0 = o[t][2 * i] * inv, y1 = o[t][2 * i + 1] * inv;
                 const size_t at = rh * HD + t * 8 + (lane & 3) * 2;
                 if (out_lo == nullptr) {         // the output projection takes IEEE half operands
-                    *reinterpret_cast<uint32_t*>(out + at) = pack_f16(y0, y1);
+                    *reinterpret_cast<uint32_t*>(out + at) = pack_f16_guard(y0, y1, err);
                 } else {
                     *reinterpret_cast<uint32_t*>(out + at) = pack_bf16(y0, y1);
                     // rounding remainder, consumed as a second bf16 operand by the output projection
@@ -641,7 +645,7 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
 // item), so that the loads do not wait for the row's suffix length; records past the row's own count are ignored.
 template <int HD>
 __device__ __forceinline__ void merge_item_warp(int lane, size_t rh, int Hq, const RowGeom& g, const PrefixPartial& part, int ct, int n_load,
-                                                __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ out_lo) {
+                                                __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ out_lo, int32_t* err) {
     constexpr int EPL = HD / 32;
     const int row = (int)(rh / Hq);
     const int slen = g.s_len[row];
@@ -690,8 +694,8 @@ __device__ __forceinline__ void merge_item_warp(int lane, size_t rh, int Hq, con
     }
     __nv_bfloat16* dst = out + rh * HD + lane * EPL;
     if (out_lo == nullptr) {                 // the output projection takes IEEE half operands: no remainder needed
-        if (EPL == 4) *reinterpret_cast<uint2*>(dst) = make_uint2(pack_f16(acc[0], acc[1]), pack_f16(acc[2], acc[3]));
-        else *reinterpret_cast<uint32_t*>(dst) = pack_f16(acc[0], acc[1]);
+        if (EPL == 4) *reinterpret_cast<uint2*>(dst) = make_uint2(pack_f16_guard(acc[0], acc[1], err), pack_f16_guard(acc[2], acc[3], err));
+        else *reinterpret_cast<uint32_t*>(dst) = pack_f16_guard(acc[0], acc[1], err);
         return;
     }
     __nv_bfloat16* dst_lo = out_lo + rh * HD + lane * EPL;
@@ -707,12 +711,12 @@ __device__ __forceinline__ void merge_item_warp(int lane, size_t rh, int Hq, con
 // Stand-alone form: the grid covers the row bound of the step.
 template <int HD>
 __global__ void __launch_bounds__(256) attn_merge_kernel(const StepDesc* __restrict__ sd, int Hq, RowGeom g, PrefixPartial part,
-                                                         __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ out_lo) {
+                                                         __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ out_lo, int32_t* err) {
     const size_t rh = (size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int n_live = sd->n_rows;
     if (rh >= (size_t)n_live * Hq) return;
     const SuffixPlan sp = suffix_plan(*g.max_slen, n_live * part.n_kv_heads, part.n_suffix_warps);
-    merge_item_warp<HD>(threadIdx.x & 31, rh, Hq, g, part, sp.ct, part.n_parts + sp.cpi, out, out_lo);
+    merge_item_warp<HD>(threadIdx.x & 31, rh, Hq, g, part, sp.ct, part.n_parts + sp.cpi, out, out_lo, err);
 }
 
 }  // namespace am

@@ -367,7 +367,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_chain_kernel(const __grid_c
                     const int tiles_n = (gd.N + gd.BN - 1) / gd.BN, n_tiles = tiles_m * tiles_n * gd.splits;
                     tc::EpiPartial e_part{nullptr, 0, 0};
                     tc::EpiResidual e_res{p.h, p.d_model};
-                    const tc::EpiSwiGLU e_glu{p.act, p.d_ff, 1};
+                    const tc::EpiSwiGLU e_glu{p.act, p.d_ff, 1, p.err};
                     const tc::EpiStoreF32 e_st{p.logits, p.vocab, nullptr};
                     int ek;                                      // 0 partial, 1 residual, 2 SwiGLU, 3 store
                     if (ph == PH_QKV) { e_part = tc::EpiPartial{p.qkv, p.n_qkv, (size_t)M * p.n_qkv}; ek = 0; }
@@ -438,7 +438,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_chain_kernel(const __grid_c
                                 }
                             }
                             if (!norm_row_cta<__nv_bfloat16>(w, lane, p.d_model, h_row, pend, (size_t)r * p.d_model, gain, p.eps,
-                                                             p.a + (size_t)r * p.d_model, 1, s_norm_red + j * 8, s_norm_cnt + j)) {
+                                                             p.a + (size_t)r * p.d_model, 1, s_norm_red + j * 8, s_norm_cnt + j, p.err)) {
                                 ok = false;
                                 break;
                             }
@@ -450,7 +450,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_chain_kernel(const __grid_c
                                 embed_row_warp<__nv_bfloat16>(lane, p.d_model,
                                                               reinterpret_cast<const __nv_bfloat16*>(p.embed) + (size_t)p.g.token[r] * p.d_model, h_row);
                             norm_row_warp<__nv_bfloat16>(lane, p.d_model, h_row, pend, (size_t)r * p.d_model, gain, p.eps,
-                                                         p.a + (size_t)r * p.d_model, nullptr, 1);
+                                                         p.a + (size_t)r * p.d_model, nullptr, 1, p.err);
                         }
                     }
                 } else if (ph == PH_POST) {
@@ -458,7 +458,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_chain_kernel(const __grid_c
                     const LayerTab& lt = p.layers[layer];
                     const QkvPostArgs<__nv_bfloat16> A{p.Hq, p.Hkv, p.hd, layer,
                                                       Partials{p.qkv, p.splits[GK_QKV], (size_t)M * p.n_qkv, p.n_qkv},
-                                                      lt.bqkv, lt.q_norm, lt.k_norm, p.eps, p.rope, p.g, p.prompt_arena, p.suffix_arena, p.q};
+                                                      lt.bqkv, lt.q_norm, lt.k_norm, p.eps, p.rope, p.g, p.prompt_arena, p.suffix_arena, p.q, p.err};
                     const int n_heads = p.Hq + 2 * p.Hkv, items = m_live * n_heads;
                     const int per_warp = (items + n_gw - 1) / n_gw;
                     const int i_end = min(items, (gw + 1) * per_warp);
@@ -482,8 +482,8 @@ __global__ void __launch_bounds__(THREADS, 1) decode_chain_kernel(const __grid_c
                     const am::SuffixPlan sp = am::suffix_plan(*p.g.max_slen, p.sd->n_rows * p.part.n_kv_heads, p.part.n_suffix_warps);
                     const int n_load = p.part.n_parts + sp.cpi;
                     for (int it = gw; it < items; it += n_gw) {
-                        if (p.hd == 128) am::merge_item_warp<128>(lane, it, p.Hq, p.g, p.part, sp.ct, n_load, p.attn, nullptr);
-                        else am::merge_item_warp<64>(lane, it, p.Hq, p.g, p.part, sp.ct, n_load, p.attn, nullptr);
+                        if (p.hd == 128) am::merge_item_warp<128>(lane, it, p.Hq, p.g, p.part, sp.ct, n_load, p.attn, nullptr, p.err);
+                        else am::merge_item_warp<64>(lane, it, p.Hq, p.g, p.part, sp.ct, n_load, p.attn, nullptr, p.err);
                     }
                 }
             }

@@ -66,8 +66,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait.  Returns false when it gave up (or when another role already raised the abort flag).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t limit = WAIT_LIMIT) {
+    for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63u) == 63u) {
             if (*abort_flag) return false;
@@ -191,7 +191,7 @@ struct EpiResidual {            // H += acc
     }
 };
 struct EpiSwiGLU {              // columns (2j, 2j+1) = (gate_j, up_j) -> out[row, j] = silu(gate) * up, bf16 (or IEEE half)
-    __nv_bfloat16* out; int ld; int half_out;
+    __nv_bfloat16* out; int ld; int half_out; int32_t* err;
     __device__ __forceinline__ void set_rows(int) {}
     __device__ __forceinline__ void operator()(int row, int col0, const float* v, int n_valid, int /*split*/) const {
         __nv_bfloat16* dst = out + (size_t)row * ld + (col0 >> 1);
@@ -202,7 +202,7 @@ struct EpiSwiGLU {              // columns (2j, 2j+1) = (gate_j, up_j) -> out[ro
                 const float g0 = v[4 * i], u0 = v[4 * i + 1], g1 = v[4 * i + 2], u1 = v[4 * i + 3];
                 const float y0 = g0 / (1.f + expf(-g0)) * u0, y1 = g1 / (1.f + expf(-g1)) * u1;
                 if (half_out) {
-                    const __half2 p = __floats2half2_rn(y0, y1);
+                    const __half2 p = __floats2half2_rn(half_guard(y0, err), half_guard(y1, err));
                     w[i] = *reinterpret_cast<const uint32_t*>(&p);
                 } else {
                     const __nv_bfloat162 p = __floats2bfloat162_rn(y0, y1);
@@ -216,7 +216,7 @@ struct EpiSwiGLU {              // columns (2j, 2j+1) = (gate_j, up_j) -> out[ro
             for (int i = 0; i < 32; i += 2)
                 if (i + 1 < n_valid) {
                     const float y = v[i] / (1.f + expf(-v[i])) * v[i + 1];
-                    if (half_out) reinterpret_cast<__half*>(dst)[i >> 1] = __float2half_rn(y);
+                    if (half_out) reinterpret_cast<__half*>(dst)[i >> 1] = __float2half_rn(half_guard(y, err));
                     else dst[i >> 1] = __float2bfloat16_rn(y);
                 }
         }
@@ -361,6 +361,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         __syncwarp();
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// Self-test of the bounded wait: one thread waits, with a short limit, on an mbarrier that nothing will ever arrive at
+// (no copy is in flight), and reports the timeout in the error flag the way the production kernels do.
+__global__ void wait_timeout_selftest_kernel(uint32_t limit, int32_t* err) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (!mbar_wait(smem_u32(&bar), 0, &abort_flag, limit)) set_error(err, DEV_ERR_WAIT_TIMEOUT);
     }
 }
 

@@ -146,10 +146,13 @@ __device__ __forceinline__ float4 bf16_remainder(float4 v) {
 // The row-wise operations below are written for ONE WARP per row (or per (row, head)), so that the stand-alone kernels
 // and the phases of the persistent decode kernel (decode_chain.cuh) run the very same arithmetic in the same order.
 
+// half_out: 0 = storage type T, 1 = IEEE half (operand of a half-precision GEMM); err = the device error flag (range guard).
 template <typename T>
-__device__ __forceinline__ void store_norm_out(T* __restrict__ a_row, T* __restrict__ a_lo_row, int i4, float4 y, int half_out) {
-    if (sizeof(T) == 2 && half_out) {          // IEEE half instead of bfloat16 (operand of a half-precision GEMM)
-        const __half2 lo = __floats2half2_rn(y.x, y.y), hi = __floats2half2_rn(y.z, y.w);
+__device__ __forceinline__ void store_norm_out(T* __restrict__ a_row, T* __restrict__ a_lo_row, int i4, float4 y, int half_out,
+                                               int32_t* err = nullptr) {
+    if (sizeof(T) == 2 && half_out) {
+        const __half2 lo = __floats2half2_rn(half_guard(y.x, err), half_guard(y.y, err)),
+                      hi = __floats2half2_rn(half_guard(y.z, err), half_guard(y.w, err));
         *reinterpret_cast<uint2*>(a_row + 4 * i4) =
             make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
     } else {
@@ -188,7 +191,7 @@ __device__ __forceinline__ float sq4(float4 v) {
 template <typename T>
 __device__ __forceinline__ void norm_row_warp(int lane, int d, float* __restrict__ h_row, Partials pend, size_t pend_row,
                                               const float* __restrict__ gain, float eps, T* __restrict__ a_row,
-                                              T* __restrict__ a_lo_row, int half_out) {
+                                              T* __restrict__ a_lo_row, int half_out, int32_t* err = nullptr) {
     const int n4 = d >> 2;
     float4* x = reinterpret_cast<float4*>(h_row);
     float seg[NORM_SEGS];
@@ -220,7 +223,7 @@ __device__ __forceinline__ void norm_row_warp(int lane, int d, float* __restrict
             if (i < n4)
                 store_norm_out<T>(a_row, a_lo_row, i,
                                   make_float4(v[k].x * rstd * gg[k].x, v[k].y * rstd * gg[k].y, v[k].z * rstd * gg[k].z, v[k].w * rstd * gg[k].w),
-                                  half_out);
+                                  half_out, err);
         }
         return;
     }
@@ -242,7 +245,7 @@ __device__ __forceinline__ void norm_row_warp(int lane, int d, float* __restrict
     const float rstd = rsqrtf(__fadd_rn(__fdiv_rn(ss, (float)d), eps));
     for (int i = lane; i < n4; i += 32) {
         const float4 v = x[i], gg = *reinterpret_cast<const float4*>(gain + 4 * i);     // this lane's own writes
-        store_norm_out<T>(a_row, a_lo_row, i, make_float4(v.x * rstd * gg.x, v.y * rstd * gg.y, v.z * rstd * gg.z, v.w * rstd * gg.w), half_out);
+        store_norm_out<T>(a_row, a_lo_row, i, make_float4(v.x * rstd * gg.x, v.y * rstd * gg.y, v.z * rstd * gg.z, v.w * rstd * gg.w), half_out, err);
     }
 }
 
@@ -255,7 +258,7 @@ __device__ __forceinline__ bool norm_row_fits_cta(int d) { return ((d >> 2) + 31
 template <typename T>
 __device__ __forceinline__ bool norm_row_cta(int w, int lane, int d, float* __restrict__ h_row, Partials pend, size_t pend_row,
                                              const float* __restrict__ gain, float eps, T* __restrict__ a_row, int half_out,
-                                             volatile float* red, int* counter) {
+                                             volatile float* red, int* counter, int32_t* err = nullptr) {
     const int n4 = d >> 2;
     float4* x = reinterpret_cast<float4*>(h_row);
     float4 v[NORM_SEG_REG4], gg[NORM_SEG_REG4];
@@ -299,7 +302,7 @@ __device__ __forceinline__ bool norm_row_cta(int w, int lane, int d, float* __re
         if (i < n4)
             store_norm_out<T>(a_row, static_cast<T*>(nullptr), i,
                               make_float4(v[kk].x * rstd * gg[kk].x, v[kk].y * rstd * gg[kk].y, v[kk].z * rstd * gg[kk].z, v[kk].w * rstd * gg[kk].w),
-                              half_out);
+                              half_out, err);
     }
     return true;
 }
@@ -320,12 +323,13 @@ constexpr int ROW_WARPS = 8;         // rows per block of the stand-alone row-wi
 template <typename T>
 __global__ void __launch_bounds__(ROW_WARPS * 32) embed_rmsnorm_kernel(const StepDesc* __restrict__ sd, int d, const int32_t* token,
                                                                         const T* __restrict__ embed, const float* __restrict__ gain, float eps,
-                                                                        float* __restrict__ h, T* __restrict__ a, T* __restrict__ a_lo, int half_out) {
+                                                                        float* __restrict__ h, T* __restrict__ a, T* __restrict__ a_lo, int half_out,
+                                                                        int32_t* err) {
     const int r = blockIdx.x * ROW_WARPS + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (r >= sd->n_rows) return;
     embed_row_warp<T>(lane, d, embed + (size_t)token[r] * d, h + (size_t)r * d);
     norm_row_warp<T>(lane, d, h + (size_t)r * d, Partials{nullptr, 0, 0, 0}, 0, gain, eps, a + (size_t)r * d,
-                     a_lo ? a_lo + (size_t)r * d : nullptr, half_out);
+                     a_lo ? a_lo + (size_t)r * d : nullptr, half_out, err);
 }
 
 // Optional residual update followed by the norm:  h[row, :] += pending partial sums of row;  a[r, :] = RMSNorm(h[row, :]; gain)
@@ -333,12 +337,12 @@ __global__ void __launch_bounds__(ROW_WARPS * 32) embed_rmsnorm_kernel(const Ste
 template <typename T>
 __global__ void __launch_bounds__(ROW_WARPS * 32) rmsnorm_kernel(const StepDesc* __restrict__ sd, int n_rows, int d, float* __restrict__ h,
                                                                   const int32_t* __restrict__ src, Partials pend, const float* __restrict__ gain,
-                                                                  float eps, T* __restrict__ a, T* __restrict__ a_lo, int half_out) {
+                                                                  float eps, T* __restrict__ a, T* __restrict__ a_lo, int half_out, int32_t* err) {
     const int r = blockIdx.x * ROW_WARPS + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (r >= (sd != nullptr ? sd->n_rows : n_rows)) return;
     const int row = src ? src[r] : r;
     norm_row_warp<T>(lane, d, h + (size_t)row * d, pend, (size_t)row * pend.ld, gain, eps, a + (size_t)r * d,
-                     a_lo ? a_lo + (size_t)r * d : nullptr, half_out);
+                     a_lo ? a_lo + (size_t)r * d : nullptr, half_out, err);
 }
 
 struct KvArena {
@@ -359,6 +363,7 @@ struct QkvPostArgs {
     RowGeom g;
     KvArena prompt_arena, suffix_arena;
     T* q_out;                     // [rows, Hq * hd]
+    int32_t* err;                 // device error flag (range guard of the half V cache)
 };
 
 // One warp per (row, head of the fused q|k|v projection); lane i handles the rotary pairs (i, i + hd/2) and, for
@@ -447,7 +452,10 @@ __device__ __forceinline__ void qkv_post_items_warp(int lane, const QkvPostArgs<
             __half* dv = reinterpret_cast<__half*>(dst);
 #pragma unroll
             for (int j = 0; j < 2; ++j)
-                if (j < npair) { dv[lane + 32 * j] = __float2half_rn(x1[b][j]); dv[lane + 32 * j + half] = __float2half_rn(x2[b][j]); }
+                if (j < npair) {
+                    dv[lane + 32 * j] = __float2half_rn(half_guard(x1[b][j], A.err));
+                    dv[lane + 32 * j + half] = __float2half_rn(half_guard(x2[b][j], A.err));
+                }
             continue;
         }
 #pragma unroll

@@ -369,7 +369,7 @@ int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, in
         count_launches(2);
         return PC_OK;
     }
-    am::attn_merge_kernel<HD><<<(M * d.n_q_heads + 7) / 8, 256, 0, st>>>(sd, d.n_q_heads, g, part, attn, attn_lo);
+    am::attn_merge_kernel<HD><<<(M * d.n_q_heads + 7) / 8, 256, 0, st>>>(sd, d.n_q_heads, g, part, attn, attn_lo, c->err);
     count_launches(3);
     return PC_OK;
 }
@@ -408,12 +408,12 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
     rope_table_kernel<<<(M * half + 255) / 256, 256, 0, st>>>(sd, half, (double)d.rope_theta, g.pos, rope);
     const int row_blocks = (M + ROW_WARPS - 1) / ROW_WARPS;
     embed_rmsnorm_kernel<T><<<row_blocks, ROW_WARPS * 32, 0, st>>>(sd, d.d_model, g.token, reinterpret_cast<const T*>(c->embed), c->attn_norm[0],
-                                               d.rms_eps, h, a, a_lo, half_gemm ? 1 : 0);
+                                               d.rms_eps, h, a, a_lo, half_gemm ? 1 : 0, c->err);
     count_launches(2);
     PC_CUDA_CHECK_LAUNCH("embed_rmsnorm");
     for (int l = 0; l < d.n_layers; ++l) {
         if (l > 0) {
-            rmsnorm_kernel<T><<<row_blocks, ROW_WARPS * 32, 0, st>>>(sd, M, d.d_model, h, nullptr, pend, c->attn_norm[l], d.rms_eps, a, a_lo, half_gemm ? 1 : 0);
+            rmsnorm_kernel<T><<<row_blocks, ROW_WARPS * 32, 0, st>>>(sd, M, d.d_model, h, nullptr, pend, c->attn_norm[l], d.rms_eps, a, a_lo, half_gemm ? 1 : 0, c->err);
             pend = none;
             count_launches(1);
         }
@@ -432,7 +432,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
         const int post_items = M * (d.n_q_heads + 2 * d.n_kv_heads);
         qkv_post_kernel<T><<<(post_items + ROW_WARPS - 1) / ROW_WARPS, ROW_WARPS * 32, 0, st>>>(
             sd, QkvPostArgs<T>{d.n_q_heads, d.n_kv_heads, d.head_dim, l, qkv_parts, bias, d.qk_norm ? c->q_norm[l] : nullptr,
-                               d.qk_norm ? c->k_norm[l] : nullptr, d.rms_eps, rope, g, prompt_arena, suffix_arena, q});
+                               d.qk_norm ? c->k_norm[l] : nullptr, d.rms_eps, rope, g, prompt_arena, suffix_arena, q, c->err});
         count_launches(2);
         if constexpr (kF32) {
             if (l == prof_layer) cudaEventRecord(c->prof_start, st);
@@ -462,7 +462,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
                     return rc2;
             }
         }
-        rmsnorm_kernel<T><<<row_blocks, ROW_WARPS * 32, 0, st>>>(sd, M, d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a, nullptr, half_gemm ? 1 : 0);
+        rmsnorm_kernel<T><<<row_blocks, ROW_WARPS * 32, 0, st>>>(sd, M, d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a, nullptr, half_gemm ? 1 : 0, c->err);
         pend = none;
         count_launches(2);
         if constexpr (kF32) {
@@ -470,7 +470,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
                                 EpiSwiGLU<T>{act, d.d_ff});
             launch_gemm_simt<T>(st, sd, act, reinterpret_cast<const T*>(c->w_down[l]), M, d.d_model, d.d_ff, EpiResidual{h, d.d_model});
         } else {
-            if (int rc = gemm_bf16(c, st, sd, c->map_a, nullptr, c->m_wgu[l], M, plan_gemm(c, GEMM_GATE_UP, c->m_wgu[l], M, false), tc::EpiSwiGLU{act, d.d_ff, half_gemm ? 1 : 0}, half_gemm))
+            if (int rc = gemm_bf16(c, st, sd, c->map_a, nullptr, c->m_wgu[l], M, plan_gemm(c, GEMM_GATE_UP, c->m_wgu[l], M, false), tc::EpiSwiGLU{act, d.d_ff, half_gemm ? 1 : 0, c->err}, half_gemm))
                 return rc;
             const GemmPlan gp = plan_gemm(c, GEMM_DOWN, c->m_wdown[l], M, true);
             if (gp.splits == 1) {
@@ -496,7 +496,7 @@ int run_lm_head(pc_ctx* c, cudaStream_t st, int n, const pc::StepDesc* sd, const
     T* a = reinterpret_cast<T*>(c->ws + c->cv.a);
     const bool half_gemm = !std::is_same<T, float>::value && d.half_gemm != 0;
     T* a_lo = std::is_same<T, float>::value || half_gemm ? nullptr : reinterpret_cast<T*>(c->ws + c->cv.a_lo);
-    rmsnorm_kernel<T><<<(n + ROW_WARPS - 1) / ROW_WARPS, ROW_WARPS * 32, 0, st>>>(sd, n, d.d_model, h, src, c->pend, c->final_norm, d.rms_eps, a, a_lo, half_gemm ? 1 : 0);
+    rmsnorm_kernel<T><<<(n + ROW_WARPS - 1) / ROW_WARPS, ROW_WARPS * 32, 0, st>>>(sd, n, d.d_model, h, src, c->pend, c->final_norm, d.rms_eps, a, a_lo, half_gemm ? 1 : 0, c->err);
     c->pend = pc::Partials{nullptr, 0, 0, 0};
     if constexpr (std::is_same<T, float>::value) {
         const T* wlm = reinterpret_cast<const T*>(d.tied_embed ? c->embed : c->lm_head);
@@ -592,6 +592,14 @@ size_t pc_chain_trace_words(const pc_ctx* ctx) {
 }
 
 uint64_t pc_capture_count(const pc_ctx* ctx) { return ctx ? ctx->captures : 0; }
+
+int pc_selftest_wait_timeout(void* stream, uint32_t spin_limit, int32_t* dev_error_flag) {
+    if (dev_error_flag == nullptr || spin_limit == 0 || spin_limit > (1u << 20)) return PC_ERR_INVALID_ARG;
+    pc::tc::wait_timeout_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(spin_limit, dev_error_flag);
+    count_launches(1);
+    PC_CUDA_CHECK_LAUNCH("wait self-test");
+    return PC_OK;
+}
 
 int pc_set_index_bounds(pc_ctx* ctx, int n_prompts, int64_t n_tokens) {
     if (ctx == nullptr || n_prompts < 0 || n_tokens < 0) return PC_ERR_INVALID_ARG;

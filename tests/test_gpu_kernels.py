@@ -214,3 +214,28 @@ def test_dapo_and_grpo_modes_through_pc_allocate():
         assert np.array_equal(var > 0, keep == 1)
         st, ex, ev, nsel, tot = _alloc_gpu(cm, cn, 0.0, 1.0, 2.0, 0, P)          # GRPO: nothing filtered
         assert np.all(st == B.PC_STATUS_COMMIT) and nsel == P
+
+
+def test_bounded_wait_gives_up_and_the_context_stays_usable():
+    """A wait on an mbarrier nobody arrives at (no copy in flight) runs out after its limit, leaves DEV_ERR_WAIT_TIMEOUT in
+    the error flag and the kernel returns; the next launches work."""
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.pc_selftest_wait_timeout(1 << 10, flag)
+    torch.cuda.synchronize()
+    assert int(flag.item()) == 3
+    # the device is still usable: an ordinary entry point gives the right answer afterwards
+    tokens = _i32([5, 9, 100, 3, 7, 0])
+    last = torch.tensor([1, 2, 5, 3], dtype=torch.int64, device="cuda")
+    r = torch.zeros(4, dtype=torch.float32, device="cuda")
+    B.pc_reward_last_token(4, tokens, last, _i32([9, 101, 0, 4]), r)
+    assert r.cpu().tolist() == [0.0, 1.0, 0.0, 1.0]
+    with pytest.raises(B.PcError):
+        B.pc_selftest_wait_timeout(0, flag)
+
+
+def test_reward_of_a_never_generated_cell_is_zero():
+    tokens = _i32([-1, 4, -1])
+    last = torch.tensor([0, 1, 2], dtype=torch.int64, device="cuda")
+    r = torch.full((3,), 7.0, device="cuda")
+    B.pc_reward_last_token(3, tokens, last, _i32([10, 10, 10]), r)
+    assert r.cpu().tolist() == [0.0, 1.0, 0.0]

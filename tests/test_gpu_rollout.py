@@ -405,3 +405,31 @@ def test_new_schedules_and_token_buffers_reuse_the_captured_steps():
     eng.run_stage(sch_prompts, longest[1:])
     assert int(eng.err_flag.item()) == 4                             # DEV_ERR_GROUP_RANGE
     eng.err_flag.zero_()
+
+
+def test_half_operands_out_of_range_are_saturated_and_flagged():
+    """IEEE-half GEMM operands: with gate / up matrices scaled until the SwiGLU output passes 65504 the step still ends with
+    in-range tokens and the device error flag holds DEV_ERR_HALF_RANGE (5) -- no silent inf / NaN logits."""
+    model = wl.SMALL_BF16
+    w = dataclasses.replace(wl.WORKLOADS["config0"], model=model, n_prompts=2, prompt_len_lo=5, prompt_len_hi=20, group_size=4,
+                            n_pilot=4, max_new=6, cap_lo=3, cap_hi=6, data_seed=2, forced_explicit=None)
+    weights = wl.gen_weights(model, seed=1, threads=2)
+    weights.put("layers.0.w_gate", weights["layers.0.w_gate"] * 64.0, True)
+    weights.put("layers.0.w_up", weights["layers.0.w_up"] * 4096.0, True)
+    batch = wl.gen_batch(w)
+    eng = RolloutEngine(model, weights, max_rows=8, max_prefill_tokens=int(batch.prompt_offsets[-1]))
+    eng.load_batch(w, batch)
+    status, n_tok = eng.run_device()
+    torch.cuda.synchronize()
+    assert int(eng.err_flag.item()) == 5
+    toks = eng.tokens.cpu().numpy().reshape(w.n_prompts, w.group_size, w.max_new)
+    for p in range(w.n_prompts):
+        for i in range(w.group_size):
+            t = toks[p, i, :batch.caps[p, i]]
+            assert t.min() >= 0 and t.max() < model.vocab
+    assert torch.isfinite(eng.last_logits).all()
+    eng.err_flag.zero_()
+    # the same model inside the range raises nothing
+    weights2 = wl.gen_weights(model, seed=1, threads=2)
+    eng2 = RolloutEngine(model, weights2, max_rows=8, max_prefill_tokens=int(batch.prompt_offsets[-1]))
+    eng2.pilot_commit_step(w, batch)
