@@ -45,6 +45,16 @@ def load_peaks():
     return 6650.0, "fallback"
 
 
+def load_tensor_peaks():
+    """(burst, sustained) dense bf16 TFLOP/s: measured on this machine when the driver's file is there, else the earlier pool figures."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p.get("bf16_tflops", 1590.0)), float(p.get("bf16_tflops_sustained", 1400.0))
+    return 1590.0, 1400.0
+
+
 class ClockSampler(threading.Thread):
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -176,6 +186,47 @@ def run_probe(args):
           flush=True)
 
 
+def phase_table(eng, B, n_layers):
+    """Per-operation device time from the sampled decode steps: every sample holds the CUDA events pc_profile_step
+    recorded around the operations of one decoder layer and of the step's tail (LM head, sampler)."""
+    names = B.PROFILE_MARKS
+    ix = {n: i for i, n in enumerate(names)}
+    layer_ops = [("norm_attn", "layer_begin", "norm_attn"), ("qkv_gemm", "norm_attn", "qkv"), ("qkv_post", "qkv", "post"),
+                 ("attn_prefix", "post", "group"), ("attn_suffix", "group", "suffix"), ("attn_merge", "suffix", "merge"),
+                 ("o_gemm", "merge", "o"), ("norm_mlp", "o", "norm_mlp"), ("gate_up_gemm", "norm_mlp", "gate_up"),
+                 ("down_gemm", "gate_up", "down")]
+    tail_ops = [("lm_head", "lm_begin", "lm_head"), ("sampler", "lm_head", "sample")]
+    tot = {k: 0.0 for k, _, _ in layer_ops + tail_ops}
+    per_sample = []
+    for evs, nr, npos in eng.profile_samples:
+        d = {}
+        for k, a, b in layer_ops + tail_ops:
+            d[k] = evs[ix[a]].elapsed_time(evs[ix[b]])
+            tot[k] += d[k]
+        per_sample.append((d, nr, npos))
+    n = max(len(per_sample), 1)
+    # one sampled step stands for its neighbours: a layer operation runs n_layers times per step, a tail operation once
+    est = {k: tot[k] / n * (1 if k in ("lm_head", "sampler") else n_layers) for k in tot}
+    return per_sample, {k: tot[k] / n for k in tot}, est
+
+
+def composite_bound_seconds(m, rows_per_step_list, caps_by_stage, prompt_lens_by_stage, peak_gbs, peak_tflops):
+    """Lower bound of a run's decode time when every phase of every step runs at its own roofline:
+    GEMMs max(weight bytes / BW, flops / tensor peak), attention KV bytes / BW."""
+    bw, tf = peak_gbs * 1e9, peak_tflops * 1e12
+    w_bytes = m.weight_bytes_per_decode_step()
+    params = w_bytes / m.elem_bytes
+    t_gemm = t_attn = 0.0
+    for rows_per_step, caps, plens in zip(rows_per_step_list, caps_by_stage, prompt_lens_by_stage):
+        rows = rows_per_step.astype(np.float64)
+        t_gemm += float(np.sum(np.maximum(w_bytes / bw, 2.0 * rows * params / tf)))
+        caps = caps.astype(np.float64)
+        suffix_tok = float(np.sum((caps - 1) * caps / 2.0))
+        prompt_tok = float(np.sum(plens))                       # prompt KV read once per group per step: sum over (group, step)
+        t_attn += (suffix_tok + prompt_tok) * m.kv_bytes_per_token / bw
+    return t_gemm, t_attn
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -184,15 +235,13 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="config2", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--also-bound", action="store_true",
-                    help="additionally time one bound pass (Section 3.4): the commit rollouts of the timed batch's survivors and the "
-                         "pilot rollouts of a second batch in one decode batch; reported as bound_pass")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the additional single-step measurements reported beside the main one: grpo_mode (all P*G rollouts "
+                         "concurrent), loop_bound (Algorithm 1 as a running loop with bound passes, Section 3.4), bf16_operands")
     ap.add_argument("--also-logprobs", action="store_true",
                     help="additionally time one step that also keeps the behaviour log-probability of every sampled token (Eq. 2's "
                          "denominator); reported as with_logprobs")
-    ap.add_argument("--also-grpo", action="store_true",
-                    help="additionally time one step with k = G (all P*G rollouts concurrent, no filter) and report it as grpo_mode")
-    ap.add_argument("--probe", default=None, metavar="rows=R,suffix=S,steps=N,prompt=L",
+    ap.add_argument("--probe", default=None, metavar="rows=R,suffix=S,steps=N,prompt=L,mode=M",
                     help="time N decode steps of R rollouts (16 groups) that already hold S suffix tokens, then exit")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -217,6 +266,7 @@ def main():
     P, G, k = w.n_prompts, w.group_size, w.n_pilot
     weights = wl.gen_weights(w.model, seed=0)
     batch = wl.gen_batch(w)
+    m = w.model
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:       # before the first GPU call
@@ -234,55 +284,47 @@ def main():
                 "status": torch.empty(P, dtype=torch.int32).pin_memory()}
     d2h_bytes = sum(t.numel() * t.element_size() for t in host_out.values())
 
-    def one_step(timed: bool):
+    def one_step(engine):
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
         ev[0].record()
-        eng.load_batch(w, batch, host_inputs)          # host -> device copies of this step's inputs
+        engine.load_batch(engine_wl[engine], batch, host_inputs)          # host -> device copies of this step's inputs
         ev[1].record()
-        status, n_tok = eng.run_device()
+        status, n_tok = engine.run_device()
         ev[2].record()
-        host_out["tokens"].copy_(eng.tokens, non_blocking=True)
-        host_out["rewards"].copy_(eng.rewards, non_blocking=True)
-        host_out["adv"].copy_(eng.adv, non_blocking=True)
-        host_out["status"].copy_(eng.status, non_blocking=True)
+        host_out["tokens"].copy_(engine.tokens, non_blocking=True)
+        host_out["rewards"].copy_(engine.rewards, non_blocking=True)
+        host_out["adv"].copy_(engine.adv, non_blocking=True)
+        host_out["status"].copy_(engine.status, non_blocking=True)
         ev[3].record()
         torch.cuda.synchronize()
-        eng.check_error_flag()
+        engine.check_error_flag()
         return n_tok, ev[1].elapsed_time(ev[2]), ev[0].elapsed_time(ev[3]), status
 
+    engine_wl = {eng: w}
+    eng.profile_every = 32                           # warm-up and timed steps take the same path
     for _ in range(args.warmup):
-        one_step(False)
-    eng.profile_every = 32
+        one_step(eng)
     eng.profile_samples = []
+    eng.stage_rows_per_step = []
     sampler = ClockSampler(local_rank)
     sampler.start()
     dist_util.barrier()
     torch.cuda.synchronize()
-    launches0 = B.pc_launch_count()
-    dev_ms, e2e_ms, tokens, status = 0.0, 0.0, 0, None
+    launches0, captures0 = B.pc_launch_count(), B.pc_capture_count(eng.ctx)
+    dev_ms, e2e_ms, tokens, status, prefill_ms = 0.0, 0.0, 0, None, 0.0
     for _ in range(args.steps):
-        n_tok, d, e, status = one_step(True)
+        n_tok, d, e, status = one_step(eng)
         dev_ms += d; e2e_ms += e; tokens += n_tok
+        prefill_ms += eng.prefill_events[0].elapsed_time(eng.prefill_events[1])
     torch.cuda.synchronize()
     dist_util.barrier()
     launches = B.pc_launch_count() - launches0
+    captures = B.pc_capture_count(eng.ctx) - captures0
     clocks = sampler.stop()
-
-    # roofline of the dominant kernel (suffix attention): algorithmic bytes of the sampled launches / their duration
-    m = w.model
-    per_pos = 2 * m.n_kv_heads * m.head_dim * m.elem_bytes                 # K and V of one position, one layer
-    per_row = 2 * m.n_q_heads * m.head_dim * m.elem_bytes                  # q read + output written
-    s_bytes = sum(nr * (npos * per_pos + per_row) for (_, _, nr, npos) in eng.profile_samples)
-    s_ms = sum(e0.elapsed_time(e1) for (e0, e1, _, _) in eng.profile_samples)
     peak, peak_kind = load_peaks()
-    achieved = s_bytes / (s_ms * 1e-3) / 1e9 if s_ms > 0 else 0.0
-    n_samp = max(len(eng.profile_samples), 1)
-    roofline = {"bound": "hbm", "kernel": "attn_suffix_kernel", "achieved": achieved, "peak": peak, "peak_kind": peak_kind,
-                "unit": "GB/s", "frac": achieved / peak,
-                "traffic": SUFFIX_TRAFFIC_PER_ALGORITHMIC_BYTE * s_bytes / n_samp, "traffic_note": "ncu capture of a smaller case scaled by algorithmic bytes", "launches_sampled": len(eng.profile_samples),
-                "avg_launch_ms": s_ms / n_samp, "avg_algorithmic_bytes": s_bytes / n_samp}
+    tf_burst, tf_sustained = load_tensor_peaks()
 
-    # whole-step HBM roofline named by the metric: (weight bytes + KV bytes) each decode step must move / peak
+    # ---- what the decode steps of this Pilot-Commit step must move (the HBM roofline the metric names)
     caps = batch.caps.astype(np.int64)
     gen = np.zeros((P, G), dtype=bool); gen[:, :k] = True; gen[status == B.PC_STATUS_COMMIT, :] = True
     kv_tok = m.kv_bytes_per_token
@@ -291,14 +333,52 @@ def main():
     steps_commit = int(caps[commit_rows].max() - 1) if commit_rows.any() else 0
     suffix_reads = float(np.sum((caps[gen] - 1) * caps[gen] / 2.0)) * kv_tok           # sum over steps of (s + 1) per rollout
     prompt_reads = 0.0
+    prompt_tok_by_stage = []
     for stage_rows, n_st in ((np.pad(gen[:, :k], ((0, 0), (0, G - k))), steps_pilot), (commit_rows, steps_commit)):
+        tok = 0.0
         for p in range(P):
             c = caps[p][stage_rows[p]]
             if c.size:
-                prompt_reads += float(c.max() - 1) * float(batch.prompt_lens[p]) * kv_tok   # once per group per step
+                tok += float(c.max() - 1) * float(batch.prompt_lens[p])             # once per group per step
+        prompt_tok_by_stage.append(np.array([tok]))
+        prompt_reads += tok * kv_tok
     weight_reads = float(steps_pilot + steps_commit) * m.weight_bytes_per_decode_step()
     kv_writes = float(np.sum(caps[gen] - 1)) * kv_tok
     step_bytes = suffix_reads + prompt_reads + weight_reads + kv_writes
+    decode_ms = dev_ms - prefill_ms
+    achieved_step = step_bytes * args.steps / (decode_ms * 1e-3) / 1e9
+
+    # ---- per-operation time from the sampled steps; roofline figures of the two heaviest kernel families
+    per_sample, per_op_ms, est_ms = phase_table(eng, B, m.n_layers)
+    per_pos = 2 * m.n_kv_heads * m.head_dim * m.elem_bytes                 # K and V of one position, one layer
+    per_row = 2 * m.n_q_heads * m.head_dim * m.elem_bytes                  # q read + output written
+    s_bytes = sum(nr * (npos * per_pos + per_row) for (_, nr, npos) in per_sample)
+    s_ms = sum(d["attn_suffix"] for (d, _, _) in per_sample)
+    n_samp = max(len(per_sample), 1)
+    layer_w_bytes = m.layer_params() * m.elem_bytes
+    g_ms = sum(d["qkv_gemm"] + d["o_gemm"] + d["gate_up_gemm"] + d["down_gemm"] for (d, _, _) in per_sample)
+    g_flops = sum(2.0 * nr * m.layer_params() for (_, nr, _) in per_sample)
+    g_bound_s = sum(max(layer_w_bytes / (peak * 1e9), 2.0 * nr * m.layer_params() / (tf_burst * 1e12)) for (_, nr, _) in per_sample)
+    kernels = {
+        "attn_suffix_kernel": {"bound": "hbm", "achieved": s_bytes / (s_ms * 1e-3) / 1e9 if s_ms > 0 else 0.0, "peak": peak, "unit": "GB/s",
+                               "frac": (s_bytes / (s_ms * 1e-3) / 1e9 / peak) if s_ms > 0 else 0.0,
+                               "traffic": SUFFIX_TRAFFIC_PER_ALGORITHMIC_BYTE * s_bytes / n_samp,
+                               "traffic_note": "ncu capture of a smaller case scaled by algorithmic bytes (profiles/attn_suffix_kernel_ncu.md)",
+                               "avg_launch_ms": s_ms / n_samp, "avg_algorithmic_bytes": s_bytes / n_samp},
+        "gemm_tc_kernel (QKV, O, gate/up, down of one layer)": {
+            "bound": "hbm below about %d rows, tensor above" % int(tf_burst * 1e12 / (peak * 1e9) / 2 * m.elem_bytes),
+            "avg_ms_per_layer": g_ms / n_samp, "weight_gbs": layer_w_bytes * n_samp / (g_ms * 1e-3) / 1e9 if g_ms > 0 else 0.0,
+            "weight_frac_of_hbm_peak": (layer_w_bytes * n_samp / (g_ms * 1e-3) / 1e9 / peak) if g_ms > 0 else 0.0,
+            "tflops": g_flops / (g_ms * 1e-3) / 1e12 if g_ms > 0 else 0.0,
+            "tensor_frac_of_bf16_burst": (g_flops / (g_ms * 1e-3) / 1e12 / tf_burst) if g_ms > 0 else 0.0,
+            "frac_of_own_bound": g_bound_s / (g_ms * 1e-3) if g_ms > 0 else 0.0, "traffic": None},
+    }
+    stage_rows = eng.stage_rows_per_step[-2:] if len(eng.stage_rows_per_step) >= 2 else eng.stage_rows_per_step
+    stage_caps = [caps[:, :k].reshape(-1), caps[commit_rows]][:len(stage_rows)]
+    t_gemm_b, t_attn_b = composite_bound_seconds(m, stage_rows, stage_caps, prompt_tok_by_stage, peak, tf_burst)
+    all_rows = np.concatenate(stage_rows) if stage_rows else np.zeros(0)
+    hist_edges = [0, 16, 32, 64, 128, 192, 256, 384, 512, 1024, 2048, 4096]
+    live_hist = {f"{a + 1}-{b}": int(np.sum((all_rows > a) & (all_rows <= b))) for a, b in zip(hist_edges[:-1], hist_edges[1:])}
 
     t_ms, n_tokens = dist_util.aggregate(dev_ms, tokens, device=dev)
     t_e2e, _ = dist_util.aggregate(e2e_ms, tokens, device=dev)
@@ -320,69 +400,100 @@ def main():
         "clocks": clocks,
         "e2e": {"value": n_tokens / (t_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d_bytes, "d2h_bytes_per_step": d2h_bytes},
         "gpu_launches": int(launches),
-        "roofline": roofline,
+        "graph_captures_in_timed_region": int(captures),
+        # the quantity the metric names: bytes every decode step of the job must move (weights + KV) over the decode time
+        "roofline": {"bound": "hbm", "kernel": "decode steps of the Pilot-Commit step, all kernels (prefill excluded)",
+                     "achieved": achieved_step, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved_step / peak,
+                     "frac_of_8tbs": achieved_step / 8000.0, "traffic": None,
+                     "bytes_per_step": step_bytes, "decode_ms_per_step": decode_ms / max(args.steps, 1),
+                     "parts": {"suffix_kv_read": suffix_reads, "prompt_kv_read": prompt_reads, "weights": weight_reads, "kv_write": kv_writes},
+                     "target": 0.60},
+        "composite_bound": {"note": "sum over decode steps of max(weight bytes / HBM peak, flops / bf16 burst peak) for the GEMMs plus KV bytes / HBM peak",
+                            "gemm_bound_s": t_gemm_b, "attention_bound_s": t_attn_b,
+                            "frac": (t_gemm_b + t_attn_b) / (decode_ms * 1e-3 / max(args.steps, 1)) if decode_ms > 0 else 0.0},
+        "kernels": kernels,
+        "phase_ms": {"prefill_per_step": prefill_ms / max(args.steps, 1),
+                     "sampled_decode_steps": len(per_sample), "per_launch_avg": per_op_ms,
+                     "estimated_per_decode_step": est_ms,
+                     "note": "CUDA events around the operations of layer %d and the LM head / sampler in every 32nd decode step; "
+                             "a layer operation is counted n_layers times" % eng.profile_layer},
+        "live_rows_histogram": live_hist,
         "hbm_step": {"bytes_per_step": step_bytes, "achieved_gbs": step_bytes * args.steps / (dev_ms * 1e-3) / 1e9,
                      "frac_of_measured": step_bytes * args.steps / (dev_ms * 1e-3) / 1e9 / peak,
                      "frac_of_8tbs": step_bytes * args.steps / (dev_ms * 1e-3) / 1e9 / 8000.0,
-                     "parts": {"suffix_kv_read": suffix_reads, "prompt_kv_read": prompt_reads, "weights": weight_reads,
-                               "kv_write": kv_writes}},
+                     "note": "as above with the prefill inside the time"},
     }
     if cpu_baseline is not None:
         line["cpu_baseline"] = cpu_baseline
+    kv_tok_f = float(kv_tok)
     if args.also_logprobs and world == 1:
         eng.profile_every = 0
         eng.collect_logprobs = True
-        one_step(False)                                       # buffers and graphs of this mode
-        n_tok, d_ms, _, _ = one_step(True)
+        one_step(eng)                                         # buffers and graphs of this mode
+        n_tok, d_ms, _, _ = one_step(eng)
         eng.collect_logprobs = False
         line["with_logprobs"] = {"tokens": n_tok, "ms_per_step": d_ms, "tokens_per_s": n_tok / (d_ms * 1e-3),
                                  "step_time_ratio": d_ms / (t_ms / max(args.steps, 1))}
-    if args.also_bound and world == 1:
-        # steady state of Section 3.4: batch A's pilot pass has just run on this engine (the timed step leaves A's prompt KV,
-        # last-position logits and statuses in place); one pass then generates A's commit rollouts and B's pilot rollouts
-        eng.profile_every = 0
-        wb = dataclasses.replace(w, data_seed=w.data_seed + 1000)
-        batch_b = wl.gen_batch(wb)
-        commit_a = np.flatnonzero(status == B.PC_STATUS_COMMIT)
-        times = []
-        for rep in range(2):                                   # first repetition: graphs and allocator
-            eng.load_batch(w, batch)
-            eng.run_device()
-            torch.cuda.synchronize()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            out_b = eng.bound_pass(w, batch, commit_a, batch_b)
-            e1.record()
-            torch.cuda.synchronize()
-            times.append(e0.elapsed_time(e1))
-        n_tok_b = int(sum(len(t) for t in out_b["a"].values()) + sum(len(t) for t in out_b["b"].values()))
-        rows_b = len(commit_a) * (G - k) + P * k
-        line["bound_pass"] = {"rows": rows_b, "commit_prompts_of_previous_batch": int(len(commit_a)), "pilot_prompts": P, "tokens": n_tok_b,
-                              "ms_per_pass": times[-1], "tokens_per_s": n_tok_b / (times[-1] * 1e-3),
-                              "note": "prefill of the new batch, decode of both row sets and the read-back of the tokens included"}
-    if args.also_grpo and world == 1:
-        # every rollout of every group at once (what plain GRPO generates for the same prompts): same kernels, k = G
-        wg = dataclasses.replace(w, n_pilot=G)
+    if not args.no_extras and world == 1:
+        eng._arenas.clear()
+        eng.prompt_kv = eng.suffix_kv = None
         del eng
         torch.cuda.empty_cache()
+        # (1) every rollout of every group at once (what plain GRPO generates for the same prompts): same kernels, k = G
+        wg = dataclasses.replace(w, n_pilot=G)
         eng2 = RolloutEngine(wg.model, weights, max_rows=P * G, max_prefill_tokens=total_prompt, device=dev)
-        eng2.load_batch(wg, batch)
-        eng2.run_device()                       # warm-up (graph capture, allocator)
-        torch.cuda.synchronize()
-        eng2.load_batch(wg, batch)
+        engine_wl[eng2] = wg
+        one_step(eng2)                           # warm-up (graph capture, allocator)
+        n_tok, ms, _, _ = one_step(eng2)
+        cg = batch.caps.astype(np.float64)
+        b = (float(np.sum((cg - 1) * cg / 2.0)) + float(np.sum(cg - 1))) * kv_tok_f \
+            + float(sum((batch.caps[p].max() - 1) * batch.prompt_lens[p] for p in range(P))) * kv_tok_f \
+            + float(batch.caps.max() - 1) * m.weight_bytes_per_decode_step()
+        tg, ta = composite_bound_seconds(m, eng2.stage_rows_per_step[-1:], [batch.caps.reshape(-1)],
+                                         [np.array([float(sum((batch.caps[p].max() - 1) * batch.prompt_lens[p] for p in range(P)))])],
+                                         peak, tf_burst)
+        line["grpo_mode"] = {"rows": P * G, "tokens": n_tok, "ms_per_step": ms, "tokens_per_s": n_tok / (ms * 1e-3),
+                             "hbm_bytes_per_step": b, "hbm_frac_of_measured": b / (ms * 1e-3) / 1e9 / peak,
+                             "composite_bound_frac": (tg + ta) / (ms * 1e-3)}
+        eng2._arenas.clear()
+        eng2.prompt_kv = eng2.suffix_kv = None
+        del eng2
+        torch.cuda.empty_cache()
+        # (2) Algorithm 1 as a running loop with bound passes (Section 3.4): three sampling batches, each pass holding the pilot
+        #     rollouts of a new batch and the commit rollouts of the previous batch's survivors on their resident prompt KV
+        from paper_2605_26606_b200.loop import RolloutLoop
+        n_b = 3
+        wd = dataclasses.replace(w, n_prompts=n_b * P)
+        data = wl.gen_batch(wd)
+        eng3 = RolloutEngine(w.model, weights, max_rows=P * k + P * (G - k), max_prefill_tokens=int(data.prompt_lens.max()) * P, device=dev)
+        loop = RolloutLoop(eng3, w, data, b_g=P, b_t=P, max_delay=1, bind=True, max_resident_prompts=3 * P)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        _, n_tok = eng2.run_device()
+        recs = loop.run(list(range(n_b * P)), 1)
         e1.record()
         torch.cuda.synchronize()
-        eng2.check_error_flag()
         ms = e0.elapsed_time(e1)
-        cg = batch.caps.astype(np.float64)
-        b = (float(np.sum((cg - 1) * cg / 2.0)) + float(np.sum(cg - 1))) * kv_tok \
-            + float(sum((batch.caps[p].max() - 1) * batch.prompt_lens[p] for p in range(P))) * kv_tok \
-            + float(batch.caps.max() - 1) * m.weight_bytes_per_decode_step()
-        line["grpo_mode"] = {"rows": P * G, "tokens": n_tok, "ms_per_step": ms, "tokens_per_s": n_tok / (ms * 1e-3),
-                             "hbm_bytes_per_step": b, "hbm_frac_of_measured": b / (ms * 1e-3) / 1e9 / peak}
+        n_tok = int(sum(len(t) for r in recs for t in r.tokens.values()))
+        line["loop_bound"] = {"training_steps": len(recs), "passes": int(sum(r.passes for r in recs)), "sampling_batch": P, "b_t": P,
+                              "committed_per_step": [len(r.plan.committed) for r in recs],
+                              "rollouts_sampled_per_step": [r.plan.rollouts_sampled for r in recs],
+                              "second_round_share": float(np.mean([r.plan.rounds > 1 for r in recs])),
+                              "tokens": n_tok, "ms_total": ms, "tokens_per_s": n_tok / (ms * 1e-3),
+                              "note": "prefills, decode passes, statistics, allocation, advantages and the read-back of every rollout included; "
+                                      "the first pass has no commit rows and the last no pilot rows"}
+        eng3._arenas.clear()
+        eng3.prompt_kv = eng3.suffix_kv = None
+        del eng3, loop
+        torch.cuda.empty_cache()
+        # (3) the main step with bfloat16 GEMM operands (value + rounding remainder for QKV / O / LM head) instead of IEEE half
+        if m.dtype == wl.DTYPE_BF16:
+            eng4 = RolloutEngine(w.model, weights, max_rows=max(P * k, P * (G - k), 1), max_prefill_tokens=total_prompt, device=dev,
+                                 half_gemm=False)
+            engine_wl[eng4] = w
+            one_step(eng4)
+            n_tok, ms, _, st4 = one_step(eng4)
+            line["bf16_operands"] = {"tokens": n_tok, "ms_per_step": ms, "tokens_per_s": n_tok / (ms * 1e-3),
+                                     "committed_prompts": int((st4 == B.PC_STATUS_COMMIT).sum())}
     print(json.dumps(line), flush=True)
 
 

@@ -75,7 +75,8 @@ enum {
     PC_STATUS_COMMIT = 0,      /* passed the filter and received n_commit more rollouts          */
     PC_STATUS_BUFFERED = 1,    /* passed the filter but b_t prompts were already selected         */
     PC_STATUS_DEFER_HARD = 2,  /* p_hat < p_lower                                                */
-    PC_STATUS_SKIP_EASY = 3    /* p_hat > p_upper                                                */
+    PC_STATUS_SKIP_EASY = 3,   /* p_hat > p_upper                                                */
+    PC_STATUS_LOW_VARIANCE = 4 /* pc_allocate_variance: pilot reward variance below the threshold */
 };
 
 typedef struct pc_ctx pc_ctx;
@@ -206,11 +207,21 @@ PC_API int pc_set_decode_mode(pc_ctx* ctx, int mode);
 PC_API int pc_set_chain_trace(pc_ctx* ctx, int64_t* trace, size_t n_words);
 PC_API size_t pc_chain_trace_words(const pc_ctx* ctx);
 
-/* Measurement aid: in the next pc_decode_step of this context, record the two CUDA events (cudaEvent_t,
- * created by the caller) around the attention kernel of `layer` that reads the rollouts' own suffix K/V
- * (for float32 models: the single attention kernel).  One-shot; the caller synchronises and reads the
- * elapsed time.  The paper has no counterpart. */
-PC_API int pc_profile_attention(pc_ctx* ctx, int layer, void* event_start, void* event_stop);
+/* Measurement aid: the next pc_decode_step of this context (issued outside any capture, one kernel per operation)
+ * records the PC_PROFILE_MARKS CUDA events (cudaEvent_t with timing, created by the caller; NULL entries are skipped) at
+ * the boundaries of the operations of decoder layer `layer` and of the step's tail, in stream order:
+ *   LAYER_BEGIN | attention RMSNorm | NORM_ATTN | QKV GEMM | QKV | bias / QK-norm / RoPE / KV append | POST |
+ *   shared-prefix attention | GROUP | per-rollout suffix attention | SUFFIX | merge | MERGE | output projection | O |
+ *   MLP RMSNorm | NORM_MLP | gate/up GEMM + SwiGLU | GATE_UP | down projection | DOWN   ... (other layers) ...
+ *   LM_BEGIN | final RMSNorm + LM head | LM_HEAD | sampler | SAMPLE
+ * so the time of an operation is the elapsed time between the marks around it.  One-shot; the caller synchronises
+ * and reads the times.  float32 models run one attention kernel: GROUP is recorded before it, SUFFIX and MERGE after
+ * it.  The paper has no counterpart. */
+enum {
+    PC_MARK_LAYER_BEGIN = 0, PC_MARK_NORM_ATTN, PC_MARK_QKV, PC_MARK_POST, PC_MARK_GROUP, PC_MARK_SUFFIX, PC_MARK_MERGE, PC_MARK_O,
+    PC_MARK_NORM_MLP, PC_MARK_GATE_UP, PC_MARK_DOWN, PC_MARK_LM_BEGIN, PC_MARK_LM_HEAD, PC_MARK_SAMPLE, PC_PROFILE_MARKS
+};
+PC_API int pc_profile_step(pc_ctx* ctx, int layer, void* const* events, int n_events);
 
 /* Shared prefill (Section 3.1: o ~ pi_theta(. | q); Section 3.3: pilot and commit rollouts of a
  * prompt are drawn from the same pi_theta(. | q), so q is evaluated once).
@@ -346,6 +357,17 @@ PC_API int pc_group_stats(void* stream, int n_groups, const float* rewards, cons
 PC_API int pc_allocate(void* stream, int n_prompts, const int32_t* pilot_success, const int32_t* pilot_n,
                 const pc_alloc_params* params, int32_t* status, int32_t* extra_rollouts, int32_t* evict,
                 int32_t* n_selected, int64_t* total_rollouts);
+
+/* The pilot filter for rewards that are not binary.  Section 3.3 motivates the filter by reward variance (for binary
+ * rewards Var = p (1 - p), so p_hat is its proxy) and states that the method applies to any scalar reward; it gives no
+ * formula for that case.  Reading taken here: keep a prompt iff the population variance of its pilot rewards (Eq. 3,
+ * the float value pc_group_stats returns, compared in double) is at least var_min; the first b_t kept prompts in batch
+ * order get status COMMIT and extra_rollouts = n_commit, later ones BUFFERED, the others PC_STATUS_LOW_VARIANCE.  There
+ * is no eviction rule in this mode.  For binary rewards and thresholds symmetric about 1/2 it decides exactly like
+ * pc_allocate with var_min = p_lower (1 - p_lower).  Outputs as pc_allocate's (no evict array). */
+PC_API int pc_allocate_variance(void* stream, int n_prompts, const float* pilot_var, const int32_t* pilot_n, double var_min,
+                                int n_commit, int b_t, int32_t* status, int32_t* extra_rollouts, int32_t* n_selected,
+                                int64_t* total_rollouts);
 
 /* Group-relative advantage A_i = (r_i - mu) / sigma (Section 3.1) over group g =
  * rewards[group_start[g] : +group_count[g]]; 0 when all rewards of the group are equal, and

@@ -26,7 +26,7 @@ from __future__ import annotations
 
 import numpy as np
 
-COMMIT, BUFFERED, DEFER_HARD, SKIP_EASY = 0, 1, 2, 3
+COMMIT, BUFFERED, DEFER_HARD, SKIP_EASY, LOW_VARIANCE = 0, 1, 2, 3, 4
 
 
 def group_stats(rewards: np.ndarray, start: np.ndarray, count: np.ndarray):
@@ -118,3 +118,27 @@ def dapo_filter(rewards: np.ndarray, start: np.ndarray, count: np.ndarray) -> np
         r = np.asarray(rewards[start[g]:start[g] + count[g]], dtype=np.float64)
         keep[g] = 1 if r.shape[0] > 0 and np.max(r) != np.min(r) else 0
     return keep
+
+
+def allocate_by_variance(pilot_var, pilot_n, var_min: float, n_commit: int, b_t: int):
+    """The pilot filter for general scalar rewards.  Section 3.3 argues from reward variance (Var = p (1 - p) for binary
+    rewards, p_hat being its proxy) and says the method applies to any scalar reward signal, without a formula for that
+    case.  Reading: keep iff the population variance of the pilot rewards (Eq. 3) is at least var_min; the variance is
+    taken in single precision, the precision in which the statistics are reported, and compared in double.  The first
+    b_t kept prompts in batch order commit, later ones are BUFFERED, the others LOW_VARIANCE.
+    Returns status, extra_rollouts, n_selected, total_rollouts."""
+    P = len(pilot_var)
+    status = np.zeros(P, dtype=np.int32)
+    extra = np.zeros(P, dtype=np.int32)
+    selected = 0
+    for p in range(P):
+        if pilot_n[p] > 0 and float(np.float32(pilot_var[p])) >= var_min:
+            if selected < b_t:
+                status[p], extra[p] = COMMIT, n_commit
+                selected += 1
+            else:
+                status[p] = BUFFERED
+        else:
+            status[p] = LOW_VARIANCE
+    total = int(np.sum(np.asarray(pilot_n, dtype=np.int64))) + selected * int(n_commit)
+    return status, extra, selected, total

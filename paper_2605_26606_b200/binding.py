@@ -20,11 +20,11 @@ PC_OK = 0
 PC_ERR_INVALID_ARG, PC_ERR_SHAPE, PC_ERR_ALIGNMENT, PC_ERR_CAPACITY = 1, 2, 3, 4
 PC_ERR_UNSUPPORTED, PC_ERR_CUDA, PC_ERR_NO_WORKSPACE = 5, 6, 7
 PC_DTYPE_F32, PC_DTYPE_BF16 = 0, 1
-PC_STATUS_COMMIT, PC_STATUS_BUFFERED, PC_STATUS_DEFER_HARD, PC_STATUS_SKIP_EASY = 0, 1, 2, 3
+PC_STATUS_COMMIT, PC_STATUS_BUFFERED, PC_STATUS_DEFER_HARD, PC_STATUS_SKIP_EASY, PC_STATUS_LOW_VARIANCE = 0, 1, 2, 3, 4
 
-EXPORTS = ["pc_status_string", "pc_last_cuda_error", "pc_launch_count", "pc_profile_attention", "pc_set_gemm_plan", "pc_set_decode_mode", "pc_set_chain_trace", "pc_chain_trace_words", "pc_capture_count", "pc_set_index_bounds", "pc_selftest_wait_timeout", "pc_create", "pc_destroy", "pc_workspace_bytes",
+EXPORTS = ["pc_status_string", "pc_last_cuda_error", "pc_launch_count", "pc_profile_step", "pc_set_gemm_plan", "pc_set_decode_mode", "pc_set_chain_trace", "pc_chain_trace_words", "pc_capture_count", "pc_set_index_bounds", "pc_selftest_wait_timeout", "pc_create", "pc_destroy", "pc_workspace_bytes",
            "pc_set_workspace", "pc_prefill_shared", "pc_decode_step", "pc_decode_run", "pc_sample", "pc_sample_static", "pc_token_logprob", "pc_set_logprob_buffer", "pc_set_prompt_keys", "pc_reward_last_token",
-           "pc_group_stats", "pc_allocate", "pc_grpo_advantage"]
+           "pc_group_stats", "pc_allocate", "pc_allocate_variance", "pc_grpo_advantage"]
 
 
 class ModelDesc(C.Structure):
@@ -78,7 +78,7 @@ def _lib():
         lib.pc_last_cuda_error.restype = C.c_char_p
         lib.pc_launch_count.restype = C.c_uint64
         lib.pc_launch_count.argtypes = []
-        lib.pc_profile_attention.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
+        lib.pc_profile_step.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_void_p), C.c_int]
         lib.pc_set_gemm_plan.argtypes = [C.c_void_p, C.c_char_p]
         lib.pc_set_decode_mode.argtypes = [C.c_void_p, C.c_int]
         lib.pc_capture_count.argtypes = [C.c_void_p]
@@ -106,6 +106,7 @@ def _lib():
         lib.pc_group_stats.argtypes = [p, i, p, p, p, p, p, p, p]
         lib.pc_allocate.argtypes = [p, i, p, p, C.POINTER(AllocParams), p, p, p, p, p]
         lib.pc_grpo_advantage.argtypes = [p, i, p, p, p, p, p]
+        lib.pc_allocate_variance.argtypes = [p, i, p, p, C.c_double, i, i, p, p, p, p]
         for name in EXPORTS[3:]:
             if name not in ("pc_destroy", "pc_chain_trace_words", "pc_capture_count"):
                 getattr(lib, name).restype = C.c_int
@@ -179,9 +180,14 @@ def pc_set_chain_trace(ctx: "Context", trace: Optional[torch.Tensor]) -> None:
     ctx._keep.append(trace)
 
 
-def pc_profile_attention(ctx: "Context", layer: int, event_start: torch.cuda.Event, event_stop: torch.cuda.Event) -> None:
-    """The events must have been created with enable_timing=True and recorded once (so that they exist)."""
-    _check(_lib().pc_profile_attention(ctx.handle, layer, event_start.cuda_event, event_stop.cuda_event), "pc_profile_attention")
+PROFILE_MARKS = ["layer_begin", "norm_attn", "qkv", "post", "group", "suffix", "merge", "o", "norm_mlp", "gate_up", "down", "lm_begin",
+                 "lm_head", "sample"]
+
+
+def pc_profile_step(ctx: "Context", layer: int, events: Sequence[torch.cuda.Event]) -> None:
+    """events: len(PROFILE_MARKS) events created with enable_timing=True and recorded once (so that they exist)."""
+    arr = (C.c_void_p * len(events))(*[e.cuda_event for e in events])
+    _check(_lib().pc_profile_step(ctx.handle, layer, arr, len(events)), "pc_profile_step")
 
 
 class Context:
@@ -318,6 +324,13 @@ def pc_allocate(n_prompts, pilot_success, pilot_n, params: AllocParams, status, 
                               C.byref(params), _ptr(status, torch.int32), _ptr(extra_rollouts, torch.int32),
                               _ptr(evict, torch.int32), _ptr(n_selected, torch.int32), _ptr(total_rollouts, torch.int64)),
            "pc_allocate")
+
+
+def pc_allocate_variance(n_prompts, pilot_var, pilot_n, var_min: float, n_commit: int, b_t: int, status, extra_rollouts, n_selected,
+                         total_rollouts) -> None:
+    _check(_lib().pc_allocate_variance(_stream(), n_prompts, _ptr(pilot_var, torch.float32), _ptr(pilot_n, torch.int32), var_min,
+                                       n_commit, b_t, _ptr(status, torch.int32), _ptr(extra_rollouts, torch.int32),
+                                       _ptr(n_selected, torch.int32), _ptr(total_rollouts, torch.int64)), "pc_allocate_variance")
 
 
 def pc_grpo_advantage(n_groups, rewards, group_start, group_count, status, adv) -> None:

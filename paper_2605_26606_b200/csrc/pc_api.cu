@@ -102,9 +102,13 @@ struct pc_ctx {
     // TMA descriptors of the KV arenas, rebuilt when a call brings another arena
     const void* prompt_arena_ptr = nullptr; int64_t prompt_arena_slots = -1; CUtensorMap map_prompt_kv;
     const void* suffix_arena_ptr = nullptr; int64_t suffix_arena_slots = -1; CUtensorMap map_suffix_kv;
-    // one-shot profiling request (pc_profile_attention)
-    int prof_layer = -1;
-    cudaEvent_t prof_start = nullptr, prof_stop = nullptr;
+    // one-shot profiling request (pc_profile_step): events recorded at the phase boundaries of one layer and of the step's tail
+    int prof_layer = -1;                     // armed when >= 0
+    int prof_active_layer = -1;              // the step being issued records into prof_ev
+    cudaEvent_t prof_ev[PC_PROFILE_MARKS] = {};
+    void mark(cudaStream_t st, int layer, int m) {      // layer < 0: a boundary of the step's tail (LM head, sampler)
+        if (prof_active_layer >= 0 && (layer < 0 || layer == prof_active_layer) && prof_ev[m] != nullptr) cudaEventRecord(prof_ev[m], st);
+    }
     float* logprobs = nullptr;       // pc_set_logprob_buffer
     const int32_t* prompt_key = nullptr;    // pc_set_prompt_keys
 
@@ -328,7 +332,7 @@ cudaError_t configure_kernels() {
 // part_out != nullptr: the records are left unmerged and described there (the caller merges them).
 template <int HD>
 int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, int layer, const AttnPlan& plan, pc::KvArena prompt_arena,
-                   pc::KvArena suffix_arena, const __nv_bfloat16* q, __nv_bfloat16* attn, bool profile,
+                   pc::KvArena suffix_arena, const __nv_bfloat16* q, __nv_bfloat16* attn,
                    pc::am::PrefixPartial* part_out = nullptr) {
     using namespace pc;
     const pc_model_desc& d = c->d;
@@ -360,16 +364,17 @@ int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, in
     am::attn_group_kernel<HD, false><<<ggrid, am::G_THREADS, am::group_smem_bytes<HD>(), st>>>(
         c->map_prompt_kv, sd, prompt_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, plan.group_row_start, g, scale_log2, part,
         attn, attn_lo, c->err);
-    if (profile) cudaEventRecord(c->prof_start, st);
+    c->mark(st, layer, PC_MARK_GROUP);
     am::attn_suffix_kernel<HD><<<sgrid, am::S_WARPS * 32, am::suffix_smem_bytes<HD>(), st>>>(
         c->map_suffix_kv, sd, suffix_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, g, scale_log2, part, c->err);
-    if (profile) cudaEventRecord(c->prof_stop, st);
+    c->mark(st, layer, PC_MARK_SUFFIX);
     if (part_out != nullptr) {
         *part_out = part;
         count_launches(2);
         return PC_OK;
     }
     am::attn_merge_kernel<HD><<<(M * d.n_q_heads + 7) / 8, 256, 0, st>>>(sd, d.n_q_heads, g, part, attn, attn_lo, c->err);
+    c->mark(st, layer, PC_MARK_MERGE);
     count_launches(3);
     return PC_OK;
 }
@@ -395,12 +400,6 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
     const RowGeom g = geom(c);
     const int half = d.head_dim / 2;
     const float scale = 1.0f / sqrtf((float)d.head_dim);
-    int prof_layer = plan.prefill ? -1 : c->prof_layer;
-    if (!plan.prefill) c->prof_layer = -1;           // one-shot (a captured step never carries the events)
-    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-    cudaStreamIsCapturing(st, &cap);
-    const bool capturing = cap != cudaStreamCaptureStatusNone;
-    if (capturing) prof_layer = -1;
     float* res_part = reinterpret_cast<float*>(w + c->cv.res_part);
     const Partials none{nullptr, 0, 0, 0};
     Partials pend = none;
@@ -412,11 +411,13 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
     count_launches(2);
     PC_CUDA_CHECK_LAUNCH("embed_rmsnorm");
     for (int l = 0; l < d.n_layers; ++l) {
+        c->mark(st, l, PC_MARK_LAYER_BEGIN);
         if (l > 0) {
             rmsnorm_kernel<T><<<row_blocks, ROW_WARPS * 32, 0, st>>>(sd, M, d.d_model, h, nullptr, pend, c->attn_norm[l], d.rms_eps, a, a_lo, half_gemm ? 1 : 0, c->err);
             pend = none;
             count_launches(1);
         }
+        c->mark(st, l, PC_MARK_NORM_ATTN);
         const float* bias = d.qkv_bias ? c->bqkv[l] : nullptr;
         Partials qkv_parts{qkv, 1, (size_t)M * c->n_qkv(), c->n_qkv()};
         if constexpr (kF32) {
@@ -429,26 +430,29 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
                                    tc::EpiPartial{qkv, c->n_qkv(), qkv_parts.stride}, half_gemm))
                 return rc;
         }
+        c->mark(st, l, PC_MARK_QKV);
         const int post_items = M * (d.n_q_heads + 2 * d.n_kv_heads);
         qkv_post_kernel<T><<<(post_items + ROW_WARPS - 1) / ROW_WARPS, ROW_WARPS * 32, 0, st>>>(
             sd, QkvPostArgs<T>{d.n_q_heads, d.n_kv_heads, d.head_dim, l, qkv_parts, bias, d.qk_norm ? c->q_norm[l] : nullptr,
                                d.qk_norm ? c->k_norm[l] : nullptr, d.rms_eps, rope, g, prompt_arena, suffix_arena, q, c->err});
         count_launches(2);
+        c->mark(st, l, PC_MARK_POST);
         if constexpr (kF32) {
-            if (l == prof_layer) cudaEventRecord(c->prof_start, st);
+            c->mark(st, l, PC_MARK_GROUP);
             if (d.head_dim == 128)
                 attn_row_simt_kernel<T, 128><<<dim3(M, d.n_kv_heads), 128, 0, st>>>(sd, d.n_q_heads, d.n_kv_heads, l, q, g,
                                                                                    prompt_arena, suffix_arena, scale, attn);
             else
                 attn_row_simt_kernel<T, 64><<<dim3(M, d.n_kv_heads), 128, 0, st>>>(sd, d.n_q_heads, d.n_kv_heads, l, q, g,
                                                                                   prompt_arena, suffix_arena, scale, attn);
-            if (l == prof_layer) cudaEventRecord(c->prof_stop, st);
+            c->mark(st, l, PC_MARK_SUFFIX);
+            c->mark(st, l, PC_MARK_MERGE);
             count_launches(1);
             launch_gemm_simt<T>(st, sd, attn, reinterpret_cast<const T*>(c->wo[l]), M, d.d_model, c->q_dim(), EpiResidual{h, d.d_model});
         } else {
             int rc = d.head_dim == 128
-                         ? attention_bf16<128>(c, st, sd, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer)
-                         : attention_bf16<64>(c, st, sd, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer);
+                         ? attention_bf16<128>(c, st, sd, M, l, plan, prompt_arena, suffix_arena, q, attn)
+                         : attention_bf16<64>(c, st, sd, M, l, plan, prompt_arena, suffix_arena, q, attn);
             if (rc) return rc;
             const GemmPlan gp = plan_gemm(c, GEMM_O, c->m_wo[l], M, true);
             if (gp.splits == 1) {
@@ -462,16 +466,20 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
                     return rc2;
             }
         }
+        c->mark(st, l, PC_MARK_O);
         rmsnorm_kernel<T><<<row_blocks, ROW_WARPS * 32, 0, st>>>(sd, M, d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a, nullptr, half_gemm ? 1 : 0, c->err);
         pend = none;
         count_launches(2);
+        c->mark(st, l, PC_MARK_NORM_MLP);
         if constexpr (kF32) {
             launch_gemm_simt<T>(st, sd, a, reinterpret_cast<const T*>(c->w_gate_up[l]), M, 2 * d.d_ff, d.d_model,
                                 EpiSwiGLU<T>{act, d.d_ff});
+            c->mark(st, l, PC_MARK_GATE_UP);
             launch_gemm_simt<T>(st, sd, act, reinterpret_cast<const T*>(c->w_down[l]), M, d.d_model, d.d_ff, EpiResidual{h, d.d_model});
         } else {
             if (int rc = gemm_bf16(c, st, sd, c->map_a, nullptr, c->m_wgu[l], M, plan_gemm(c, GEMM_GATE_UP, c->m_wgu[l], M, false), tc::EpiSwiGLU{act, d.d_ff, half_gemm ? 1 : 0, c->err}, half_gemm))
                 return rc;
+            c->mark(st, l, PC_MARK_GATE_UP);
             const GemmPlan gp = plan_gemm(c, GEMM_DOWN, c->m_wdown[l], M, true);
             if (gp.splits == 1) {
                 if (int rc = gemm_bf16(c, st, sd, c->map_act, nullptr, c->m_wdown[l], M, gp, tc::EpiResidual{h, d.d_model}, half_gemm)) return rc;
@@ -481,6 +489,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
             }
         }
         count_launches(2);
+        c->mark(st, l, PC_MARK_DOWN);
         PC_CUDA_CHECK_LAUNCH("decoder layer");
     }
     c->pend = pend;        // folded into h by the final norm
@@ -496,6 +505,7 @@ int run_lm_head(pc_ctx* c, cudaStream_t st, int n, const pc::StepDesc* sd, const
     T* a = reinterpret_cast<T*>(c->ws + c->cv.a);
     const bool half_gemm = !std::is_same<T, float>::value && d.half_gemm != 0;
     T* a_lo = std::is_same<T, float>::value || half_gemm ? nullptr : reinterpret_cast<T*>(c->ws + c->cv.a_lo);
+    c->mark(st, -1, PC_MARK_LM_BEGIN);
     rmsnorm_kernel<T><<<(n + ROW_WARPS - 1) / ROW_WARPS, ROW_WARPS * 32, 0, st>>>(sd, n, d.d_model, h, src, c->pend, c->final_norm, d.rms_eps, a, a_lo, half_gemm ? 1 : 0, c->err);
     c->pend = pc::Partials{nullptr, 0, 0, 0};
     if constexpr (std::is_same<T, float>::value) {
@@ -507,6 +517,7 @@ int run_lm_head(pc_ctx* c, cudaStream_t st, int n, const pc::StepDesc* sd, const
             return rc;
     }
     count_launches(2);
+    c->mark(st, -1, PC_MARK_LM_HEAD);
     PC_CUDA_CHECK_LAUNCH("lm head");
     return PC_OK;
 }
@@ -626,12 +637,10 @@ int pc_token_logprob(void* stream, int n_rows, int vocab, const float* logits, c
     return PC_OK;
 }
 
-int pc_profile_attention(pc_ctx* ctx, int layer, void* event_start, void* event_stop) {
-    if (ctx == nullptr || layer < 0 || layer >= ctx->d.n_layers || event_start == nullptr || event_stop == nullptr)
-        return PC_ERR_INVALID_ARG;
+int pc_profile_step(pc_ctx* ctx, int layer, void* const* events, int n_events) {
+    if (ctx == nullptr || layer < 0 || layer >= ctx->d.n_layers || events == nullptr || n_events != PC_PROFILE_MARKS) return PC_ERR_INVALID_ARG;
+    for (int i = 0; i < PC_PROFILE_MARKS; ++i) ctx->prof_ev[i] = static_cast<cudaEvent_t>(events[i]);
     ctx->prof_layer = layer;
-    ctx->prof_start = static_cast<cudaEvent_t>(event_start);
-    ctx->prof_stop = static_cast<cudaEvent_t>(event_stop);
     return PC_OK;
 }
 
@@ -956,11 +965,6 @@ int run_decode_chained(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd
     char* w = c->ws;
     const RowGeom g = geom(c);
     const int half = d.head_dim / 2;
-    int prof_layer = c->prof_layer;
-    c->prof_layer = -1;                               // one-shot (a captured step never carries the events)
-    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-    cudaStreamIsCapturing(st, &cap);
-    if (cap != cudaStreamCaptureStatusNone) prof_layer = -1;
     rope_table_kernel<<<(M * half + 255) / 256, 256, 0, st>>>(sd, half, (double)d.rope_theta, g.pos, reinterpret_cast<float2*>(w + c->cv.rope));
     count_launches(1);
     PC_CUDA_CHECK_LAUNCH("rope table");
@@ -969,8 +973,8 @@ int run_decode_chained(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd
     __nv_bfloat16* attn = reinterpret_cast<__nv_bfloat16*>(w + c->cv.attn);
     for (int l = 0; l < d.n_layers; ++l) {
         am::PrefixPartial part;
-        int rc = d.head_dim == 128 ? attention_bf16<128>(c, st, sd, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer, &part)
-                                   : attention_bf16<64>(c, st, sd, M, l, plan, prompt_arena, suffix_arena, q, attn, l == prof_layer, &part);
+        int rc = d.head_dim == 128 ? attention_bf16<128>(c, st, sd, M, l, plan, prompt_arena, suffix_arena, q, attn, &part)
+                                   : attention_bf16<64>(c, st, sd, M, l, plan, prompt_arena, suffix_arena, q, attn, &part);
         if (rc) return rc;
         if ((rc = launch_chain(c, st, M, sd, l, prompt_arena, suffix_arena, &part, logits))) return rc;
     }
@@ -986,6 +990,12 @@ int decode_launches(pc_ctx* ctx, cudaStream_t st, int m_bound, int groups_bound,
     const pc::RowKeys keys = row_keys(ctx);
     const pc::StepDesc* sd = reinterpret_cast<const pc::StepDesc*>(ctx->ws + ctx->cv.step_desc);
     const pc::DecodeArgsDev* da = reinterpret_cast<const pc::DecodeArgsDev*>(ctx->ws + ctx->cv.dargs);
+    // a profiling request is served by the first step issued outside a capture (a captured step never carries the events)
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    cudaStreamIsCapturing(st, &cap);
+    ctx->prof_active_layer = -1;
+    if (cap == cudaStreamCaptureStatusNone && ctx->prof_layer >= 0) { ctx->prof_active_layer = ctx->prof_layer; ctx->prof_layer = -1; }
+    struct Disarm { pc_ctx* c; ~Disarm() { c->prof_active_layer = -1; } } disarm{ctx};
     pc::prep_decode_rows<<<(m_bound + 128) / 128, 128, 0, st>>>(sd, da, a.prompt_slots, a.suffix_slots, ctx->d.vocab, g, keys, ctx->err);
     count_launches(1);
     PC_CUDA_CHECK_LAUNCH("prep_decode_rows");
@@ -1023,6 +1033,7 @@ int decode_launches(pc_ctx* ctx, cudaStream_t st, int m_bound, int groups_bound,
                                                               keys.out_index, 0, da);
             count_launches(1);
         }
+        ctx->mark(st, -1, PC_MARK_SAMPLE);
         PC_CUDA_CHECK_LAUNCH("sample");
     }
     return PC_OK;
@@ -1217,10 +1228,23 @@ int pc_allocate(void* stream, int n_prompts, const int32_t* pilot_success, const
                           evict == nullptr))
         return PC_ERR_INVALID_ARG;
     pc::allocate_kernel<<<1, 1024, 0, static_cast<cudaStream_t>(stream)>>>(
-        n_prompts, pilot_success, pilot_n, params->p_lower, params->p_upper, params->p_solve, params->n_commit, params->b_t, status,
-        extra_rollouts, evict, n_selected, reinterpret_cast<long long*>(total_rollouts));
+        n_prompts, pilot_success, pilot_n, nullptr, 0.0, params->p_lower, params->p_upper, params->p_solve, params->n_commit, params->b_t,
+        status, extra_rollouts, evict, n_selected, reinterpret_cast<long long*>(total_rollouts));
     count_launches(1);
     PC_CUDA_CHECK_LAUNCH("allocate");
+    return PC_OK;
+}
+
+int pc_allocate_variance(void* stream, int n_prompts, const float* pilot_var, const int32_t* pilot_n, double var_min, int n_commit,
+                         int b_t, int32_t* status, int32_t* extra_rollouts, int32_t* n_selected, int64_t* total_rollouts) {
+    if (n_prompts < 0 || n_commit < 0 || b_t < 0 || !(var_min >= 0.0) || n_selected == nullptr || total_rollouts == nullptr)
+        return PC_ERR_INVALID_ARG;
+    if (n_prompts > 0 && (pilot_var == nullptr || pilot_n == nullptr || status == nullptr || extra_rollouts == nullptr)) return PC_ERR_INVALID_ARG;
+    pc::allocate_kernel<<<1, 1024, 0, static_cast<cudaStream_t>(stream)>>>(
+        n_prompts, nullptr, pilot_n, pilot_var, var_min, 0.0, 0.0, 0.0, n_commit, b_t, status, extra_rollouts, nullptr, n_selected,
+        reinterpret_cast<long long*>(total_rollouts));
+    count_launches(1);
+    PC_CUDA_CHECK_LAUNCH("allocate (variance filter)");
     return PC_OK;
 }
 

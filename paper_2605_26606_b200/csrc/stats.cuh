@@ -7,7 +7,7 @@
 
 namespace pc {
 
-constexpr int STATUS_COMMIT = 0, STATUS_BUFFERED = 1, STATUS_DEFER_HARD = 2, STATUS_SKIP_EASY = 3;
+constexpr int STATUS_COMMIT = 0, STATUS_BUFFERED = 1, STATUS_DEFER_HARD = 2, STATUS_SKIP_EASY = 3, STATUS_LOW_VARIANCE = 4;
 
 __global__ void group_stats_kernel(int n_groups, const float* __restrict__ rewards, const int32_t* __restrict__ start,
                                    const int32_t* __restrict__ count, int32_t* __restrict__ n_out,
@@ -34,8 +34,11 @@ __global__ void group_stats_kernel(int n_groups, const float* __restrict__ rewar
 }
 
 // Single block.  Prompts are taken in batch order; the first b_t that pass the filter commit.
+// pilot_var != nullptr selects the filter for general scalar rewards: keep iff the pilot variance (Eq. 3, as float) is at
+// least var_min; the success-rate thresholds and the eviction rule are then not used (evict = 0).
 __global__ void __launch_bounds__(1024) allocate_kernel(int n_prompts, const int32_t* __restrict__ success,
-                                                        const int32_t* __restrict__ pilot_n, double p_lower, double p_upper,
+                                                        const int32_t* __restrict__ pilot_n, const float* __restrict__ pilot_var,
+                                                        double var_min, double p_lower, double p_upper,
                                                         double p_solve, int n_commit, int b_t, int32_t* __restrict__ status,
                                                         int32_t* __restrict__ extra, int32_t* __restrict__ evict,
                                                         int32_t* __restrict__ n_selected, long long* __restrict__ total_rollouts) {
@@ -50,10 +53,15 @@ __global__ void __launch_bounds__(1024) allocate_kernel(int n_prompts, const int
         int keep = 0, st = STATUS_DEFER_HARD, ev = 0, np = 0;
         if (p < n_prompts) {
             np = max(pilot_n[p], 0);
-            const double p_hat = np > 0 ? (double)success[p] / (double)np : 0.0;   // IEEE division, same as the host's
-            keep = (p_lower <= p_hat) && (p_hat <= p_upper);
-            ev = p_hat >= p_solve;
-            st = keep ? STATUS_COMMIT : (p_hat < p_lower ? STATUS_DEFER_HARD : STATUS_SKIP_EASY);
+            if (pilot_var != nullptr) {
+                keep = np > 0 && (double)pilot_var[p] >= var_min;
+                st = keep ? STATUS_COMMIT : STATUS_LOW_VARIANCE;
+            } else {
+                const double p_hat = np > 0 ? (double)success[p] / (double)np : 0.0;   // IEEE division, same as the host's
+                keep = (p_lower <= p_hat) && (p_hat <= p_upper);
+                ev = p_hat >= p_solve;
+                st = keep ? STATUS_COMMIT : (p_hat < p_lower ? STATUS_DEFER_HARD : STATUS_SKIP_EASY);
+            }
         }
         // exclusive prefix count of `keep` in batch order
         const unsigned ballot = __ballot_sync(0xffffffffu, keep);
@@ -68,7 +76,7 @@ __global__ void __launch_bounds__(1024) allocate_kernel(int n_prompts, const int
             if (keep && before >= b_t) st = STATUS_BUFFERED;
             status[p] = st;
             extra[p] = st == STATUS_COMMIT ? n_commit : 0;
-            evict[p] = ev;
+            if (evict != nullptr) evict[p] = ev;
         }
         __syncthreads();
         if (threadIdx.x == 0) {

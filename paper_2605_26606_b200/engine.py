@@ -102,7 +102,7 @@ class RolloutEngine:
         self.err_flag = torch.zeros(1, dtype=torch.int32, device=dev)
         B.pc_set_workspace(self.ctx, self.workspace, max_rows, max_prefill_tokens, self.err_flag)
         self.kv_dtype = torch.float32 if m.dtype == DTYPE_F32 else torch.bfloat16
-        # measurement: every `profile_every`-th decode step, time the suffix-attention kernel of one layer
+        # measurement: every `profile_every`-th decode step, time the operations of one layer and of the step's tail
         self._arenas: Dict[str, Optional[torch.Tensor]] = {}
         self.profile_every = 0
         self.use_graphs = True
@@ -112,7 +112,8 @@ class RolloutEngine:
         self.record_commit_logits: Optional[dict] = None    # the same for the commit stage
         self.record_rows: Optional[set] = None              # keep only the logits rows of these (prompt, rollout) pairs
         self.profile_layer = m.n_layers // 2
-        self.profile_samples: List[tuple] = []      # (start event, stop event, rows, suffix slots read per row)
+        self.stage_rows_per_step: List[np.ndarray] = []      # live rows of every decode step, one array per stage run so far
+        self.profile_samples: List[tuple] = []      # (events at the marks of binding.PROFILE_MARKS, rows, suffix slots read per row)
 
     # ------------------------------------------------------------------------------------------
     def kv_arena(self, n_slots: int, which: str) -> torch.Tensor:
@@ -260,10 +261,11 @@ class RolloutEngine:
                 logits_out = torch.empty((nr, self.model.vocab), dtype=torch.float32, device=dev)
                 record_logits[s] = (logits_out, sch.row_prompt[o:o + nr].cpu().numpy(), sch.row_rollout[o:o + nr].cpu().numpy())
             if profiled(s):
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record(); e1.record()             # creates the underlying CUDA events
-                B.pc_profile_attention(self.ctx, self.profile_layer, e0, e1)
-                self.profile_samples.append((e0, e1, nr, s + 1))
+                evs = [torch.cuda.Event(enable_timing=True) for _ in B.PROFILE_MARKS]
+                for e in evs:
+                    e.record()                       # creates the underlying CUDA events
+                B.pc_profile_step(self.ctx, self.profile_layer, evs)
+                self.profile_samples.append((evs, nr, s + 1))
             B.pc_decode_step(self.ctx, nr, pr + 4 * o, rr + 4 * o, rs + 4 * o, rk + 8 * o, self.tokens, rt + 8 * o,
                              int(sch.groups_per_step[s]), gs + 4 * go, int(sch.max_group_rows[s]), self.prompt_len,
                              self.prompt_kv, self.total_prompt_tokens, self.prompt_kv_start, self.suffix_kv,
@@ -295,6 +297,7 @@ class RolloutEngine:
                             self.prompt_kv_start, self.suffix_kv, self.suffix_slots, sp)
             s = e
         self._keep_schedule = sch
+        self.stage_rows_per_step.append(sch.rows_per_step.copy())
         return int(self.batch.caps[prompts, rollouts].sum())
 
     # ------------------------------------------------------------------------------------------
@@ -313,7 +316,10 @@ class RolloutEngine:
         wl = self.wl
         P, G, k = wl.n_prompts, wl.group_size, wl.n_pilot
         b_t = P if b_t is None else b_t
+        self.prefill_events = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+        self.prefill_events[0].record()
         self.prefill()
+        self.prefill_events[1].record()
         pp, rr = np.repeat(np.arange(P), k), np.tile(np.arange(k), P)
         n_tok = self.run_stage(pp, rr, record_logits=self.record_pilot_logits)
         pilot_count = torch.full((P,), k, dtype=torch.int32, device=self.device)

@@ -239,3 +239,25 @@ def test_reward_of_a_never_generated_cell_is_zero():
     r = torch.full((3,), 7.0, device="cuda")
     B.pc_reward_last_token(3, tokens, last, _i32([10, 10, 10]), r)
     assert r.cpu().tolist() == [0.0, 1.0, 0.0]
+
+
+def test_variance_filter_for_scalar_rewards_matches_oracle():
+    """pc_allocate_variance on the variances pc_group_stats returns: decisions identical to the oracle's, for continuous
+    rewards and for binary ones (where it reproduces the success-rate band)."""
+    rng = np.random.default_rng(11)
+    P, k = 300, 16
+    for binary in (False, True):
+        r = (rng.random((P, k)) < rng.random((P, 1))).astype(np.float64) if binary else rng.normal(size=(P, k)) * rng.uniform(0, 2, size=(P, 1))
+        start, count = np.arange(P) * k, np.full(P, k)
+        n, m, mean, var = _stats_gpu(r.reshape(-1), start, count)
+        var_min = 0.1875 if binary else 0.7
+        status, extra = torch.zeros(P, dtype=torch.int32, device="cuda"), torch.zeros(P, dtype=torch.int32, device="cuda")
+        nsel, total = torch.zeros(1, dtype=torch.int32, device="cuda"), torch.zeros(1, dtype=torch.int64, device="cuda")
+        B.pc_allocate_variance(P, torch.from_numpy(var).cuda(), _i32(n), var_min, 48, 100, status, extra, nsel, total)
+        _, _, _, ovar = ostats.group_stats(r.astype(np.float32).astype(np.float64).reshape(-1), start, count)
+        st, ex, sel, tot = ostats.allocate_by_variance(ovar, n, var_min, 48, 100)
+        assert np.array_equal(status.cpu().numpy(), st) and np.array_equal(extra.cpu().numpy(), ex)
+        assert int(nsel.item()) == sel and int(total.item()) == tot
+        if binary:
+            keep = (m / k >= 0.25) & (m / k <= 0.75)
+            assert np.array_equal(st != ostats.LOW_VARIANCE, keep)

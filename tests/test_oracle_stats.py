@@ -185,3 +185,27 @@ def test_dapo_filter_is_the_pilot_filter_with_k_equal_n():
     # GRPO: every prompt of the training batch gets n rollouts, none is filtered
     st, *_ , total = stats.allocate(np.array([0, 3, 8]), np.full(3, 8), 0.0, 1.0, 2.0, 0, 3)
     assert np.all(st == stats.COMMIT) and total == 24 == stats.sampling_cost("grpo", 3, 3, 8, 0)
+
+
+def test_variance_filter_equals_the_success_rate_filter_for_binary_rewards_and_symmetric_thresholds():
+    """Section 3.3: Var[r | q] = p (1 - p), so for binary rewards a variance threshold v is the success-rate band
+    [p_lo, 1 - p_lo] with p_lo (1 - p_lo) = v.  Checked for every (m, k) with k a power of two (all values exact)."""
+    from oracle import stats as S
+    for k in (2, 4, 8, 16, 32):
+        for p_lo in (0.125, 0.25, 0.375):
+            m = np.arange(k + 1)
+            n = np.full(k + 1, k)
+            var = (m / k) * (1 - m / k)
+            st_v, ex_v, sel_v, tot_v = S.allocate_by_variance(var, n, p_lo * (1 - p_lo), 5, k + 1)
+            st_p, ex_p, ev_p, sel_p, tot_p = S.allocate(m, n, p_lo, 1 - p_lo, 2.0, 5, k + 1)
+            assert np.array_equal(st_v == S.COMMIT, st_p == S.COMMIT), (k, p_lo)
+            assert np.array_equal(ex_v, ex_p) and sel_v == sel_p and tot_v == tot_p
+            assert np.all(st_v[st_p != S.COMMIT] == S.LOW_VARIANCE)
+    # continuous rewards: the decision is the plain definition, a population variance (numpy) against the threshold
+    rng = np.random.default_rng(4)
+    r = rng.normal(size=(40, 8)) * rng.uniform(0, 2, size=(40, 1))
+    var = r.var(axis=1)
+    st, ex, sel, tot = S.allocate_by_variance(var, np.full(40, 8), 0.5, 3, 7)
+    kept = np.flatnonzero(var.astype(np.float32) >= 0.5)
+    assert np.array_equal(np.flatnonzero(st == S.COMMIT), kept[:7]) and np.array_equal(np.flatnonzero(st == S.BUFFERED), kept[7:])
+    assert sel == min(7, len(kept)) and tot == 40 * 8 + sel * 3 and ex.sum() == sel * 3
