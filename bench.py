@@ -159,7 +159,8 @@ def run_probe(args):
     batch = wl.gen_batch(w)
     eng = RolloutEngine(w.model, weights, max_rows=P * G, max_prefill_tokens=int(batch.prompt_offsets[-1]))
     eng.use_graphs = kv.get("graphs", "1") != "0"
-    B.pc_set_decode_mode(eng.ctx, int(kv.get("mode", 1)))
+    B.pc_set_decode_mode(eng.ctx, int(kv.get("mode", 0)))
+    B.pc_set_attention_overlap(eng.ctx, int(kv.get("overlap", 1)))
     eng.load_batch(w, batch)
     eng.suffix_kv.zero_()
     eng.tokens.random_(0, w.model.vocab)

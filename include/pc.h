@@ -100,7 +100,7 @@ typedef struct pc_model_desc {
                           * bfloat16 for the token lookup).  A bfloat16 weight converts to half exactly
                           * unless it is below 2^-14 in magnitude (then to within 2^-25).  Activations
                           * and V values that do not fit half (|x| > 65504, or NaN) are stored saturated
-                          * (NaN as 0) and reported as code 5 in *dev_error_flag.                        */
+                          * and reported as code 5 in *dev_error_flag.                                    */
 } pc_model_desc;
 
 /* Device pointers to the weights.  The per-layer members are HOST arrays of n_layers
@@ -189,6 +189,12 @@ PC_API int pc_selftest_wait_timeout(void* stream, uint32_t spin_limit, int32_t* 
  * the decode steps can check row_prompt and row_tok_index against them (see "Device-side anomalies" above).  0 = not
  * stated, not checked (the default). */
 PC_API int pc_set_index_bounds(pc_ctx* ctx, int n_prompts, int64_t n_tokens);
+
+/* bf16 models, decode steps: 1 (the default) issues the shared-prefix attention kernel and the per-rollout suffix attention
+ * kernel of a layer on two streams (the second one is created by the context on first use and released by pc_destroy), so
+ * that they can overlap; 0 (the default: measured no faster, both kernels fill the SMs) issues them one after the other.
+ * Results are identical.  Drops captured decode steps. */
+PC_API int pc_set_attention_overlap(pc_ctx* ctx, int on);
 
 /* How the decode steps of a bf16 model with half_gemm = 1 are issued.  mode 1: everything between two
  * attention calls of a step -- output projection, residual + RMSNorm, gate/up + SwiGLU, down projection, residual +

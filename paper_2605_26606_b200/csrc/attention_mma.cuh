@@ -641,14 +641,16 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
 // One warp per (row, head); a lane owns HD/32 consecutive dims.
 // ---------------------------------------------------------------------------------------------
 // rh = row * Hq + head (the caller keeps it below n_live * Hq).  ct = tiles per suffix chunk of this step (suffix_plan);
-// n_load = how many records to request: every record index the step can have produced (part.n_parts + chunk slots per
+// n_load > 0 = how many records to request: every record index the step can have produced (part.n_parts + chunk slots per
 // item), so that the loads do not wait for the row's suffix length; records past the row's own count are ignored.
+// n_load <= 0: wait for the suffix length and request the row's own records only.
 template <int HD>
 __device__ __forceinline__ void merge_item_warp(int lane, size_t rh, int Hq, const RowGeom& g, const PrefixPartial& part, int ct, int n_load,
                                                 __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ out_lo, int32_t* err) {
     constexpr int EPL = HD / 32;
     const int row = (int)(rh / Hq);
     const int slen = g.s_len[row];
+    if (n_load <= 0) n_load = part.n_parts + suffix_chunks(slen, ct);      // large batches: request only the row's own records
     float mi[MAX_RECORDS], li[MAX_RECORDS];
     float ov[MAX_RECORDS][EPL];
 #pragma unroll
@@ -716,7 +718,8 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const StepDesc* __restr
     const int n_live = sd->n_rows;
     if (rh >= (size_t)n_live * Hq) return;
     const SuffixPlan sp = suffix_plan(*g.max_slen, n_live * part.n_kv_heads, part.n_suffix_warps);
-    merge_item_warp<HD>(threadIdx.x & 31, rh, Hq, g, part, sp.ct, part.n_parts + sp.cpi, out, out_lo, err);
+    // few items: request every record slot of the step at once (latency); many items: only the row's own records (bytes)
+    merge_item_warp<HD>(threadIdx.x & 31, rh, Hq, g, part, sp.ct, n_live * Hq <= 8192 ? part.n_parts + sp.cpi : 0, out, out_lo, err);
 }
 
 }  // namespace am

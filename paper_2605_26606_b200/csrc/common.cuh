@@ -14,7 +14,7 @@ enum DevError : int32_t {
     DEV_ERR_TOKEN_RANGE = 2,    // a token id outside [0, vocab)
     DEV_ERR_WAIT_TIMEOUT = 3,   // a bounded wait on an mbarrier ran out
     DEV_ERR_GROUP_RANGE = 4,    // group / row bookkeeping inconsistent
-    DEV_ERR_HALF_RANGE = 5,     // a GEMM operand or V value did not fit IEEE half (stored saturated, NaN as 0)
+    DEV_ERR_HALF_RANGE = 5,     // a GEMM operand or V value did not fit IEEE half (stored saturated)
 };
 
 // What one forward pass covers, kept in device memory so that a captured CUDA graph can be replayed for
@@ -63,14 +63,14 @@ __device__ __forceinline__ void set_error(int32_t* flag, int32_t code) {
     if (flag != nullptr) atomicCAS(flag, 0, code);
 }
 
-// Values headed for IEEE half storage: anything beyond the largest finite half is stored saturated and reported.
+// Values headed for IEEE half storage: anything beyond the largest finite half is stored saturated (NaN as the largest
+// finite value) and reported.  half_clamp is branch-free; callers OR half_bad over a batch of values and report once.
 constexpr float HALF_MAX_F = 65504.f;
+__device__ __forceinline__ float half_clamp(float x) { return fminf(fmaxf(x, -HALF_MAX_F), HALF_MAX_F); }
+__device__ __forceinline__ int half_bad(float x) { return !(fabsf(x) <= HALF_MAX_F); }
 __device__ __forceinline__ float half_guard(float x, int32_t* err) {
-    if (!(fabsf(x) <= HALF_MAX_F)) {
-        set_error(err, DEV_ERR_HALF_RANGE);
-        x = x != x ? 0.f : copysignf(HALF_MAX_F, x);
-    }
-    return x;
+    if (half_bad(x)) set_error(err, DEV_ERR_HALF_RANGE);
+    return half_clamp(x);
 }
 
 template <typename T> __device__ __forceinline__ float to_f32(T v);

@@ -427,8 +427,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_chain_kernel(const __grid_c
                             float* h_row = p.h + (size_t)r * p.d_model;
                             if (ph == PH_EMBED) {
                                 const __nv_bfloat16* e_row = reinterpret_cast<const __nv_bfloat16*>(p.embed) + (size_t)p.g.token[r] * p.d_model;
-#pragma unroll
-                                for (int kk = 0; kk < NORM_SEG_REG4; ++kk) {
+                                for (int kk = 0; kk < 8; ++kk) {
                                     const int i = lane + 32 * (w + NORM_SEGS * kk);
                                     if (i < (p.d_model >> 2)) {
                                         float v[4];
@@ -438,7 +437,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_chain_kernel(const __grid_c
                                 }
                             }
                             if (!norm_row_cta<__nv_bfloat16>(w, lane, p.d_model, h_row, pend, (size_t)r * p.d_model, gain, p.eps,
-                                                             p.a + (size_t)r * p.d_model, 1, s_norm_red + j * 8, s_norm_cnt + j, p.err)) {
+                                                             p.a + (size_t)r * p.d_model, nullptr, 1, s_norm_red + j * 8, s_norm_cnt + j, p.err)) {
                                 ok = false;
                                 break;
                             }

@@ -197,12 +197,14 @@ struct EpiSwiGLU {              // columns (2j, 2j+1) = (gate_j, up_j) -> out[ro
         __nv_bfloat16* dst = out + (size_t)row * ld + (col0 >> 1);
         if (n_valid == 32 && (ld & 7) == 0) {
             uint32_t w[8];
+            int bad = 0;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const float g0 = v[4 * i], u0 = v[4 * i + 1], g1 = v[4 * i + 2], u1 = v[4 * i + 3];
                 const float y0 = g0 / (1.f + expf(-g0)) * u0, y1 = g1 / (1.f + expf(-g1)) * u1;
                 if (half_out) {
-                    const __half2 p = __floats2half2_rn(half_guard(y0, err), half_guard(y1, err));
+                    bad |= half_bad(y0) | half_bad(y1);
+                    const __half2 p = __floats2half2_rn(half_clamp(y0), half_clamp(y1));
                     w[i] = *reinterpret_cast<const uint32_t*>(&p);
                 } else {
                     const __nv_bfloat162 p = __floats2bfloat162_rn(y0, y1);
@@ -211,6 +213,7 @@ struct EpiSwiGLU {              // columns (2j, 2j+1) = (gate_j, up_j) -> out[ro
             }
             *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
             *reinterpret_cast<uint4*>(dst + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+            if (bad) set_error(err, DEV_ERR_HALF_RANGE);
         } else {
 #pragma unroll
             for (int i = 0; i < 32; i += 2)

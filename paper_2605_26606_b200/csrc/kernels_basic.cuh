@@ -151,8 +151,8 @@ template <typename T>
 __device__ __forceinline__ void store_norm_out(T* __restrict__ a_row, T* __restrict__ a_lo_row, int i4, float4 y, int half_out,
                                                int32_t* err = nullptr) {
     if (sizeof(T) == 2 && half_out) {
-        const __half2 lo = __floats2half2_rn(half_guard(y.x, err), half_guard(y.y, err)),
-                      hi = __floats2half2_rn(half_guard(y.z, err), half_guard(y.w, err));
+        if (half_bad(y.x) | half_bad(y.y) | half_bad(y.z) | half_bad(y.w)) set_error(err, DEV_ERR_HALF_RANGE);
+        const __half2 lo = __floats2half2_rn(half_clamp(y.x), half_clamp(y.y)), hi = __floats2half2_rn(half_clamp(y.z), half_clamp(y.w));
         *reinterpret_cast<uint2*>(a_row + 4 * i4) =
             make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
     } else {
@@ -249,22 +249,20 @@ __device__ __forceinline__ void norm_row_warp(int lane, int d, float* __restrict
     }
 }
 
-// The same row handled by NORM_SEGS warps of one CTA, warp w taking segment w.  The segment sums are exchanged through
-// shared memory: red[NORM_SEGS] floats and one counter, both used once (zero before); the wait on the counter is
-// bounded and returns false when it ran out.  Rows whose segments do not fit NORM_SEG_REG4 blocks per warp are not
-// handled here (the caller falls back to one warp per row).
-constexpr int NORM_SEG_REG4 = 2;
-__device__ __forceinline__ bool norm_row_fits_cta(int d) { return ((d >> 2) + 31) / 32 <= NORM_SEGS * NORM_SEG_REG4; }
-template <typename T>
-__device__ __forceinline__ bool norm_row_cta(int w, int lane, int d, float* __restrict__ h_row, Partials pend, size_t pend_row,
-                                             const float* __restrict__ gain, float eps, T* __restrict__ a_row, int half_out,
-                                             volatile float* red, int* counter, int32_t* err = nullptr) {
+// The same row handled by NORM_SEGS warps of one CTA, warp w taking segment w: every load of the row is in flight at once,
+// which is what a latency-bound batch wants.  The segment sums are exchanged through shared memory: red[NORM_SEGS] floats
+// and one counter, both used once (zero before); the wait on the counter is bounded and returns false when it ran out.
+// KK = blocks per warp kept in registers; rows need (d / 128) <= NORM_SEGS * KK.
+template <typename T, int KK>
+__device__ __forceinline__ bool norm_row_cta_kk(int w, int lane, int d, float* __restrict__ h_row, Partials pend, size_t pend_row,
+                                                const float* __restrict__ gain, float eps, T* __restrict__ a_row, T* __restrict__ a_lo_row,
+                                                int half_out, volatile float* red, int* counter, int32_t* err) {
     const int n4 = d >> 2;
     float4* x = reinterpret_cast<float4*>(h_row);
-    float4 v[NORM_SEG_REG4], gg[NORM_SEG_REG4];
+    float4 v[KK], gg[KK];
     float part = 0.f;
 #pragma unroll
-    for (int kk = 0; kk < NORM_SEG_REG4; ++kk) {
+    for (int kk = 0; kk < KK; ++kk) {
         const int i = lane + 32 * (w + NORM_SEGS * kk);
         if (i < n4) {
             gg[kk] = *reinterpret_cast<const float4*>(gain + 4 * i);
@@ -274,7 +272,7 @@ __device__ __forceinline__ bool norm_row_cta(int w, int lane, int d, float* __re
     }
     if (pend.n > 0) {
 #pragma unroll
-        for (int kk = 0; kk < NORM_SEG_REG4; ++kk) {
+        for (int kk = 0; kk < KK; ++kk) {
             const int i = lane + 32 * (w + NORM_SEGS * kk);
             if (i < n4) x[i] = v[kk];
         }
@@ -297,14 +295,24 @@ __device__ __forceinline__ bool norm_row_cta(int w, int lane, int d, float* __re
     for (int g = 0; g < NORM_SEGS; ++g) ss = __fadd_rn(ss, red[g]);
     const float rstd = rsqrtf(__fadd_rn(__fdiv_rn(ss, (float)d), eps));
 #pragma unroll
-    for (int kk = 0; kk < NORM_SEG_REG4; ++kk) {
+    for (int kk = 0; kk < KK; ++kk) {
         const int i = lane + 32 * (w + NORM_SEGS * kk);
         if (i < n4)
-            store_norm_out<T>(a_row, static_cast<T*>(nullptr), i,
+            store_norm_out<T>(a_row, a_lo_row, i,
                               make_float4(v[kk].x * rstd * gg[kk].x, v[kk].y * rstd * gg[kk].y, v[kk].z * rstd * gg[kk].z, v[kk].w * rstd * gg[kk].w),
                               half_out, err);
     }
     return true;
+}
+__device__ __forceinline__ bool norm_row_fits_cta(int d) { return ((d >> 2) + 31) / 32 <= NORM_SEGS * 8; }
+template <typename T>
+__device__ __forceinline__ bool norm_row_cta(int w, int lane, int d, float* __restrict__ h_row, Partials pend, size_t pend_row,
+                                             const float* __restrict__ gain, float eps, T* __restrict__ a_row, T* __restrict__ a_lo_row,
+                                             int half_out, volatile float* red, int* counter, int32_t* err = nullptr) {
+    const int nk = ((d >> 2) + 31) / 32;
+    if (nk <= NORM_SEGS * 2) return norm_row_cta_kk<T, 2>(w, lane, d, h_row, pend, pend_row, gain, eps, a_row, a_lo_row, half_out, red, counter, err);
+    if (nk <= NORM_SEGS * 4) return norm_row_cta_kk<T, 4>(w, lane, d, h_row, pend, pend_row, gain, eps, a_row, a_lo_row, half_out, red, counter, err);
+    return norm_row_cta_kk<T, 8>(w, lane, d, h_row, pend, pend_row, gain, eps, a_row, a_lo_row, half_out, red, counter, err);
 }
 
 // h_row[:] = E[token, :] as float (the residual stream), one warp per row; d is a multiple of 8.
@@ -317,32 +325,56 @@ __device__ __forceinline__ void embed_row_warp(int lane, int d, const T* __restr
     }
 }
 
-constexpr int ROW_WARPS = 8;         // rows per block of the stand-alone row-wise kernels
+constexpr int ROW_WARPS = 8;         // items per block of the stand-alone per-(row, head) kernels
+constexpr int NORM_THREADS = NORM_SEGS * 32;
 
-// h[r, :] = E[token[r], :] (float residual stream); a[r, :] = RMSNorm(h[r, :]; gain) in storage type T.
+// h[r, :] = E[token[r], :] (float residual stream); a[r, :] = RMSNorm(h[r, :]; gain) in storage type T.  One block per row.
 template <typename T>
-__global__ void __launch_bounds__(ROW_WARPS * 32) embed_rmsnorm_kernel(const StepDesc* __restrict__ sd, int d, const int32_t* token,
-                                                                        const T* __restrict__ embed, const float* __restrict__ gain, float eps,
-                                                                        float* __restrict__ h, T* __restrict__ a, T* __restrict__ a_lo, int half_out,
-                                                                        int32_t* err) {
-    const int r = blockIdx.x * ROW_WARPS + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+__global__ void __launch_bounds__(NORM_THREADS) embed_rmsnorm_kernel(const StepDesc* __restrict__ sd, int d, const int32_t* token,
+                                                                     const T* __restrict__ embed, const float* __restrict__ gain, float eps,
+                                                                     float* __restrict__ h, T* __restrict__ a, T* __restrict__ a_lo, int half_out,
+                                                                     int32_t* err) {
+    __shared__ float red[8];
+    __shared__ int counter;
+    const int r = blockIdx.x, w = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (r >= sd->n_rows) return;
-    embed_row_warp<T>(lane, d, embed + (size_t)token[r] * d, h + (size_t)r * d);
-    norm_row_warp<T>(lane, d, h + (size_t)r * d, Partials{nullptr, 0, 0, 0}, 0, gain, eps, a + (size_t)r * d,
-                     a_lo ? a_lo + (size_t)r * d : nullptr, half_out, err);
+    if (threadIdx.x == 0) counter = 0;
+    const T* e_row = embed + (size_t)token[r] * d;
+    float* h_row = h + (size_t)r * d;
+    for (int i = threadIdx.x; i < (d >> 2); i += NORM_THREADS) {
+        float v[4];
+        VecLoad<T, 4>::load(e_row + 4 * i, v);
+        reinterpret_cast<float4*>(h_row)[i] = make_float4(v[0], v[1], v[2], v[3]);
+    }
+    __syncthreads();
+    if (norm_row_fits_cta(d))
+        norm_row_cta<T>(w, lane, d, h_row, Partials{nullptr, 0, 0, 0}, 0, gain, eps, a + (size_t)r * d, a_lo ? a_lo + (size_t)r * d : nullptr,
+                        half_out, red, &counter, err);
+    else if (w == 0)
+        norm_row_warp<T>(lane, d, h_row, Partials{nullptr, 0, 0, 0}, 0, gain, eps, a + (size_t)r * d, a_lo ? a_lo + (size_t)r * d : nullptr,
+                         half_out, err);
 }
 
 // Optional residual update followed by the norm:  h[row, :] += pending partial sums of row;  a[r, :] = RMSNorm(h[row, :]; gain)
 // with row = src ? src[r] : r.  The partial sums are indexed by row, like h.  n_rows bounds r when there is no step descriptor.
+// One block per row.
 template <typename T>
-__global__ void __launch_bounds__(ROW_WARPS * 32) rmsnorm_kernel(const StepDesc* __restrict__ sd, int n_rows, int d, float* __restrict__ h,
-                                                                  const int32_t* __restrict__ src, Partials pend, const float* __restrict__ gain,
-                                                                  float eps, T* __restrict__ a, T* __restrict__ a_lo, int half_out, int32_t* err) {
-    const int r = blockIdx.x * ROW_WARPS + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+__global__ void __launch_bounds__(NORM_THREADS) rmsnorm_kernel(const StepDesc* __restrict__ sd, int n_rows, int d, float* __restrict__ h,
+                                                               const int32_t* __restrict__ src, Partials pend, const float* __restrict__ gain,
+                                                               float eps, T* __restrict__ a, T* __restrict__ a_lo, int half_out, int32_t* err) {
+    __shared__ float red[8];
+    __shared__ int counter;
+    const int r = blockIdx.x, w = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (r >= (sd != nullptr ? sd->n_rows : n_rows)) return;
+    if (threadIdx.x == 0) counter = 0;
+    __syncthreads();
     const int row = src ? src[r] : r;
-    norm_row_warp<T>(lane, d, h + (size_t)row * d, pend, (size_t)row * pend.ld, gain, eps, a + (size_t)r * d,
-                     a_lo ? a_lo + (size_t)r * d : nullptr, half_out, err);
+    if (norm_row_fits_cta(d))
+        norm_row_cta<T>(w, lane, d, h + (size_t)row * d, pend, (size_t)row * pend.ld, gain, eps, a + (size_t)r * d,
+                        a_lo ? a_lo + (size_t)r * d : nullptr, half_out, red, &counter, err);
+    else if (w == 0)
+        norm_row_warp<T>(lane, d, h + (size_t)row * d, pend, (size_t)row * pend.ld, gain, eps, a + (size_t)r * d,
+                         a_lo ? a_lo + (size_t)r * d : nullptr, half_out, err);
 }
 
 struct KvArena {

@@ -123,6 +123,10 @@ struct pc_ctx {
     int32_t n_prompts_hint = 0;              // pc_set_index_bounds: sizes of the caller's per-prompt arrays and token buffer (0: unknown)
     int64_t n_tokens_hint = 0;
 
+    int attn_overlap = 0;                    // decode: shared-prefix and suffix attention kernels of a layer on two streams
+    cudaStream_t side_stream = nullptr;      // second branch of that fork (created on first use)
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+
     std::vector<GraphEntry> graphs;
     cudaStream_t capture_stream = nullptr;      // decode steps are captured here (the caller's stream may be the default one)
     void drop_graphs() {
@@ -132,6 +136,9 @@ struct pc_ctx {
     ~pc_ctx() {
         drop_graphs();
         if (capture_stream) cudaStreamDestroy(capture_stream);
+        if (side_stream) cudaStreamDestroy(side_stream);
+        if (ev_fork) cudaEventDestroy(ev_fork);
+        if (ev_join) cudaEventDestroy(ev_join);
     }
 
     int n_qkv() const { return (d.n_q_heads + 2 * d.n_kv_heads) * d.head_dim; }
@@ -361,12 +368,29 @@ int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, in
         count_launches(1);
         return PC_OK;
     }
-    am::attn_group_kernel<HD, false><<<ggrid, am::G_THREADS, am::group_smem_bytes<HD>(), st>>>(
+    // The two kernels are independent (both read q, each leaves its own records), so outside profiled steps they are issued
+    // on two streams -- a fork and a join inside the captured step -- and share the GPU.
+    const bool overlap = c->attn_overlap != 0 && c->prof_active_layer < 0;
+    cudaStream_t gst = st;
+    if (overlap) {
+        if (c->side_stream == nullptr) {
+            cudaError_t e = cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming);
+            if (e != cudaSuccess) return cuda_fail(e, "side stream of the attention fork");
+        }
+        cudaEventRecord(c->ev_fork, st);
+        cudaStreamWaitEvent(c->side_stream, c->ev_fork, 0);
+        gst = c->side_stream;
+    }
+    am::attn_group_kernel<HD, false><<<ggrid, am::G_THREADS, am::group_smem_bytes<HD>(), gst>>>(
         c->map_prompt_kv, sd, prompt_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, plan.group_row_start, g, scale_log2, part,
         attn, attn_lo, c->err);
+    if (overlap) cudaEventRecord(c->ev_join, gst);
     c->mark(st, layer, PC_MARK_GROUP);
     am::attn_suffix_kernel<HD><<<sgrid, am::S_WARPS * 32, am::suffix_smem_bytes<HD>(), st>>>(
         c->map_suffix_kv, sd, suffix_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, g, scale_log2, part, c->err);
+    if (overlap) cudaStreamWaitEvent(st, c->ev_join, 0);
     c->mark(st, layer, PC_MARK_SUFFIX);
     if (part_out != nullptr) {
         *part_out = part;
@@ -405,15 +429,14 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
     Partials pend = none;
 
     rope_table_kernel<<<(M * half + 255) / 256, 256, 0, st>>>(sd, half, (double)d.rope_theta, g.pos, rope);
-    const int row_blocks = (M + ROW_WARPS - 1) / ROW_WARPS;
-    embed_rmsnorm_kernel<T><<<row_blocks, ROW_WARPS * 32, 0, st>>>(sd, d.d_model, g.token, reinterpret_cast<const T*>(c->embed), c->attn_norm[0],
+    embed_rmsnorm_kernel<T><<<M, NORM_THREADS, 0, st>>>(sd, d.d_model, g.token, reinterpret_cast<const T*>(c->embed), c->attn_norm[0],
                                                d.rms_eps, h, a, a_lo, half_gemm ? 1 : 0, c->err);
     count_launches(2);
     PC_CUDA_CHECK_LAUNCH("embed_rmsnorm");
     for (int l = 0; l < d.n_layers; ++l) {
         c->mark(st, l, PC_MARK_LAYER_BEGIN);
         if (l > 0) {
-            rmsnorm_kernel<T><<<row_blocks, ROW_WARPS * 32, 0, st>>>(sd, M, d.d_model, h, nullptr, pend, c->attn_norm[l], d.rms_eps, a, a_lo, half_gemm ? 1 : 0, c->err);
+            rmsnorm_kernel<T><<<M, NORM_THREADS, 0, st>>>(sd, M, d.d_model, h, nullptr, pend, c->attn_norm[l], d.rms_eps, a, a_lo, half_gemm ? 1 : 0, c->err);
             pend = none;
             count_launches(1);
         }
@@ -467,7 +490,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
             }
         }
         c->mark(st, l, PC_MARK_O);
-        rmsnorm_kernel<T><<<row_blocks, ROW_WARPS * 32, 0, st>>>(sd, M, d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a, nullptr, half_gemm ? 1 : 0, c->err);
+        rmsnorm_kernel<T><<<M, NORM_THREADS, 0, st>>>(sd, M, d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a, nullptr, half_gemm ? 1 : 0, c->err);
         pend = none;
         count_launches(2);
         c->mark(st, l, PC_MARK_NORM_MLP);
@@ -506,7 +529,7 @@ int run_lm_head(pc_ctx* c, cudaStream_t st, int n, const pc::StepDesc* sd, const
     const bool half_gemm = !std::is_same<T, float>::value && d.half_gemm != 0;
     T* a_lo = std::is_same<T, float>::value || half_gemm ? nullptr : reinterpret_cast<T*>(c->ws + c->cv.a_lo);
     c->mark(st, -1, PC_MARK_LM_BEGIN);
-    rmsnorm_kernel<T><<<(n + ROW_WARPS - 1) / ROW_WARPS, ROW_WARPS * 32, 0, st>>>(sd, n, d.d_model, h, src, c->pend, c->final_norm, d.rms_eps, a, a_lo, half_gemm ? 1 : 0, c->err);
+    rmsnorm_kernel<T><<<n, NORM_THREADS, 0, st>>>(sd, n, d.d_model, h, src, c->pend, c->final_norm, d.rms_eps, a, a_lo, half_gemm ? 1 : 0, c->err);
     c->pend = pc::Partials{nullptr, 0, 0, 0};
     if constexpr (std::is_same<T, float>::value) {
         const T* wlm = reinterpret_cast<const T*>(d.tied_embed ? c->embed : c->lm_head);
@@ -579,6 +602,13 @@ int pc_set_gemm_plan(pc_ctx* ctx, const char* spec) {
     }
     for (int k = 0; k < 5; ++k) { ctx->plan_bn[k] = bn[k]; ctx->plan_splits[k] = sp[k]; }
     ctx->drop_graphs();          // captured steps carry the old choice
+    return PC_OK;
+}
+
+int pc_set_attention_overlap(pc_ctx* ctx, int on) {
+    if (ctx == nullptr || (on != 0 && on != 1)) return PC_ERR_INVALID_ARG;
+    if (on != ctx->attn_overlap) ctx->drop_graphs();
+    ctx->attn_overlap = on;
     return PC_OK;
 }
 
