@@ -160,7 +160,8 @@ def run_probe(args):
     eng = RolloutEngine(w.model, weights, max_rows=P * G, max_prefill_tokens=int(batch.prompt_offsets[-1]))
     eng.use_graphs = kv.get("graphs", "1") != "0"
     B.pc_set_decode_mode(eng.ctx, int(kv.get("mode", 0)))
-    B.pc_set_attention_overlap(eng.ctx, int(kv.get("overlap", 1)))
+    B.pc_set_attention_overlap(eng.ctx, int(kv.get("overlap", 0)))
+    B.pc_set_fused_sampler(eng.ctx, int(kv.get("fused", 0)))
     eng.load_batch(w, batch)
     eng.suffix_kv.zero_()
     eng.tokens.random_(0, w.model.vocab)

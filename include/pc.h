@@ -28,7 +28,7 @@
  *    statistics are float; dot products accumulate in float.
  *  - KV arena layout (prompt arena and suffix arena alike):
  *        [n_layers][2 (0 = K after RoPE, 1 = V)][n_kv_heads][n_slots][head_dim]
- *    in the model's storage type (bf16 models: K planes bfloat16, V planes IEEE half, both
+ *    in the model's storage type (bf16 models: K and V planes IEEE half, still
  *    2 bytes per element); a "slot" holds one token position.  A prompt or a
  *    rollout owns a contiguous range of slots given by its first slot (int64).
  *  - Index arrays are int32, slot numbers and token-buffer indices int64.
@@ -190,7 +190,16 @@ PC_API int pc_selftest_wait_timeout(void* stream, uint32_t spin_limit, int32_t* 
  * stated, not checked (the default). */
 PC_API int pc_set_index_bounds(pc_ctx* ctx, int n_prompts, int64_t n_tokens);
 
-/* bf16 models, decode steps: 1 (the default) issues the shared-prefix attention kernel and the per-rollout suffix attention
+/* bf16 models, decode steps that only sample (no logits_out, no log-probability buffer): 1 draws the token in
+ * the epilogue of the LM-head GEMM -- per 256-column tile of the vocabulary the largest and second-largest perturbed score
+ * and the arg-max, folded per row by a small second kernel -- so the step's [rows, vocab] logits are never written or read
+ * back; 0 (the default) stores the logits and runs the stand-alone sampler on them.  Both draw exactly the same tokens
+ * (Section 4.2: T = 1.0, top_p = 1.0; pc_sample states the rule).  The epilogue form scores a row per thread, without the
+ * warp-shared bound of the stand-alone sampler, and is the slower of the two on B200 (measured: +1.3 ms per step at 256
+ * rows, +5.9 ms at 2048); it is kept for callers that cannot afford the [rows, vocab] logits buffer.  Drops captured steps. */
+PC_API int pc_set_fused_sampler(pc_ctx* ctx, int on);
+
+/* bf16 models, decode steps: 1 issues the shared-prefix attention kernel and the per-rollout suffix attention
  * kernel of a layer on two streams (the second one is created by the context on first use and released by pc_destroy), so
  * that they can overlap; 0 (the default: measured no faster, both kernels fill the SMs) issues them one after the other.
  * Results are identical.  Drops captured decode steps. */

@@ -1,6 +1,6 @@
 // Shared-prefix decode attention for bf16 models, on tensor cores, with K/V tiles staged by TMA.
 //
-// The K/V arenas are viewed as 2-D bf16 tensors [planes * n_slots, head_dim]; a tile of TP consecutive
+// The K/V arenas are viewed as 2-D tensors of 16-bit elements (IEEE half) [planes * n_slots, head_dim]; a tile of TP consecutive
 // slots is fetched as head_dim/64 boxes of [TP rows x 64 columns] with the 128-byte swizzle, which makes
 // the ldmatrix reads below bank-conflict free.
 //
@@ -58,7 +58,7 @@ __device__ __forceinline__ void mma_bf16(float* c, uint32_t a0, uint32_t a1, uin
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-// P V product with P and V in IEEE half (V is stored as half in the arenas, see qkv_post_kernel)
+// Both attention products take IEEE half operands: q, K and V are stored as half (see qkv_post_kernel), P is rounded to half
 __device__ __forceinline__ void mma_f16(float* c, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
     asm volatile(
         "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
@@ -243,8 +243,8 @@ attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __
                 const int r = np * 16 + (lane & 7) + ((mat >> 1) << 3), d = ks * 16 + ((mat & 1) << 3);
                 uint32_t b0, b1, b2, b3;
                 ldsm_x4(kb + tile_off<G_TK>(r, d), b0, b1, b2, b3);
-                mma_bf16(s[2 * np], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
-                mma_bf16(s[2 * np + 1], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b2, b3);
+                mma_f16(s[2 * np], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
+                mma_f16(s[2 * np + 1], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b2, b3);
             }
         }
         // mask, online softmax (rows lane/4 and lane/4 + 8; a row lives in the four lanes of a quad)
@@ -527,7 +527,7 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
                         const int r = mt * 16 + (lane & 7) + ((mat & 1) << 3), d = ks * 16 + ((mat >> 1) << 3);
                         uint32_t a0, a1, a2, a3;
                         ldsm_x4(kb + tile_off<S_TP>(r, d), a0, a1, a2, a3);
-                        mma_bf16(s[mt], a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
+                        mma_f16(s[mt], a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
                     }
                 }
             }

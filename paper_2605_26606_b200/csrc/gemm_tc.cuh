@@ -18,6 +18,8 @@
 #include <cuda.h>
 #include <cuda_fp16.h>
 
+#include <cstring>
+
 #include "common.cuh"
 
 namespace pc {
@@ -137,7 +139,8 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n, bool half_operan
 // ---------------------------------------------------------------------------------------------
 // Epilogues: called once per (row, 32 consecutive columns); n_valid columns are inside N.
 // ---------------------------------------------------------------------------------------------
-struct EpiStoreF32 {            // C = acc (+ bias)
+struct EpiStoreF32 {
+    static constexpr bool kWholeTile = false;            // C = acc (+ bias)
     float* C; int ldc; const float* bias;
     __device__ __forceinline__ void set_rows(int) {}
     __device__ __forceinline__ void operator()(int row, int col0, const float* v, int n_valid, int /*split*/) const {
@@ -156,7 +159,8 @@ struct EpiStoreF32 {            // C = acc (+ bias)
         }
     }
 };
-struct EpiPartial {             // P[split][row][col] = acc   (raw K-slice sums; the consumer adds the slices in order)
+struct EpiPartial {
+    static constexpr bool kWholeTile = false;             // P[split][row][col] = acc   (raw K-slice sums; the consumer adds the slices in order)
     float* P; int ld; size_t split_stride;
     __device__ __forceinline__ void set_rows(int m) { split_stride = (size_t)m * ld; }     // slices packed by the row bound
     __device__ __forceinline__ void operator()(int row, int col0, const float* v, int n_valid, int split) const {
@@ -171,7 +175,8 @@ struct EpiPartial {             // P[split][row][col] = acc   (raw K-slice sums;
         }
     }
 };
-struct EpiResidual {            // H += acc
+struct EpiResidual {
+    static constexpr bool kWholeTile = false;            // H += acc
     float* H; int ldc;
     __device__ __forceinline__ void set_rows(int) {}
     __device__ __forceinline__ void operator()(int row, int col0, const float* v, int n_valid, int /*split*/) const {
@@ -190,7 +195,8 @@ struct EpiResidual {            // H += acc
         }
     }
 };
-struct EpiSwiGLU {              // columns (2j, 2j+1) = (gate_j, up_j) -> out[row, j] = silu(gate) * up, bf16 (or IEEE half)
+struct EpiSwiGLU {
+    static constexpr bool kWholeTile = false;              // columns (2j, 2j+1) = (gate_j, up_j) -> out[row, j] = silu(gate) * up, bf16 (or IEEE half)
     __nv_bfloat16* out; int ld; int half_out; int32_t* err;
     __device__ __forceinline__ void set_rows(int) {}
     __device__ __forceinline__ void operator()(int row, int col0, const float* v, int n_valid, int /*split*/) const {
@@ -274,20 +280,46 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (warp == 0) {
         if (lane == 0) {
             // ---------------- TMA producer ----------------
+            // The weight tiles of the first k-blocks are requested first, their activation tiles right after.
             uint32_t stage = 0, phase = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
-                const int m0 = (t % tiles_m) * BM, sp = (t / tiles_m) % splits, n0 = (t / (tiles_m * splits)) * BN;
-                const int kb0 = sp * k_blocks_total / splits, kb1 = (sp + 1) * k_blocks_total / splits;
-                for (int kb = kb0; kb < kb1; ++kb) {
-                    if (!mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-                    const uint32_t sa = tiles_u32 + stage * (A_BYTES + B_BYTES), sb = sa + A_BYTES;
-                    mbar_arrive_expect_tx(full0 + 8 * stage, A_BYTES + B_BYTES);
-                    tma_load_2d(sa, &map_a, full0 + 8 * stage, kb * BK, m0);
-                    if (DUAL) tma_load_2d(sa + A1_BYTES, &map_a_lo, full0 + 8 * stage, kb * BK, m0);
-                    tma_load_2d(sb, &map_w, full0 + 8 * stage, kb * BK, n0);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            struct Cursor { int t, kb, kb1, m0, n0; };
+            auto seek = [&](Cursor& c) {
+                if (c.t >= n_tiles) return;
+                const int sp = (c.t / tiles_m) % splits;
+                c.m0 = (c.t % tiles_m) * BM; c.n0 = (c.t / (tiles_m * splits)) * BN;
+                c.kb = sp * k_blocks_total / splits; c.kb1 = (sp + 1) * k_blocks_total / splits;
+            };
+            auto advance = [&](Cursor& c) { if (++c.kb == c.kb1) { c.t += gridDim.x; seek(c); } };
+            Cursor cb{(int)blockIdx.x, 0, 0, 0, 0};
+            seek(cb);
+            {
+                Cursor ca = cb;
+                int ahead = 0;
+                uint32_t stage_b = 0;
+                while (cb.t < n_tiles && ahead < STAGES) {          // the ring is empty: no wait needed
+                    mbar_arrive_expect_tx(full0 + 8 * stage_b, A_BYTES + B_BYTES);
+                    tma_load_2d(tiles_u32 + stage_b * (A_BYTES + B_BYTES) + A_BYTES, &map_w, full0 + 8 * stage_b, cb.kb * BK, cb.n0);
+                    ++ahead; ++stage_b;
+                    advance(cb);
                 }
+                for (; ahead > 0; --ahead) {
+                    const uint32_t sa = tiles_u32 + stage * (A_BYTES + B_BYTES);
+                    tma_load_2d(sa, &map_a, full0 + 8 * stage, ca.kb * BK, ca.m0);
+                    if (DUAL) tma_load_2d(sa + A1_BYTES, &map_a_lo, full0 + 8 * stage, ca.kb * BK, ca.m0);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    advance(ca);
+                }
+            }
+            while (cb.t < n_tiles) {
+                if (!mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                const uint32_t sa = tiles_u32 + stage * (A_BYTES + B_BYTES), sb = sa + A_BYTES;
+                mbar_arrive_expect_tx(full0 + 8 * stage, A_BYTES + B_BYTES);
+                tma_load_2d(sa, &map_a, full0 + 8 * stage, cb.kb * BK, cb.m0);
+                if (DUAL) tma_load_2d(sa + A1_BYTES, &map_a_lo, full0 + 8 * stage, cb.kb * BK, cb.m0);
+                tma_load_2d(sb, &map_w, full0 + 8 * stage, cb.kb * BK, cb.n0);
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                advance(cb);
             }
             if (!ok) { *abort_flag = 1; set_error(err, DEV_ERR_WAIT_TIMEOUT); }
         }
@@ -338,12 +370,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
             tc_fence_after();
             const int row = m0 + quarter * 32 + lane;
+            if constexpr (Epi::kWholeTile) {
+                // the epilogue walks the accumulator tile itself (more than one pass over its columns)
+                epi.template tile<BN>(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN, row, row < m_live, n0, N);
+            } else {
 #pragma unroll 1
-            for (int c = 0; c < BN; c += 32) {
-                if (n0 + c >= N) break;                 // warp-uniform
-                float v[32];
-                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + c, v);
-                if (row < m_live) epi(row, n0 + c, v, min(32, N - (n0 + c)), sp);
+                for (int c = 0; c < BN; c += 32) {
+                    if (n0 + c >= N) break;                 // warp-uniform
+                    float v[32];
+                    tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + c, v);
+                    if (row < m_live) epi(row, n0 + c, v, min(32, N - (n0 + c)), sp);
+                }
             }
             tc_fence_before();
             __syncwarp();
@@ -389,13 +426,16 @@ inline cudaError_t configure() {
 // Host launcher.  map_w must have been encoded with box_rows = BN; map_a_lo is ignored unless DUAL.
 template <int BN, bool DUAL, class Epi>
 inline cudaError_t launch(cudaStream_t st, const CUtensorMap& map_a, const CUtensorMap& map_a_lo, const CUtensorMap& map_w,
-                          const StepDesc* sd, int M, int N, int K, int splits, Epi epi, int32_t* err, int num_sms, bool half_operands = false) {
+                          const StepDesc* sd, int M, int N, int K, int splits, Epi epi, int32_t* err, int num_sms, bool half_operands = false,
+                          bool /*unused*/ = false) {
     auto kern = gemm_tc_kernel<BN, DUAL, Epi>;
     const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN) * splits;
     if (tiles == 0) return cudaSuccess;
-    kern<<<tiles < num_sms ? tiles : num_sms, NUM_THREADS, smem_bytes(BN, DUAL), st>>>(map_a, map_a_lo, map_w, sd, M, N, K, splits, epi, err,
-                                                                                       half_operands ? 1 : 0);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)(tiles < num_sms ? tiles : num_sms)); cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = smem_bytes(BN, DUAL); cfg.stream = st;
+    return cudaLaunchKernelEx(&cfg, kern, map_a, map_a_lo, map_w, sd, M, N, K, splits, epi, err, half_operands ? 1 : 0);
 }
 
 }  // namespace tc

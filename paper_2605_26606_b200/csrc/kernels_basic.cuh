@@ -466,11 +466,22 @@ __device__ __forceinline__ void qkv_post_items_warp(int lane, const QkvPostArgs<
                     x1[b][j] = y1; x2[b][j] = y2;
                 }
         }
+        // 16-bit models keep q, K and V as IEEE half (same two bytes, three more mantissa bits than bfloat16): the rounding of
+        // V, and for models with QK-norm that of q and K (their scores are of order one), is the largest single error source
+        // of the logits.  Values outside half's range are stored saturated and reported.
         if (is_q) {
             T* dst = A.q_out + (size_t)r * A.Hq * A.hd + (size_t)head * A.hd;
 #pragma unroll
             for (int j = 0; j < 2; ++j)
-                if (j < npair) { dst[lane + 32 * j] = from_f32<T>(x1[b][j]); dst[lane + 32 * j + half] = from_f32<T>(x2[b][j]); }
+                if (j < npair) {
+                    if (sizeof(T) == 2) {
+                        reinterpret_cast<__half*>(dst)[lane + 32 * j] = __float2half_rn(half_guard(x1[b][j], A.err));
+                        reinterpret_cast<__half*>(dst)[lane + 32 * j + half] = __float2half_rn(half_guard(x2[b][j], A.err));
+                    } else {
+                        dst[lane + 32 * j] = from_f32<T>(x1[b][j]);
+                        dst[lane + 32 * j + half] = from_f32<T>(x2[b][j]);
+                    }
+                }
             continue;
         }
         if (slot[b] < 0) continue;
@@ -478,9 +489,7 @@ __device__ __forceinline__ void qkv_post_items_warp(int lane, const QkvPostArgs<
         const int kvh = is_k ? head - A.Hq : head - A.Hq - A.Hkv;
         const int64_t plane = ((int64_t)A.layer * 2 + (is_k ? 0 : 1)) * A.Hkv + kvh;
         T* dst = reinterpret_cast<T*>(ar.base) + (plane * ar.n_slots + slot[b]) * A.hd;
-        if (!is_k && sizeof(T) == 2) {
-            // 16-bit models keep V as IEEE half (same two bytes, three more mantissa bits than bfloat16): V is a linear map
-            // of a unit-RMS vector, far inside half's range, and its rounding is the largest single error source of the logits
+        if (sizeof(T) == 2) {
             __half* dv = reinterpret_cast<__half*>(dst);
 #pragma unroll
             for (int j = 0; j < 2; ++j)

@@ -11,6 +11,7 @@
 #include <new>
 #include <string>
 #include <type_traits>
+#include <utility>
 #include <vector>
 
 #include "attention_mma.cuh"
@@ -20,6 +21,7 @@
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "kernels_basic.cuh"
+#include "lm_sample.cuh"
 #include "sampler.cuh"
 #include "stats.cuh"
 #include "tensor_map.h"
@@ -45,6 +47,15 @@ int cuda_fail(cudaError_t e, const char* what) {
         if (e__ != cudaSuccess) return cuda_fail(e__, what);        \
     } while (0)
 
+// Kernel launch through the extensible launch call (one place to add launch attributes).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -54,7 +65,7 @@ constexpr int kMaxSplits = pc::PARTIALS_MAX;
 struct Carve {
     size_t h, a, qkv, q, attn, act, logits, rope, pos, wslot, warena, p_start, p_len, s_start, s_len, token, last_row,
         part_m, part_l, part_o, res_part, step_desc, step_counter, max_slen, sample_scratch, a_lo, attn_lo, chain_layers, chain_glob,
-        chain_bar, dargs, key_prompt, key_rollout, key_step, out_index, group_start, total;
+        chain_bar, dargs, key_prompt, key_rollout, key_step, out_index, group_start, sample_tiles, total;
 };
 
 // A captured decode step, replayable for every step that fits the same upper bounds on the same KV arenas.  The
@@ -123,6 +134,7 @@ struct pc_ctx {
     int32_t n_prompts_hint = 0;              // pc_set_index_bounds: sizes of the caller's per-prompt arrays and token buffer (0: unknown)
     int64_t n_tokens_hint = 0;
 
+    int fused_sampler = 0;                   // decode steps that only sample: Gumbel-max in the LM head's epilogue, no logits stored
     int attn_overlap = 0;                    // decode: shared-prefix and suffix attention kernels of a layer on two streams
     cudaStream_t side_stream = nullptr;      // second branch of that fork (created on first use)
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
@@ -190,6 +202,8 @@ Carve carve(const pc_ctx* c, int max_rows, int max_prefill) {
     v.key_step = take(M * 4);
     v.out_index = take(M * 8);
     v.group_start = take((M + 1) * 4);
+    // fused LM head + sampler: one record per (vocabulary tile of the narrowest tile width, row)
+    v.sample_tiles = take((size_t)((d.vocab + 63) / 64) * (size_t)std::max(max_rows, 1) * sizeof(pc::Top2Rec));
     // prefix part of the shared-prefix attention: (max, sum, unnormalised output) per (row, query head)
     const size_t R = (size_t)std::max(max_rows, 1);
     v.part_m = take(pc::am::MAX_RECORDS * R * d.n_q_heads * 4);
@@ -331,6 +345,10 @@ cudaError_t configure_kernels() {
     if (e == cudaSuccess) e = tc::configure<64, true, tc::EpiStoreF32>();
     if (e == cudaSuccess) e = tc::configure<256, false, tc::EpiStoreF32>();
     if (e == cudaSuccess) e = tc::configure<64, false, tc::EpiStoreF32>();
+    if (e == cudaSuccess) e = tc::configure<256, true, EpiSample>();
+    if (e == cudaSuccess) e = tc::configure<64, true, EpiSample>();
+    if (e == cudaSuccess) e = tc::configure<256, false, EpiSample>();
+    if (e == cudaSuccess) e = tc::configure<64, false, EpiSample>();
     if (e == cudaSuccess) e = configure_attention<128>();
     if (e == cudaSuccess) e = configure_attention<64>();
     return e;
@@ -362,7 +380,7 @@ int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, in
                            d.n_kv_heads, sgrid * am::S_WARPS};
     const dim3 ggrid(q_tiles * n_parts, d.n_kv_heads, plan.n_groups);
     if (plan.prefill) {
-        am::attn_group_kernel<HD, true><<<ggrid, am::G_THREADS, am::group_smem_bytes<HD>(), st>>>(
+        launch_k(am::attn_group_kernel<HD, true>, dim3(ggrid), dim3(am::G_THREADS), am::group_smem_bytes<HD>(), st, 
             c->map_prompt_kv, sd, prompt_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, plan.group_row_start, g, scale_log2,
             part, attn, attn_lo, c->err);
         count_launches(1);
@@ -383,12 +401,12 @@ int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, in
         cudaStreamWaitEvent(c->side_stream, c->ev_fork, 0);
         gst = c->side_stream;
     }
-    am::attn_group_kernel<HD, false><<<ggrid, am::G_THREADS, am::group_smem_bytes<HD>(), gst>>>(
+    launch_k(am::attn_group_kernel<HD, false>, dim3(ggrid), dim3(am::G_THREADS), am::group_smem_bytes<HD>(), gst, 
         c->map_prompt_kv, sd, prompt_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, plan.group_row_start, g, scale_log2, part,
         attn, attn_lo, c->err);
     if (overlap) cudaEventRecord(c->ev_join, gst);
     c->mark(st, layer, PC_MARK_GROUP);
-    am::attn_suffix_kernel<HD><<<sgrid, am::S_WARPS * 32, am::suffix_smem_bytes<HD>(), st>>>(
+    launch_k(am::attn_suffix_kernel<HD>, dim3(sgrid), dim3(am::S_WARPS * 32), am::suffix_smem_bytes<HD>(), st, 
         c->map_suffix_kv, sd, suffix_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, g, scale_log2, part, c->err);
     if (overlap) cudaStreamWaitEvent(st, c->ev_join, 0);
     c->mark(st, layer, PC_MARK_SUFFIX);
@@ -397,7 +415,7 @@ int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, in
         count_launches(2);
         return PC_OK;
     }
-    am::attn_merge_kernel<HD><<<(M * d.n_q_heads + 7) / 8, 256, 0, st>>>(sd, d.n_q_heads, g, part, attn, attn_lo, c->err);
+    launch_k(am::attn_merge_kernel<HD>, dim3((M * d.n_q_heads + 7) / 8), dim3(256), 0, st, sd, d.n_q_heads, g, part, attn, attn_lo, c->err);
     c->mark(st, layer, PC_MARK_MERGE);
     count_launches(3);
     return PC_OK;
@@ -428,15 +446,15 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
     const Partials none{nullptr, 0, 0, 0};
     Partials pend = none;
 
-    rope_table_kernel<<<(M * half + 255) / 256, 256, 0, st>>>(sd, half, (double)d.rope_theta, g.pos, rope);
-    embed_rmsnorm_kernel<T><<<M, NORM_THREADS, 0, st>>>(sd, d.d_model, g.token, reinterpret_cast<const T*>(c->embed), c->attn_norm[0],
+    launch_k(rope_table_kernel, dim3((M * half + 255) / 256), dim3(256), 0, st, sd, half, (double)d.rope_theta, g.pos, rope);
+    launch_k(embed_rmsnorm_kernel<T>, dim3(M), dim3(NORM_THREADS), 0, st, sd, d.d_model, g.token, reinterpret_cast<const T*>(c->embed), c->attn_norm[0],
                                                d.rms_eps, h, a, a_lo, half_gemm ? 1 : 0, c->err);
     count_launches(2);
     PC_CUDA_CHECK_LAUNCH("embed_rmsnorm");
     for (int l = 0; l < d.n_layers; ++l) {
         c->mark(st, l, PC_MARK_LAYER_BEGIN);
         if (l > 0) {
-            rmsnorm_kernel<T><<<M, NORM_THREADS, 0, st>>>(sd, M, d.d_model, h, nullptr, pend, c->attn_norm[l], d.rms_eps, a, a_lo, half_gemm ? 1 : 0, c->err);
+            launch_k(rmsnorm_kernel<T>, dim3(M), dim3(NORM_THREADS), 0, st, sd, M, d.d_model, h, nullptr, pend, c->attn_norm[l], d.rms_eps, a, a_lo, half_gemm ? 1 : 0, c->err);
             pend = none;
             count_launches(1);
         }
@@ -455,7 +473,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
         }
         c->mark(st, l, PC_MARK_QKV);
         const int post_items = M * (d.n_q_heads + 2 * d.n_kv_heads);
-        qkv_post_kernel<T><<<(post_items + ROW_WARPS - 1) / ROW_WARPS, ROW_WARPS * 32, 0, st>>>(
+        launch_k(qkv_post_kernel<T>, dim3((post_items + ROW_WARPS - 1) / ROW_WARPS), dim3(ROW_WARPS * 32), 0, st, 
             sd, QkvPostArgs<T>{d.n_q_heads, d.n_kv_heads, d.head_dim, l, qkv_parts, bias, d.qk_norm ? c->q_norm[l] : nullptr,
                                d.qk_norm ? c->k_norm[l] : nullptr, d.rms_eps, rope, g, prompt_arena, suffix_arena, q, c->err});
         count_launches(2);
@@ -490,7 +508,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
             }
         }
         c->mark(st, l, PC_MARK_O);
-        rmsnorm_kernel<T><<<M, NORM_THREADS, 0, st>>>(sd, M, d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a, nullptr, half_gemm ? 1 : 0, c->err);
+        launch_k(rmsnorm_kernel<T>, dim3(M), dim3(NORM_THREADS), 0, st, sd, M, d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a, nullptr, half_gemm ? 1 : 0, c->err);
         pend = none;
         count_launches(2);
         c->mark(st, l, PC_MARK_NORM_MLP);
@@ -529,7 +547,7 @@ int run_lm_head(pc_ctx* c, cudaStream_t st, int n, const pc::StepDesc* sd, const
     const bool half_gemm = !std::is_same<T, float>::value && d.half_gemm != 0;
     T* a_lo = std::is_same<T, float>::value || half_gemm ? nullptr : reinterpret_cast<T*>(c->ws + c->cv.a_lo);
     c->mark(st, -1, PC_MARK_LM_BEGIN);
-    rmsnorm_kernel<T><<<n, NORM_THREADS, 0, st>>>(sd, n, d.d_model, h, src, c->pend, c->final_norm, d.rms_eps, a, a_lo, half_gemm ? 1 : 0, c->err);
+    launch_k(rmsnorm_kernel<T>, dim3(n), dim3(NORM_THREADS), 0, st, sd, n, d.d_model, h, src, c->pend, c->final_norm, d.rms_eps, a, a_lo, half_gemm ? 1 : 0, c->err);
     c->pend = pc::Partials{nullptr, 0, 0, 0};
     if constexpr (std::is_same<T, float>::value) {
         const T* wlm = reinterpret_cast<const T*>(d.tied_embed ? c->embed : c->lm_head);
@@ -542,6 +560,34 @@ int run_lm_head(pc_ctx* c, cudaStream_t st, int n, const pc::StepDesc* sd, const
     count_launches(2);
     c->mark(st, -1, PC_MARK_LM_HEAD);
     PC_CUDA_CHECK_LAUNCH("lm head");
+    return PC_OK;
+}
+
+// Final norm, LM head and the Gumbel-max draw in the GEMM's epilogue (lm_sample.cuh): the step's logits are not stored.
+int run_lm_head_sample(pc_ctx* c, cudaStream_t st, int n, const pc::StepDesc* sd, const pc::RowKeys& keys, const pc::DecodeArgsDev* da) {
+    using namespace pc;
+    using T = __nv_bfloat16;
+    const pc_model_desc& d = c->d;
+    float* h = reinterpret_cast<float*>(c->ws + c->cv.h);
+    T* a = reinterpret_cast<T*>(c->ws + c->cv.a);
+    const bool half_gemm = d.half_gemm != 0;
+    T* a_lo = half_gemm ? nullptr : reinterpret_cast<T*>(c->ws + c->cv.a_lo);
+    c->mark(st, -1, PC_MARK_LM_BEGIN);
+    launch_k(rmsnorm_kernel<T>, dim3(n), dim3(NORM_THREADS), 0, st, sd, n, d.d_model, h, nullptr, c->pend, c->final_norm, d.rms_eps, a, a_lo,
+             half_gemm ? 1 : 0, c->err);
+    c->pend = pc::Partials{nullptr, 0, 0, 0};
+    const GemmPlan gp = plan_gemm(c, GEMM_LM_HEAD, c->m_lm, n, false);
+    Top2Rec* rec = reinterpret_cast<Top2Rec*>(c->ws + c->cv.sample_tiles);
+    const int m_stride = std::max(c->max_rows, 1);
+    if (int rc = gemm_bf16(c, st, sd, c->map_a, half_gemm ? nullptr : &c->map_a_lo, c->m_lm, n, gp,
+                           EpiSample{rec, m_stride, keys.key_prompt, keys.rollout, keys.step_key, da}, half_gemm))
+        return rc;
+    c->mark(st, -1, PC_MARK_LM_HEAD);
+    const int bn = gp.wide ? 256 : 64;
+    launch_k(sample_tiles_reduce_kernel, dim3((n + 7) / 8), dim3(256), 0, st, sd, (d.vocab + bn - 1) / bn, rec, m_stride, keys.out_index, da);
+    count_launches(3);
+    c->mark(st, -1, PC_MARK_SAMPLE);
+    PC_CUDA_CHECK_LAUNCH("lm head with sampler");
     return PC_OK;
 }
 
@@ -605,6 +651,13 @@ int pc_set_gemm_plan(pc_ctx* ctx, const char* spec) {
     return PC_OK;
 }
 
+int pc_set_fused_sampler(pc_ctx* ctx, int on) {
+    if (ctx == nullptr || (on != 0 && on != 1)) return PC_ERR_INVALID_ARG;
+    if (on != ctx->fused_sampler) ctx->drop_graphs();
+    ctx->fused_sampler = on;
+    return PC_OK;
+}
+
 int pc_set_attention_overlap(pc_ctx* ctx, int on) {
     if (ctx == nullptr || (on != 0 && on != 1)) return PC_ERR_INVALID_ARG;
     if (on != ctx->attn_overlap) ctx->drop_graphs();
@@ -660,7 +713,7 @@ int pc_token_logprob(void* stream, int n_rows, int vocab, const float* logits, c
     if (n_rows < 0 || vocab <= 0 || !(temperature > 0.f)) return PC_ERR_INVALID_ARG;
     if (n_rows == 0) return PC_OK;
     if (logits == nullptr || tokens == nullptr || out_logprob == nullptr) return PC_ERR_INVALID_ARG;
-    pc::token_logprob_kernel<<<n_rows, 256, 0, static_cast<cudaStream_t>(stream)>>>(nullptr, vocab, logits, logits_row, temperature, tokens,
+    launch_k(pc::token_logprob_kernel, dim3(n_rows), dim3(256), 0, static_cast<cudaStream_t>(stream), nullptr, vocab, logits, logits_row, temperature, tokens,
                                                                                    tok_index, 0, out_logprob, out_index, 0, nullptr);
     count_launches(1);
     PC_CUDA_CHECK_LAUNCH("token_logprob");
@@ -828,7 +881,7 @@ int pc_prefill_shared(pc_ctx* ctx, void* stream, int n_prompts, const int32_t* p
     int32_t* last_row = reinterpret_cast<int32_t*>(ctx->ws + ctx->cv.last_row);
     pc::StepDesc* sd = reinterpret_cast<pc::StepDesc*>(ctx->ws + ctx->cv.step_desc);
     pc::set_step_desc<<<1, pc::STEP_DESC_THREADS, 0, st>>>(sd, total_tokens, n_prompts, max_prompt_len, g.max_slen, nullptr, 0);
-    pc::prep_prefill_rows<<<n_prompts, 256, 0, st>>>(n_prompts, prompt_tokens, prompt_offsets, prompt_kv_start, prompt_slots,
+    launch_k(pc::prep_prefill_rows, dim3(n_prompts), dim3(256), 0, st, n_prompts, prompt_tokens, prompt_offsets, prompt_kv_start, prompt_slots,
                                                      ctx->d.vocab, g, last_row, ctx->err);
     count_launches(2);
     PC_CUDA_CHECK_LAUNCH("prep_prefill_rows");
@@ -995,7 +1048,7 @@ int run_decode_chained(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd
     char* w = c->ws;
     const RowGeom g = geom(c);
     const int half = d.head_dim / 2;
-    rope_table_kernel<<<(M * half + 255) / 256, 256, 0, st>>>(sd, half, (double)d.rope_theta, g.pos, reinterpret_cast<float2*>(w + c->cv.rope));
+    launch_k(rope_table_kernel, dim3((M * half + 255) / 256), dim3(256), 0, st, sd, half, (double)d.rope_theta, g.pos, reinterpret_cast<float2*>(w + c->cv.rope));
     count_launches(1);
     PC_CUDA_CHECK_LAUNCH("rope table");
     if (int rc = launch_chain(c, st, M, sd, -1, prompt_arena, suffix_arena, nullptr, logits)) return rc;
@@ -1026,7 +1079,7 @@ int decode_launches(pc_ctx* ctx, cudaStream_t st, int m_bound, int groups_bound,
     ctx->prof_active_layer = -1;
     if (cap == cudaStreamCaptureStatusNone && ctx->prof_layer >= 0) { ctx->prof_active_layer = ctx->prof_layer; ctx->prof_layer = -1; }
     struct Disarm { pc_ctx* c; ~Disarm() { c->prof_active_layer = -1; } } disarm{ctx};
-    pc::prep_decode_rows<<<(m_bound + 128) / 128, 128, 0, st>>>(sd, da, a.prompt_slots, a.suffix_slots, ctx->d.vocab, g, keys, ctx->err);
+    launch_k(pc::prep_decode_rows, dim3((m_bound + 128) / 128), dim3(128), 0, st, sd, da, a.prompt_slots, a.suffix_slots, ctx->d.vocab, g, keys, ctx->err);
     count_launches(1);
     PC_CUDA_CHECK_LAUNCH("prep_decode_rows");
     const pc::KvArena pa{const_cast<void*>(a.prompt_kv), a.prompt_slots}, sa{a.suffix_kv, a.suffix_slots};
@@ -1040,6 +1093,10 @@ int decode_launches(pc_ctx* ctx, cudaStream_t st, int m_bound, int groups_bound,
     } else {
         rc = f32 ? run_layers<float>(ctx, st, m_bound, sd, pa, sa, plan) : run_layers<__nv_bfloat16>(ctx, st, m_bound, sd, pa, sa, plan);
         if (rc) return rc;
+        if (!f32 && a.sample && logits_out == nullptr && a.logprobs == nullptr && ctx->fused_sampler) {
+            // nobody asked for the logits: the draw happens in the LM head's epilogue and they are never stored
+            return run_lm_head_sample(ctx, st, m_bound, sd, keys, da);
+        }
         rc = f32 ? run_lm_head<float>(ctx, st, m_bound, sd, nullptr, logits) : run_lm_head<__nv_bfloat16>(ctx, st, m_bound, sd, nullptr, logits);
         if (rc) return rc;
     }
@@ -1047,19 +1104,19 @@ int decode_launches(pc_ctx* ctx, cudaStream_t st, int m_bound, int groups_bound,
         // keys, output positions, token buffer, temperature and seed come from the workspace copies / the argument block
         const int chunks = pc::sample_chunks(m_bound, ctx->num_sms);
         if (chunks == 1) {
-            pc::sample_kernel<<<m_bound, 256, 0, st>>>(sd, ctx->d.vocab, logits, nullptr, 1.f, 0u, 0u, keys.key_prompt, keys.rollout,
+            launch_k(pc::sample_kernel, dim3(m_bound), dim3(256), 0, st, sd, ctx->d.vocab, logits, nullptr, 1.f, 0u, 0u, keys.key_prompt, keys.rollout,
                                                        keys.step_key, 0, nullptr, keys.out_index, 0, nullptr, nullptr, da);
             count_launches(1);
         } else {
             pc::Top2Rec* scratch = reinterpret_cast<pc::Top2Rec*>(ctx->ws + ctx->cv.sample_scratch);
-            pc::sample_partial_kernel<<<dim3(m_bound, chunks), 256, 0, st>>>(sd, ctx->d.vocab, chunks, logits, nullptr, 1.f, 0u, 0u,
+            launch_k(pc::sample_partial_kernel, dim3(dim3(m_bound, chunks)), dim3(256), 0, st, sd, ctx->d.vocab, chunks, logits, nullptr, 1.f, 0u, 0u,
                                                                              keys.key_prompt, keys.rollout, keys.step_key, 0, scratch, nullptr, da);
-            pc::sample_reduce_kernel<<<(m_bound + 127) / 128, 128, 0, st>>>(sd, m_bound, chunks, scratch, nullptr, keys.out_index, 0,
+            launch_k(pc::sample_reduce_kernel, dim3((m_bound + 127) / 128), dim3(128), 0, st, sd, m_bound, chunks, scratch, nullptr, keys.out_index, 0,
                                                                             nullptr, da);
             count_launches(2);
         }
         if (a.logprobs != nullptr) {
-            pc::token_logprob_kernel<<<m_bound, 256, 0, st>>>(sd, ctx->d.vocab, logits, nullptr, 1.f, nullptr, keys.out_index, 0, nullptr,
+            launch_k(pc::token_logprob_kernel, dim3(m_bound), dim3(256), 0, st, sd, ctx->d.vocab, logits, nullptr, 1.f, nullptr, keys.out_index, 0, nullptr,
                                                               keys.out_index, 0, da);
             count_launches(1);
         }
@@ -1208,14 +1265,14 @@ int pc_sample(void* stream, int n_rows, int vocab, const float* logits, const in
         while (chunks > 1 && (size_t)n_rows * chunks * sizeof(pc::Top2Rec) > scratch_bytes) --chunks;    // use what fits
     }
     if (chunks == 1) {
-        pc::sample_kernel<<<n_rows, 256, 0, st>>>(nullptr, vocab, logits, logits_row, temperature, k0, k1, row_prompt, row_rollout,
+        launch_k(pc::sample_kernel, dim3(n_rows), dim3(256), 0, st, nullptr, vocab, logits, logits_row, temperature, k0, k1, row_prompt, row_rollout,
                                                   row_step, 0, out_tokens, out_index, 0, out_top2_gap, nullptr, nullptr);
         count_launches(1);
     } else {
         pc::Top2Rec* rec = static_cast<pc::Top2Rec*>(scratch);
-        pc::sample_partial_kernel<<<dim3(n_rows, chunks), 256, 0, st>>>(nullptr, vocab, chunks, logits, logits_row, temperature, k0, k1,
+        launch_k(pc::sample_partial_kernel, dim3(dim3(n_rows, chunks)), dim3(256), 0, st, nullptr, vocab, chunks, logits, logits_row, temperature, k0, k1,
                                                                         row_prompt, row_rollout, row_step, 0, rec, nullptr, nullptr);
-        pc::sample_reduce_kernel<<<(n_rows + 127) / 128, 128, 0, st>>>(nullptr, n_rows, chunks, rec, out_tokens, out_index, 0,
+        launch_k(pc::sample_reduce_kernel, dim3((n_rows + 127) / 128), dim3(128), 0, st, nullptr, n_rows, chunks, rec, out_tokens, out_index, 0,
                                                                        out_top2_gap, nullptr);
         count_launches(2);
     }
@@ -1345,9 +1402,9 @@ int pc_sample_static(void* stream, int n_rows, int vocab, const float* logits, c
     const uint32_t k0 = (uint32_t)(seed & 0xffffffffu), k1 = (uint32_t)(seed >> 32);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // every record the second kernel reads is written by the first one in this same call: nothing has to start at zero
-    pc::sample_partial_kernel<<<dim3(n_rows, chunks), 256, 0, st>>>(nullptr, vocab, chunks, logits, logits_row, temperature, k0, k1,
+    launch_k(pc::sample_partial_kernel, dim3(dim3(n_rows, chunks)), dim3(256), 0, st, nullptr, vocab, chunks, logits, logits_row, temperature, k0, k1,
                                                                     row_prompt, row_rollout, row_step, 0, rec, nullptr, nullptr);
-    pc::sample_reduce_kernel<<<(n_rows + 127) / 128, 128, 0, st>>>(nullptr, n_rows, chunks, rec, out_tokens, out_index, 0, out_top2_gap, nullptr);
+    launch_k(pc::sample_reduce_kernel, dim3((n_rows + 127) / 128), dim3(128), 0, st, nullptr, n_rows, chunks, rec, out_tokens, out_index, 0, out_top2_gap, nullptr);
     count_launches(2);
     PC_CUDA_CHECK_LAUNCH("sample (static scratch)");
     return PC_OK;

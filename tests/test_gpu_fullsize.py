@@ -71,7 +71,7 @@ def compare_rollout_windows(dec, w, batch, out, p, i, windows, records, last_log
     toks = out["tokens"][p][i]
     Lp = int(batch.prompt_lens[p])
     pt = batch.prompt_tokens[batch.prompt_offsets[p]:batch.prompt_offsets[p + 1]]
-    steps = [s for s0 in windows for s in range(s0, s0 + WINDOW) if s + 1 < len(toks)]
+    steps = [s for s0 in windows for s in range(s0, s0 + WINDOW) if s + 1 < len(toks) and s in records]
     assert steps, (p, i, len(toks), windows)
     upto = max(steps) + 1                                       # decode step s consumes generated token s
     positions = [Lp + s for s in steps] + ([Lp - 1] if last_logits is not None else [])
@@ -195,3 +195,4 @@ def test_config1_full_step(shape_1p5b):
     w2, n2, _ = compare_rollout_windows(dec, w, batch, out, pa, cand[pa][1], windows, eng.record_commit_logits)
     assert n1 + n2 == 2 * WINDOW + 1 and max(w1, w2) <= 5e-2, (n1, n2, w1, w2)
     _free(eng)
+

@@ -1,0 +1,53 @@
+"""BASELINE configs 3 and 4 (Qwen3-8B and 14B shapes) at full width and depth, kept in a module of their own so that the host
+memory of the 1.5B-shape tests is released first."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle.decoder import Decoder
+from paper_2605_26606_b200 import workloads as wl
+from paper_2605_26606_b200.engine import RolloutEngine
+
+from gpu_util import ensure_built
+from test_gpu_fullsize import _free, check_step_invariants, compare_rollout_windows
+
+pytestmark = pytest.mark.gpu
+
+
+def _large_model_slice(workload_name, n_check_steps=6):
+    """BASELINE configs 3 and 4 at full width and depth: the whole Pilot-Commit step (every rollout to its cap) with the
+    invariants that hold at any size, and the logits of one pilot rollout at the first decode steps against the oracle
+    (single precision here: the 8B / 14B shapes would otherwise take many minutes of float64 host arithmetic; 5e-2 is two
+    orders of magnitude above float32's own error)."""
+    ensure_built()
+    w = wl.WORKLOADS[workload_name]
+    weights = wl.gen_weights(w.model, seed=0, threads=16)
+    batch = wl.gen_batch(w)
+    P, G, k = w.n_prompts, w.group_size, w.n_pilot
+    eng = RolloutEngine(w.model, weights, max_rows=max(P * k, P * (G - k)), max_prefill_tokens=int(batch.prompt_offsets[-1]))
+    eng.record_pilot_logits = {s: None for s in range(n_check_steps)}
+    p0 = 0
+    i0 = int(np.argmax(batch.caps[p0, :k]))
+    eng.record_rows = {(p0, i0)}
+    out = eng.pilot_commit_step(w, batch)
+    check_step_invariants(out, w, batch)
+    last_logits = eng.last_logits.cpu().numpy()
+    records = eng.record_pilot_logits
+    _free(eng)
+    dec = Decoder(w.model, weights, dtype=np.float32, cache_weights=False)
+    worst, n_cmp, _ = compare_rollout_windows(dec, w, batch, out, p0, i0, [0], {s: records[s] for s in range(n_check_steps)}, last_logits)
+    assert n_cmp >= n_check_steps and worst <= 5e-2, (n_cmp, worst)
+    return out
+
+
+def test_config3_qwen3_8b_shape_full_step(cuda_device):
+    out = _large_model_slice("config3")
+    assert out["generated_tokens"] > 0
+
+
+@pytest.mark.skipif(os.environ.get("PC_SKIP_CONFIG4") == "1",
+                    reason="the 14B shape needs about 30 GB of host memory for its weights and three more minutes; PC_SKIP_CONFIG4=1 leaves it out")
+def test_config4_qwen3_14b_shape_full_step(cuda_device):
+    out = _large_model_slice("config4")
+    assert out["generated_tokens"] > 0

@@ -433,3 +433,33 @@ def test_half_operands_out_of_range_are_saturated_and_flagged():
     weights2 = wl.gen_weights(model, seed=1, threads=2)
     eng2 = RolloutEngine(model, weights2, max_rows=8, max_prefill_tokens=int(batch.prompt_offsets[-1]))
     eng2.pilot_commit_step(w, batch)
+
+
+@pytest.mark.parametrize("vocab,half_gemm", [(4096, True), (20004, True), (20004, False)], ids=["narrow-tiles", "wide-tiles-ragged-vocab", "bf16-operands"])
+def test_sampler_in_the_lm_head_epilogue_draws_the_same_tokens(vocab, half_gemm):
+    """pc_set_fused_sampler: the Gumbel-max draw inside the LM-head GEMM (no logits stored) against the stand-alone sampler on
+    stored logits, free running over a whole Pilot-Commit step: every token identical, and the oracle's tokens wherever its
+    top-two gap is clear (checked teacher-forced by the tests above for the stored-logits path)."""
+    from paper_2605_26606_b200 import binding as B
+    model = dataclasses.replace(wl.SMALL_BF16, name=f"small-bf16-v{vocab}", vocab=vocab)
+    w = dataclasses.replace(wl.WORKLOADS["config0"], model=model, n_prompts=5, prompt_len_lo=3, prompt_len_hi=90, group_size=40,
+                            n_pilot=8, max_new=30, cap_lo=1, cap_hi=30, data_seed=23,
+                            forced_explicit=((0, 0.5), (1, 0.5), (2, 0.5), (3, 0.0), (4, 0.5)))
+    weights = wl.gen_weights(model, seed=0, threads=2, gain_jitter=0.1)
+    batch = wl.gen_batch(w)
+    eng = RolloutEngine(model, weights, max_rows=200, max_prefill_tokens=int(batch.prompt_offsets[-1]), half_gemm=half_gemm)
+    outs = []
+    for fused in (0, 1):
+        B.pc_set_fused_sampler(eng.ctx, fused)
+        n0 = B.pc_launch_count()
+        outs.append(eng.pilot_commit_step(w, batch))
+    a, b = outs
+    assert np.array_equal(a["status"], b["status"]) and np.any(a["status"] == ostats.COMMIT)
+    n_tok = 0
+    for p in range(w.n_prompts):
+        for i in range(w.group_size):
+            if a["generated"][p, i]:
+                assert np.array_equal(a["tokens"][p][i], b["tokens"][p][i]), (p, i)
+                n_tok += len(a["tokens"][p][i])
+    assert n_tok > 1000
+    assert np.array_equal(a["advantages"], b["advantages"])
