@@ -162,6 +162,7 @@ def run_probe(args):
     B.pc_set_decode_mode(eng.ctx, int(kv.get("mode", 0)))
     B.pc_set_attention_overlap(eng.ctx, int(kv.get("overlap", 0)))
     B.pc_set_fused_sampler(eng.ctx, int(kv.get("fused", 0)))
+    B.pc_set_fused_epilogues(eng.ctx, int(kv.get("epi", 1)))
     eng.load_batch(w, batch)
     eng.suffix_kv.zero_()
     eng.tokens.random_(0, w.model.vocab)

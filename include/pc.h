@@ -190,6 +190,15 @@ PC_API int pc_selftest_wait_timeout(void* stream, uint32_t spin_limit, int32_t* 
  * stated, not checked (the default). */
 PC_API int pc_set_index_bounds(pc_ctx* ctx, int n_prompts, int64_t n_tokens);
 
+/* bf16 models with half_gemm = 1 and head_dim 128, passes of more than 256 rows.  1 (the default): two row-wise kernels
+ * of every layer run inside GEMM epilogues instead -- bias / QK-norm / RoPE / KV append in the QKV projection's, and the residual add, the operand of the
+ * gate/up projection and the RMSNorm's sum of squares in the output projection's, the norm's 1/rms being applied by the
+ * gate/up epilogue (RMSNorm(h; g) W^T = rstd * ((h * g) W^T)).  The two projections then run without K split, which is why
+ * smaller passes keep the separate kernels (their projections need the split to fill the GPU).  0: one kernel per
+ * operation throughout, as for every other model type.  Same mathematics, different rounding order (both inside the
+ * tolerances the tests state).  Drops captured decode steps.  The paper has no counterpart. */
+PC_API int pc_set_fused_epilogues(pc_ctx* ctx, int on);
+
 /* bf16 models, decode steps that only sample (no logits_out, no log-probability buffer): 1 draws the token in
  * the epilogue of the LM-head GEMM -- per 256-column tile of the vocabulary the largest and second-largest perturbed score
  * and the arg-max, folded per row by a small second kernel -- so the step's [rows, vocab] logits are never written or read

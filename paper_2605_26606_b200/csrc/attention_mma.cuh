@@ -643,14 +643,39 @@ attn_suffix_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* _
 // rh = row * Hq + head (the caller keeps it below n_live * Hq).  ct = tiles per suffix chunk of this step (suffix_plan);
 // n_load > 0 = how many records to request: every record index the step can have produced (part.n_parts + chunk slots per
 // item), so that the loads do not wait for the row's suffix length; records past the row's own count are ignored.
-// n_load <= 0: wait for the suffix length and request the row's own records only.
-template <int HD>
+// STREAM: wait for the suffix length and request the row's own records only, one after the other (n_load is not used).
+template <int HD, bool STREAM = false>
 __device__ __forceinline__ void merge_item_warp(int lane, size_t rh, int Hq, const RowGeom& g, const PrefixPartial& part, int ct, int n_load,
                                                 __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ out_lo, int32_t* err) {
     constexpr int EPL = HD / 32;
     const int row = (int)(rh / Hq);
     const int slen = g.s_len[row];
-    if (n_load <= 0) n_load = part.n_parts + suffix_chunks(slen, ct);      // large batches: request only the row's own records
+    float M = -INFINITY;
+    float acc[EPL];
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+    float denom = 0.f;
+    if constexpr (STREAM) {
+        // Large batches: the row's own records only, streamed (few registers, so many warps are resident): first the
+        // largest m, then the weighted sums in index order -- the same operations in the same order as below.
+        const int n_own = part.n_parts + suffix_chunks(slen, ct);
+        for (int i = 0; i < n_own; ++i) M = fmaxf(M, part.m[(size_t)i * part.stride + rh]);
+#pragma unroll 2
+        for (int i = 0; i < n_own; ++i) {
+            const float w = exp2_safe(part.m[(size_t)i * part.stride + rh], M);
+            if (w > 0.f) {
+                denom += part.l[(size_t)i * part.stride + rh] * w;
+                const float* src = part.o + ((size_t)i * part.stride + rh) * HD + lane * EPL;
+                if (EPL == 4) {
+                    const float4 v = *reinterpret_cast<const float4*>(src);
+                    acc[0] += v.x * w; acc[1] += v.y * w; acc[2] += v.z * w; acc[3] += v.w * w;
+                } else {
+                    const float2 v = *reinterpret_cast<const float2*>(src);
+                    acc[0] += v.x * w; acc[1] += v.y * w;
+                }
+            }
+        }
+    } else {
     float mi[MAX_RECORDS], li[MAX_RECORDS];
     float ov[MAX_RECORDS][EPL];
 #pragma unroll
@@ -671,13 +696,8 @@ __device__ __forceinline__ void merge_item_warp(int lane, size_t rh, int Hq, con
 #pragma unroll
     for (int i = 0; i < MAX_RECORDS; ++i)
         if (i >= n_rec) mi[i] = -INFINITY;           // not a record of this row (stale memory)
-    float M = -INFINITY;
 #pragma unroll
     for (int i = 0; i < MAX_RECORDS; ++i) M = fmaxf(M, mi[i]);
-    float acc[EPL];
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
-    float denom = 0.f;
 #pragma unroll
     for (int i = 0; i < MAX_RECORDS; ++i) {
         const float w = exp2_safe(mi[i], M);
@@ -686,6 +706,7 @@ __device__ __forceinline__ void merge_item_warp(int lane, size_t rh, int Hq, con
 #pragma unroll
             for (int e = 0; e < EPL; ++e) acc[e] += ov[i][e] * w;
         }
+    }
     }
     const float inv = denom > 0.f ? 1.f / denom : 0.f;
     float lo[EPL];
@@ -711,15 +732,16 @@ __device__ __forceinline__ void merge_item_warp(int lane, size_t rh, int Hq, con
 }
 
 // Stand-alone form: the grid covers the row bound of the step.
-template <int HD>
+template <int HD, bool STREAM>
 __global__ void __launch_bounds__(256) attn_merge_kernel(const StepDesc* __restrict__ sd, int Hq, RowGeom g, PrefixPartial part,
                                                          __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ out_lo, int32_t* err) {
     const size_t rh = (size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int n_live = sd->n_rows;
     if (rh >= (size_t)n_live * Hq) return;
     const SuffixPlan sp = suffix_plan(*g.max_slen, n_live * part.n_kv_heads, part.n_suffix_warps);
-    // few items: request every record slot of the step at once (latency); many items: only the row's own records (bytes)
-    merge_item_warp<HD>(threadIdx.x & 31, rh, Hq, g, part, sp.ct, n_live * Hq <= 8192 ? part.n_parts + sp.cpi : 0, out, out_lo, err);
+    // few items (host: STREAM = false): request every record slot of the step at once (latency); many items: only the row's
+    // own records, with few registers (occupancy)
+    merge_item_warp<HD, STREAM>(threadIdx.x & 31, rh, Hq, g, part, sp.ct, part.n_parts + sp.cpi, out, out_lo, err);
 }
 
 }  // namespace am

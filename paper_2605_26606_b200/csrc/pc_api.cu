@@ -19,6 +19,7 @@
 #include "common.cuh"
 #include "decode_chain.cuh"
 #include "gemm_simt.cuh"
+#include "gemm_epilogues.cuh"
 #include "gemm_tc.cuh"
 #include "kernels_basic.cuh"
 #include "lm_sample.cuh"
@@ -65,7 +66,7 @@ constexpr int kMaxSplits = pc::PARTIALS_MAX;
 struct Carve {
     size_t h, a, qkv, q, attn, act, logits, rope, pos, wslot, warena, p_start, p_len, s_start, s_len, token, last_row,
         part_m, part_l, part_o, res_part, step_desc, step_counter, max_slen, sample_scratch, a_lo, attn_lo, chain_layers, chain_glob,
-        chain_bar, dargs, key_prompt, key_rollout, key_step, out_index, group_start, sample_tiles, total;
+        chain_bar, dargs, key_prompt, key_rollout, key_step, out_index, group_start, sample_tiles, ssq, total;
 };
 
 // A captured decode step, replayable for every step that fits the same upper bounds on the same KV arenas.  The
@@ -134,6 +135,7 @@ struct pc_ctx {
     int32_t n_prompts_hint = 0;              // pc_set_index_bounds: sizes of the caller's per-prompt arrays and token buffer (0: unknown)
     int64_t n_tokens_hint = 0;
 
+    int fused_epilogues = 1;                 // half-operand models with head_dim 128: QKV post-processing and the MLP norm inside GEMM epilogues
     int fused_sampler = 0;                   // decode steps that only sample: Gumbel-max in the LM head's epilogue, no logits stored
     int attn_overlap = 0;                    // decode: shared-prefix and suffix attention kernels of a layer on two streams
     cudaStream_t side_stream = nullptr;      // second branch of that fork (created on first use)
@@ -202,6 +204,7 @@ Carve carve(const pc_ctx* c, int max_rows, int max_prefill) {
     v.key_step = take(M * 4);
     v.out_index = take(M * 8);
     v.group_start = take((M + 1) * 4);
+    v.ssq = take((size_t)((d.d_model + 63) / 64) * M * 4);       // per-tile sums of squares of the residual rows (EpiResNorm)
     // fused LM head + sampler: one record per (vocabulary tile of the narrowest tile width, row)
     v.sample_tiles = take((size_t)((d.vocab + 63) / 64) * (size_t)std::max(max_rows, 1) * sizeof(pc::Top2Rec));
     // prefix part of the shared-prefix attention: (max, sum, unnormalised output) per (row, query head)
@@ -286,6 +289,18 @@ int gemm_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, const CUtensor
     return PC_OK;
 }
 
+// Unsplit GEMM with an explicit tile width (the fused epilogues need complete sums in a tile).
+template <int BN, class Epi>
+int gemm_half_bn(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, const CUtensorMap& map_a, const WMap& w, int M, Epi epi) {
+    const CUtensorMap& mw = BN == 256 ? w.wide : (BN == 128 ? w.mid : w.narrow);
+    const cudaError_t e = pc::tc::launch<BN, false>(st, map_a, map_a, mw, sd, M, w.N, w.K, 1, epi, c->err, c->num_sms, true);
+    if (e != cudaSuccess) return cuda_fail(e, "tensor-core gemm (fused epilogue)");
+    return PC_OK;
+}
+inline bool wide_tiles_fill_the_gpu(const pc_ctx* c, int M, int N) {
+    return ((M + pc::tc::BM - 1) / pc::tc::BM) * ((N + 255) / 256) >= c->num_sms / 2;
+}
+
 // How the rows of a forward pass group for attention.
 struct AttnPlan {
     bool prefill;                      // true: causal attention inside each prompt, no suffix part
@@ -345,6 +360,12 @@ cudaError_t configure_kernels() {
     if (e == cudaSuccess) e = tc::configure<64, true, tc::EpiStoreF32>();
     if (e == cudaSuccess) e = tc::configure<256, false, tc::EpiStoreF32>();
     if (e == cudaSuccess) e = tc::configure<64, false, tc::EpiStoreF32>();
+    if (e == cudaSuccess) e = tc::configure<128, false, EpiQkvPost>();
+    if (e == cudaSuccess) e = tc::configure<256, false, EpiQkvPost>();
+    if (e == cudaSuccess) e = tc::configure<64, false, EpiResNorm>();
+    if (e == cudaSuccess) e = tc::configure<256, false, EpiResNorm>();
+    if (e == cudaSuccess) e = tc::configure<64, false, EpiSwiGLUNorm>();
+    if (e == cudaSuccess) e = tc::configure<256, false, EpiSwiGLUNorm>();
     if (e == cudaSuccess) e = tc::configure<256, true, EpiSample>();
     if (e == cudaSuccess) e = tc::configure<64, true, EpiSample>();
     if (e == cudaSuccess) e = tc::configure<256, false, EpiSample>();
@@ -415,7 +436,10 @@ int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, in
         count_launches(2);
         return PC_OK;
     }
-    launch_k(am::attn_merge_kernel<HD>, dim3((M * d.n_q_heads + 7) / 8), dim3(256), 0, st, sd, d.n_q_heads, g, part, attn, attn_lo, c->err);
+    if ((long long)M * d.n_q_heads > 8192)
+        launch_k(am::attn_merge_kernel<HD, true>, dim3((M * d.n_q_heads + 7) / 8), dim3(256), 0, st, sd, d.n_q_heads, g, part, attn, attn_lo, c->err);
+    else
+        launch_k(am::attn_merge_kernel<HD, false>, dim3((M * d.n_q_heads + 7) / 8), dim3(256), 0, st, sd, d.n_q_heads, g, part, attn, attn_lo, c->err);
     c->mark(st, layer, PC_MARK_MERGE);
     count_launches(3);
     return PC_OK;
@@ -437,6 +461,13 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
     T* attn = reinterpret_cast<T*>(w + c->cv.attn);
     T* act = reinterpret_cast<T*>(w + c->cv.act);
     const bool half_gemm = !kF32 && d.half_gemm != 0;      // every GEMM operand in IEEE half
+    // QKV post-processing in the QKV GEMM's epilogue; residual add, operand of the gate/up GEMM and the norm's sum of squares
+    // in the output projection's epilogue, its 1/rms applied by the gate/up epilogue (gemm_epilogues.cuh)
+    // From three row tiles on: below that the two projections need their K split to keep the SMs busy (measured: unsplit they
+    // lose more than the two small kernels cost), and a split GEMM's tile does not hold complete sums.
+    const bool fused = half_gemm && d.head_dim == 128 && d.d_model % 64 == 0 && c->fused_epilogues != 0 && M > 2 * tc::BM;
+    float* ssq = reinterpret_cast<float*>(w + c->cv.ssq);
+    const int m_stride = std::max(std::max(c->max_rows, c->max_prefill), 1);
     T* a_lo = kF32 || half_gemm ? nullptr : reinterpret_cast<T*>(w + c->cv.a_lo);          // rounding remainders (bf16 operands only)
     float2* rope = reinterpret_cast<float2*>(w + c->cv.rope);
     const RowGeom g = geom(c);
@@ -445,6 +476,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
     float* res_part = reinterpret_cast<float*>(w + c->cv.res_part);
     const Partials none{nullptr, 0, 0, 0};
     Partials pend = none;
+    int n_ssq = 0;
 
     launch_k(rope_table_kernel, dim3((M * half + 255) / 256), dim3(256), 0, st, sd, half, (double)d.rope_theta, g.pos, rope);
     launch_k(embed_rmsnorm_kernel<T>, dim3(M), dim3(NORM_THREADS), 0, st, sd, d.d_model, g.token, reinterpret_cast<const T*>(c->embed), c->attn_norm[0],
@@ -464,6 +496,12 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
         if constexpr (kF32) {
             launch_gemm_simt<T>(st, sd, a, reinterpret_cast<const T*>(c->wqkv[l]), M, c->n_qkv(), d.d_model,
                                 EpiStoreF32{qkv, c->n_qkv(), nullptr});
+        } else if (fused) {
+            const EpiQkvPost epi{d.n_q_heads, d.n_kv_heads, l, bias, d.qk_norm ? c->q_norm[l] : nullptr, d.qk_norm ? c->k_norm[l] : nullptr,
+                                 d.rms_eps, rope, g, prompt_arena, suffix_arena, reinterpret_cast<__half*>(q), c->err};
+            const int rc = wide_tiles_fill_the_gpu(c, M, c->n_qkv()) ? gemm_half_bn<256>(c, st, sd, c->map_a, c->m_wqkv[l], M, epi)
+                                                                     : gemm_half_bn<128>(c, st, sd, c->map_a, c->m_wqkv[l], M, epi);
+            if (rc) return rc;
         } else {
             const GemmPlan gp = plan_gemm(c, GEMM_QKV, c->m_wqkv[l], M, true);
             qkv_parts.n = gp.splits;
@@ -473,10 +511,10 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
         }
         c->mark(st, l, PC_MARK_QKV);
         const int post_items = M * (d.n_q_heads + 2 * d.n_kv_heads);
-        launch_k(qkv_post_kernel<T>, dim3((post_items + ROW_WARPS - 1) / ROW_WARPS), dim3(ROW_WARPS * 32), 0, st, 
+        if (!fused) launch_k(qkv_post_kernel<T>, dim3((post_items + ROW_WARPS - 1) / ROW_WARPS), dim3(ROW_WARPS * 32), 0, st, 
             sd, QkvPostArgs<T>{d.n_q_heads, d.n_kv_heads, d.head_dim, l, qkv_parts, bias, d.qk_norm ? c->q_norm[l] : nullptr,
                                d.qk_norm ? c->k_norm[l] : nullptr, d.rms_eps, rope, g, prompt_arena, suffix_arena, q, c->err});
-        count_launches(2);
+        count_launches(fused ? 1 : 2);
         c->mark(st, l, PC_MARK_POST);
         if constexpr (kF32) {
             c->mark(st, l, PC_MARK_GROUP);
@@ -496,7 +534,14 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
                          : attention_bf16<64>(c, st, sd, M, l, plan, prompt_arena, suffix_arena, q, attn);
             if (rc) return rc;
             const GemmPlan gp = plan_gemm(c, GEMM_O, c->m_wo[l], M, true);
-            if (gp.splits == 1) {
+            if (fused) {
+                const bool wide = wide_tiles_fill_the_gpu(c, M, d.d_model);
+                n_ssq = (d.d_model + (wide ? 256 : 64) - 1) / (wide ? 256 : 64);
+                const EpiResNorm epi{h, d.d_model, c->mlp_norm[l], reinterpret_cast<__half*>(a), ssq, m_stride, c->err};
+                const int rc2 = wide ? gemm_half_bn<256>(c, st, sd, c->map_attn, c->m_wo[l], M, epi)
+                                     : gemm_half_bn<64>(c, st, sd, c->map_attn, c->m_wo[l], M, epi);
+                if (rc2) return rc2;
+            } else if (gp.splits == 1) {
                 if (int rc2 = gemm_bf16(c, st, sd, c->map_attn, half_gemm ? nullptr : &c->map_attn_lo, c->m_wo[l], M, gp,
                                         tc::EpiResidual{h, d.d_model}, half_gemm))
                     return rc2;
@@ -508,15 +553,28 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
             }
         }
         c->mark(st, l, PC_MARK_O);
-        launch_k(rmsnorm_kernel<T>, dim3(M), dim3(NORM_THREADS), 0, st, sd, M, d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a, nullptr, half_gemm ? 1 : 0, c->err);
+        if (!fused) launch_k(rmsnorm_kernel<T>, dim3(M), dim3(NORM_THREADS), 0, st, sd, M, d.d_model, h, nullptr, pend, c->mlp_norm[l], d.rms_eps, a, nullptr, half_gemm ? 1 : 0, c->err);
         pend = none;
-        count_launches(2);
+        count_launches(fused ? 1 : 2);
         c->mark(st, l, PC_MARK_NORM_MLP);
         if constexpr (kF32) {
             launch_gemm_simt<T>(st, sd, a, reinterpret_cast<const T*>(c->w_gate_up[l]), M, 2 * d.d_ff, d.d_model,
                                 EpiSwiGLU<T>{act, d.d_ff});
             c->mark(st, l, PC_MARK_GATE_UP);
             launch_gemm_simt<T>(st, sd, act, reinterpret_cast<const T*>(c->w_down[l]), M, d.d_model, d.d_ff, EpiResidual{h, d.d_model});
+        } else if (fused) {
+            const EpiSwiGLUNorm epi{reinterpret_cast<__half*>(act), d.d_ff, ssq, n_ssq, m_stride, d.d_model, d.rms_eps, c->err};
+            const int rc = plan_gemm(c, GEMM_GATE_UP, c->m_wgu[l], M, false).wide ? gemm_half_bn<256>(c, st, sd, c->map_a, c->m_wgu[l], M, epi)
+                                                                                  : gemm_half_bn<64>(c, st, sd, c->map_a, c->m_wgu[l], M, epi);
+            if (rc) return rc;
+            c->mark(st, l, PC_MARK_GATE_UP);
+            const GemmPlan gp = plan_gemm(c, GEMM_DOWN, c->m_wdown[l], M, true);
+            if (gp.splits == 1) {
+                if (int rc2 = gemm_bf16(c, st, sd, c->map_act, nullptr, c->m_wdown[l], M, gp, tc::EpiResidual{h, d.d_model}, half_gemm)) return rc2;
+            } else {
+                pend = Partials{res_part, gp.splits, (size_t)M * d.d_model, d.d_model};
+                if (int rc2 = gemm_bf16(c, st, sd, c->map_act, nullptr, c->m_wdown[l], M, gp, tc::EpiPartial{res_part, d.d_model, pend.stride}, half_gemm)) return rc2;
+            }
         } else {
             if (int rc = gemm_bf16(c, st, sd, c->map_a, nullptr, c->m_wgu[l], M, plan_gemm(c, GEMM_GATE_UP, c->m_wgu[l], M, false), tc::EpiSwiGLU{act, d.d_ff, half_gemm ? 1 : 0, c->err}, half_gemm))
                 return rc;
@@ -648,6 +706,13 @@ int pc_set_gemm_plan(pc_ctx* ctx, const char* spec) {
     }
     for (int k = 0; k < 5; ++k) { ctx->plan_bn[k] = bn[k]; ctx->plan_splits[k] = sp[k]; }
     ctx->drop_graphs();          // captured steps carry the old choice
+    return PC_OK;
+}
+
+int pc_set_fused_epilogues(pc_ctx* ctx, int on) {
+    if (ctx == nullptr || (on != 0 && on != 1)) return PC_ERR_INVALID_ARG;
+    if (on != ctx->fused_epilogues) ctx->drop_graphs();
+    ctx->fused_epilogues = on;
     return PC_OK;
 }
 

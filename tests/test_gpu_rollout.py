@@ -348,6 +348,7 @@ def test_persistent_decode_kernel_equals_one_kernel_per_operation(model):
     weights = wl.gen_weights(model, seed=0, threads=2, gain_jitter=0.1)
     batch = wl.gen_batch(w)
     eng = RolloutEngine(model, weights, max_rows=200, max_prefill_tokens=int(batch.prompt_offsets[-1]))
+    B.pc_set_fused_epilogues(eng.ctx, 0)              # the persistent kernel shares its arithmetic with the one-kernel-per-operation form
     outs, logits = [], []
     for mode in (0, 1, 1):
         B.pc_set_decode_mode(eng.ctx, mode)
