@@ -195,7 +195,8 @@ PC_API int pc_set_index_bounds(pc_ctx* ctx, int n_prompts, int64_t n_tokens);
  * gate/up projection and the RMSNorm's sum of squares in the output projection's, the norm's 1/rms being applied by the
  * gate/up epilogue (RMSNorm(h; g) W^T = rstd * ((h * g) W^T)).  The two projections then run without K split, which is why
  * smaller passes keep the separate kernels (their projections need the split to fill the GPU).  0: one kernel per
- * operation throughout, as for every other model type.  Same mathematics, different rounding order (both inside the
+ * operation throughout, as for every other model type.  A value n > 1: the fused form from passes of n rows on (a
+ * measurement aid: below 257 rows it is slower).  Same mathematics, different rounding order (both inside the
  * tolerances the tests state).  Drops captured decode steps.  The paper has no counterpart. */
 PC_API int pc_set_fused_epilogues(pc_ctx* ctx, int on);
 

@@ -57,7 +57,15 @@ struct RowKeys {
     int32_t* step_key;       // [M] step counter of the key: suffix tokens cached + 1
     int64_t* out_index;      // [M] where the drawn token goes in the token buffer
     int32_t* group_start;    // [groups + 1] first row of every group of the step
+    int32_t* sample_bound;   // [M] largest second-best score any vocabulary tile of the row has reported so far (ordered-int form)
 };
+
+// float <-> int with the same order (atomicMax on scores of either sign); -infinity maps to the smallest value in use
+__device__ __forceinline__ int32_t score_to_ordered(float f) {
+    const int32_t i = __float_as_int(f);
+    return i ^ ((i >> 31) & 0x7fffffff);
+}
+__device__ __forceinline__ float ordered_to_score(int32_t i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
 
 __device__ __forceinline__ void set_error(int32_t* flag, int32_t code) {
     if (flag != nullptr) atomicCAS(flag, 0, code);

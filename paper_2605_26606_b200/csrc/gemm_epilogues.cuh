@@ -31,35 +31,52 @@ struct EpiResNorm {
     float* ssq; int m_stride;          // [tiles of this GEMM][m_stride]
     int32_t* err;
     __device__ __forceinline__ void set_rows(int) {}
+    // The residual values of the next 32 columns are requested before the current 32 are worked on: a thread owns a
+    // row, so its loads are a latency chain of their own and one chunk's round trip at a time would dominate the tile.
     template <int BN>
     __device__ __forceinline__ void tile(uint32_t taddr, int row, bool live, int n0, int N) const {
         float ss = 0.f;
         int bad = 0;
+        const int n_chunks = min(BN, N - n0) >> 5;      // warp-uniform (N is a multiple of 32)
+        float* hrow = h + (size_t)(live ? row : 0) * ld + n0;
+        float4 cur[8], nxt[8];
+        if (live) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) cur[i] = reinterpret_cast<const float4*>(hrow)[i];
+        }
 #pragma unroll 1
-        for (int c = 0; c < BN; c += 32) {
-            if (n0 + c >= N) break;                 // warp-uniform (N is a multiple of 32)
+        for (int ci = 0; ci < n_chunks; ++ci) {
+            const int c = ci << 5;
+            if (live && ci + 1 < n_chunks) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) nxt[i] = reinterpret_cast<const float4*>(hrow + c + 32)[i];
+            }
             float v[32];
             tc::tmem_ld32(taddr + c, v);
-            if (!live) continue;
-            float4* hp = reinterpret_cast<float4*>(h + (size_t)row * ld + n0 + c);
-            const float4* gp = reinterpret_cast<const float4*>(gain + n0 + c);
-            uint32_t w[16];
+            if (live) {
+                const float4* gp = reinterpret_cast<const float4*>(gain + n0 + c);
+                uint32_t w[16];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                float4 x = hp[i];
-                const float4 g = gp[i];
-                x.x += v[4 * i]; x.y += v[4 * i + 1]; x.z += v[4 * i + 2]; x.w += v[4 * i + 3];
-                hp[i] = x;
-                ss += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
-                const float y0 = x.x * g.x, y1 = x.y * g.y, y2 = x.z * g.z, y3 = x.w * g.w;
-                bad |= half_bad(y0) | half_bad(y1) | half_bad(y2) | half_bad(y3);
-                const __half2 p0 = __floats2half2_rn(half_clamp(y0), half_clamp(y1)), p1 = __floats2half2_rn(half_clamp(y2), half_clamp(y3));
-                w[2 * i] = *reinterpret_cast<const uint32_t*>(&p0);
-                w[2 * i + 1] = *reinterpret_cast<const uint32_t*>(&p1);
+                for (int i = 0; i < 8; ++i) {
+                    float4 x = cur[i];
+                    const float4 g = __ldg(gp + i);
+                    x.x += v[4 * i]; x.y += v[4 * i + 1]; x.z += v[4 * i + 2]; x.w += v[4 * i + 3];
+                    cur[i] = x;
+                    ss += x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+                    const float y0 = x.x * g.x, y1 = x.y * g.y, y2 = x.z * g.z, y3 = x.w * g.w;
+                    bad |= half_bad(y0) | half_bad(y1) | half_bad(y2) | half_bad(y3);
+                    const __half2 p0 = __floats2half2_rn(half_clamp(y0), half_clamp(y1)), p1 = __floats2half2_rn(half_clamp(y2), half_clamp(y3));
+                    w[2 * i] = *reinterpret_cast<const uint32_t*>(&p0);
+                    w[2 * i + 1] = *reinterpret_cast<const uint32_t*>(&p1);
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) reinterpret_cast<float4*>(hrow + c)[i] = cur[i];
+                uint4* ap = reinterpret_cast<uint4*>(a + (size_t)row * ld + n0 + c);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) ap[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) cur[i] = nxt[i];
             }
-            uint4* ap = reinterpret_cast<uint4*>(a + (size_t)row * ld + n0 + c);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) ap[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
         }
         if (live) {
             ssq[(size_t)(n0 / BN) * m_stride + row] = ss;

@@ -19,6 +19,7 @@
 #include <cuda_fp16.h>
 
 #include <cstring>
+#include <type_traits>
 
 #include "common.cuh"
 
@@ -176,9 +177,13 @@ struct EpiPartial {
     }
 };
 struct EpiResidual {
-    static constexpr bool kWholeTile = false;            // H += acc
+    static constexpr bool kWholeTile = true;             // H += acc
     float* H; int ldc;
     __device__ __forceinline__ void set_rows(int) {}
+    // Whole tile of the thread's row: the residual values of the next 32 columns are requested before the current 32
+    // are added and stored (a thread owns a row, so one chunk's round trip at a time would dominate a one-tile CTA).
+    template <int BN>
+    __device__ __forceinline__ void tile(uint32_t taddr, int row, bool live, int n0, int N) const;
     __device__ __forceinline__ void operator()(int row, int col0, const float* v, int n_valid, int /*split*/) const {
         float* dst = H + (size_t)row * ldc + col0;
         if (n_valid == 32 && (ldc & 3) == 0) {
@@ -195,6 +200,44 @@ struct EpiResidual {
         }
     }
 };
+template <int BN>
+__device__ __forceinline__ void EpiResidual::tile(uint32_t taddr, int row, bool live, int n0, int N) const {
+    const int n_cols = min(BN, N - n0);
+    float* hrow = H + (size_t)(live ? row : 0) * ldc + n0;
+    if ((ldc & 3) != 0 || (n_cols & 31) != 0) {              // ragged or unaligned: one chunk at a time
+#pragma unroll 1
+        for (int c = 0; c < n_cols; c += 32) {
+            float v[32];
+            tmem_ld32(taddr + c, v);
+            if (live) (*this)(row, n0 + c, v, min(32, n_cols - c), 0);
+        }
+        return;
+    }
+    float4 cur[8], nxt[8];
+    if (live) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) cur[i] = reinterpret_cast<const float4*>(hrow)[i];
+    }
+#pragma unroll 1
+    for (int c = 0; c < n_cols; c += 32) {
+        if (live && c + 32 < n_cols) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) nxt[i] = reinterpret_cast<const float4*>(hrow + c + 32)[i];
+        }
+        float v[32];
+        tmem_ld32(taddr + c, v);
+        if (live) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float4 o = cur[i];
+                o.x += v[4 * i]; o.y += v[4 * i + 1]; o.z += v[4 * i + 2]; o.w += v[4 * i + 3];
+                reinterpret_cast<float4*>(hrow + c)[i] = o;
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) cur[i] = nxt[i];
+        }
+    }
+}
 struct EpiSwiGLU {
     static constexpr bool kWholeTile = false;              // columns (2j, 2j+1) = (gate_j, up_j) -> out[row, j] = silu(gate) * up, bf16 (or IEEE half)
     __nv_bfloat16* out; int ld; int half_out; int32_t* err;
@@ -235,8 +278,15 @@ struct EpiSwiGLU {
 // ---------------------------------------------------------------------------------------------
 // Kernel
 // ---------------------------------------------------------------------------------------------
+// Epilogue warps of a kernel instance: four (one per 32-lane quarter of the accumulator) unless the epilogue asks for eight
+// (Epi::kEpiWarps = 8: two warps per quarter, each walking half of the tile's columns -- for epilogues whose arithmetic,
+// not their memory traffic, is what has to hide behind the next tile's main loop).
+template <class E, class = void> struct EpiWarps { static constexpr int value = 4; };
+template <class E> struct EpiWarps<E, std::void_t<decltype(E::kEpiWarps)>> { static constexpr int value = E::kEpiWarps; };
+template <class E> constexpr int block_threads() { return 64 + 32 * EpiWarps<E>::value; }
+
 template <int BN, bool DUAL, class Epi>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(block_threads<Epi>(), 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_a_lo,
                const __grid_constant__ CUtensorMap map_w, const StepDesc* __restrict__ sd, int M, int N, int K, int splits, Epi epi,
                int32_t* err, int half_operands) {
@@ -262,7 +312,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(tfull0 + 8 * b, 1); mbar_init(tempty0 + 8 * b, 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull0 + 8 * b, 1); mbar_init(tempty0 + 8 * b, EpiWarps<Epi>::value); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -370,7 +420,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
             tc_fence_after();
             const int row = m0 + quarter * 32 + lane;
-            if constexpr (Epi::kWholeTile) {
+            if constexpr (EpiWarps<Epi>::value == 8) {
+                // two warps per quarter: warps 2..5 take the first half of the tile's columns, warps 6..9 the second
+                epi.template tile_part<BN>(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN, row, row < m_live, n0, N, (warp - 2) >> 2);
+            } else if constexpr (Epi::kWholeTile) {
                 // the epilogue walks the accumulator tile itself (more than one pass over its columns)
                 epi.template tile<BN>(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN, row, row < m_live, n0, N);
             } else {
@@ -433,7 +486,7 @@ inline cudaError_t launch(cudaStream_t st, const CUtensorMap& map_a, const CUten
     if (tiles == 0) return cudaSuccess;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
-    cfg.gridDim = dim3((unsigned)(tiles < num_sms ? tiles : num_sms)); cfg.blockDim = dim3(NUM_THREADS);
+    cfg.gridDim = dim3((unsigned)(tiles < num_sms ? tiles : num_sms)); cfg.blockDim = dim3(block_threads<Epi>());
     cfg.dynamicSmemBytes = smem_bytes(BN, DUAL); cfg.stream = st;
     return cudaLaunchKernelEx(&cfg, kern, map_a, map_a_lo, map_w, sd, M, N, K, splits, epi, err, half_operands ? 1 : 0);
 }

@@ -81,6 +81,7 @@ __global__ void prep_decode_rows(const StepDesc* __restrict__ sd, const DecodeAr
     keys.rollout[r] = da->row_rollout[ro];
     keys.step_key[r] = step + 1;
     keys.out_index[r] = ok ? ti + 1 : -1;            // -1: nothing is stored for this row
+    keys.sample_bound[r] = score_to_ordered(-INFINITY);      // no tile of the row has reported a second-best score yet
     if (ok) atomicMax(g.max_slen, step + 1);
 }
 

@@ -66,7 +66,7 @@ constexpr int kMaxSplits = pc::PARTIALS_MAX;
 struct Carve {
     size_t h, a, qkv, q, attn, act, logits, rope, pos, wslot, warena, p_start, p_len, s_start, s_len, token, last_row,
         part_m, part_l, part_o, res_part, step_desc, step_counter, max_slen, sample_scratch, a_lo, attn_lo, chain_layers, chain_glob,
-        chain_bar, dargs, key_prompt, key_rollout, key_step, out_index, group_start, sample_tiles, ssq, total;
+        chain_bar, dargs, key_prompt, key_rollout, key_step, out_index, group_start, sample_tiles, sample_bound, ssq, total;
 };
 
 // A captured decode step, replayable for every step that fits the same upper bounds on the same KV arenas.  The
@@ -206,7 +206,8 @@ Carve carve(const pc_ctx* c, int max_rows, int max_prefill) {
     v.group_start = take((M + 1) * 4);
     v.ssq = take((size_t)((d.d_model + 63) / 64) * M * 4);       // per-tile sums of squares of the residual rows (EpiResNorm)
     // fused LM head + sampler: one record per (vocabulary tile of the narrowest tile width, row)
-    v.sample_tiles = take((size_t)((d.vocab + 63) / 64) * (size_t)std::max(max_rows, 1) * sizeof(pc::Top2Rec));
+    v.sample_tiles = take(2 * (size_t)((d.vocab + 63) / 64) * (size_t)std::max(max_rows, 1) * sizeof(pc::Top2Rec));   // one record per half tile
+    v.sample_bound = take((size_t)std::max(max_rows, 1) * sizeof(int32_t));
     // prefix part of the shared-prefix attention: (max, sum, unnormalised output) per (row, query head)
     const size_t R = (size_t)std::max(max_rows, 1);
     v.part_m = take(pc::am::MAX_RECORDS * R * d.n_q_heads * 4);
@@ -465,7 +466,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
     // in the output projection's epilogue, its 1/rms applied by the gate/up epilogue (gemm_epilogues.cuh)
     // From three row tiles on: below that the two projections need their K split to keep the SMs busy (measured: unsplit they
     // lose more than the two small kernels cost), and a split GEMM's tile does not hold complete sums.
-    const bool fused = half_gemm && d.head_dim == 128 && d.d_model % 64 == 0 && c->fused_epilogues != 0 && M > 2 * tc::BM;
+    const bool fused = half_gemm && d.head_dim == 128 && d.d_model % 64 == 0 && c->fused_epilogues != 0 && M >= (c->fused_epilogues == 1 ? 2 * tc::BM + 1 : c->fused_epilogues);
     float* ssq = reinterpret_cast<float*>(w + c->cv.ssq);
     const int m_stride = std::max(std::max(c->max_rows, c->max_prefill), 1);
     T* a_lo = kF32 || half_gemm ? nullptr : reinterpret_cast<T*>(w + c->cv.a_lo);          // rounding remainders (bf16 operands only)
@@ -638,11 +639,11 @@ int run_lm_head_sample(pc_ctx* c, cudaStream_t st, int n, const pc::StepDesc* sd
     Top2Rec* rec = reinterpret_cast<Top2Rec*>(c->ws + c->cv.sample_tiles);
     const int m_stride = std::max(c->max_rows, 1);
     if (int rc = gemm_bf16(c, st, sd, c->map_a, half_gemm ? nullptr : &c->map_a_lo, c->m_lm, n, gp,
-                           EpiSample{rec, m_stride, keys.key_prompt, keys.rollout, keys.step_key, da}, half_gemm))
+                           EpiSample{rec, m_stride, keys.key_prompt, keys.rollout, keys.step_key, keys.sample_bound, da}, half_gemm))
         return rc;
     c->mark(st, -1, PC_MARK_LM_HEAD);
     const int bn = gp.wide ? 256 : 64;
-    launch_k(sample_tiles_reduce_kernel, dim3((n + 7) / 8), dim3(256), 0, st, sd, (d.vocab + bn - 1) / bn, rec, m_stride, keys.out_index, da);
+    launch_k(sample_tiles_reduce_kernel, dim3((n + 7) / 8), dim3(256), 0, st, sd, 2 * ((d.vocab + bn - 1) / bn), rec, m_stride, keys.out_index, da);
     count_launches(3);
     c->mark(st, -1, PC_MARK_SAMPLE);
     PC_CUDA_CHECK_LAUNCH("lm head with sampler");
@@ -710,7 +711,7 @@ int pc_set_gemm_plan(pc_ctx* ctx, const char* spec) {
 }
 
 int pc_set_fused_epilogues(pc_ctx* ctx, int on) {
-    if (ctx == nullptr || (on != 0 && on != 1)) return PC_ERR_INVALID_ARG;
+    if (ctx == nullptr || on < 0) return PC_ERR_INVALID_ARG;
     if (on != ctx->fused_epilogues) ctx->drop_graphs();
     ctx->fused_epilogues = on;
     return PC_OK;
@@ -1001,7 +1002,7 @@ pc::RowKeys row_keys(const pc_ctx* c) {
     char* w = c->ws;
     return pc::RowKeys{reinterpret_cast<int32_t*>(w + c->cv.key_prompt), reinterpret_cast<int32_t*>(w + c->cv.key_rollout),
                        reinterpret_cast<int32_t*>(w + c->cv.key_step), reinterpret_cast<int64_t*>(w + c->cv.out_index),
-                       reinterpret_cast<int32_t*>(w + c->cv.group_start)};
+                       reinterpret_cast<int32_t*>(w + c->cv.group_start), reinterpret_cast<int32_t*>(w + c->cv.sample_bound)};
 }
 
 // Upper bounds of a step's group geometry, rounded up to classes so that steps of similar shape share a captured graph
