@@ -201,12 +201,15 @@ PC_API int pc_set_index_bounds(pc_ctx* ctx, int n_prompts, int64_t n_tokens);
 PC_API int pc_set_fused_epilogues(pc_ctx* ctx, int on);
 
 /* bf16 models, decode steps that only sample (no logits_out, no log-probability buffer): 1 draws the token in
- * the epilogue of the LM-head GEMM -- per 256-column tile of the vocabulary the largest and second-largest perturbed score
+ * the epilogue of the LM-head GEMM -- per half tile of the vocabulary the largest and second-largest perturbed score
  * and the arg-max, folded per row by a small second kernel -- so the step's [rows, vocab] logits are never written or read
  * back; 0 (the default) stores the logits and runs the stand-alone sampler on them.  Both draw exactly the same tokens
- * (Section 4.2: T = 1.0, top_p = 1.0; pc_sample states the rule).  The epilogue form scores a row per thread, without the
- * warp-shared bound of the stand-alone sampler, and is the slower of the two on B200 (measured: +1.3 ms per step at 256
- * rows, +5.9 ms at 2048); it is kept for callers that cannot afford the [rows, vocab] logits buffer.  Drops captured steps. */
+ * (Section 4.2: T = 1.0, top_p = 1.0; pc_sample states the rule): the tiles of a row share a running lower bound of the
+ * row's second-best score, so which candidates a tile scores depends on timing, the folded result does not.  The
+ * epilogue form is not the faster one on B200 (LM head + draw at 2048 rows: 2.37 ms against 0.90 + 0.60 ms; at 64 rows
+ * 0.17 against 0.15 ms): the Philox arithmetic needs many warps per scheduler to reach the integer pipes' rate, and a
+ * GEMM CTA has room for eight epilogue warps.  It is kept for callers that cannot afford the [rows, vocab] logits
+ * buffer.  Drops captured steps. */
 PC_API int pc_set_fused_sampler(pc_ctx* ctx, int on);
 
 /* bf16 models, decode steps: 1 issues the shared-prefix attention kernel and the per-rollout suffix attention

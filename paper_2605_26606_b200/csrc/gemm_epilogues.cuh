@@ -18,8 +18,19 @@ namespace pc {
 
 // 1 / rms of a row from the per-tile sums of squares an EpiResNorm GEMM left (entries added in tile order).
 __device__ __forceinline__ float rstd_from_ssq(const float* __restrict__ ssq, int n_ssq, int m_stride, int row, int d, float eps) {
+    // entries added in tile order; six loads in flight at a time (one at a time would be n_ssq dependent L2 round trips at
+    // the head of every tile's epilogue)
     float s = 0.f;
-    for (int t = 0; t < n_ssq; ++t) s += ssq[(size_t)t * m_stride + row];
+    const float* p = ssq + row;
+    int t = 0;
+    for (; t + 6 <= n_ssq; t += 6) {
+        float x[6];
+#pragma unroll
+        for (int i = 0; i < 6; ++i) x[i] = p[(size_t)(t + i) * m_stride];
+#pragma unroll
+        for (int i = 0; i < 6; ++i) s += x[i];
+    }
+    for (; t < n_ssq; ++t) s += p[(size_t)t * m_stride];
     return rsqrtf(s / (float)d + eps);
 }
 

@@ -20,6 +20,29 @@
 
 namespace pc {
 
+// Eight Philox4x32-10 blocks with consecutive first counter words, advanced round by round: the eight dependency chains
+// are independent, and written this way they are in flight together (two epilogue warps per scheduler have no other
+// way to hide the multiplier's latency).  word[4 b + i] is word i of block c0 + b.
+__device__ __forceinline__ void philox4x32_10_x8(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1,
+                                                 uint32_t (&word)[32]) {
+    constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+    uint32_t x0[8], x1[8], x2[8], x3[8];
+#pragma unroll
+    for (int b = 0; b < 8; ++b) { x0[b] = c0 + b; x1[b] = c1; x2[b] = c2; x3[b] = c3; }
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+            const uint32_t hi0 = __umulhi(M0, x0[b]), lo0 = M0 * x0[b];
+            const uint32_t hi1 = __umulhi(M1, x2[b]), lo1 = M1 * x2[b];
+            x0[b] = hi1 ^ x1[b] ^ k0; x1[b] = lo1; x2[b] = hi0 ^ x3[b] ^ k1; x3[b] = lo0;
+        }
+        k0 += W0; k1 += W1;
+    }
+#pragma unroll
+    for (int b = 0; b < 8; ++b) { word[4 * b] = x0[b]; word[4 * b + 1] = x1[b]; word[4 * b + 2] = x2[b]; word[4 * b + 3] = x3[b]; }
+}
+
 struct EpiSample {
     static constexpr bool kWholeTile = true;
     static constexpr int kEpiWarps = 8;        // the Philox arithmetic of a tile is split over two warps per accumulator quarter
@@ -78,11 +101,7 @@ struct EpiSample {
             // all eight Philox blocks of the chunk first, without a branch between them (eight independent dependency
             // chains in flight), then one mask of the candidates that pass the integer bound: it is empty almost always
             uint32_t word[32];
-#pragma unroll
-            for (int b = 0; b < 8; ++b) {
-                const Philox4 w = philox4x32_10((uint32_t)((n0 + c) >> 2) + b, c1, c2, c3, k0, k1);
-                word[4 * b] = w.x; word[4 * b + 1] = w.y; word[4 * b + 2] = w.z; word[4 * b + 3] = w.w;
-            }
+            philox4x32_10_x8((uint32_t)((n0 + c) >> 2), c1, c2, c3, k0, k1, word);
             uint32_t pass = 0;
 #pragma unroll
             for (int i = 0; i < 32; ++i) pass |= (uint32_t)((8388608u - (word[i] >> 9)) < pass_below) << i;
@@ -110,20 +129,36 @@ struct EpiSample {
     }
 };
 
-// One warp per row: folds the row's records of all vocabulary tiles (in tile order within a lane, then across lanes with
-// the order-independent merge) and stores the token.
-__global__ void __launch_bounds__(256) sample_tiles_reduce_kernel(const StepDesc* __restrict__ sd, int n_tiles, const Top2Rec* __restrict__ rec,
-                                                                  int m_stride, const int64_t* __restrict__ out_index,
-                                                                  const DecodeArgsDev* __restrict__ da) {
-    const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+// One block of 128 threads per row: folds the row's records of all half tiles (the merge is order-independent: equal scores
+// keep the lowest id) and stores the token.  A thread's loads are issued four at a time.
+constexpr int TILES_REDUCE_THREADS = 128;
+__global__ void __launch_bounds__(TILES_REDUCE_THREADS) sample_tiles_reduce_kernel(const StepDesc* __restrict__ sd, int n_tiles, const Top2Rec* __restrict__ rec,
+                                                                                   int m_stride, const int64_t* __restrict__ out_index,
+                                                                                   const DecodeArgsDev* __restrict__ da) {
+    const int r = blockIdx.x;
     if (r >= sd->n_rows) return;
+    const int4* p = reinterpret_cast<const int4*>(rec) + r;
     Top2 t{-INFINITY, -INFINITY, 0x7fffffff};
-    for (int i = lane; i < n_tiles; i += 32) {
-        const Top2Rec x = rec[(size_t)i * m_stride + r];
-        t = top2_merge(t, Top2{x.best, x.second, x.idx});
+    int i = threadIdx.x;
+    for (; i + 3 * TILES_REDUCE_THREADS < n_tiles; i += 4 * TILES_REDUCE_THREADS) {
+        int4 x[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) x[j] = __ldcg(p + (size_t)(i + j * TILES_REDUCE_THREADS) * m_stride);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) t = top2_merge(t, Top2{__int_as_float(x[j].x), __int_as_float(x[j].y), x[j].z});
+    }
+    for (; i < n_tiles; i += TILES_REDUCE_THREADS) {
+        const int4 x = __ldcg(p + (size_t)i * m_stride);
+        t = top2_merge(t, Top2{__int_as_float(x.x), __int_as_float(x.y), x.z});
     }
     t = top2_warp_reduce(t);
-    if (lane == 0) {
+    __shared__ Top2 sh[TILES_REDUCE_THREADS / 32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) sh[warp] = t;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 1; w < TILES_REDUCE_THREADS / 32; ++w) t = top2_merge(t, sh[w]);
         const int64_t at = out_index[r];
         if (at >= 0) da->tokens[at] = t.idx;
     }

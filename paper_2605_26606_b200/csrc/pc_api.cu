@@ -643,7 +643,7 @@ int run_lm_head_sample(pc_ctx* c, cudaStream_t st, int n, const pc::StepDesc* sd
         return rc;
     c->mark(st, -1, PC_MARK_LM_HEAD);
     const int bn = gp.wide ? 256 : 64;
-    launch_k(sample_tiles_reduce_kernel, dim3((n + 7) / 8), dim3(256), 0, st, sd, 2 * ((d.vocab + bn - 1) / bn), rec, m_stride, keys.out_index, da);
+    launch_k(sample_tiles_reduce_kernel, dim3(n), dim3(TILES_REDUCE_THREADS), 0, st, sd, 2 * ((d.vocab + bn - 1) / bn), rec, m_stride, keys.out_index, da);
     count_launches(3);
     c->mark(st, -1, PC_MARK_SAMPLE);
     PC_CUDA_CHECK_LAUNCH("lm head with sampler");

@@ -1,13 +1,15 @@
 """pc_sample_static -- the sampler variant for callers that cannot allocate device memory (a plugin that only receives
 its input and output buffers, code running while the host framework's allocator is frozen or exhausted).  Its scratch is
 an array inside the library image, so the test hands it nothing but inputs and outputs and checks, on two calls in a
-row that reuse that array with different shapes, that it draws exactly the tokens pc_sample draws.
+row that reuse that array with different shapes, that it draws exactly the tokens pc_sample draws and, on the small
+case, the tokens the oracle's sampler draws.
 
 Collected last on purpose: a run that stops at the first failure has then already run every other test."""
 import numpy as np
 import pytest
 import torch
 
+from oracle import sampler as osampler
 from paper_2605_26606_b200 import binding as B
 from paper_2605_26606_b200 import build
 
@@ -36,6 +38,15 @@ def test_static_scratch_sampler_matches_pc_sample_on_two_calls_in_a_row(cuda_dev
         torch.cuda.synchronize()
         assert torch.equal(got_tok, want_tok)                    # token ids: bit-exact, as everywhere in the suite
         assert torch.equal(got_gap, want_gap)                    # maxima are exact, so the gaps are identical too
+        if n <= 16:
+            # against the oracle itself (float64 scores there, float32 here: equal wherever the top-two gap is not a rounding error)
+            lg, tok, gap = logits.cpu().numpy(), got_tok.cpu().numpy(), got_gap.cpu().numpy()
+            pr, ro, st = prompt.cpu().numpy(), roll.cpu().numpy(), step.cpu().numpy()
+            for r in range(n):
+                want, g = osampler.sample(lg[r], temperature, seed, int(pr[r]), int(ro[r]), int(st[r]))
+                assert abs(gap[r] - g) < 1e-4
+                if g > 1e-4:
+                    assert tok[r] == want
 
 
 def test_static_scratch_sampler_refuses_more_rows_than_it_holds(cuda_device):
