@@ -163,6 +163,8 @@ def run_probe(args):
     B.pc_set_attention_overlap(eng.ctx, int(kv.get("overlap", 0)))
     B.pc_set_fused_sampler(eng.ctx, int(kv.get("fused", 0)))
     B.pc_set_fused_epilogues(eng.ctx, int(kv.get("epi", 1)))
+    if "plan" in kv:            # forced GEMM plans, e.g. plan=qkv:128x1+o:64x1
+        B.pc_set_gemm_plan(eng.ctx, kv["plan"].replace(":", "=").replace("+", ","))
     eng.load_batch(w, batch)
     eng.suffix_kv.zero_()
     eng.tokens.random_(0, w.model.vocab)
@@ -244,7 +246,7 @@ def main():
     ap.add_argument("--also-logprobs", action="store_true",
                     help="additionally time one step that also keeps the behaviour log-probability of every sampled token (Eq. 2's "
                          "denominator); reported as with_logprobs")
-    ap.add_argument("--probe", default=None, metavar="rows=R,suffix=S,steps=N,prompt=L,mode=M",
+    ap.add_argument("--probe", default=None, metavar="rows=R,suffix=S,steps=N,prompt=L,mode=M,plan=qkv:128x1+o:64x1",
                     help="time N decode steps of R rollouts (16 groups) that already hold S suffix tokens, then exit")
     args = ap.parse_args()
     if args.impl == "reference":

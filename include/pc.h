@@ -176,8 +176,10 @@ PC_API int pc_set_workspace(pc_ctx* ctx, void* dev_ws, size_t bytes, int max_row
  * GEMMs instead of the built-in choice.  spec (host string) is a comma-separated list of name=WIDTHxSLICES with name
  * in {qkv, o, gu, dn, lm} (QKV, output, gate/up, down projection, LM head), e.g. "dn=256x4,o=64x2"; names left out,
  * NULL or "" keep the built-in choice.  The slice count is clamped to what the workspace holds for the step's row
- * bound; gate/up and the LM head never split.  Results stay deterministic for a fixed plan.  Drops captured decode
- * steps.  The paper has no counterpart. */
+ * bound; gate/up and the LM head never split.  Where the QKV and output projections run with the fused epilogues
+ * (pc_set_fused_epilogues) only the width applies to them: 128 or 256 for QKV (whole heads per tile; 128 is accepted for
+ * this case only and otherwise read as 64), 64 or 256 for the output projection.  Results stay deterministic for a
+ * fixed plan.  Drops captured decode steps.  The paper has no counterpart. */
 PC_API int pc_set_gemm_plan(pc_ctx* ctx, const char* spec);
 
 /* Self-test of the bounded waits every kernel here uses on its mbarriers: launches one warp that waits, for at most

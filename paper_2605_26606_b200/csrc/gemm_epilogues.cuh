@@ -9,6 +9,8 @@
 //   EpiSwiGLUNorm gate/up projection of such an operand: (gate, up) *= rstd, then silu(gate) * up.
 //   EpiQkvPost    QKV projection: bias, per-head RMSNorm of q and k (Qwen3), RoPE, q to its buffer, K / V to the row's
 //                 KV slot -- the arithmetic of qkv_post_kernel, one thread per row and one head (128 columns) at a time.
+//                 When the previous layer's down projection ran with EpiResNorm (unsplit: large passes), it also applies
+//                 the attention norm's 1/rms, and that layer boundary has no norm kernel either.
 #pragma once
 
 #include "gemm_tc.cuh"
@@ -142,13 +144,20 @@ struct EpiQkvPost {
     KvArena prompt_arena, suffix_arena;
     __half* q_out;                     // [rows, Hq * HD]
     int32_t* err;
+    // n_ssq > 0: the operand is half(h * gain) without the attention norm's 1/rms (left by an EpiResNorm down projection
+    // together with the row's sums of squares); the accumulators are scaled by it before the bias is added
+    const float* ssq; int n_ssq, m_stride, d_model;
     __device__ __forceinline__ void set_rows(int) {}
     template <int BN>
     __device__ __forceinline__ void tile(uint32_t taddr, int row, bool live, int n0, int N) const {
         static_assert(BN % HD == 0, "QKV tiles must hold whole heads");
         int64_t slot = -1;
         int to_suffix = 0;
-        if (live) { slot = g.wslot[row]; to_suffix = g.warena[row]; }
+        float rstd = 1.f;
+        if (live) {
+            slot = g.wslot[row]; to_suffix = g.warena[row];
+            if (n_ssq > 0) rstd = rstd_from_ssq(ssq, n_ssq, m_stride, row, d_model, eps);
+        }
 #pragma unroll 1
         for (int ho = 0; ho < BN; ho += HD) {
             if (n0 + ho >= N) break;                 // warp-uniform
@@ -158,6 +167,10 @@ struct EpiQkvPost {
             if (!live) continue;
             const int head = (n0 + ho) / HD;
             const bool is_q = head < Hq, is_k = !is_q && head < Hq + Hkv;
+            if (n_ssq > 0) {
+#pragma unroll
+                for (int i = 0; i < HD; ++i) x[i] *= rstd;
+            }
             if (bias != nullptr) {
                 const float4* bp = reinterpret_cast<const float4*>(bias + (size_t)head * HD);
 #pragma unroll

@@ -33,8 +33,9 @@ __device__ __forceinline__ void philox4x32_10_x8(uint32_t c0, uint32_t c1, uint3
     for (int r = 0; r < 10; ++r) {
 #pragma unroll
         for (int b = 0; b < 8; ++b) {
-            const uint32_t hi0 = __umulhi(M0, x0[b]), lo0 = M0 * x0[b];
-            const uint32_t hi1 = __umulhi(M1, x2[b]), lo1 = M1 * x2[b];
+            const uint64_t p0 = (uint64_t)M0 * x0[b], p1 = (uint64_t)M1 * x2[b];
+            const uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
+            const uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
             x0[b] = hi1 ^ x1[b] ^ k0; x1[b] = lo1; x2[b] = hi0 ^ x3[b] ^ k1; x3[b] = lo0;
         }
         k0 += W0; k1 += W1;

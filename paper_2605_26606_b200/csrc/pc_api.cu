@@ -478,6 +478,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
     const Partials none{nullptr, 0, 0, 0};
     Partials pend = none;
     int n_ssq = 0;
+    int n_ssq_attn = 0;          // > 0: the previous layer's down projection left half(h * gain) and sums of squares for this layer's attention norm
 
     launch_k(rope_table_kernel, dim3((M * half + 255) / 256), dim3(256), 0, st, sd, half, (double)d.rope_theta, g.pos, rope);
     launch_k(embed_rmsnorm_kernel<T>, dim3(M), dim3(NORM_THREADS), 0, st, sd, d.d_model, g.token, reinterpret_cast<const T*>(c->embed), c->attn_norm[0],
@@ -486,7 +487,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
     PC_CUDA_CHECK_LAUNCH("embed_rmsnorm");
     for (int l = 0; l < d.n_layers; ++l) {
         c->mark(st, l, PC_MARK_LAYER_BEGIN);
-        if (l > 0) {
+        if (l > 0 && n_ssq_attn == 0) {
             launch_k(rmsnorm_kernel<T>, dim3(M), dim3(NORM_THREADS), 0, st, sd, M, d.d_model, h, nullptr, pend, c->attn_norm[l], d.rms_eps, a, a_lo, half_gemm ? 1 : 0, c->err);
             pend = none;
             count_launches(1);
@@ -499,9 +500,11 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
                                 EpiStoreF32{qkv, c->n_qkv(), nullptr});
         } else if (fused) {
             const EpiQkvPost epi{d.n_q_heads, d.n_kv_heads, l, bias, d.qk_norm ? c->q_norm[l] : nullptr, d.qk_norm ? c->k_norm[l] : nullptr,
-                                 d.rms_eps, rope, g, prompt_arena, suffix_arena, reinterpret_cast<__half*>(q), c->err};
-            const int rc = wide_tiles_fill_the_gpu(c, M, c->n_qkv()) ? gemm_half_bn<256>(c, st, sd, c->map_a, c->m_wqkv[l], M, epi)
-                                                                     : gemm_half_bn<128>(c, st, sd, c->map_a, c->m_wqkv[l], M, epi);
+                                 d.rms_eps, rope, g, prompt_arena, suffix_arena, reinterpret_cast<__half*>(q), c->err, ssq, n_ssq_attn, m_stride, d.d_model};
+            n_ssq_attn = 0;
+            const bool wide_qkv = c->plan_bn[GEMM_QKV] != 0 ? c->plan_bn[GEMM_QKV] == 256 : wide_tiles_fill_the_gpu(c, M, c->n_qkv());
+            const int rc = wide_qkv ? gemm_half_bn<256>(c, st, sd, c->map_a, c->m_wqkv[l], M, epi)
+                                    : gemm_half_bn<128>(c, st, sd, c->map_a, c->m_wqkv[l], M, epi);
             if (rc) return rc;
         } else {
             const GemmPlan gp = plan_gemm(c, GEMM_QKV, c->m_wqkv[l], M, true);
@@ -536,7 +539,7 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
             if (rc) return rc;
             const GemmPlan gp = plan_gemm(c, GEMM_O, c->m_wo[l], M, true);
             if (fused) {
-                const bool wide = wide_tiles_fill_the_gpu(c, M, d.d_model);
+                const bool wide = c->plan_bn[GEMM_O] != 0 ? c->plan_bn[GEMM_O] == 256 : wide_tiles_fill_the_gpu(c, M, d.d_model);
                 n_ssq = (d.d_model + (wide ? 256 : 64) - 1) / (wide ? 256 : 64);
                 const EpiResNorm epi{h, d.d_model, c->mlp_norm[l], reinterpret_cast<__half*>(a), ssq, m_stride, c->err};
                 const int rc2 = wide ? gemm_half_bn<256>(c, st, sd, c->map_attn, c->m_wo[l], M, epi)
@@ -570,7 +573,15 @@ int run_layers(pc_ctx* c, cudaStream_t st, int M, const pc::StepDesc* sd, pc::Kv
             if (rc) return rc;
             c->mark(st, l, PC_MARK_GATE_UP);
             const GemmPlan gp = plan_gemm(c, GEMM_DOWN, c->m_wdown[l], M, true);
-            if (gp.splits == 1) {
+            if (gp.splits == 1 && l + 1 < d.n_layers) {
+                // complete sums in every tile: the next layer's attention norm moves into this epilogue and the QKV epilogue
+                // (the sums of squares of the MLP norm were consumed by the gate/up projection above)
+                n_ssq_attn = (d.d_model + (gp.wide ? 256 : 64) - 1) / (gp.wide ? 256 : 64);
+                const EpiResNorm epi2{h, d.d_model, c->attn_norm[l + 1], reinterpret_cast<__half*>(a), ssq, m_stride, c->err};
+                const int rc2 = gp.wide ? gemm_half_bn<256>(c, st, sd, c->map_act, c->m_wdown[l], M, epi2)
+                                        : gemm_half_bn<64>(c, st, sd, c->map_act, c->m_wdown[l], M, epi2);
+                if (rc2) return rc2;
+            } else if (gp.splits == 1) {
                 if (int rc2 = gemm_bf16(c, st, sd, c->map_act, nullptr, c->m_wdown[l], M, gp, tc::EpiResidual{h, d.d_model}, half_gemm)) return rc2;
             } else {
                 pend = Partials{res_part, gp.splits, (size_t)M * d.d_model, d.d_model};
@@ -699,7 +710,7 @@ int pc_set_gemm_plan(pc_ctx* ctx, const char* spec) {
         if (kind < 0) return PC_ERR_INVALID_ARG;
         int w = 0, s = 0, used = 0;
         if (std::sscanf(p + len, "%dx%d%n", &w, &s, &used) != 2) return PC_ERR_INVALID_ARG;
-        if ((w != 64 && w != 256) || s < 1 || s > kMaxSplits) return PC_ERR_INVALID_ARG;
+        if ((w != 64 && w != 128 && w != 256) || s < 1 || s > kMaxSplits) return PC_ERR_INVALID_ARG;      // 128: fused QKV epilogue only
         bn[kind] = w; sp[kind] = s;
         p += len + used;
         if (*p == ',') ++p;
