@@ -28,10 +28,11 @@ if ROOT not in sys.path:
 from paper_2605_26606_b200 import dist_util  # noqa: E402
 from paper_2605_26606_b200 import workloads as wl  # noqa: E402
 
-# DRAM traffic of the suffix attention kernel per algorithmic byte, from the ncu capture summarised in
-# profiles/attn_suffix_kernel_ncu.md (304 rollouts x 513 slots: 168.98 MB moved for 161.6 MB algorithmic).  The kernel
-# streams every (rollout, KV head) suffix once, so traffic grows in proportion to the algorithmic bytes of a launch.
-SUFFIX_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.046
+# DRAM traffic of the suffix attention kernel per algorithmic byte, from the ncu captures summarised in
+# profiles/attn_suffix_kernel_ncu.md (current build: 143.5 MB moved for 136.0 MB algorithmic at 256 rollouts x 513 slots, 1,157 MB
+# for 1,088 MB at 2048 x 513).  The kernel streams every (rollout, KV head) suffix once, so traffic grows in proportion to the
+# algorithmic bytes of a launch.
+SUFFIX_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.06
 METRIC = "generated tokens/s"
 UNIT = "tokens/s"
 
@@ -185,10 +186,40 @@ def run_probe(args):
     m = w.model
     bytes_step = m.weight_bytes_per_decode_step() + (P * G * (suffix + 1) + P * plen) * m.kv_bytes_per_token
     peak, kind = load_peaks()
-    print(json.dumps({"probe": {"rows": P * G, "suffix": suffix, "steps": steps, "prompt_len": plen}, "ms_per_decode_step": ms, "host_issue_ms_per_step": host_ms,
-                      "tokens_per_s": P * G / (ms * 1e-3), "launches_per_step": (B.pc_launch_count() - l0) / steps,
-                      "hbm_bytes_per_step": bytes_step, "hbm_frac": bytes_step / (ms * 1e-3) / 1e9 / peak, "peak_kind": kind}),
-          flush=True)
+    line = {"probe": {"rows": P * G, "suffix": suffix, "steps": steps, "prompt_len": plen}, "ms_per_decode_step": ms, "host_issue_ms_per_step": host_ms,
+            "tokens_per_s": P * G / (ms * 1e-3), "launches_per_step": (B.pc_launch_count() - l0) / steps,
+            "hbm_bytes_per_step": bytes_step, "hbm_frac": bytes_step / (ms * 1e-3) / 1e9 / peak, "peak_kind": kind}
+    if kv.get("trace") == "1" and int(kv.get("mode", 0)) == 1:
+        line["chain_trace_us"] = chain_trace(eng, B, torch, pp, rr, suffix + steps)
+    print(json.dumps(line), flush=True)
+
+
+def chain_trace(eng, B, torch, pp, rr, step):
+    """SM-clock stamps of the persistent decode kernel (pc_set_decode_mode 1) for one more decode step, as microseconds from the
+    start of the launch that holds the middle layers: per phase of one layer, when the row-wise warps (W), the GEMM producer
+    (P), the MMA issuer (M) and the epilogue (E) began, passed their grid barrier and finished."""
+    eng.use_graphs = False
+    n = B.pc_chain_trace_words(eng.ctx)
+    tr = torch.zeros(n, dtype=torch.int64, device="cuda")
+    B.pc_set_chain_trace(eng.ctx, tr)
+    eng.run_stage(pp, rr, step_range=(step, step + 1))
+    torch.cuda.synchronize()
+    eng.check_error_flag()
+    B.pc_set_chain_trace(eng.ctx, None)
+    t = tr.cpu().numpy().reshape(-1, 10, 4, 16)             # [launch segment][phase][traced CTA][stamp]
+    names = ["W_BEGIN", "W_WAITED", "W_DONE", "P_BEGIN", "P_BARRIER", "P_DONE", "M_FIRST", "M_DONE", "E_FIRST", "E_DONE"]
+    ghz = 1.965
+    seg = t.shape[0] // 2
+    out = {}
+    for cta in (0, 3):
+        t0 = t[seg, 0, cta, 10]
+        d = {"kernel_us": round(float(t[seg, 0, cta, 11] - t0) / ghz / 1e3, 1)}
+        for j in range(9):
+            ev = t[seg, j, cta]
+            if ev[:10].any():
+                d[f"phase{j}"] = {names[e]: round(float(ev[e] - t0) / ghz / 1e3, 1) for e in range(10) if ev[e]}
+        out[f"cta{cta}"] = d
+    return out
 
 
 def phase_table(eng, B, n_layers):
@@ -397,7 +428,7 @@ def main():
         "dtype": ("f16" if eng.half_gemm else "bf16") if m.dtype == wl.DTYPE_BF16 else "f32", "data": "synthetic",
         "config": {"workload": w.name, "model": m.name, "prompts": P, "group_size": G, "n_pilot": k, "max_new": w.max_new,
                    "mode": "pilot-commit",
-                   "arithmetic": "16-bit storage (bf16 model); GEMM operands IEEE half, K / q / embedding bfloat16, float32 accumulation"
+                   "arithmetic": "16-bit storage (bf16 model); GEMM operands, q, K and V IEEE half, embedding bfloat16, float32 accumulation and residual stream"
                                  if m.dtype == wl.DTYPE_BF16 and eng.half_gemm else "model storage type, float32 accumulation", "committed_prompts": int((status == B.PC_STATUS_COMMIT).sum()),
                    "rollouts_generated": n_roll, "rollouts_per_s": n_roll * world / (t_ms * 1e-3 / max(args.steps, 1)),
                    "l2": "inputs larger than L2 (3.1 GB of weights and tens of GB of KV per step); no flush",
@@ -410,6 +441,8 @@ def main():
         "roofline": {"bound": "hbm", "kernel": "decode steps of the Pilot-Commit step, all kernels (prefill excluded)",
                      "achieved": achieved_step, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved_step / peak,
                      "frac_of_8tbs": achieved_step / 8000.0, "traffic": None,
+                     "traffic_note": "not captured for the 4,100-step job; ncu captures of single decode steps moved 1.22 x (256 rows x 512) "
+                                     "and 1.26 x (2048 rows x 512) their algorithmic bytes (profiles/decode_step_launch_list_config2.md)",
                      "bytes_per_step": step_bytes, "decode_ms_per_step": decode_ms / max(args.steps, 1),
                      "parts": {"suffix_kv_read": suffix_reads, "prompt_kv_read": prompt_reads, "weights": weight_reads, "kv_write": kv_writes},
                      "target": 0.60},
