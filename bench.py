@@ -190,7 +190,7 @@ def run_probe(args):
             "tokens_per_s": P * G / (ms * 1e-3), "launches_per_step": (B.pc_launch_count() - l0) / steps,
             "hbm_bytes_per_step": bytes_step, "hbm_frac": bytes_step / (ms * 1e-3) / 1e9 / peak, "peak_kind": kind}
     if kv.get("trace") == "1" and int(kv.get("mode", 0)) == 1:
-        line["chain_trace_us"] = chain_trace(eng, B, torch, pp, rr, suffix + steps)
+        line["chain_trace_us"] = chain_trace(eng, B, torch, pp, rr, suffix + steps - 1)        # the last timed step once more
     print(json.dumps(line), flush=True)
 
 

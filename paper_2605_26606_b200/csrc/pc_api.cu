@@ -246,6 +246,7 @@ bool make_wmap(WMap* w, const void* base, int N, int K) {
 struct GemmPlan {
     bool wide;
     int splits;
+    bool mid = false;      // 128-column tiles (split-K partial sums and the SwiGLU epilogue with one operand matrix only)
 };
 enum GemmKind { GEMM_QKV = 0, GEMM_O = 1, GEMM_GATE_UP = 2, GEMM_DOWN = 3, GEMM_LM_HEAD = 4 };
 GemmPlan plan_gemm(const pc_ctx* c, GemmKind kind, const WMap& w, int M, bool may_split) {
@@ -256,11 +257,19 @@ GemmPlan plan_gemm(const pc_ctx* c, GemmKind kind, const WMap& w, int M, bool ma
     GemmPlan p{true, 1};
     if (c->plan_bn[kind] != 0) {
         p.wide = c->plan_bn[kind] == 256;
+        p.mid = c->plan_bn[kind] == 128;
         p.splits = std::max(1, std::min(c->plan_splits[kind], max_splits));
         return p;
     }
     const int tiles_wide = tiles_m * ((w.N + 255) / 256);
     if (tiles_wide >= c->num_sms / 2) return p;
+    // gate/up with one row tile: 128-column tiles give one tile per SM (140 for the 1.5B shape), where 256 columns leave half
+    // the SMs without a weight stream and 64 columns fetch the activation tile twice as often (measured: -4 % of a 64-row step)
+    if (kind == GEMM_GATE_UP && !may_split && tiles_m * ((w.N + 127) / 128) <= c->num_sms) {
+        p.wide = false;
+        p.mid = true;
+        return p;
+    }
     // Too few wide tiles to keep the SMs busy.  A wide tile moves half as many bytes from L2 into shared memory per
     // flop as a narrow one, so from three row tiles on (and enough K per tile for that traffic to matter; crossover
     // measured on the 1.5B shape at 128..896 rows) the wide tile stays and K is split until about every SM has a CTA.
@@ -283,7 +292,12 @@ int gemm_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, const CUtensor
     if (map_a_lo != nullptr)
         e = p.wide ? pc::tc::launch<256, true>(st, map_a, *map_a_lo, w.wide, sd, M, w.N, w.K, p.splits, epi, c->err, c->num_sms)
                    : pc::tc::launch<64, true>(st, map_a, *map_a_lo, w.narrow, sd, M, w.N, w.K, p.splits, epi, c->err, c->num_sms);
-    else
+    else if (p.mid && !p.wide && (std::is_same<Epi, pc::tc::EpiPartial>::value || std::is_same<Epi, pc::tc::EpiSwiGLU>::value)) {
+        if constexpr (std::is_same<Epi, pc::tc::EpiPartial>::value || std::is_same<Epi, pc::tc::EpiSwiGLU>::value)
+            e = pc::tc::launch<128, false>(st, map_a, map_a, w.mid, sd, M, w.N, w.K, p.splits, epi, c->err, c->num_sms, half_operands);
+        else
+            e = cudaErrorInvalidValue;
+    } else
         e = p.wide ? pc::tc::launch<256, false>(st, map_a, map_a, w.wide, sd, M, w.N, w.K, p.splits, epi, c->err, c->num_sms, half_operands)
                    : pc::tc::launch<64, false>(st, map_a, map_a, w.narrow, sd, M, w.N, w.K, p.splits, epi, c->err, c->num_sms, half_operands);
     if (e != cudaSuccess) return cuda_fail(e, "tensor-core gemm");
@@ -357,6 +371,8 @@ cudaError_t configure_kernels() {
     if (e == cudaSuccess) e = tc::configure<64, false, tc::EpiResidual>();
     if (e == cudaSuccess) e = tc::configure<256, false, tc::EpiSwiGLU>();
     if (e == cudaSuccess) e = tc::configure<64, false, tc::EpiSwiGLU>();
+    if (e == cudaSuccess) e = tc::configure<128, false, tc::EpiSwiGLU>();
+    if (e == cudaSuccess) e = tc::configure<128, false, tc::EpiPartial>();
     if (e == cudaSuccess) e = tc::configure<256, true, tc::EpiStoreF32>();
     if (e == cudaSuccess) e = tc::configure<64, true, tc::EpiStoreF32>();
     if (e == cudaSuccess) e = tc::configure<256, false, tc::EpiStoreF32>();
