@@ -170,8 +170,33 @@ def test_all_rollouts_at_once_2048_rows(shape_1p5b):
     _free(eng)
 
 
+def test_headline_shape_with_bf16_operands(shape_1p5b):
+    """The other operand mode at the 1.5B shape (bfloat16 GEMM operands, value + rounding remainder for QKV / output projection /
+    LM head): pilot stage of a short-cap variant of config2, logits of two rollouts over one window against the oracle."""
+    model, weights, dec = shape_1p5b
+    w = dataclasses.replace(wl.WORKLOADS["config2"], max_new=24, cap_lo=12, cap_hi=24)
+    batch = wl.gen_batch(w)
+    P, G, k = w.n_prompts, w.group_size, w.n_pilot
+    eng = RolloutEngine(w.model, weights, max_rows=max(P * k, P * (G - k)), max_prefill_tokens=int(batch.prompt_offsets[-1]), half_gemm=False)
+    eng.record_pilot_logits = {s: None for s in range(2, 2 + WINDOW)}
+    pa = int(np.argsort(batch.prompt_lens)[0])
+    long_of = sorted(range(k), key=lambda i: -int(batch.caps[pa, i]))
+    rows = [(pa, long_of[0]), (pa, long_of[1])]
+    eng.record_rows = set(rows)
+    out = eng.pilot_commit_step(w, batch)
+    check_step_invariants(out, w, batch)
+    last_logits = eng.last_logits.cpu().numpy()
+    worst, n_cmp = 0.0, 0
+    for p, i in rows:
+        wv, n, _ = compare_rollout_windows(dec, w, batch, out, p, i, [2], eng.record_pilot_logits, last_logits)
+        worst, n_cmp = max(worst, wv), n_cmp + n
+    print("bf16 operands, 1.5B shape: max |dlogit|", worst)
+    assert n_cmp == 2 * (WINDOW + 1) and worst <= 5e-2, (n_cmp, worst)
+    _free(eng)
+
+
 def test_config1_full_step(shape_1p5b):
-    """BASELINE config 1 in full (32 prompts of 256 tokens, G = 16, k = 4, up to 512 new tokens): 128 pilot rows, then 12 rows
+    """Workload config1 in full (32 prompts of 256 tokens, G = 16, k = 4, up to 512 new tokens): 128 pilot rows, then 12 rows
     per committed prompt."""
     model, weights, dec = shape_1p5b
     w = wl.WORKLOADS["config1"]

@@ -1,4 +1,4 @@
-"""BASELINE configs 3 and 4 (Qwen3-8B and 14B shapes) at full width and depth, kept in a module of their own so that the host
+"""Workloads config3 and config4 (Qwen3-8B and 14B shapes) at full width and depth, kept in a module of their own so that the host
 memory of the 1.5B-shape tests is released first."""
 import os
 
@@ -16,7 +16,7 @@ pytestmark = pytest.mark.gpu
 
 
 def _large_model_slice(workload_name, n_check_steps=6):
-    """BASELINE configs 3 and 4 at full width and depth: the whole Pilot-Commit step (every rollout to its cap) with the
+    """Workloads config3 and config4 at full width and depth: the whole Pilot-Commit step (every rollout to its cap) with the
     invariants that hold at any size, and the logits of one pilot rollout at the first decode steps against the oracle
     (single precision here: the 8B / 14B shapes would otherwise take many minutes of float64 host arithmetic; 5e-2 is two
     orders of magnitude above float32's own error)."""
