@@ -164,6 +164,7 @@ def run_probe(args):
     B.pc_set_attention_overlap(eng.ctx, int(kv.get("overlap", 0)))
     B.pc_set_fused_sampler(eng.ctx, int(kv.get("fused", 0)))
     B.pc_set_fused_epilogues(eng.ctx, int(kv.get("epi", 1)))
+    B.pc_set_dependent_launch(eng.ctx, int(kv.get("dep", 1)))
     if "plan" in kv:            # forced GEMM plans, e.g. plan=qkv:128x1+o:64x1
         B.pc_set_gemm_plan(eng.ctx, kv["plan"].replace(":", "=").replace("+", ","))
     eng.load_batch(w, batch)

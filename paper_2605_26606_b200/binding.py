@@ -22,7 +22,7 @@ PC_ERR_UNSUPPORTED, PC_ERR_CUDA, PC_ERR_NO_WORKSPACE = 5, 6, 7
 PC_DTYPE_F32, PC_DTYPE_BF16 = 0, 1
 PC_STATUS_COMMIT, PC_STATUS_BUFFERED, PC_STATUS_DEFER_HARD, PC_STATUS_SKIP_EASY, PC_STATUS_LOW_VARIANCE = 0, 1, 2, 3, 4
 
-EXPORTS = ["pc_status_string", "pc_last_cuda_error", "pc_launch_count", "pc_profile_step", "pc_set_gemm_plan", "pc_set_decode_mode", "pc_set_attention_overlap", "pc_set_fused_sampler", "pc_set_fused_epilogues", "pc_set_chain_trace", "pc_chain_trace_words", "pc_capture_count", "pc_set_index_bounds", "pc_selftest_wait_timeout", "pc_create", "pc_destroy", "pc_workspace_bytes",
+EXPORTS = ["pc_status_string", "pc_last_cuda_error", "pc_launch_count", "pc_profile_step", "pc_set_gemm_plan", "pc_set_decode_mode", "pc_set_attention_overlap", "pc_set_fused_sampler", "pc_set_fused_epilogues", "pc_set_dependent_launch", "pc_set_chain_trace", "pc_chain_trace_words", "pc_capture_count", "pc_set_index_bounds", "pc_selftest_wait_timeout", "pc_create", "pc_destroy", "pc_workspace_bytes",
            "pc_set_workspace", "pc_prefill_shared", "pc_decode_step", "pc_decode_run", "pc_sample", "pc_sample_static", "pc_token_logprob", "pc_set_logprob_buffer", "pc_set_prompt_keys", "pc_reward_last_token",
            "pc_group_stats", "pc_allocate", "pc_allocate_variance", "pc_grpo_advantage"]
 
@@ -84,6 +84,7 @@ def _lib():
         lib.pc_set_attention_overlap.argtypes = [C.c_void_p, C.c_int]
         lib.pc_set_fused_sampler.argtypes = [C.c_void_p, C.c_int]
         lib.pc_set_fused_epilogues.argtypes = [C.c_void_p, C.c_int]
+        lib.pc_set_dependent_launch.argtypes = [C.c_void_p, C.c_int]
         lib.pc_capture_count.argtypes = [C.c_void_p]
         lib.pc_capture_count.restype = C.c_uint64
         lib.pc_set_index_bounds.argtypes = [C.c_void_p, C.c_int, C.c_int64]
@@ -163,6 +164,10 @@ def pc_set_decode_mode(ctx: "Context", mode: int) -> None:
 
 def pc_set_fused_epilogues(ctx: "Context", on: int) -> None:
     _check(_lib().pc_set_fused_epilogues(ctx.handle, on), "pc_set_fused_epilogues")
+
+
+def pc_set_dependent_launch(ctx: "Context", mask: int) -> None:
+    _check(_lib().pc_set_dependent_launch(ctx.handle, mask), "pc_set_dependent_launch")
 
 
 def pc_set_fused_sampler(ctx: "Context", on: int) -> None:

@@ -736,6 +736,7 @@ template <int HD, bool STREAM>
 __global__ void __launch_bounds__(256) attn_merge_kernel(const StepDesc* __restrict__ sd, int Hq, RowGeom g, PrefixPartial part,
                                                          __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ out_lo, int32_t* err) {
     const size_t rh = (size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    grid_dep_launch_dependents();          // the output projection may set itself up and request its first weight tiles
     const int n_live = sd->n_rows;
     if (rh >= (size_t)n_live * Hq) return;
     const SuffixPlan sp = suffix_plan(*g.max_slen, n_live * part.n_kv_heads, part.n_suffix_warps);

@@ -67,6 +67,14 @@ __device__ __forceinline__ int32_t score_to_ordered(float f) {
 }
 __device__ __forceinline__ float ordered_to_score(int32_t i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
 
+// Programmatic dependent launch (griddepcontrol): a kernel launched with the programmatic-serialization attribute may
+// start while the kernel before it in the stream is still running; it must not touch anything that kernel writes until
+// grid_dep_wait() has returned (which is when that kernel has finished and its writes are visible).  Launched without
+// the attribute, both instructions do nothing.  The rule followed here: before the wait a kernel only sets up its own
+// shared / tensor memory and reads weights (never written during a pass); every CTA executes the wait on every path.
+__device__ __forceinline__ void grid_dep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void set_error(int32_t* flag, int32_t code) {
     if (flag != nullptr) atomicCAS(flag, 0, code);
 }

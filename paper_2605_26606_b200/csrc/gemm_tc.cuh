@@ -322,6 +322,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // The kernel after this one may start its own set-up now.  This kernel, if it was launched as a programmatic dependent,
+    // may be running beside the one before it: everything but the weight stream waits for that kernel here.
+    grid_dep_launch_dependents();
+    if (threadIdx.x != 0) grid_dep_wait();
 
     // work item t = ((n_tile * splits) + split) * tiles_m + m_tile; split s covers k-blocks [s*KB/splits, (s+1)*KB/splits)
     const int tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN - 1) / BN, n_tiles = tiles_m * tiles_n * splits;
@@ -353,6 +357,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     ++ahead; ++stage_b;
                     advance(cb);
                 }
+                grid_dep_wait();          // the activations are the previous kernel's output; the weights above are not
                 for (; ahead > 0; --ahead) {
                     const uint32_t sa = tiles_u32 + stage * (A_BYTES + B_BYTES);
                     tma_load_2d(sa, &map_a, full0 + 8 * stage, ca.kb * BK, ca.m0);
@@ -480,7 +485,7 @@ inline cudaError_t configure() {
 template <int BN, bool DUAL, class Epi>
 inline cudaError_t launch(cudaStream_t st, const CUtensorMap& map_a, const CUtensorMap& map_a_lo, const CUtensorMap& map_w,
                           const StepDesc* sd, int M, int N, int K, int splits, Epi epi, int32_t* err, int num_sms, bool half_operands = false,
-                          bool /*unused*/ = false) {
+                          bool programmatic = false) {
     auto kern = gemm_tc_kernel<BN, DUAL, Epi>;
     const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN) * splits;
     if (tiles == 0) return cudaSuccess;
@@ -488,6 +493,13 @@ inline cudaError_t launch(cudaStream_t st, const CUtensorMap& map_a, const CUten
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)(tiles < num_sms ? tiles : num_sms)); cfg.blockDim = dim3(block_threads<Epi>());
     cfg.dynamicSmemBytes = smem_bytes(BN, DUAL); cfg.stream = st;
+    // programmatic: this launch may begin (set-up, first weight tiles) before the previous kernel of the stream has ended
+    cudaLaunchAttribute attr[1];
+    if (programmatic) {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+    }
     return cudaLaunchKernelEx(&cfg, kern, map_a, map_a_lo, map_w, sd, M, N, K, splits, epi, err, half_operands ? 1 : 0);
 }
 

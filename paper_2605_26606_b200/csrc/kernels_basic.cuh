@@ -338,6 +338,7 @@ __global__ void __launch_bounds__(NORM_THREADS) embed_rmsnorm_kernel(const StepD
     __shared__ float red[8];
     __shared__ int counter;
     const int r = blockIdx.x, w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    grid_dep_launch_dependents();          // the projection that follows may set itself up and request its first weight tiles
     if (r >= sd->n_rows) return;
     if (threadIdx.x == 0) counter = 0;
     const T* e_row = embed + (size_t)token[r] * d;
@@ -366,6 +367,7 @@ __global__ void __launch_bounds__(NORM_THREADS) rmsnorm_kernel(const StepDesc* _
     __shared__ float red[8];
     __shared__ int counter;
     const int r = blockIdx.x, w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    grid_dep_launch_dependents();          // the projection that follows may set itself up and request its first weight tiles
     if (r >= (sd != nullptr ? sd->n_rows : n_rows)) return;
     if (threadIdx.x == 0) counter = 0;
     __syncthreads();

@@ -85,8 +85,9 @@ __device__ __forceinline__ void scan_blocks(Top2& t, const float* __restrict__ l
     // below it can change neither the winner nor the gap.  Candidates that pass are not scored where they are found (a
     // lane or two would drag the whole warp through the logarithms on most draws) but parked in a warp-private queue
     // and scored 32 at a time, one per lane.  Trip counts are warp-uniform (shuffles and ballots need every lane).
-    uint32_t pass_below = 0xffffffffu;          // a candidate is scored iff (2^23 - (w >> 9)) < pass_below
+    int pass_above = -1;                        // a candidate is scored iff (int)(w >> 9) > pass_above  (-1: every candidate)
     float bound_for = -INFINITY;                // warp-wide score the bound was computed for
+    bool stale = true;                          // a score was folded since the bound was computed (warp-uniform)
     const int lane = threadIdx.x & 31;
     const uint32_t lt_mask = (1u << lane) - 1u;
     int queued = 0;                             // warp-uniform
@@ -99,26 +100,35 @@ __device__ __forceinline__ void scan_blocks(Top2& t, const float* __restrict__ l
                 top2_push_unordered(t, lg[c.x] / temperature + gumbel_from_word(c.y), (int)c.x);
             }
             queued -= take;
+            stale = true;
             __syncwarp();
         }
     };
     for (int base = b_begin + (threadIdx.x - lane); base < b_end; base += blockDim.x) {
-        const float ws = warp_max(t.second);
-        if (ws > bound_for) {
-            bound_for = ws;
-            const float T = ws - lmax - 1e-3f * (1.f + fabsf(ws) + fabsf(lmax));     // conservative
-            // (1 - U0) * 2^23 with U0 = exp(-exp(-T)); expm1f keeps the relative accuracy when U0 is close to 1
-            const float d = -expm1f(-expf(-T)) * 8388608.f;
-            pass_below = d >= 8388608.f ? 0xffffffffu : (uint32_t)(d * 1.001f + 2.f);
+        if (stale) {                             // the second-best scores only move when candidates were scored
+            stale = false;
+            const float ws = warp_max(t.second);
+            if (ws > bound_for) {
+                bound_for = ws;
+                const float T = ws - lmax - 1e-3f * (1.f + fabsf(ws) + fabsf(lmax));     // conservative
+                // (1 - U0) * 2^23 with U0 = exp(-exp(-T)); expm1f keeps the relative accuracy when U0 is close to 1
+                const float d = -expm1f(-expf(-T)) * 8388608.f;
+                // scored iff 2^23 - (w >> 9) < d * 1.001 + 2, i.e. iff (w >> 9) > 2^23 - (that bound)
+                pass_above = d >= 8388608.f ? -1 : 8388608 - (int)(uint32_t)(d * 1.001f + 2.f);
+            }
         }
         const int b = base + lane;
         Philox4 w{0, 0, 0, 0};
         if (b < b_end) w = philox4x32_10((uint32_t)b, c1, c2, c3, k0, k1);
+        // Almost every block holds no candidate above the bound: one comparison on the block's largest word and one vote
+        // decide that for the whole warp; only blocks that may hold one go through the per-word test and the queue.
+        const uint32_t top = max(max(w.x, w.y), max(w.z, w.w));
+        if (!__any_sync(0xffffffffu, b < b_end && (int)(top >> 9) > pass_above)) continue;
         const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int v = b * 4 + i;
-            const bool pass = b < b_end && v < vocab && (8388608u - (ww[i] >> 9)) < pass_below;
+            const bool pass = b < b_end && v < vocab && (int)(ww[i] >> 9) > pass_above;
             const uint32_t m = __ballot_sync(0xffffffffu, pass);
             if (pass) queue[queued + __popc(m & lt_mask)] = make_uint2((uint32_t)v, ww[i]);
             queued += __popc(m);

@@ -370,6 +370,41 @@ def test_persistent_decode_kernel_equals_one_kernel_per_operation(model):
         assert np.array_equal(a["advantages"], b["advantages"])
 
 
+@pytest.mark.parametrize("model,group_size", [(wl.SMALL_BF16, 40), (wl.SMALL_QKNORM_BF16, 40), (wl.SMALL_BF16, 90)],
+                         ids=["small-batch-kernels", "qk-norm", "fused-epilogues"])
+def test_dependent_launch_of_the_projections_changes_no_bit(model, group_size):
+    """pc_set_dependent_launch: a projection launched as a programmatic dependent sets itself up and requests weight tiles
+    while the kernel before it still runs, and waits for that kernel before it reads activations.  Tokens, recorded logits
+    and advantages of a free-running Pilot-Commit step must be identical with the switch on (every projection), on for the
+    gate/up projection only, and off; a projection that read its operand early would show up as a difference.  The
+    90-rollout groups take the commit stage above 256 rows, where the fused epilogues run."""
+    from paper_2605_26606_b200 import binding as B
+    w = dataclasses.replace(wl.WORKLOADS["config0"], model=model, n_prompts=5, prompt_len_lo=3, prompt_len_hi=90, group_size=group_size,
+                            n_pilot=8, max_new=40, cap_lo=1, cap_hi=40, data_seed=21,
+                            forced_explicit=((0, 0.5), (1, 0.5), (2, 0.5), (3, 0.0), (4, 0.5)))
+    weights = wl.gen_weights(model, seed=0, threads=2, gain_jitter=0.1)
+    batch = wl.gen_batch(w)
+    eng = RolloutEngine(model, weights, max_rows=5 * group_size, max_prefill_tokens=int(batch.prompt_offsets[-1]))
+    outs, logits = [], []
+    for mask in (0, 31, 4, 31):
+        B.pc_set_dependent_launch(eng.ctx, mask)
+        eng.record_pilot_logits = {s: None for s in (0, 5, 17)}
+        outs.append(eng.pilot_commit_step(w, batch))
+        logits.append({s: v[0].clone() for s, v in eng.record_pilot_logits.items()})
+    eng.record_pilot_logits = None
+    a = outs[0]
+    assert np.any(a["status"] == ostats.COMMIT)
+    for b, lg in zip(outs[1:], logits[1:]):
+        assert np.array_equal(a["status"], b["status"])
+        for p in range(w.n_prompts):
+            for i in range(w.group_size):
+                if a["generated"][p, i]:
+                    assert np.array_equal(a["tokens"][p][i], b["tokens"][p][i]), (p, i)
+        for s in lg:
+            assert torch.equal(lg[s], logits[0][s]), s
+        assert np.array_equal(a["advantages"], b["advantages"])
+
+
 def test_new_schedules_and_token_buffers_reuse_the_captured_steps():
     """pc_decode_run keys its captured steps on shapes and arenas only: running the same step again (fresh schedule tensors, a
     fresh token buffer, another sampling seed) captures nothing new, and a bad row index is caught on the device."""
