@@ -202,15 +202,16 @@ PC_API int pc_set_index_bounds(pc_ctx* ctx, int n_prompts, int64_t n_tokens);
  * tolerances the tests state).  Drops captured decode steps.  The paper has no counterpart. */
 PC_API int pc_set_fused_epilogues(pc_ctx* ctx, int on);
 
-/* bf16 models.  mask: one bit per projection (1 QKV, 2 output, 4 gate/up, 8 down, 16 LM head), 0 .. 31; the default is
- * 31.  A projection whose bit is set is launched as a programmatic dependent of the kernel before it (a row norm, the
- * attention merge or another projection, all of which signal their dependents as soon as they start): its CTAs set up
- * their barriers and tensor memory and request their first weight tiles -- data no kernel of a pass writes -- while
- * that kernel is still running, and wait for it (griddepcontrol.wait) before they touch activations, the step
- * descriptor or any output.  Results are bit-identical to mask 0 (plain stream order); only the start of each projection
- * moves.  Passes of 129 .. 256 rows (two row tiles: measured slower with it) and steps that record phase events
- * (pc_profile_step) run in plain stream order whatever the mask.  Drops captured decode steps.  The paper has no
- * counterpart. */
+/* bf16 models.  mask: one bit per kernel (1 QKV, 2 output, 4 gate/up, 8 down projection, 16 LM head, 32 shared-prefix
+ * attention of decode steps), 0 .. 63; the default is 63.  A kernel whose bit is set is launched as a programmatic
+ * dependent of the kernel before it (a row norm, the QKV post-processing, the attention merge or a projection, all of
+ * which signal their dependents as soon as they start).  A projection's CTAs set up their barriers and tensor memory
+ * and request their first weight tiles while that kernel is still running; the attention kernel requests its first
+ * prompt K/V tiles (written by an earlier call).  Both wait for the kernel before them (griddepcontrol.wait) before they
+ * touch activations or any output.  Results are bit-identical to mask 0 (plain stream order); only the start of each
+ * kernel moves.  Projections of passes of 129 .. 256 rows (two row tiles: measured slower with it) and steps that record
+ * phase events (pc_profile_step) run in plain stream order whatever the mask.  Drops captured decode steps.  The paper
+ * has no counterpart. */
 PC_API int pc_set_dependent_launch(pc_ctx* ctx, int mask);
 
 /* bf16 models, decode steps that only sample (no logits_out, no log-probability buffer): 1 draws the token in

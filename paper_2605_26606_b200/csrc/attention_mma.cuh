@@ -123,7 +123,12 @@ attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __
     constexpr int DT = HD / 8;           // dim n-tiles of the output
     constexpr int TILE_BYTES = G_TK * HD * 2;
     const int grp = blockIdx.z, kvh = blockIdx.y;
-    if (grp >= sd->n_groups) return;
+    // Decode steps launch this kernel as a programmatic dependent of the QKV post-processing: the step descriptor, the row
+    // geometry and the prompt K/V were all written before that kernel started, so the first K/V tiles are requested while
+    // it still runs; q is read after grid_dep_wait().  Every CTA waits on every path (a grid that ended before the kernel
+    // it depends on would let the next kernel start too early).  The prefill form reads K/V of this very pass: it waits first.
+    if (FINAL) grid_dep_wait();
+    if (grp >= sd->n_groups) { grid_dep_wait(); return; }
     // group_row_start holds this pass's groups from entry 0 on (decode: the copy prep_decode_rows leaves in the workspace)
     const int row0 = group_row_start[grp], n_rows = group_row_start[grp + 1] - row0;
     const int n_rep = Hq / Hkv;
@@ -131,7 +136,7 @@ attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __
     const int q_tiles = gridDim.x / n_parts;
     const int my_part = blockIdx.x / q_tiles;
     const int q0 = (blockIdx.x - my_part * q_tiles) * G_QROWS;
-    if (q0 >= n_rows * n_rep) return;
+    if (q0 >= n_rows * n_rep) { grid_dep_wait(); return; }
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -177,6 +182,7 @@ attn_group_kernel(const __grid_constant__ CUtensorMap kv_map, const StepDesc* __
         set_range(g.p_len[row0]);
         if (threadIdx.x == 0)
             for (int t = 0; t < G_STAGES && t < n_tiles; ++t) issue(tile0 + t, t);
+        grid_dep_wait();
     }
 
     // this thread's two query rows: qr = q0 + warp*16 + lane/4 (+8); query row qr = (rollout row qr / n_rep, head qr % n_rep)

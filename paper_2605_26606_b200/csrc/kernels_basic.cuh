@@ -513,6 +513,7 @@ template <typename T>
 __global__ void __launch_bounds__(ROW_WARPS * 32) qkv_post_kernel(const StepDesc* __restrict__ sd, QkvPostArgs<T> A) {
     const int n_heads = A.Hq + 2 * A.Hkv;
     const int item = blockIdx.x * ROW_WARPS + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    grid_dep_launch_dependents();          // the shared-prefix attention kernel may request its first prompt K/V tiles
     if (item >= sd->n_rows * n_heads) return;
     const int row = item / n_heads, head = item - row * n_heads;
     qkv_post_items_warp<T, 1>(lane, A, &row, &head, 1);

@@ -57,6 +57,21 @@ inline cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_
     return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
 }
 
+// The same launch as a programmatic dependent of the kernel before it in the stream (see grid_dep_wait in common.cuh).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k_dep(bool dep, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    if (dep) {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+    }
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -137,7 +152,7 @@ struct pc_ctx {
 
     int fused_epilogues = 1;                 // half-operand models with head_dim 128: QKV post-processing and the MLP norm inside GEMM epilogues
     int fused_sampler = 0;                   // decode steps that only sample: Gumbel-max in the LM head's epilogue, no logits stored
-    int dep_launch = 31;                     // bit per projection (1 QKV, 2 output, 4 gate/up, 8 down, 16 LM head): launched as a programmatic dependent of the kernel before it
+    int dep_launch = 63;                     // bit per kernel (1 QKV, 2 output, 4 gate/up, 8 down projection, 16 LM head, 32 shared-prefix attention): launched as a programmatic dependent of the kernel before it
     int attn_overlap = 0;                    // decode: shared-prefix and suffix attention kernels of a layer on two streams
     cudaStream_t side_stream = nullptr;      // second branch of that fork (created on first use)
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
@@ -250,7 +265,7 @@ struct GemmPlan {
     bool mid = false;      // 128-column tiles (split-K partial sums and the SwiGLU epilogue with one operand matrix only)
 };
 enum GemmKind { GEMM_QKV = 0, GEMM_O = 1, GEMM_GATE_UP = 2, GEMM_DOWN = 3, GEMM_LM_HEAD = 4 };
-enum DepBit { DEP_QKV = 1, DEP_O = 2, DEP_GATE_UP = 4, DEP_DOWN = 8, DEP_LM_HEAD = 16 };      // bits of pc_ctx::dep_launch
+enum DepBit { DEP_QKV = 1, DEP_O = 2, DEP_GATE_UP = 4, DEP_DOWN = 8, DEP_LM_HEAD = 16, DEP_GROUP = 32 };      // bits of pc_ctx::dep_launch
 GemmPlan plan_gemm(const pc_ctx* c, GemmKind kind, const WMap& w, int M, bool may_split) {
     const int tiles_m = (M + pc::tc::BM - 1) / pc::tc::BM;
     const int k_blocks = w.K / pc::tc::BK;
@@ -290,7 +305,7 @@ GemmPlan plan_gemm(const pc_ctx* c, GemmKind kind, const WMap& w, int M, bool ma
 // measured on the 1.5B shape, decode steps of 16 / 64 / 128 rows take 6.7 / 5.4 / 4.4 % less time with it, steps of 192 and
 // 256 rows 1.8 % more, 384 rows the same, 560 rows 2 % less.
 inline bool dependent_launch(const pc_ctx* c, int dep_bit, int M) {
-    return (c->dep_launch & dep_bit) != 0 && c->prof_active_layer < 0 && !(M > pc::tc::BM && M <= 2 * pc::tc::BM);
+    return (c->dep_launch & dep_bit) != 0 && c->prof_active_layer < 0 && (dep_bit == DEP_GROUP || !(M > pc::tc::BM && M <= 2 * pc::tc::BM));
 }
 
 // map_a_lo != nullptr: the activations come as a high bf16 part and its rounding remainder, both multiplied with the
@@ -454,7 +469,10 @@ int attention_bf16(pc_ctx* c, cudaStream_t st, const pc::StepDesc* sd, int M, in
         cudaStreamWaitEvent(c->side_stream, c->ev_fork, 0);
         gst = c->side_stream;
     }
-    launch_k(am::attn_group_kernel<HD, false>, dim3(ggrid), dim3(am::G_THREADS), am::group_smem_bytes<HD>(), gst, 
+    // after the QKV post-processing kernel or the QKV projection (both signal their dependents early); not on the side stream
+    // of the fork and not after the persistent kernel
+    const bool group_dep = !overlap && part_out == nullptr && dependent_launch(c, DEP_GROUP, M);
+    launch_k_dep(group_dep, am::attn_group_kernel<HD, false>, dim3(ggrid), dim3(am::G_THREADS), am::group_smem_bytes<HD>(), gst, 
         c->map_prompt_kv, sd, prompt_arena.n_slots, d.n_q_heads, d.n_kv_heads, layer, q, plan.group_row_start, g, scale_log2, part,
         attn, attn_lo, c->err);
     if (overlap) cudaEventRecord(c->ev_join, gst);
@@ -767,7 +785,7 @@ int pc_set_fused_sampler(pc_ctx* ctx, int on) {
 }
 
 int pc_set_dependent_launch(pc_ctx* ctx, int mask) {
-    if (ctx == nullptr || mask < 0 || mask > 31) return PC_ERR_INVALID_ARG;
+    if (ctx == nullptr || mask < 0 || mask > 63) return PC_ERR_INVALID_ARG;
     if (mask != ctx->dep_launch) ctx->drop_graphs();
     ctx->dep_launch = mask;
     return PC_OK;

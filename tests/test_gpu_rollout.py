@@ -375,8 +375,8 @@ def test_persistent_decode_kernel_equals_one_kernel_per_operation(model):
 def test_dependent_launch_of_the_projections_changes_no_bit(model, group_size):
     """pc_set_dependent_launch: a projection launched as a programmatic dependent sets itself up and requests weight tiles
     while the kernel before it still runs, and waits for that kernel before it reads activations.  Tokens, recorded logits
-    and advantages of a free-running Pilot-Commit step must be identical with the switch on (every projection), on for the
-    gate/up projection only, and off; a projection that read its operand early would show up as a difference.  The
+    and advantages of a free-running Pilot-Commit step must be identical with the switch on (every projection and the shared-prefix attention), on for the
+    gate/up projection only, on for the attention kernel only, and off; a projection that read its operand early would show up as a difference.  The
     90-rollout groups take the commit stage above 256 rows, where the fused epilogues run."""
     from paper_2605_26606_b200 import binding as B
     w = dataclasses.replace(wl.WORKLOADS["config0"], model=model, n_prompts=5, prompt_len_lo=3, prompt_len_hi=90, group_size=group_size,
@@ -386,7 +386,7 @@ def test_dependent_launch_of_the_projections_changes_no_bit(model, group_size):
     batch = wl.gen_batch(w)
     eng = RolloutEngine(model, weights, max_rows=5 * group_size, max_prefill_tokens=int(batch.prompt_offsets[-1]))
     outs, logits = [], []
-    for mask in (0, 31, 4, 31):
+    for mask in (0, 63, 4, 32, 63):
         B.pc_set_dependent_launch(eng.ctx, mask)
         eng.record_pilot_logits = {s: None for s in (0, 5, 17)}
         outs.append(eng.pilot_commit_step(w, batch))
