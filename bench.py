@@ -455,7 +455,8 @@ def main():
                      "sampled_decode_steps": len(per_sample), "per_launch_avg": per_op_ms,
                      "estimated_per_decode_step": est_ms,
                      "note": "CUDA events around the operations of layer %d and the LM head / sampler in every 32nd decode step; "
-                             "a layer operation is counted n_layers times" % eng.profile_layer},
+                             "a layer operation is counted n_layers times; the sampled steps run in plain stream order (an event between "
+                             "two kernels rules out the dependent launches the other steps use)" % eng.profile_layer},
         "live_rows_histogram": live_hist,
         "hbm_step": {"bytes_per_step": step_bytes, "achieved_gbs": step_bytes * args.steps / (dev_ms * 1e-3) / 1e9,
                      "frac_of_measured": step_bytes * args.steps / (dev_ms * 1e-3) / 1e9 / peak,
